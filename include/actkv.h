@@ -1,0 +1,219 @@
+/*
+ * actkv.h — C ABI of the action-guided KV-cache compression hot path (ActKV) for one B200.
+ *
+ * The library runs the three page-aware primitives the paper distils every eviction method
+ * into (Section 3.3: CalAttn -> Eviction -> Compaction) plus the confidence monitor that sets
+ * the budget (Section 6, Algorithm 2), directly on a paged bf16 KV cache
+ * PagedKVCache[2, B, BS, H, D] addressed through a block table (Section 2.5).
+ *
+ * Conventions that hold for every entry point
+ *   - `extern "C"`, plain pointers and sizes.  Unless a parameter says "host", a pointer is a
+ *     DEVICE pointer owned by the caller.  The two descriptor structs and the parameter struct
+ *     are HOST structs (passed by pointer, read during the call) that hold device pointers.
+ *   - Every call is asynchronous on `stream`, never synchronises, never allocates or frees
+ *     device memory.  Scratch comes from the caller: `ws` of at least
+ *     `actkv_*_workspace_bytes(...)` bytes, 256-byte aligned.
+ *   - Return value: ACTKV_OK or a negative code for what the host can see (bad argument,
+ *     workspace too small, launch failure).  What only the device can see (a page id out of
+ *     range, a free list that is too short) is written to the caller's `status[4]` int32 words:
+ *     status[0] = first error code (0 while clean), status[1..2] = where (request / unit,
+ *     offending value).  Kernels never trap; an out-of-range page id is replaced by page 0 for
+ *     the access and reported.  When the plan step of actkv_compact reports ACTKV_E_NOFREE the
+ *     copy and table-update steps of that call do nothing, so pool and tables stay unmodified.
+ *   - All indices are int32.  Strides are in ELEMENTS (bf16), the head dimension is contiguous.
+ *   - "unit" = one (layer, KV head, request); units are independent in score and select.
+ *   - Arrays with a leading layer axis are RELATIVE to `layer_begin`: slab 0 belongs to layer
+ *     `layer_begin`.  Only the pool is indexed by absolute layer.
+ */
+#ifndef ACTKV_H_
+#define ACTKV_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define ACTKV_OK            0
+#define ACTKV_E_INVALID    -1   /* bad argument / unsupported shape (host-detected)              */
+#define ACTKV_E_WORKSPACE  -2   /* `ws_bytes` smaller than the matching *_workspace_bytes()     */
+#define ACTKV_E_CUDA       -3   /* a CUDA runtime call or launch failed                          */
+#define ACTKV_E_BADPAGE    -4   /* device: page id outside [0, n_pages) met in a page table      */
+#define ACTKV_E_NOFREE     -5   /* device: free list holds fewer pages than compaction needs     */
+#define ACTKV_E_BADINDEX   -6   /* device: selected token index outside [0, seq_len)             */
+#define ACTKV_E_TIMEOUT    -7   /* device: a bounded wait inside a kernel gave up                */
+
+/* CUDA stream handle (identical to cudaStream_t; spelled out so the header needs no CUDA). */
+typedef struct CUstream_st* actkv_stream_t;
+
+/*
+ * The paged pool, Section 2.5: PagedKVCache[2, B, BS, H, D] per layer.
+ * Element (layer l, kv in {0 = K, 1 = V}, page p, slot s, head h, dim d) lives at
+ *   base + l*stride_layer + kv*stride_kv + p*stride_page + s*stride_slot + h*stride_head + d.
+ * The tensor-core score path needs page_size 16, head_dim 128, stride_head == head_dim,
+ * stride_slot == n_kv_heads*head_dim, stride_page == page_size*stride_slot and a 128-byte
+ * aligned base; other layouts take the FMA path.
+ */
+typedef struct {
+  void*   base;                 /* device, bf16 */
+  int32_t n_layers, n_pages, page_size, n_kv_heads, head_dim;
+  int64_t stride_layer, stride_kv, stride_page, stride_slot, stride_head;
+} actkv_pool_t;
+
+/*
+ * Block table and allocator state, Section 2.5 (block_table, seqused_k) plus the free list the
+ * freed blocks go back to (Section 7.2, last paragraph).  Logical token j of request r sits in
+ * physical slot page_table[r][j / page_size] * page_size + j % page_size.
+ * free_list is a LIFO stack of page ids, the top at free_list[*free_count - 1].
+ */
+typedef struct {
+  int32_t  n_req, max_pages;
+  int32_t* page_table;          /* [n_req, max_pages], unused entries -1 */
+  int32_t* seq_len;             /* [n_req] */
+  int32_t* free_list;           /* [n_pages] */
+  int32_t* free_count;          /* [1] */
+} actkv_tables_t;
+
+/*
+ * Parameters of the confidence monitor, Section 6.1 and Algorithm 2; defaults of Section 8.1
+ * (Configuration): k=20, w=64, s=8, b=10, scale_up=1.75, B_upper=30000.
+ * The clamp is an addition of this library (off when clamp_hi_ppm <= 0): after the update,
+ * B' = min(max(B', ceil(L*clamp_lo_ppm/1e6)), floor(L*clamp_hi_ppm/1e6)), L = seq_len, in
+ * exact integer arithmetic.
+ */
+typedef struct {
+  int32_t k;                    /* top-k tokens per distribution                         */
+  int32_t w, s;                 /* min-pooling window and stride                         */
+  double  b_percent;            /* bottom-b% of the pooled sequence is kept               */
+  double  scale_up;             /* B' = floor(B*scale_up) when the fitted slope is < 0    */
+  int32_t B_upper;              /* cap on B'                                              */
+  int32_t clamp_lo_ppm, clamp_hi_ppm;
+} actkv_budget_params_t;
+
+/* Per-unit report of actkv_select: the n-th largest score and how ties at it were resolved. */
+typedef struct {
+  float   threshold;            /* score of the last entry kept (0 if none kept)          */
+  int32_t n_equal_kept;         /* entries equal to threshold that were kept              */
+  int32_t n_equal_total;        /* entries equal to threshold in the unit                 */
+  int32_t n_keep;               /* min(budget, seq_len)                                   */
+} actkv_tie_t;
+
+/* ---------------------------------------------------------------------------------------
+ * actkv_budget — confidence monitor and budget update (Section 6.1 equations, Algorithm 2).
+ *
+ * For every new token i of request r (rows tok_indptr[r] .. tok_indptr[r+1] of `logits`):
+ *   T_i = -(1/k) sum_{j<=k} log P_i(j)  over the k most probable tokens
+ *       = logsumexp(z_i) - mean(top-k z_i),
+ * appended (as float32) to the request's history conf_hist[r][hist_len[r] ...].  Then over the
+ * whole history (length Lh): R'_m = min T[m*s .. m*s+w), m = 0..floor((Lh-w)/s); R = the values
+ * of R' not above its b-th percentile (nearest rank: the max(1, ceil(b/100*M))-th smallest), in
+ * time order; alpha = least-squares slope of R against 0..|R|-1 (0 when |R| < 2 or Lh < w);
+ *   B' = alpha < 0 ? min(floor(B*scale_up), B_upper) : B,   then the optional clamp.
+ * logits     float32 [n_rows, vocab] row-major, n_rows = tok_indptr[n_req] (passed as n_rows).
+ * tok_indptr int32 [n_req+1].  conf_hist float32 [n_req, hist_cap]; hist_len int32 [n_req]
+ *            (updated).  Tokens that do not fit in hist_cap are dropped and reported as
+ *            ACTKV_E_INVALID in status.
+ * seq_len    int32 [n_req] (only read when the clamp is on; may be NULL otherwise).
+ * budget_in / budget_out int32 [n_req] (may alias).  slope_out double [n_req] or NULL.
+ * logits == NULL with n_rows == 0 runs only the trend / update step on the stored history.
+ */
+size_t actkv_budget_workspace_bytes(int32_t n_rows, int32_t vocab, int32_t n_req);
+int actkv_budget(const float* logits, const int32_t* tok_indptr, int32_t n_rows, int32_t vocab,
+                 float* conf_hist, int32_t* hist_len, int32_t hist_cap,
+                 const actkv_budget_params_t* params /* host */,
+                 const int32_t* seq_len, const int32_t* budget_in, int32_t* budget_out,
+                 double* slope_out, int32_t n_req, void* ws, size_t ws_bytes,
+                 int32_t* status, actkv_stream_t stream);
+
+/* ---------------------------------------------------------------------------------------
+ * actkv_score — action-region attention score of every cached entry
+ * (Section 2.3 attention definition; Section 7.1 LSE identity; Algorithm 3 pooling).
+ *
+ * For layer l, request r, KV head h, key j < L_r, window row w < W_r and q-head
+ * qh = h*G + g (G = n_q_heads / n_kv_heads, contiguous GQA groups):
+ *   s      = sm_scale * <q[l, win_indptr[r]+w, qh, :], K[l, slot(r, j), h, :]>
+ *   lse    = log sum_{j visible} exp(s)              (or lse_in when supplied)
+ *   a      = exp(s - lse)                            (Section 7.1: A = exp(s - LSE))
+ *   score[l, h, tok_indptr[r]+j] = (1/W_r) * sum_w max_g a      (Algorithm 3 steps 4-5)
+ * causal == 0: every row sees every key.  causal != 0: the window is the last W_r cached
+ * tokens, row w sees keys j <= L_r - W_r + w; a masked (w, j) pair contributes 0 and the
+ * divisor stays W_r.
+ * q          bf16 [NLs, sum_win, n_q_heads, head_dim], NLs = layer_end - layer_begin.
+ * win_indptr int32 [n_req+1]; tok_indptr int32 [n_req+1] (exclusive prefix sums of W_r, L_r).
+ * lse_in     float32 [NLs, sum_win, n_q_heads] natural-log units of the scaled logits, or NULL
+ *            to compute it here (one extra pass over K).  lse_out: same shape or NULL.
+ * score_out  float32 [NLs, n_kv_heads, sum_tok].
+ * sum_win, max_win, sum_tok, max_tok: host copies of win_indptr[n_req], max W_r,
+ *            tok_indptr[n_req], max L_r (upper bounds are accepted for the two maxima).
+ * W_r == 0 for a request with L_r > 0 is reported as ACTKV_E_INVALID in status.
+ */
+size_t actkv_score_workspace_bytes(const actkv_pool_t* pool /* host */, int32_t n_req,
+                                   int32_t n_layers_sub, int32_t n_q_heads, int32_t sum_win,
+                                   int32_t max_win, int32_t max_tok);
+int actkv_score(const actkv_pool_t* pool /* host */, const actkv_tables_t* tables /* host */,
+                int32_t layer_begin, int32_t layer_end,
+                const void* q, const int32_t* win_indptr, int32_t n_q_heads,
+                const float* lse_in, float sm_scale, int32_t causal,
+                const int32_t* tok_indptr, float* score_out, float* lse_out,
+                int32_t sum_win, int32_t max_win, int32_t sum_tok, int32_t max_tok,
+                void* ws, size_t ws_bytes, int32_t* status, actkv_stream_t stream);
+
+/* ---------------------------------------------------------------------------------------
+ * actkv_keep_indptr — helper: keep_indptr[r] = sum_{r'<r} min(budget[r'], seq_len[r']),
+ * keep_indptr[n_req] = total (Algorithm 1 step 5 keeps min(B, L) entries).  One tiny kernel.
+ */
+int actkv_keep_indptr(const int32_t* seq_len, const int32_t* budget, int32_t n_req,
+                      int32_t* keep_indptr, actkv_stream_t stream);
+
+/* ---------------------------------------------------------------------------------------
+ * actkv_select — TopK(score, k = B) per unit (Algorithm 1 step 5, applied to the pooled
+ * score, independently per layer and KV head).
+ *
+ * For unit (o, r), o < n_outer (= layers * KV heads), over score[o, tok_indptr[r] ..
+ * tok_indptr[r+1]): keep the n_r = min(budget[r], L_r) largest float32 scores; among equal
+ * scores the lower token index wins; emit the kept token indices (0-based within the
+ * request) in ascending order to sel_idx[o*sel_stride + keep_indptr[r] ...].
+ * score      float32 [n_outer, sum_tok] (values must be >= 0, as pooled probabilities are;
+ *            -0.0 and NaN are treated by their bit pattern order).
+ * keep_mask  optional uint32 bitmap [n_outer, ceil(sum_tok/32)]: bit (tok_indptr[r]+j) set
+ *            iff kept; must be zero-filled by the caller.  NULL to skip.
+ * tie_report optional [n_outer, n_req].
+ */
+size_t actkv_select_workspace_bytes(int32_t n_outer, int32_t n_req, int32_t max_tok);
+int actkv_select(const float* score, const int32_t* tok_indptr, int32_t sum_tok,
+                 const int32_t* budget, int32_t n_outer, int32_t n_req,
+                 const int32_t* keep_indptr, int32_t* sel_idx, int64_t sel_stride,
+                 uint32_t* keep_mask, actkv_tie_t* tie_report,
+                 void* ws, size_t ws_bytes, int32_t* status, actkv_stream_t stream);
+
+/* ---------------------------------------------------------------------------------------
+ * actkv_compact — pack the survivors into fresh pages and free the old ones
+ * (Section 7.2 / Algorithm 4: survivors packed contiguously, pure copy, freed blocks returned;
+ *  here into pages popped from the free list instead of the tail of the old ones).
+ *
+ * Requests with budget[r] >= seq_len[r] are left untouched.  For the others, in ascending r,
+ * n_r = budget[r], X_r = ceil(n_r / page_size), off_r = sum of X over earlier compacting
+ * requests:  new_page[r][i] = free_list[free_count - 1 - (off_r + i)],  i < X_r.
+ * For every layer in [layer_begin, layer_end), head h, i < n_r: the K row and the V row of
+ * token sel_idx[(l-layer_begin)*H + h][keep_indptr[r] + i] move to logical slot i of the new
+ * pages.  When layer_end == pool->n_layers the tables are updated after the copies:
+ * page_table[r] = new pages then -1, seq_len[r] = n_r, free_count -= sum X, then for r
+ * ascending and i ascending free_list[free_count++] = old page i of r.
+ * Calls on layer sub-ranges recompute the same plan from the still-unchanged tables.
+ * max_keep: host upper bound on n_r (<= max_pages*page_size).
+ */
+size_t actkv_compact_workspace_bytes(int32_t n_req, int32_t max_pages);
+int actkv_compact(const actkv_pool_t* pool /* host */, const actkv_tables_t* tables /* host */,
+                  int32_t layer_begin, int32_t layer_end,
+                  const int32_t* sel_idx, int64_t sel_stride, const int32_t* keep_indptr,
+                  const int32_t* budget, int32_t max_keep,
+                  void* ws, size_t ws_bytes, int32_t* status, actkv_stream_t stream);
+
+/* Library version string (host pointer to static storage). */
+const char* actkv_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* ACTKV_H_ */
