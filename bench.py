@@ -1,0 +1,418 @@
+#!/usr/bin/env python
+"""Benchmark of the ActKV compression hot path on B200.
+
+One step = one pass of the whole path over one batch of synthetic input:
+  actkv_budget (64 action-token logit rows per request) -> actkv_keep_indptr ->
+  actkv_score_lse + actkv_score -> actkv_select -> actkv_compact   over all layers.
+Metric: KV tokens compressed per second (tokens = cached tokens examined, counted once per
+request whatever the number of layers and heads).  Default workload: the 8 x 35000-token
+Qwen3-30B-A3B attention shape (48 layers, 32 q / 4 KV heads, head_dim 128, page 16, window 64,
+budget 26%).
+
+  python bench.py --gpus 1 --steps 5 --warmup 3
+  python -m torch.distributed.run --nproc-per-node N ... bench.py --gpus N   (N independent replicas)
+  python bench.py --impl reference     (the CPU oracle on a bounded sample of the same workload)
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+import torch
+
+from paper_2609_31395_b200 import synth
+
+METRIC = "KV tokens compressed/s (score+select+compact)"
+UNIT = "tokens/s"
+VOCAB = 151936
+LOGIT_ROWS = 64          # action-token logit rows per request fed to actkv_budget each step
+BUDGET_PPM = 260000      # config: budget 26% of the length (clamp of the monitor's output)
+
+
+def peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return {"hbm_gbs": d["hbm_gbs"], "tf_burst": d["bf16_tflops"], "tf_sustained": d["bf16_tflops_sustained"],
+                "source": "measured"}
+    return {"hbm_gbs": 6650.0, "tf_burst": 1590.0, "tf_sustained": 1400.0, "source": "fallback"}
+
+
+def make_workload(name: str, layers):
+    if name == "c3":
+        wl = synth.config3(48 if layers is None else layers)
+    elif name == "c2":
+        wl = synth.config2(36 if layers is None else layers)
+    elif name == "c1":
+        wl = synth.config1()
+    else:
+        raise SystemExit(f"unknown workload {name}")
+    return wl
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.proc = None
+        self.lines = []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                                          "-lms", "100", "-i", str(self.index)], stdout=subprocess.PIPE, text=True)
+            threading.Thread(target=self._read, daemon=True).start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for ln in self.lines:
+            f = [x.strip() for x in ln.split(",")]
+            if len(f) < 7:
+                continue
+            try:
+                sm.append(float(f[0])); mx.append(float(f[1]))
+            except ValueError:
+                continue
+            for n, v in zip(names, f[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def visible_gpu_index(local_rank: int) -> int:
+    vis = os.environ.get("CUDA_VISIBLE_DEVICES")
+    if vis:
+        try:
+            return int(vis.split(",")[local_rank])
+        except Exception:
+            return local_rank
+    return local_rank
+
+
+# ---------------------------------------------------------------------------------------------
+# the CPU oracle on a bounded sample (cpu_baseline and --impl reference)
+
+
+def oracle_sample(wl, n_heads_sample: int = 2):
+    """Draws a one-layer, one-request instance of `wl`'s shape on the CPU and returns a closure that
+    runs the oracle's budget + score + select + compact on it, plus the scaling to the metric."""
+    from oracle import actkv_oracle as O
+    small = synth.Workload(wl.name + "_sample", 1, n_heads_sample, wl.group, wl.seq_lens[:1], wl.windows[:1],
+                           wl.budgets[:1], head_dim=wl.head_dim, page_size=wl.page_size, causal=wl.causal,
+                           table_style="permutation", n_topics=wl.n_topics, seed=wl.seed)
+    inst = synth.generate(small, "cpu")
+    bits = lambda t: t.contiguous().view(torch.int16).numpy().view(np.uint16)
+    pool_b, q_b = bits(inst.pool), bits(inst.q)
+    pt, sl = inst.page_table.numpy(), inst.seq_len.numpy()
+    logits, tind = synth.confidence_logits(1, LOGIT_ROWS, VOCAB, seed=wl.seed, device="cpu")
+    logits_np = logits.numpy()
+    bp = O.BudgetParams(clamp_lo_ppm=BUDGET_PPM, clamp_hi_ppm=BUDGET_PPM)
+
+    def run():
+        hist = np.zeros((1, 4096), dtype=np.float32)
+        _, _, bud, _, _ = O.budget(logits_np, tind.numpy(), hist, [0], small.budgets, bp, sl)
+        sc, _, tok = O.score(pool_b, pt, sl, q_b, inst.win_indptr.numpy(), small.n_q_heads, small.sm_scale,
+                             small.causal)
+        sel = [[[O.select_unit(sc[0, h], int(bud[0]))] for h in range(n_heads_sample)]]
+        tables = O.Tables(pt.copy(), sl.copy(), inst.free_list.numpy().copy(), int(inst.free_count))
+        O.compact(pool_b, tables, sel, bud)
+
+    # the sample covers 1 request x n_heads_sample heads x 1 layer of the (R x Hkv x NL) workload
+    frac = (1.0 / wl.n_req) * (n_heads_sample / wl.n_kv_heads) * (1.0 / wl.n_layers)
+    tokens_equiv = sum(wl.seq_lens) * frac
+    desc = (f"1 request x {n_heads_sample} of {wl.n_kv_heads} KV heads x 1 of {wl.n_layers} layers "
+            f"({wl.seq_lens[0]} tokens, window {wl.windows[0]}, budget {wl.budgets[0]}) + {LOGIT_ROWS} logit rows; "
+            f"tokens/s scaled by the unit count")
+    return run, tokens_equiv, desc
+
+
+def timed_cpu(fn, reps: int = 1):
+    """Runs fn `reps` times; returns (seconds per run, threads actually busy = CPU time / wall time)."""
+    w0, c0 = time.perf_counter(), time.process_time()
+    for _ in range(reps):
+        fn()
+    w, c = time.perf_counter() - w0, time.process_time() - c0
+    return w / reps, max(1, int(round(c / max(w, 1e-9))))
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    wl = make_workload(args.workload, args.layers)
+    run, tokens_equiv, desc = oracle_sample(wl)
+    for _ in range(args.warmup):
+        run()
+    dt, cores = timed_cpu(run, args.steps)
+    v = tokens_equiv / dt
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": v, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": wl.name, "note": "CPU oracle on a bounded sample per step: " + desc},
+        "cpu_baseline": {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": desc},
+        "e2e": {"value": v, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0}))
+
+
+# ---------------------------------------------------------------------------------------------
+# the CUDA path
+
+
+def run_ours(args):
+    from paper_2609_31395_b200 import binding as B
+    from paper_2609_31395_b200 import harness as H
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py: no CUDA device; the CUDA path has no CPU fallback")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+    B.load()
+    pk = peaks()
+
+    wl = make_workload(args.workload, args.layers)
+    wl.seed += 100 * rank                      # every replica draws its own batch
+    R, NL, Hkv, G, D = wl.n_req, wl.n_layers, wl.n_kv_heads, wl.group, wl.head_dim
+    inst = synth.generate(wl, dev)
+    sz = H.sizes_of(inst)
+    comp = H.Compressor(inst.pool, inst.page_table, inst.seq_len, inst.free_list, inst.free_count, wl.n_q_heads, sz,
+                        layers_per_call=args.layers_per_call, want_lse=True)
+    # budget inputs: LOGIT_ROWS action-token logit rows per request
+    logits, ltok = synth.confidence_logits(R, LOGIT_ROWS, VOCAB, seed=wl.seed, device=dev)
+    n_rows = logits.shape[0]
+    hist_cap = 4096
+    conf_hist = torch.zeros((R, hist_cap), dtype=torch.float32, device=dev)
+    hist_len = torch.zeros(R, dtype=torch.int32, device=dev)
+    budget_in = torch.full((R,), 512, dtype=torch.int32, device=dev)
+    budget_dev = torch.zeros(R, dtype=torch.int32, device=dev)
+    ws_budget = torch.empty(B.actkv_budget_workspace_bytes(n_rows, R, hist_cap) + 256, dtype=torch.uint8, device=dev)
+    bparams = B.BudgetParams.paper_defaults(clamp_lo_ppm=BUDGET_PPM, clamp_hi_ppm=BUDGET_PPM)
+    assert all(b == L * BUDGET_PPM // 1000000 for b, L in zip(wl.budgets, wl.seq_lens)) or args.workload != "c3"
+    if args.workload != "c3":                  # other shapes: fixed budgets, the monitor still runs
+        bparams = B.BudgetParams.paper_defaults()
+
+    saved = [t.clone() for t in (inst.page_table, inst.seq_len, inst.free_list, inst.free_count)]
+
+    def restore():
+        for dst, src in zip((inst.page_table, inst.seq_len, inst.free_list, inst.free_count), saved):
+            dst.copy_(src)
+        hist_len.zero_()
+        comp.status.zero_()
+
+    lse_supplied = None
+    stage_names = ["budget", "lse", "score", "select", "compact"]
+
+    def one_step(events=None):
+        def mark(name):
+            if events is not None:
+                e = torch.cuda.Event(enable_timing=True)
+                e.record()
+                events.append((name, e))
+        mark("start")
+        B.actkv_budget(logits, ltok, n_rows, VOCAB, conf_hist, hist_len, hist_cap, bparams, inst.seq_len, budget_in,
+                       budget_dev, None, R, ws_budget, comp.status)
+        bud = budget_dev if args.workload == "c3" else inst.budget
+        mark("budget")
+        n = comp.step(inst.q, inst.win_indptr, inst.tok_indptr, bud, wl.sm_scale, wl.causal,
+                      lse_in=lse_supplied, marks=(lambda nm: mark(nm)) if events is not None else (lambda nm: None))
+        return n + 2
+
+    for _ in range(args.warmup):
+        restore()
+        one_step()
+    torch.cuda.synchronize()
+    comp.check_status()
+    if args.lse == "supplied":
+        lse_supplied = comp.lse.clone()
+
+    sampler = ClockSampler(visible_gpu_index(local_rank))
+    sampler.start()
+    if dist is not None:
+        dist.barrier()
+    torch.cuda.synchronize()
+    all_events, launches = [], 0
+    t_wall0 = time.perf_counter()
+    for _ in range(args.steps):
+        restore()
+        ev = []
+        launches = one_step(ev)
+        all_events.append(ev)
+    torch.cuda.synchronize()
+    if dist is not None:
+        dist.barrier()
+    t_wall = time.perf_counter() - t_wall0
+    clocks = sampler.stop()
+    comp.check_status()
+
+    stage_ms = {k: 0.0 for k in stage_names}
+    total_ms = 0.0
+    for ev in all_events:
+        total_ms += ev[0][1].elapsed_time(ev[-1][1])
+        prev = ev[0][1]
+        for name, e in ev[1:]:
+            if name == "begin":
+                continue
+            stage_ms[name] += prev.elapsed_time(e)
+            prev = e
+    ms_per_step = total_ms / args.steps
+    stage_ms = {k: v / args.steps for k, v in stage_ms.items()}
+    t = torch.tensor([ms_per_step], dtype=torch.float64, device=dev)
+    if dist is not None:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    ms_max = float(t.item())
+    tokens = sum(wl.seq_lens)
+    value = world * tokens / (ms_max * 1e-3)
+
+    # ---- roofline of the dominant kernel --------------------------------------------------------
+    rho = sum(min(b, L) for b, L in zip(wl.budgets, wl.seq_lens)) / max(1, tokens)
+    flops_pass = 2.0 * sum(W * G * L for W, L in zip(wl.windows, wl.seq_lens)) * D * Hkv * NL
+    bytes_k = 2.0 * D * tokens * Hkv * NL
+    alg_bytes = (264.0 + 1032.0 * rho) * tokens * Hkv * NL
+    n_calls = -(-NL // comp.lpc)
+    stages = {
+        "lse": {"bound": "tensor", "achieved": flops_pass / (stage_ms["lse"] * 1e-3) / 1e12 if stage_ms["lse"] else None,
+                "peak": pk["tf_sustained"], "unit": "TFLOP/s"},
+        "score": {"bound": "tensor", "achieved": flops_pass / (stage_ms["score"] * 1e-3) / 1e12, "peak": pk["tf_sustained"],
+                  "unit": "TFLOP/s"},
+        "compact": {"bound": "hbm", "achieved": 1024.0 * rho * tokens * Hkv * NL / (stage_ms["compact"] * 1e-3) / 1e9,
+                    "peak": pk["hbm_gbs"], "unit": "GB/s"},
+        "budget": {"bound": "hbm", "achieved": 4.0 * n_rows * VOCAB / (stage_ms["budget"] * 1e-3) / 1e9,
+                   "peak": pk["hbm_gbs"], "unit": "GB/s"},
+    }
+    for s in stages.values():
+        s["frac"] = None if s["achieved"] is None else s["achieved"] / s["peak"]
+    dom = max(("lse", "score", "compact"), key=lambda k: stage_ms[k])
+    roofline = dict(stages[dom])
+    roofline.update({"kernel": dom, "launches_per_step": n_calls, "ms_per_launch": stage_ms[dom] / n_calls,
+                     "traffic": None, "peak_source": pk["source"] + (" sustained bf16" if stages[dom]["bound"] == "tensor" else " copy")})
+    hbm_frac_whole = alg_bytes / (ms_max * 1e-3) / 1e9 / pk["hbm_gbs"]
+
+    # ---- end to end: host buffers in, host results out, every step -------------------------------
+    e2e = None
+    if not args.no_e2e:
+        q_host = inst.q.cpu().pin_memory()
+        logits_host = logits.cpu().pin_memory()
+        tabs_host = [t.cpu().pin_memory() for t in saved]
+        bin_host = budget_in.cpu().pin_memory()
+        out_host = [torch.empty_like(t).pin_memory() for t in tabs_host[:2]] + \
+                   [torch.empty(1, dtype=torch.int32).pin_memory(), torch.empty(4, dtype=torch.int32).pin_memory(),
+                    torch.empty(R, dtype=torch.int32).pin_memory()]
+        h2d = q_host.numel() * 2 + logits_host.numel() * 4 + sum(t.numel() * 4 for t in tabs_host) + bin_host.numel() * 4
+        d2h = sum(t.numel() * 4 for t in out_host)
+        e2e_ms = []
+        for it in range(1 + min(args.steps, 3)):
+            hist_len.zero_(); comp.status.zero_()
+            torch.cuda.synchronize()
+            if dist is not None:
+                dist.barrier()
+            t0 = time.perf_counter()
+            inst.q.copy_(q_host, non_blocking=True)
+            logits.copy_(logits_host, non_blocking=True)
+            for dst, src in zip((inst.page_table, inst.seq_len, inst.free_list, inst.free_count), tabs_host):
+                dst.copy_(src, non_blocking=True)
+            budget_in.copy_(bin_host, non_blocking=True)
+            one_step()
+            out_host[0].copy_(inst.page_table, non_blocking=True)
+            out_host[1].copy_(inst.seq_len, non_blocking=True)
+            out_host[2].copy_(inst.free_count, non_blocking=True)
+            out_host[3].copy_(comp.status, non_blocking=True)
+            out_host[4].copy_(budget_dev, non_blocking=True)
+            torch.cuda.synchronize()
+            if it > 0:
+                e2e_ms.append((time.perf_counter() - t0) * 1e3)
+        te = torch.tensor([sum(e2e_ms) / len(e2e_ms)], dtype=torch.float64, device=dev)
+        if dist is not None:
+            dist.all_reduce(te, op=dist.ReduceOp.MAX)
+        e2e = {"value": world * tokens / (float(te.item()) * 1e-3), "unit": UNIT, "ms_per_step": float(te.item()),
+               "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h),
+               "note": "KV pool stays resident in HBM (it is the cache being compressed); queries, logits, tables "
+                       "and budgets come from pinned host memory, new tables / budgets / status go back"}
+
+    # ---- the oracle on the host cores (rank 0, single GPU only) ----------------------------------
+    cpu_baseline = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        run, tokens_equiv, desc = oracle_sample(wl, n_heads_sample=wl.n_kv_heads)
+        dt, cores = timed_cpu(run, 2)
+        cpu_baseline = {"value": tokens_equiv / dt, "unit": UNIT, "cores": cores, "kind": "oracle",
+                        "sample": desc, "seconds": 2 * dt}
+
+    if rank == 0:
+        out = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms_max, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": wl.name, "requests": R, "tokens_per_request": wl.seq_lens[0], "layers": NL,
+                       "kv_heads": Hkv, "q_heads": wl.n_q_heads, "head_dim": D, "page": wl.page_size,
+                       "window": wl.windows[0], "budget": wl.budgets[0], "lse": args.lse,
+                       "layers_per_call": comp.lpc, "replicas": world,
+                       "l2": "inputs (KV pool %.1f GB) far larger than the 126 MB L2" % (inst.pool.numel() * 2 / 1e9)},
+            "stage_ms": stage_ms, "hbm_roofline_frac_whole_step": hbm_frac_whole,
+            "algorithmic_bytes_per_step": alg_bytes, "k_bytes_per_pass": bytes_k,
+            "roofline": roofline, "roofline_stages": stages, "cpu_baseline": cpu_baseline, "e2e": e2e,
+            "clocks": clocks, "gpu_launches": launches, "wall_s_timed_region": t_wall,
+        }
+        print(json.dumps(out))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="c3", choices=["c1", "c2", "c3"])
+    ap.add_argument("--layers", type=int, default=None, help="override the layer count (debugging only)")
+    ap.add_argument("--layers-per-call", type=int, default=None)
+    ap.add_argument("--lse", default="internal", choices=["internal", "supplied"])
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.warmup < 3 and args.impl == "ours":
+        print("note: fewer than 3 warm-up steps", file=sys.stderr)
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -117,8 +117,9 @@ typedef struct {
  * seq_len    int32 [n_req] (only read when the clamp is on; may be NULL otherwise).
  * budget_in / budget_out int32 [n_req] (may alias).  slope_out double [n_req] or NULL.
  * logits == NULL with n_rows == 0 runs only the trend / update step on the stored history.
+ * hist_cap <= 65536.
  */
-size_t actkv_budget_workspace_bytes(int32_t n_rows, int32_t vocab, int32_t n_req);
+size_t actkv_budget_workspace_bytes(int32_t n_rows, int32_t n_req, int32_t hist_cap);
 int actkv_budget(const float* logits, const int32_t* tok_indptr, int32_t n_rows, int32_t vocab,
                  float* conf_hist, int32_t* hist_len, int32_t hist_cap,
                  const actkv_budget_params_t* params /* host */,
@@ -158,6 +159,19 @@ int actkv_score(const actkv_pool_t* pool /* host */, const actkv_tables_t* table
                 const int32_t* tok_indptr, float* score_out, float* lse_out,
                 int32_t sum_win, int32_t max_win, int32_t sum_tok, int32_t max_tok,
                 void* ws, size_t ws_bytes, int32_t* status, actkv_stream_t stream);
+
+/* ---------------------------------------------------------------------------------------
+ * actkv_score_lse — only the log-sum-exp of actkv_score (Section 7.1, LSE equation): what a
+ * paged attention backend would hand over as a by-product.  Same arguments and workspace as
+ * actkv_score; writes lse_out float32 [NLs, sum_win, n_q_heads] (required) and no score.
+ * actkv_score_lse followed by actkv_score(lse_in = that) equals actkv_score(lse_in = NULL).
+ */
+int actkv_score_lse(const actkv_pool_t* pool /* host */, const actkv_tables_t* tables /* host */,
+                    int32_t layer_begin, int32_t layer_end,
+                    const void* q, const int32_t* win_indptr, int32_t n_q_heads,
+                    float sm_scale, int32_t causal, const int32_t* tok_indptr, float* lse_out,
+                    int32_t sum_win, int32_t max_win, int32_t sum_tok, int32_t max_tok,
+                    void* ws, size_t ws_bytes, int32_t* status, actkv_stream_t stream);
 
 /* ---------------------------------------------------------------------------------------
  * actkv_keep_indptr — helper: keep_indptr[r] = sum_{r'<r} min(budget[r'], seq_len[r']),

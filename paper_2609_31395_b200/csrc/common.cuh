@@ -1,0 +1,78 @@
+// Shared device/host helpers of the ActKV CUDA library (sm_100a).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <stdint.h>
+
+#include "../../include/actkv.h"
+
+#define ACTKV_CHECK_LAUNCH()                                   \
+  do {                                                         \
+    if (cudaGetLastError() != cudaSuccess) return ACTKV_E_CUDA; \
+  } while (0)
+
+namespace actkv {
+
+// First device-detected error wins; later ones are dropped.
+__device__ __forceinline__ void report(int32_t* status, int32_t code, int32_t where, int32_t what) {
+  if (status == nullptr) return;
+  if (atomicCAS(status, 0, code) == 0) {
+    status[1] = where;
+    status[2] = what;
+  }
+}
+
+__device__ __forceinline__ bool status_set(const int32_t* status) {
+  return status != nullptr && *((const volatile int32_t*)status) != 0;
+}
+
+// Plain-value copy of actkv_pool_t for kernel parameters.
+struct PoolView {
+  const __nv_bfloat16* base;
+  int32_t n_layers, n_pages, page_size, n_kv_heads, head_dim;
+  int64_t stride_layer, stride_kv, stride_page, stride_slot, stride_head;
+};
+
+struct TablesView {
+  int32_t n_req, max_pages;
+  int32_t* page_table;
+  int32_t* seq_len;
+  int32_t* free_list;
+  int32_t* free_count;
+};
+
+inline PoolView make_view(const actkv_pool_t* p) {
+  PoolView v;
+  v.base = (const __nv_bfloat16*)p->base;
+  v.n_layers = p->n_layers; v.n_pages = p->n_pages; v.page_size = p->page_size;
+  v.n_kv_heads = p->n_kv_heads; v.head_dim = p->head_dim;
+  v.stride_layer = p->stride_layer; v.stride_kv = p->stride_kv; v.stride_page = p->stride_page;
+  v.stride_slot = p->stride_slot; v.stride_head = p->stride_head;
+  return v;
+}
+
+inline TablesView make_view(const actkv_tables_t* t) {
+  TablesView v;
+  v.n_req = t->n_req; v.max_pages = t->max_pages; v.page_table = t->page_table;
+  v.seq_len = t->seq_len; v.free_list = t->free_list; v.free_count = t->free_count;
+  return v;
+}
+
+inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+// Page id of logical page `lp` of request r; out-of-range ids are reported and replaced by 0.
+__device__ __forceinline__ int32_t checked_page(const TablesView& t, int32_t n_pages, int32_t r,
+                                                int32_t lp, int32_t* status) {
+  int32_t id = t.page_table[(int64_t)r * t.max_pages + lp];
+  if ((uint32_t)id >= (uint32_t)n_pages) {
+    report(status, ACTKV_E_BADPAGE, r, id);
+    id = 0;
+  }
+  return id;
+}
+
+constexpr float kLog2e = 1.4426950408889634f;
+constexpr float kLn2 = 0.6931471805599453f;
+
+}  // namespace actkv

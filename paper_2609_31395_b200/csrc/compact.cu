@@ -1,0 +1,219 @@
+// actkv_compact: pack survivors into fresh pages, free the old pages (Section 7.2, Algorithm 4:
+// plan first, then one-shot parallel copies whose sources and destinations are disjoint, then
+// return the freed blocks).  Three kernels on one stream:
+//   plan     : per request X_r, offsets into the run of pages popped from the free-list stack,
+//              the new page ids; detects a short free list (nothing is modified in that case);
+//   copy     : one CTA per (destination page, request, layer) gathers the 16-byte vectors of the
+//              K and V rows of the survivors of every head into the page — destination pages are
+//              written whole and coalesced, sources are 256-byte row gathers;
+//   finalize : new page table / seq_len, pop and push on the free list (only on the call whose
+//              layer range ends at the pool's last layer).
+#include "common.cuh"
+
+namespace actkv {
+
+struct CompactWs {
+  int32_t plan_ok;       // 1 when the copy / finalize kernels may run
+  int32_t total_new;     // pages popped
+  int32_t pad[2];
+  // followed by int32 new_off[R], push_off[R], new_pages[R * max_pages]
+};
+
+__device__ __forceinline__ int32_t* ws_new_off(CompactWs* w) { return reinterpret_cast<int32_t*>(w + 1); }
+__device__ __forceinline__ int32_t* ws_push_off(CompactWs* w, int R) { return ws_new_off(w) + R; }
+__device__ __forceinline__ int32_t* ws_new_pages(CompactWs* w, int R) { return ws_new_off(w) + 2 * R; }
+
+__global__ void compact_plan_kernel(TablesView tab, int32_t page_size, int32_t n_pages,
+                                    const int32_t* __restrict__ budget, int32_t max_keep,
+                                    CompactWs* ws, int32_t* status) {
+  const int R = tab.n_req;
+  int32_t* new_off = ws_new_off(ws);
+  int32_t* push_off = ws_push_off(ws, R);
+  int32_t* new_pages = ws_new_pages(ws, R);
+  __shared__ int32_t s_total, s_ok;
+  if (threadIdx.x == 0) {
+    int32_t off = 0, poff = 0;
+    bool ok = !status_set(status);
+    for (int r = 0; r < R; ++r) {
+      const int32_t L = tab.seq_len[r];
+      int32_t B = budget[r] < 0 ? 0 : budget[r];
+      if (B < L) {
+        new_off[r] = off;
+        push_off[r] = poff;
+        off += (B + page_size - 1) / page_size;
+        poff += (L + page_size - 1) / page_size;
+        if ((L + page_size - 1) / page_size > tab.max_pages) { report(status, ACTKV_E_INVALID, r, L); ok = false; }
+        if (B > max_keep) { report(status, ACTKV_E_INVALID, r, B); ok = false; }   // host bound too small
+      } else {
+        new_off[r] = -1;
+        push_off[r] = -1;
+      }
+    }
+    const int32_t fc = *tab.free_count;
+    if (fc < 0 || fc > n_pages) { report(status, ACTKV_E_INVALID, -1, fc); ok = false; }
+    else if (off > fc) { report(status, ACTKV_E_NOFREE, off, fc); ok = false; }
+    s_total = off;
+    s_ok = ok ? 1 : 0;
+  }
+  __syncthreads();
+  const int32_t total = s_total;
+  if (s_ok) {
+    const int32_t fc = *tab.free_count;
+    for (int i = threadIdx.x; i < total; i += blockDim.x) {
+      int32_t id = tab.free_list[fc - 1 - i];
+      if ((uint32_t)id >= (uint32_t)n_pages) { report(status, ACTKV_E_BADPAGE, -1, id); s_ok = 0; }
+      new_pages[i] = id;
+    }
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) { ws->plan_ok = s_ok; ws->total_new = total; }
+}
+
+constexpr int CP_NT = 256;
+constexpr int CP_UNROLL = 8;
+
+__global__ void __launch_bounds__(CP_NT) compact_copy_kernel(
+    PoolView pool, TablesView tab, int32_t layer_begin, const int32_t* __restrict__ sel_idx,
+    int64_t sel_stride, const int32_t* __restrict__ keep_indptr, const int32_t* __restrict__ budget,
+    CompactWs* ws, int32_t* status) {
+  if (!ws->plan_ok) return;
+  const int R = tab.n_req;
+  const int r = blockIdx.y, slab = blockIdx.z, dp = blockIdx.x;
+  const int32_t noff = ws_new_off(ws)[r];
+  if (noff < 0) return;
+  const int P = pool.page_size, H = pool.n_kv_heads, D = pool.head_dim;
+  const int32_t n = budget[r] < 0 ? 0 : budget[r];
+  const int X = (n + P - 1) / P;
+  if (dp >= X) return;
+  const int32_t L = tab.seq_len[r];
+  const int32_t dst_page = ws_new_pages(ws, R)[noff + dp];
+  const int n_slots = min(P, n - dp * P);
+  const int vpr = D / 8;                                  // 16-byte vectors per row
+  const int per_kv = n_slots * H * vpr;
+  const int total = 2 * per_kv;
+  __nv_bfloat16* lbase = const_cast<__nv_bfloat16*>(pool.base) + (int64_t)(layer_begin + slab) * pool.stride_layer;
+  const int32_t* sel_base = sel_idx + (int64_t)slab * H * sel_stride + keep_indptr[r] + dp * P;
+
+  for (int v0 = threadIdx.x; v0 < total; v0 += CP_NT * CP_UNROLL) {
+    uint4 val[CP_UNROLL];
+    int64_t dst_off[CP_UNROLL];
+#pragma unroll
+    for (int k = 0; k < CP_UNROLL; ++k) {
+      const int v = v0 + k * CP_NT;
+      dst_off[k] = -1;
+      if (v < total) {
+        const int kv = v / per_kv;
+        int rem = v - kv * per_kv;
+        const int slot = rem / (H * vpr);
+        rem -= slot * (H * vpr);
+        const int h = rem / vpr, dv = rem - h * vpr;
+        const int32_t tok = sel_base[(int64_t)h * sel_stride + slot];
+        if ((uint32_t)tok >= (uint32_t)L) {
+          report(status, ACTKV_E_BADINDEX, r, tok);
+        } else {
+          const int32_t sp = checked_page(tab, pool.n_pages, r, tok / P, status);
+          const int64_t src = (int64_t)kv * pool.stride_kv + (int64_t)sp * pool.stride_page +
+                              (int64_t)(tok % P) * pool.stride_slot + (int64_t)h * pool.stride_head + dv * 8;
+          val[k] = *reinterpret_cast<const uint4*>(lbase + src);
+          dst_off[k] = (int64_t)kv * pool.stride_kv + (int64_t)dst_page * pool.stride_page +
+                       (int64_t)slot * pool.stride_slot + (int64_t)h * pool.stride_head + dv * 8;
+        }
+      }
+    }
+#pragma unroll
+    for (int k = 0; k < CP_UNROLL; ++k)
+      if (dst_off[k] >= 0) *reinterpret_cast<uint4*>(lbase + dst_off[k]) = val[k];
+  }
+}
+
+__global__ void compact_finalize_kernel(TablesView tab, int32_t page_size,
+                                        const int32_t* __restrict__ budget, CompactWs* ws,
+                                        const int32_t* status) {
+  // an error met by the copies (bad index, bad page) leaves the tables as they were: the fresh
+  // pages that were written are still on the free list
+  if (!ws->plan_ok || status_set(status)) return;
+  const int R = tab.n_req;
+  const int32_t* new_off = ws_new_off(ws);
+  const int32_t* push_off = ws_push_off(ws, R);
+  const int32_t* new_pages = ws_new_pages(ws, R);
+  const int32_t fc_new = *tab.free_count - ws->total_new;
+  __shared__ int32_t s_pushed;
+  if (threadIdx.x == 0) s_pushed = 0;
+  __syncthreads();
+  // push the old pages (reads the old table), request by request in ascending order
+  for (int r = 0; r < R; ++r) {
+    if (new_off[r] < 0) continue;
+    const int Y = (tab.seq_len[r] + page_size - 1) / page_size;
+    for (int i = threadIdx.x; i < Y; i += blockDim.x)
+      tab.free_list[fc_new + push_off[r] + i] = tab.page_table[(int64_t)r * tab.max_pages + i];
+    if (threadIdx.x == 0) s_pushed += Y;
+  }
+  __syncthreads();
+  // then rewrite the tables
+  for (int r = 0; r < R; ++r) {
+    if (new_off[r] < 0) continue;
+    const int32_t n = budget[r] < 0 ? 0 : budget[r];
+    const int X = (n + page_size - 1) / page_size;
+    for (int i = threadIdx.x; i < tab.max_pages; i += blockDim.x)
+      tab.page_table[(int64_t)r * tab.max_pages + i] = i < X ? new_pages[new_off[r] + i] : -1;
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    for (int r = 0; r < R; ++r)
+      if (new_off[r] >= 0) tab.seq_len[r] = budget[r] < 0 ? 0 : budget[r];
+    *tab.free_count = fc_new + s_pushed;
+  }
+}
+
+}  // namespace actkv
+
+extern "C" {
+
+size_t actkv_compact_workspace_bytes(int32_t n_req, int32_t max_pages) {
+  if (n_req < 0 || max_pages < 0) return 0;
+  return actkv::align_up(sizeof(actkv::CompactWs) + sizeof(int32_t) * ((size_t)2 * n_req + (size_t)n_req * max_pages), 256);
+}
+
+int actkv_compact(const actkv_pool_t* pool, const actkv_tables_t* tables, int32_t layer_begin,
+                  int32_t layer_end, const int32_t* sel_idx, int64_t sel_stride,
+                  const int32_t* keep_indptr, const int32_t* budget, int32_t max_keep,
+                  void* ws, size_t ws_bytes, int32_t* status, actkv_stream_t stream) {
+  if (!pool || !tables || !pool->base) return ACTKV_E_INVALID;
+  if (layer_begin < 0 || layer_end > pool->n_layers || layer_begin > layer_end) return ACTKV_E_INVALID;
+  if (pool->page_size <= 0 || pool->head_dim <= 0 || pool->head_dim % 8 != 0 || pool->n_kv_heads <= 0)
+    return ACTKV_E_INVALID;
+  // 16-byte vector moves need every row start 16-byte aligned
+  if (((uintptr_t)pool->base & 15) || pool->stride_layer % 8 || pool->stride_kv % 8 || pool->stride_page % 8 ||
+      pool->stride_slot % 8 || pool->stride_head % 8)
+    return ACTKV_E_INVALID;
+  const int R = tables->n_req;
+  if (R < 0 || tables->max_pages < 0 || max_keep < 0 || sel_stride < 0) return ACTKV_E_INVALID;
+  if (R == 0) return ACTKV_OK;
+  if (!tables->page_table || !tables->seq_len || !tables->free_list || !tables->free_count || !budget ||
+      !keep_indptr || !sel_idx || !ws)
+    return ACTKV_E_INVALID;
+  if (ws_bytes < actkv_compact_workspace_bytes(R, tables->max_pages)) return ACTKV_E_WORKSPACE;
+  if (R > 65535 || layer_end - layer_begin > 65535) return ACTKV_E_INVALID;
+  cudaStream_t s = (cudaStream_t)stream;
+  actkv::PoolView pv = actkv::make_view(pool);
+  actkv::TablesView tv = actkv::make_view(tables);
+  actkv::CompactWs* w = (actkv::CompactWs*)ws;
+  actkv::compact_plan_kernel<<<1, 256, 0, s>>>(tv, pool->page_size, pool->n_pages, budget, max_keep, w, status);
+  ACTKV_CHECK_LAUNCH();
+  const int nl = layer_end - layer_begin;
+  int max_x = (max_keep + pool->page_size - 1) / pool->page_size;
+  if (max_x > tables->max_pages) max_x = tables->max_pages;
+  if (nl > 0 && max_x > 0) {
+    dim3 grid((unsigned)max_x, (unsigned)R, (unsigned)nl);
+    actkv::compact_copy_kernel<<<grid, actkv::CP_NT, 0, s>>>(pv, tv, layer_begin, sel_idx, sel_stride,
+                                                              keep_indptr, budget, w, status);
+    ACTKV_CHECK_LAUNCH();
+  }
+  if (layer_end == pool->n_layers) {
+    actkv::compact_finalize_kernel<<<1, 1024, 0, s>>>(tv, pool->page_size, budget, w, status);
+    ACTKV_CHECK_LAUNCH();
+  }
+  return ACTKV_OK;
+}
+
+}  // extern "C"

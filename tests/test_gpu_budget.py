@@ -1,0 +1,146 @@
+"""GPU parity of actkv_budget against the oracle's confidence monitor."""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import actkv_oracle as O
+from paper_2609_31395_b200 import binding as B
+from paper_2609_31395_b200 import synth
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+T_ATOL = 2e-5          # float32 logsumexp / mean against float64, values of order 10
+
+
+def _run(logits, tok_indptr, hist, hist_len, budget_in, params, seq_len=None):
+    R = hist.shape[0]
+    cap = hist.shape[1]
+    n_rows = 0 if logits is None else logits.shape[0]
+    vocab = 0 if logits is None else logits.shape[1]
+    ws = torch.empty(B.actkv_budget_workspace_bytes(n_rows, R, cap) + 256, dtype=torch.uint8, device=DEV)
+    status = torch.zeros(4, dtype=torch.int32, device=DEV)
+    out = torch.zeros(R, dtype=torch.int32, device=DEV)
+    slopes = torch.zeros(R, dtype=torch.float64, device=DEV)
+    B.actkv_budget(logits, tok_indptr, n_rows, vocab, hist, hist_len, cap, params, seq_len, budget_in, out, slopes,
+                   R, ws, status)
+    torch.cuda.synchronize()
+    return out.cpu().numpy(), slopes.cpu().numpy(), status.cpu().tolist()
+
+
+def _oracle_params(p: B.BudgetParams) -> O.BudgetParams:
+    return O.BudgetParams(p.k, p.w, p.s, p.b_percent, p.scale_up, p.B_upper, p.clamp_lo_ppm, p.clamp_hi_ppm)
+
+
+def _compare(logits, tok, hist0, len0, budget_in, params, seq_len=None):
+    R = hist0.shape[0]
+    hist = hist0.clone().to(DEV)
+    hist_len = len0.clone().to(DEV)
+    got_B, got_a, st = _run(logits, tok, hist, hist_len, budget_in.to(DEV), params,
+                            None if seq_len is None else seq_len.to(DEV))
+    assert st[0] == 0
+    op = _oracle_params(params)
+    tok_np = tok.cpu().numpy()
+    oh, ol, oB, oa, oT = O.budget(logits.cpu().numpy(), tok_np, hist0.numpy(), len0.numpy(), budget_in.numpy(), op,
+                                  None if seq_len is None else seq_len.numpy())
+    gh = hist.cpu().numpy()
+    gl = hist_len.cpu().numpy()
+    assert np.array_equal(gl, ol)
+    for r in range(R):
+        assert np.abs(gh[r, :gl[r]].astype(np.float64) - oh[r, :ol[r]]).max() <= T_ATOL
+    # the decision part on the GPU's own stored history must match the oracle exactly
+    borderline = 0
+    for r in range(R):
+        Rr = O.trace_confidence(gh[r, :gl[r]], op.w, op.s, op.b_percent)
+        a = O.fit_slope(Rr)
+        assert abs(got_a[r] - a) <= 1e-12 * max(1.0, abs(a))
+        want = O.budget_update(int(budget_in[r]), a, op, None if seq_len is None else int(seq_len[r]))
+        assert got_B[r] == want
+        if got_B[r] != oB[r]:
+            borderline += 1
+            assert abs(oa[r]) < 1e-4           # full-pipeline disagreement only when the slope is ~0
+    return got_B, got_a, borderline
+
+
+def test_uniform_rows_give_log_vocab_and_zero_slope():
+    V, T, R = 151936, 80, 2
+    logits = torch.full((R * T, V), 0.37, dtype=torch.float32, device=DEV)
+    tok = torch.arange(0, (R + 1) * T, T, dtype=torch.int32, device=DEV)
+    hist = torch.zeros((R, 256), dtype=torch.float32)
+    p = B.BudgetParams.paper_defaults()
+    hist_d = hist.clone().to(DEV)
+    len_d = torch.zeros(R, dtype=torch.int32, device=DEV)
+    got_B, got_a, st = _run(logits, tok, hist_d, len_d, torch.tensor([512, 896], dtype=torch.int32, device=DEV), p)
+    assert st[0] == 0
+    h = hist_d.cpu().numpy()
+    assert np.abs(h[:, :T] - math.log(V)).max() < T_ATOL
+    assert (got_a == 0.0).all() and got_B.tolist() == [512, 896]
+
+
+@pytest.mark.parametrize("vocab,R,T", [(151936, 3, 96), (1000, 6, 400), (37, 6, 400)])
+def test_against_oracle_gaussian_logits(vocab, R, T):
+    logits, tok = synth.confidence_logits(R, T, vocab, seed=vocab, device=DEV)
+    hist0 = torch.zeros((R, 512), dtype=torch.float32)
+    len0 = torch.zeros(R, dtype=torch.int32)
+    budget_in = torch.tensor([512, 896, 1568, 20000, 29000, 100][:R], dtype=torch.int32)
+    p = B.BudgetParams.paper_defaults()
+    got_B, got_a, _ = _compare(logits, tok, hist0, len0, budget_in, p)
+    if vocab == 1000:
+        assert (got_a < 0).any() and (got_a == 0).any()      # both outcomes occur in this draw
+    for r in range(R):
+        if got_a[r] < 0:
+            assert got_B[r] == min(int(budget_in[r] * 1.75), 30000)
+
+
+def test_history_accumulates_across_calls_and_clamp():
+    R, T, V = 4, 40, 2048
+    p = B.BudgetParams.paper_defaults(clamp_lo_ppm=150000, clamp_hi_ppm=400000)
+    seq_len = torch.tensor([35000, 8192, 65536, 1000], dtype=torch.int32)
+    budget_in = torch.tensor([7000, 100, 30000, 500], dtype=torch.int32)
+    hist = torch.zeros((R, 128), dtype=torch.float32)
+    lens = torch.zeros(R, dtype=torch.int32)
+    op = _oracle_params(p)
+    hist_d, len_d = hist.clone().to(DEV), lens.clone().to(DEV)
+    oh, ol = hist.numpy(), lens.numpy()
+    for call in range(3):
+        logits, tok = synth.confidence_logits(R, T, V, seed=100 + call, device=DEV)
+        got_B, got_a, st = _run(logits, tok, hist_d, len_d, budget_in.to(DEV), p, seq_len.to(DEV))
+        oh, ol, oB, oa, _ = O.budget(logits.cpu().numpy(), tok.cpu().numpy(), oh, ol, budget_in.numpy(), op,
+                                     seq_len.numpy())
+        assert st[0] == 0
+        assert np.array_equal(len_d.cpu().numpy(), ol)
+        assert np.abs(hist_d.cpu().numpy() - oh).max() <= T_ATOL
+        lo = [-(-int(L) * 150000 // 1000000) for L in seq_len]
+        hi = [int(L) * 400000 // 1000000 for L in seq_len]
+        assert all(lo[r] <= got_B[r] <= hi[r] for r in range(R))
+    assert ol.tolist() == [120] * R
+
+
+def test_history_overflow_is_reported():
+    R, T, V = 1, 50, 64
+    logits, tok = synth.confidence_logits(R, T, V, seed=1, device=DEV)
+    hist = torch.zeros((R, 32), dtype=torch.float32, device=DEV)
+    lens = torch.zeros(R, dtype=torch.int32, device=DEV)
+    _, _, st = _run(logits, tok, hist, lens, torch.tensor([10], dtype=torch.int32, device=DEV),
+                    B.BudgetParams.paper_defaults())
+    assert st[0] == B.E_INVALID
+    assert lens.cpu().tolist() == [32]
+
+
+def test_trend_only_call_and_ties_at_top_k():
+    # top-k boundary inside a run of equal logits: 30 logits at 2.0, k = 20
+    V = 500
+    z = torch.zeros((70, V), dtype=torch.float32, device=DEV)
+    z[:, 100:130] = 2.0
+    z[:, 7] = 5.0
+    tok = torch.tensor([0, 70], dtype=torch.int32, device=DEV)
+    hist0 = torch.zeros((1, 128), dtype=torch.float32)
+    len0 = torch.zeros(1, dtype=torch.int32)
+    p = B.BudgetParams.paper_defaults()
+    _compare(z, tok, hist0, len0, torch.tensor([512], dtype=torch.int32), p)
+    # trend-only call on a stored decreasing history
+    hist = torch.linspace(9.0, 3.0, 512).view(1, 512).contiguous().to(DEV)
+    lens = torch.tensor([512], dtype=torch.int32, device=DEV)
+    got_B, got_a, st = _run(None, None, hist, lens, torch.tensor([512], dtype=torch.int32, device=DEV), p)
+    assert st[0] == 0 and got_a[0] < 0 and got_B[0] == 896 and lens.cpu().tolist() == [512]

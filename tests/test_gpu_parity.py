@@ -1,0 +1,231 @@
+"""GPU parity: every step of the CUDA path, called through the C ABI, against the CPU oracle."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import actkv_oracle as O
+from paper_2609_31395_b200 import binding as B
+from paper_2609_31395_b200 import harness as H
+from paper_2609_31395_b200 import synth
+
+import parity_util as U
+
+pytestmark = pytest.mark.gpu
+
+DEV = "cuda:0"
+
+
+def _small(causal=False, head_dim=128, page=16, G=4, seed=0, **kw):
+    """Several tiles and ragged tails: lengths not multiples of the page, the 64-key FMA tile or
+    the 128-key tensor tile; ragged windows."""
+    return synth.Workload("small", 2, 2, G, [1000, 333, 130, 17], [8, 5, 16, 3], [250, 100, 130, 4],
+                          head_dim=head_dim, page_size=page, causal=causal, table_style="fragmented",
+                          seed=seed, poison_tail=True, **kw)
+
+
+def _full_check(inst, lse_in=None, layers_per_call=None):
+    wl = inst.wl
+    pool_before = U.bits(inst.pool)
+    tables_before = U.oracle_tables(inst)
+    comp = U.run_step(inst, lse_in=lse_in, layers_per_call=layers_per_call)
+    comp.check_status()
+    keep_indptr = comp.keep_indptr.cpu().numpy()
+    sel_idx = comp.sel_idx.cpu().numpy()
+    want_keep = np.concatenate([[0], np.cumsum([min(b, L) for b, L in zip(wl.budgets, wl.seq_lens)])])
+    assert np.array_equal(keep_indptr, want_keep)
+    out = {}
+    if layers_per_call is None:
+        lse_np = None if lse_in is None else lse_in.cpu().numpy().astype(np.float64)
+        want, lse, tok, err = U.check_scores(inst, comp, lse_in=lse_np)
+        if lse_in is None:
+            got_lse = comp.lse.cpu().numpy()
+            m = ~np.isnan(lse)
+            assert np.abs(got_lse[m] - lse[m]).max() < 1e-4
+        score_gpu = comp.score.cpu().numpy().reshape(-1, comp.score.shape[-1])
+        U.check_select_exact(score_gpu, tok, wl.budgets, sel_idx, keep_indptr)
+        out["ties"] = U.check_select_vs_oracle_scores(want.reshape(-1, want.shape[-1]), tok, wl.budgets, sel_idx,
+                                                      keep_indptr)
+        out["lse"] = lse
+        out["err"] = err
+        U.check_compaction(inst, pool_before, tables_before, sel_idx, keep_indptr, wl.budgets)
+    out["comp"] = comp
+    return out
+
+
+@pytest.mark.parametrize("causal", [False, True])
+@pytest.mark.parametrize("head_dim,page,G", [(128, 16, 4), (64, 8, 2), (128, 16, 8)])
+def test_pipeline_small(causal, head_dim, page, G):
+    wl = _small(causal=causal, head_dim=head_dim, page=page, G=G)
+    if causal:
+        wl.windows = [min(w, L) for w, L in zip(wl.windows, wl.seq_lens)]
+    inst = synth.generate(wl, DEV)
+    _full_check(inst)
+
+
+def test_pipeline_supplied_lse_matches_internal():
+    inst = synth.generate(_small(), DEV)
+    r1 = _full_check(inst)
+    lse = r1["comp"].lse.clone()
+    score_internal = r1["comp"].score.clone()
+    inst2 = synth.generate(_small(), DEV)
+    r2 = _full_check(inst2, lse_in=lse)
+    # the same LSE values give the same scores bit for bit
+    assert torch.equal(score_internal, r2["comp"].score)
+
+
+def test_layer_sub_ranges_give_the_same_result():
+    a = synth.generate(_small(), DEV)
+    b = synth.generate(_small(), DEV)
+    _full_check(a)
+    _full_check(b, layers_per_call=1)
+    assert torch.equal(a.pool.view(torch.int16), b.pool.view(torch.int16))
+    assert torch.equal(a.page_table, b.page_table) and torch.equal(a.seq_len, b.seq_len)
+    assert torch.equal(a.free_list, b.free_list) and torch.equal(a.free_count, b.free_count)
+
+
+def test_config1_all_units_and_planted_keys():
+    inst = synth.generate(synth.config1(), DEV)
+    res = _full_check(inst)
+    comp = res["comp"]
+    sel = comp.sel_idx.cpu().numpy()
+    planted = set(inst.planted[0].tolist())
+    assert len(planted) == 82
+    for o in range(sel.shape[0]):
+        assert planted <= set(sel[o, :1024].tolist())
+
+
+def test_window_rows_at_tensor_tile_sizes():
+    """window x group = 128 .. 512 rows (multiples and non-multiples of the 128-row tile)."""
+    for W, G in [(32, 4), (64, 8), (33, 4), (96, 4), (20, 8)]:
+        wl = synth.Workload("rows", 1, 2, G, [700, 257], [W, max(1, W // 2)], [200, 64], table_style="permutation",
+                            seed=W * 10 + G, poison_tail=True)
+        _full_check(synth.generate(wl, DEV))
+
+
+def test_long_request_many_chunks():
+    """More keys than one LSE chunk and several key tiles per CTA; ragged last page."""
+    wl = synth.Workload("long", 1, 1, 4, [9000 + 7], [32], [2300], table_style="fragmented", seed=5, poison_tail=True)
+    _full_check(synth.generate(wl, DEV))
+
+
+def test_duplicate_keys_make_exact_ties():
+    """Duplicated key rows give bit-equal scores; the lower index must win at the threshold."""
+    wl = synth.Workload("dups", 1, 2, 4, [512], [16], [100], table_style="permutation", seed=9, plant_frac=0.0)
+    inst = synth.generate(wl, DEV)
+    P = wl.page_size
+    kflat = inst.pool[0, 0].view(-1, wl.n_kv_heads, wl.head_dim)
+    pt = inst.page_table[0].to(torch.int64)
+    j = torch.arange(512, device=DEV)
+    slots = pt[j // P] * P + j % P
+    kflat[slots[256:]] = kflat[slots[:256]]            # second half duplicates the first
+    res = _full_check(inst)
+    comp = res["comp"]
+    ties = comp.ties.cpu().numpy().reshape(-1, 4)
+    score = comp.score.cpu().numpy().reshape(-1, 512)
+    assert np.array_equal(score[:, :256], score[:, 256:])
+    # every unit: threshold value appears at j and j+256; only consistent counts are possible
+    for u in range(ties.shape[0]):
+        thr = ties[u, 0:1].view(np.float32)[0]
+        assert ties[u, 3] == 100
+        assert ties[u, 2] == int((score[u] == thr).sum()) and ties[u, 2] >= 2
+        assert 1 <= ties[u, 1] <= ties[u, 2]
+
+
+def test_budget_covers_length_is_noop_and_budget_zero_empties():
+    wl = _small()
+    wl.budgets = [5000, 333, 0, 17]
+    inst = synth.generate(wl, DEV)
+    before = inst.pool.clone()
+    pt_before = inst.page_table.clone()
+    fc_before = int(inst.free_count.cpu())
+    res = _full_check(inst)
+    assert torch.equal(before.view(torch.int16), inst.pool.view(torch.int16))      # nothing copied at all
+    assert torch.equal(inst.page_table[0], pt_before[0]) and torch.equal(inst.page_table[1], pt_before[1])
+    assert inst.seq_len.cpu().tolist() == [1000, 333, 0, 17]
+    assert (inst.page_table[2] == -1).all()
+    assert int(inst.free_count.cpu()) == fc_before + -(-130 // 16)
+
+
+def test_free_list_short_modifies_nothing():
+    inst = synth.generate(_small(), DEV)
+    inst.free_count.fill_(3)
+    before = inst.pool.clone()
+    pt, sl, fl = inst.page_table.clone(), inst.seq_len.clone(), inst.free_list.clone()
+    comp = U.run_step(inst)
+    st = comp.status.cpu().tolist()
+    assert st[0] == B.E_NOFREE
+    assert torch.equal(before.view(torch.int16), inst.pool.view(torch.int16))
+    assert torch.equal(pt, inst.page_table) and torch.equal(sl, inst.seq_len) and torch.equal(fl, inst.free_list)
+    assert int(inst.free_count.cpu()) == 3
+
+
+def test_bad_page_id_is_reported_not_trapped():
+    inst = synth.generate(_small(), DEV)
+    inst.page_table[1, 2] = 10**6
+    before_pt = inst.page_table.clone()
+    comp = U.run_step(inst)
+    st = comp.status.cpu().tolist()
+    assert st[0] == B.E_BADPAGE and st[1] == 1 and st[2] == 10**6
+    assert torch.equal(before_pt, inst.page_table)           # compaction refused to run
+    # the context is still usable
+    assert torch.ones(4, device=DEV).sum().item() == 4.0
+
+
+def test_host_argument_errors():
+    inst = synth.generate(_small(), DEV)
+    sz = H.sizes_of(inst)
+    comp = H.Compressor(inst.pool, inst.page_table, inst.seq_len, inst.free_list, inst.free_count,
+                        inst.wl.n_q_heads, sz)
+    tiny = torch.empty(256, dtype=torch.uint8, device=DEV)
+    with pytest.raises(B.ActKVError) as e:
+        B.actkv_score(comp.pd, comp.td, 0, 2, inst.q, inst.win_indptr, inst.wl.n_q_heads, None, 0.1, 0,
+                      inst.tok_indptr, comp.score, None, sz.sum_win, sz.max_win, sz.sum_tok, sz.max_tok, tiny,
+                      comp.status)
+    assert e.value.code == B.E_WORKSPACE
+    with pytest.raises(B.ActKVError) as e:
+        B.actkv_score(comp.pd, comp.td, 0, 3, inst.q, inst.win_indptr, inst.wl.n_q_heads, None, 0.1, 0,
+                      inst.tok_indptr, comp.score, None, sz.sum_win, sz.max_win, sz.sum_tok, sz.max_tok,
+                      comp.ws_score, comp.status)
+    assert e.value.code == B.E_INVALID
+    with pytest.raises(B.ActKVError) as e:                   # 7 q-heads do not divide over 2 KV heads
+        B.actkv_score(comp.pd, comp.td, 0, 2, inst.q, inst.win_indptr, 7, None, 0.1, 0,
+                      inst.tok_indptr, comp.score, None, sz.sum_win, sz.max_win, sz.sum_tok, sz.max_tok,
+                      comp.ws_score, comp.status)
+    assert e.value.code == B.E_INVALID
+
+
+def test_zero_window_is_reported():
+    wl = _small()
+    wl.windows = [8, 0, 16, 3]
+    inst = synth.generate(wl, DEV)
+    comp = U.run_step(inst)
+    st = comp.status.cpu().tolist()
+    assert st[0] == B.E_INVALID and st[1] == 1
+
+
+def test_empty_request_is_skipped():
+    wl = synth.Workload("empty", 1, 2, 4, [300, 0, 64], [8, 4, 8], [100, 10, 10], table_style="fragmented", seed=4)
+    inst = synth.generate(wl, DEV)
+    _full_check(inst)
+
+
+def test_keep_mask_bitmap():
+    inst = synth.generate(_small(), DEV)
+    wl = inst.wl
+    sz = H.sizes_of(inst)
+    comp = H.Compressor(inst.pool, inst.page_table, inst.seq_len, inst.free_list, inst.free_count, wl.n_q_heads, sz,
+                        want_mask=True)
+    B.actkv_keep_indptr(inst.seq_len, inst.budget, wl.n_req, comp.keep_indptr)
+    comp.run_score(inst.q, inst.win_indptr, inst.tok_indptr, wl.sm_scale, False)
+    comp.run_select(inst.tok_indptr, inst.budget, wl.n_layers)
+    torch.cuda.synchronize()
+    mask = comp.mask.cpu().numpy().view(np.uint32)
+    sel = comp.sel_idx.cpu().numpy()
+    ki = comp.keep_indptr.cpu().numpy()
+    tok = inst.tok_indptr.cpu().numpy()
+    for o in range(mask.shape[0]):
+        bitsv = np.unpackbits(mask[o].view(np.uint8), bitorder="little")[: tok[-1]]
+        want = np.zeros(tok[-1], dtype=np.uint8)
+        for r in range(wl.n_req):
+            want[tok[r] + sel[o, ki[r]:ki[r + 1]]] = 1
+        assert np.array_equal(bitsv, want)
