@@ -27,12 +27,14 @@ def max_rel(got: np.ndarray, want: np.ndarray) -> float:
     return float(np.max(np.abs(got - want) / np.maximum(np.abs(want), SCORE_ATOL))) if got.size else 0.0
 
 
-def check_scores(inst, comp: H.Compressor, units=None, layers=None, lse_in=None):
-    """GPU scores (comp.score, first slabs) against the oracle on `units` (default: all)."""
+def check_scores(inst, comp: H.Compressor, pool_before: np.ndarray, tables_before: O.Tables, units=None,
+                 layers=None, lse_in=None):
+    """GPU scores (comp.score, first slabs) against the oracle on `units` (default: all), on the
+    pool and tables as they were BEFORE the step (compaction rewrites the tables)."""
     wl = inst.wl
-    pool_b = bits(inst.pool)
+    pool_b = pool_before
     q_b = bits(inst.q if layers is None else inst.q[layers])
-    want, lse, tok = O.score(pool_b, inst.page_table.cpu().numpy(), inst.seq_len.cpu().numpy(), q_b,
+    want, lse, tok = O.score(pool_b, tables_before.page_table, tables_before.seq_len, q_b,
                              inst.win_indptr.cpu().numpy(), wl.n_q_heads, wl.sm_scale, wl.causal,
                              layers=layers, lse_in=lse_in, units=units)
     got = comp.score[: want.shape[0]].cpu().numpy()

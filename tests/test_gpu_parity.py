@@ -36,7 +36,7 @@ def _full_check(inst, lse_in=None, layers_per_call=None):
     out = {}
     if layers_per_call is None:
         lse_np = None if lse_in is None else lse_in.cpu().numpy().astype(np.float64)
-        want, lse, tok, err = U.check_scores(inst, comp, lse_in=lse_np)
+        want, lse, tok, err = U.check_scores(inst, comp, pool_before, tables_before, lse_in=lse_np)
         if lse_in is None:
             got_lse = comp.lse.cpu().numpy()
             m = ~np.isnan(lse)
