@@ -43,6 +43,7 @@ extern "C" {
 #define ACTKV_E_NOFREE     -5   /* device: free list holds fewer pages than compaction needs     */
 #define ACTKV_E_BADINDEX   -6   /* device: selected token index outside [0, seq_len)             */
 #define ACTKV_E_TIMEOUT    -7   /* device: a bounded wait inside a kernel gave up                */
+#define ACTKV_E_TOOBIG     -8   /* sizes beyond the fixed scratch of a *_noalloc entry point    */
 
 /* CUDA stream handle (identical to cudaStream_t; spelled out so the header needs no CUDA). */
 typedef struct CUstream_st* actkv_stream_t;
@@ -223,6 +224,39 @@ int actkv_compact(const actkv_pool_t* pool /* host */, const actkv_tables_t* tab
                   const int32_t* sel_idx, int64_t sel_stride, const int32_t* keep_indptr,
                   const int32_t* budget, int32_t max_keep,
                   void* ws, size_t ws_bytes, int32_t* status, actkv_stream_t stream);
+
+/* ---------------------------------------------------------------------------------------
+ * actkv_compact_noalloc — actkv_compact without a caller-supplied workspace.
+ * (The paper has no counterpart; this is a convenience of the library.)
+ *
+ * Who it is for: a serving engine normally claims almost all of HBM for its KV block pool when
+ * it starts, so a later cudaMalloc for a few hundred KB of plan scratch can fail outright, and
+ * even when it succeeds cudaMalloc stalls the whole device, which a decode loop cannot afford
+ * between two steps.  Plug-in style callers (a C host without torch's caching allocator) are in
+ * the same position: they have device pointers to the pool and the tables and nothing to
+ * allocate with.  For them the plan scratch lives in a fixed array inside the library's device
+ * image (ACTKV_COMPACT_NOALLOC_BYTES on every GPU that loads the library, held until exit).
+ *
+ * Same arguments, semantics, status reporting and result as actkv_compact, minus ws/ws_bytes.
+ * Limits and rules:
+ *   - actkv_compact_workspace_bytes(n_req, max_pages) must not exceed
+ *     ACTKV_COMPACT_NOALLOC_BYTES (about n_req*(max_pages+2) <= 262 000 table entries, e.g.
+ *     64 requests x 4000 pages); larger tables return ACTKV_E_TOOBIG and launch nothing.
+ *   - The first call on each device looks up the array's device address (once, with that device
+ *     current) before launching; make that first call outside any stream capture.
+ *   - It calls no cudaMalloc / cudaFree and no allocating library routine.
+ *   - All calls on a device share the one array.  The plan kernel of a call rewrites every word
+ *     the later kernels of that call read, so stale contents are harmless, but two calls whose
+ *     kernels overlap on the GPU (different streams without an ordering between them) race on
+ *     it: serialise them, or give the second one actkv_compact with its own workspace.
+ */
+#define ACTKV_COMPACT_NOALLOC_BYTES (1u << 20)
+size_t actkv_compact_noalloc_max_bytes(void);
+int actkv_compact_noalloc(const actkv_pool_t* pool /* host */, const actkv_tables_t* tables /* host */,
+                          int32_t layer_begin, int32_t layer_end,
+                          const int32_t* sel_idx, int64_t sel_stride, const int32_t* keep_indptr,
+                          const int32_t* budget, int32_t max_keep,
+                          int32_t* status, actkv_stream_t stream);
 
 /* Library version string (host pointer to static storage). */
 const char* actkv_version(void);

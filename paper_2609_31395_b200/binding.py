@@ -16,14 +16,16 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libactkv.so")
 
 OK, E_INVALID, E_WORKSPACE, E_CUDA, E_BADPAGE, E_NOFREE, E_BADINDEX, E_TIMEOUT = 0, -1, -2, -3, -4, -5, -6, -7
+E_TOOBIG = -8
 ERROR_NAMES = {E_INVALID: "ACTKV_E_INVALID", E_WORKSPACE: "ACTKV_E_WORKSPACE", E_CUDA: "ACTKV_E_CUDA",
                E_BADPAGE: "ACTKV_E_BADPAGE", E_NOFREE: "ACTKV_E_NOFREE", E_BADINDEX: "ACTKV_E_BADINDEX",
-               E_TIMEOUT: "ACTKV_E_TIMEOUT"}
+               E_TIMEOUT: "ACTKV_E_TIMEOUT", E_TOOBIG: "ACTKV_E_TOOBIG"}
 
 EXPORTS = ["actkv_budget_workspace_bytes", "actkv_budget", "actkv_score_workspace_bytes", "actkv_score",
            "actkv_score_lse",
            "actkv_keep_indptr", "actkv_select_workspace_bytes", "actkv_select",
-           "actkv_compact_workspace_bytes", "actkv_compact", "actkv_version"]
+           "actkv_compact_workspace_bytes", "actkv_compact", "actkv_compact_noalloc",
+           "actkv_compact_noalloc_max_bytes", "actkv_version"]
 
 
 class ActKVError(RuntimeError):
@@ -103,6 +105,11 @@ def load():
     lib.actkv_compact.restype = i32
     lib.actkv_compact.argtypes = [C.POINTER(PoolDesc), C.POINTER(TablesDesc), i32, i32, vp, i64, vp, vp, i32,
                                   vp, sz, vp, vp]
+    lib.actkv_compact_noalloc_max_bytes.restype = sz
+    lib.actkv_compact_noalloc_max_bytes.argtypes = []
+    lib.actkv_compact_noalloc.restype = i32
+    lib.actkv_compact_noalloc.argtypes = [C.POINTER(PoolDesc), C.POINTER(TablesDesc), i32, i32, vp, i64, vp, vp, i32,
+                                          vp, vp]
     _lib = lib
     return lib
 
@@ -235,3 +242,22 @@ def actkv_compact(pool: PoolDesc, tables: TablesDesc, layer_begin, layer_end, se
                               max_keep, _ptr(ws, None, "ws"), ws.numel() * ws.element_size(),
                               _ptr(status, torch.int32, "status"), _stream(stream))
     _check("actkv_compact", rc)
+
+
+def actkv_compact_noalloc_max_bytes() -> int:
+    return load().actkv_compact_noalloc_max_bytes()
+
+
+def actkv_compact_noalloc(pool: PoolDesc, tables: TablesDesc, layer_begin, layer_end, sel_idx, sel_stride,
+                          keep_indptr, budget, max_keep, status, stream=None):
+    """actkv_compact for callers that cannot allocate the plan scratch: a serving engine that has
+    handed all of HBM to its KV pool (cudaMalloc may fail, and it stalls the device), or a host
+    without an allocator of its own.  The scratch is a fixed 1 MiB array inside the library, shared
+    by every call on the device, so calls that overlap on the GPU race; tables larger than the
+    array are refused with ACTKV_E_TOOBIG."""
+    rc = load().actkv_compact_noalloc(C.byref(pool), C.byref(tables), layer_begin, layer_end,
+                                      _ptr(sel_idx, torch.int32, "sel_idx"), sel_stride,
+                                      _ptr(keep_indptr, torch.int32, "keep_indptr"),
+                                      _ptr(budget, torch.int32, "budget"), max_keep,
+                                      _ptr(status, torch.int32, "status"), _stream(stream))
+    _check("actkv_compact_noalloc", rc)

@@ -217,3 +217,55 @@ int actkv_compact(const actkv_pool_t* pool, const actkv_tables_t* tables, int32_
 }
 
 }  // extern "C"
+
+// ---------------------------------------------------------------------------------------------
+// actkv_compact_noalloc: the same compaction for callers that have no device allocator to ask
+// for the plan scratch.  The scratch is a fixed array in the library's own device image.
+
+#include <mutex>
+
+// Plan scratch of actkv_compact_noalloc.  One copy lives on every GPU that loads the library, from
+// load until the process exits.  Device code could name it directly; host code may only use the
+// address that cudaGetSymbolAddress returns for the current device (the host-side symbol is a
+// stand-in, not a device pointer).
+static __device__ __align__(256) unsigned char g_compact_scratch[ACTKV_COMPACT_NOALLOC_BYTES];
+
+namespace {
+constexpr int kMaxDevices = 64;
+std::mutex g_scratch_mutex;
+void* g_scratch_addr[kMaxDevices] = {nullptr};
+}  // namespace
+
+extern "C" {
+
+size_t actkv_compact_noalloc_max_bytes(void) { return ACTKV_COMPACT_NOALLOC_BYTES; }
+
+int actkv_compact_noalloc(const actkv_pool_t* pool, const actkv_tables_t* tables, int32_t layer_begin,
+                          int32_t layer_end, const int32_t* sel_idx, int64_t sel_stride,
+                          const int32_t* keep_indptr, const int32_t* budget, int32_t max_keep,
+                          int32_t* status, actkv_stream_t stream) {
+  if (!tables) return ACTKV_E_INVALID;
+  if (tables->n_req < 0 || tables->max_pages < 0) return ACTKV_E_INVALID;
+  if (actkv_compact_workspace_bytes(tables->n_req, tables->max_pages) > ACTKV_COMPACT_NOALLOC_BYTES)
+    return ACTKV_E_TOOBIG;
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return ACTKV_E_CUDA;
+  void* scratch = nullptr;
+  {
+    std::lock_guard<std::mutex> lock(g_scratch_mutex);
+    if (g_scratch_addr[dev] == nullptr) {
+      // once per device, with that device current: resolve the array's address on THIS device
+      void* p = nullptr;
+      if (cudaGetSymbolAddress(&p, g_compact_scratch) != cudaSuccess || p == nullptr) return ACTKV_E_CUDA;
+      g_scratch_addr[dev] = p;
+    }
+    scratch = g_scratch_addr[dev];
+  }
+  // Every word of the plan that the copy and table-update kernels read is rewritten by the plan
+  // kernel of this same call (flags, per-request offsets, the page ids it pops), so what an earlier
+  // call left in the array is never read and nothing needs clearing.
+  return actkv_compact(pool, tables, layer_begin, layer_end, sel_idx, sel_stride, keep_indptr, budget, max_keep,
+                       scratch, ACTKV_COMPACT_NOALLOC_BYTES, status, stream);
+}
+
+}  // extern "C"
