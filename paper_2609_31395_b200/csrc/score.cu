@@ -89,7 +89,7 @@ static int score_impl(int mode, const actkv_pool_t* pool, const actkv_tables_t* 
   a.scale_log2 = sm_scale * kLog2e;
   a.causal = causal;
   const int64_t units = (int64_t)nls * Hkv * R;
-  const bool use_tc = score_tc_supported(pool, G, max_win);
+  const bool use_tc = score_tc_supported(pool, G, max_win, sm_scale, q);
 
   const float* lse = lse_in;
   if (mode & 1) {

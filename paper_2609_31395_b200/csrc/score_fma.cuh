@@ -14,7 +14,7 @@ namespace actkv {
 constexpr int FMA_TK = 64;        // keys per tile
 constexpr int FMA_RQ = 32;        // window x group rows per chunk (at most)
 constexpr int FMA_NT = 256;       // threads per CTA
-constexpr int LSE_CHUNK = 2048;   // keys per partial (m, sum) of the LSE pass (both paths)
+constexpr int LSE_CHUNK = 4096;   // keys per partial (m, sum) of the LSE pass (both paths)
 
 struct ScoreArgs {
   PoolView pool;
