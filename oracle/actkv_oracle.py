@@ -230,11 +230,13 @@ def compact(pool_bits: np.ndarray, tables: Tables, sel, budget, layers=None):
             for h in range(Hkv):
                 idx = np.asarray(sel[a][h][r], dtype=np.int64)
                 assert idx.shape[0] == n
-                for i in range(n):
-                    d = new_page[i // P] * P + i % P
-                    sslot = src_slot_of[idx[i]]
-                    dst[0, d, h, :] = src[0, sslot, h, :]
-                    dst[1, d, h, :] = src[1, sslot, h, :]
+                # survivor i (token idx[i]) goes to logical slot i of the new pages; the same
+                # copy for every i at once (sources and destinations are disjoint pages)
+                i = np.arange(n)
+                d = np.asarray(new_page, dtype=np.int64)[i // P] * P + i % P
+                sslot = src_slot_of[idx]
+                dst[0, d, h, :] = src[0, sslot, h, :]
+                dst[1, d, h, :] = src[1, sslot, h, :]
         pt[r, :] = -1
         pt[r, :X] = new_page
         sl[r] = n

@@ -72,10 +72,16 @@ __global__ void compact_plan_kernel(TablesView tab, int32_t page_size, int32_t n
 constexpr int CP_NT = 256;
 constexpr int CP_UNROLL = 8;
 
+// One CTA per (destination page, request, layer).  The (slot, head) -> source / destination row
+// offsets are resolved once into shared memory; the copy loop then costs two shared loads and a few
+// integer ops per 16-byte vector, with CP_UNROLL independent loads in flight per thread.
+// VPR_SHIFT >= 0: 16-byte vectors per row = 1 << VPR_SHIFT (head_dim 64 / 128 / 256); -1: any head_dim.
+template <int VPR_SHIFT>
 __global__ void __launch_bounds__(CP_NT) compact_copy_kernel(
     PoolView pool, TablesView tab, int32_t layer_begin, const int32_t* __restrict__ sel_idx,
     int64_t sel_stride, const int32_t* __restrict__ keep_indptr, const int32_t* __restrict__ budget,
     CompactWs* ws, int32_t* status) {
+  extern __shared__ __align__(16) int64_t cp_smem[];     // [2][P*H]: source offsets, destination offsets
   if (!ws->plan_ok) return;
   const int R = tab.n_req;
   const int r = blockIdx.y, slab = blockIdx.z, dp = blockIdx.x;
@@ -88,41 +94,51 @@ __global__ void __launch_bounds__(CP_NT) compact_copy_kernel(
   const int32_t L = tab.seq_len[r];
   const int32_t dst_page = ws_new_pages(ws, R)[noff + dp];
   const int n_slots = min(P, n - dp * P);
-  const int vpr = D / 8;                                  // 16-byte vectors per row
-  const int per_kv = n_slots * H * vpr;
-  const int total = 2 * per_kv;
-  __nv_bfloat16* lbase = const_cast<__nv_bfloat16*>(pool.base) + (int64_t)(layer_begin + slab) * pool.stride_layer;
+  const int nsh = n_slots * H;
+  int64_t* src_off = cp_smem;
+  int64_t* dst_off = cp_smem + P * H;
   const int32_t* sel_base = sel_idx + (int64_t)slab * H * sel_stride + keep_indptr[r] + dp * P;
-
+  for (int i = threadIdx.x; i < nsh; i += CP_NT) {
+    const int slot = i / H, h = i - slot * H;
+    const int32_t tok = sel_base[(int64_t)h * sel_stride + slot];
+    int64_t so = -1;
+    if ((uint32_t)tok >= (uint32_t)L) {
+      report(status, ACTKV_E_BADINDEX, r, tok);
+    } else {
+      const int32_t sp = checked_page(tab, pool.n_pages, r, tok / P, status);
+      so = (int64_t)sp * pool.stride_page + (int64_t)(tok % P) * pool.stride_slot + (int64_t)h * pool.stride_head;
+    }
+    src_off[i] = so;
+    dst_off[i] = (int64_t)dst_page * pool.stride_page + (int64_t)slot * pool.stride_slot + (int64_t)h * pool.stride_head;
+  }
+  __syncthreads();
+  __nv_bfloat16* lbase = const_cast<__nv_bfloat16*>(pool.base) + (int64_t)(layer_begin + slab) * pool.stride_layer;
+  const int vpr = D / 8;
+  const int per_kv = (VPR_SHIFT >= 0) ? (nsh << VPR_SHIFT) : nsh * vpr;
+  const int total = 2 * per_kv;
   for (int v0 = threadIdx.x; v0 < total; v0 += CP_NT * CP_UNROLL) {
     uint4 val[CP_UNROLL];
-    int64_t dst_off[CP_UNROLL];
+    int64_t doff[CP_UNROLL];
 #pragma unroll
     for (int k = 0; k < CP_UNROLL; ++k) {
       const int v = v0 + k * CP_NT;
-      dst_off[k] = -1;
+      doff[k] = -1;
       if (v < total) {
-        const int kv = v / per_kv;
-        int rem = v - kv * per_kv;
-        const int slot = rem / (H * vpr);
-        rem -= slot * (H * vpr);
-        const int h = rem / vpr, dv = rem - h * vpr;
-        const int32_t tok = sel_base[(int64_t)h * sel_stride + slot];
-        if ((uint32_t)tok >= (uint32_t)L) {
-          report(status, ACTKV_E_BADINDEX, r, tok);
-        } else {
-          const int32_t sp = checked_page(tab, pool.n_pages, r, tok / P, status);
-          const int64_t src = (int64_t)kv * pool.stride_kv + (int64_t)sp * pool.stride_page +
-                              (int64_t)(tok % P) * pool.stride_slot + (int64_t)h * pool.stride_head + dv * 8;
-          val[k] = *reinterpret_cast<const uint4*>(lbase + src);
-          dst_off[k] = (int64_t)kv * pool.stride_kv + (int64_t)dst_page * pool.stride_page +
-                       (int64_t)slot * pool.stride_slot + (int64_t)h * pool.stride_head + dv * 8;
+        const int kv = v >= per_kv ? 1 : 0;
+        const int rem = v - kv * per_kv;
+        const int i = (VPR_SHIFT >= 0) ? (rem >> VPR_SHIFT) : rem / vpr;
+        const int dv = (VPR_SHIFT >= 0) ? (rem & ((1 << VPR_SHIFT) - 1)) : rem - i * vpr;
+        const int64_t so = src_off[i];
+        if (so >= 0) {
+          const int64_t kvo = (int64_t)kv * pool.stride_kv + dv * 8;
+          val[k] = *reinterpret_cast<const uint4*>(lbase + so + kvo);
+          doff[k] = dst_off[i] + kvo;
         }
       }
     }
 #pragma unroll
     for (int k = 0; k < CP_UNROLL; ++k)
-      if (dst_off[k] >= 0) *reinterpret_cast<uint4*>(lbase + dst_off[k]) = val[k];
+      if (doff[k] >= 0) *reinterpret_cast<uint4*>(lbase + doff[k]) = val[k];
   }
 }
 
@@ -205,8 +221,21 @@ int actkv_compact(const actkv_pool_t* pool, const actkv_tables_t* tables, int32_
   if (max_x > tables->max_pages) max_x = tables->max_pages;
   if (nl > 0 && max_x > 0) {
     dim3 grid((unsigned)max_x, (unsigned)R, (unsigned)nl);
-    actkv::compact_copy_kernel<<<grid, actkv::CP_NT, 0, s>>>(pv, tv, layer_begin, sel_idx, sel_stride,
-                                                              keep_indptr, budget, w, status);
+    const size_t sm = (size_t)2 * pool->page_size * pool->n_kv_heads * sizeof(int64_t);
+    if (sm > 48 * 1024) return ACTKV_E_INVALID;
+    const int vpr = pool->head_dim / 8;
+    if (vpr == 16)
+      actkv::compact_copy_kernel<4><<<grid, actkv::CP_NT, sm, s>>>(pv, tv, layer_begin, sel_idx, sel_stride,
+                                                                    keep_indptr, budget, w, status);
+    else if (vpr == 8)
+      actkv::compact_copy_kernel<3><<<grid, actkv::CP_NT, sm, s>>>(pv, tv, layer_begin, sel_idx, sel_stride,
+                                                                    keep_indptr, budget, w, status);
+    else if (vpr == 32)
+      actkv::compact_copy_kernel<5><<<grid, actkv::CP_NT, sm, s>>>(pv, tv, layer_begin, sel_idx, sel_stride,
+                                                                    keep_indptr, budget, w, status);
+    else
+      actkv::compact_copy_kernel<-1><<<grid, actkv::CP_NT, sm, s>>>(pv, tv, layer_begin, sel_idx, sel_stride,
+                                                                     keep_indptr, budget, w, status);
     ACTKV_CHECK_LAUNCH();
   }
   if (layer_end == pool->n_layers) {

@@ -1,0 +1,249 @@
+// Pooled-score pass of the tensor-core score path (Section 7.1 recovery identity A = exp(s - LSE);
+// Algorithm 3 steps 3-5: max over the GQA group, mean over the action tokens).
+//
+// D[key, row] = K Q^T: the 128 keys of a tile sit on the TMEM lanes, row = w*G + g on the columns,
+// 256 columns per accumulator, two accumulators in the 512 TMEM columns.  A "job" is one (key tile,
+// 256-row chunk) accumulator.  Two epilogue warpgroups take the jobs of even / odd parity, so one
+// drains accumulator 0 while the tensor pipe fills accumulator 1 and the other warpgroup drains it.
+// With two row chunks per tile the warpgroups hold partial sums over different action tokens of the
+// same keys; warpgroup 1 hands its partial to warpgroup 0 through shared memory.
+#pragma once
+
+#include "tc_common.cuh"
+
+namespace actkv {
+namespace tc {
+
+constexpr int POOL_EPI_WARPS = 8;
+constexpr int POOL_THREADS = (2 + POOL_EPI_WARPS) * 32;
+
+struct PoolBarriers {
+  uint64_t k_full[8];
+  uint64_t k_empty[8];
+  uint64_t q_full;
+  uint64_t tmem_full[2];
+  uint64_t tmem_empty[2];
+  uint64_t part_full;         // warpgroup 1 -> warpgroup 0: partial sums of a tile are in `exch`
+  uint64_t part_empty;        // warpgroup 0 -> warpgroup 1: `exch` has been read
+  uint64_t drained;
+  uint32_t tmem_base;
+  int abort_flag;
+  float exch[TK];
+};
+
+// One accumulator: columns [0, 32*n_cg) hold s for rows n0 .. of this key (lane).  nlse = -lse*log2(e)
+// per row (-inf for padding rows).  Adds sum_w exp2(max_g(s*c + nlse)) over the live rows to `acc`.
+// TMEM loads are software-pipelined against the arithmetic of the previous 32 columns.
+template <int G>
+__device__ __forceinline__ void pool_job(uint32_t taddr, const float* nlse, int n_cg, int w_first, int w_min, float c,
+                                         float& acc) {
+  float v[2][32];
+  tmem_ld32(taddr, v[0]);
+#pragma unroll
+  for (int cg = 0; cg < 8; ++cg) {
+    if (cg < n_cg) {
+      tmem_ld_wait();
+      if (cg + 1 < n_cg) tmem_ld32(taddr + (cg + 1) * 32, v[(cg + 1) & 1]);
+      float* x = v[cg & 1];
+      const float4* l4 = reinterpret_cast<const float4*>(nlse + cg * 32);
+#pragma unroll
+      for (int q4 = 0; q4 < 8; ++q4) {
+        const float4 l = l4[q4];
+        ffma2(x[q4 * 4 + 0], x[q4 * 4 + 1], x[q4 * 4 + 0], x[q4 * 4 + 1], c, l.x, l.y);
+        ffma2(x[q4 * 4 + 2], x[q4 * 4 + 3], x[q4 * 4 + 2], x[q4 * 4 + 3], c, l.z, l.w);
+      }
+      constexpr int WPG = 32 / G;                 // action tokens per 32-column group
+#pragma unroll
+      for (int i = 0; i < WPG; ++i) {
+        const float mx = max_of<G>(x + i * G);
+        const int w = w_first + cg * WPG + i;
+        acc += (w >= w_min) ? exp2f(mx) : 0.f;    // padding rows: mx = -inf -> 0
+      }
+    }
+  }
+}
+
+template <int G>
+__global__ void __launch_bounds__(POOL_THREADS, 1)
+score_tc_pool_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constant__ CUtensorMap qmap, const TcArgs ta) {
+  extern __shared__ __align__(1024) uint8_t smem[];
+  const ScoreArgs& a = ta.a;
+  const int R = a.tab.n_req, Hkv = a.pool.n_kv_heads;
+  const int u = blockIdx.x / ta.n_kchunks;
+  const int kchunk = blockIdx.x - u * ta.n_kchunks;
+  const int r = u % R, h = (u / R) % Hkv, slab = u / (R * Hkv);
+  const int L = a.tab.seq_len[r];
+  const int w0 = a.win_indptr[r], W = a.win_indptr[r + 1] - w0;
+  const int rows = W * G;
+  const int t_begin = kchunk * ta.tiles_per_cta;
+  if (t_begin * TK >= L) return;
+  if (W <= 0 || (a.causal && W > L)) {
+    if (threadIdx.x == 0 && kchunk == 0) report(a.status, ACTKV_E_INVALID, r, W);
+    return;
+  }
+  const int t_end = min((L + TK - 1) / TK, t_begin + ta.tiles_per_cta);
+  const int n_tiles = t_end - t_begin;
+  const int rows_pad = (rows + 127) & ~127;               // <= MAX_ROWS (checked by the host)
+  const int n_rc = (rows_pad + 255) / 256;                // 256-row chunks per key tile: 1 or 2
+  const int n_qblk = rows_pad / 128;
+  const int n_jobs = n_tiles * n_rc;
+  const int S = ta.n_stages;
+
+  const uint32_t smem_base = smem_u32(smem);
+  const uint32_t q_bytes = (uint32_t)n_rc * 2 * QBLK_BYTES;     // per chunk: [2 halves][256 rows x 128 B]
+  const uint32_t q_smem = smem_base;
+  const uint32_t k_smem = smem_base + q_bytes;
+  float* nlse = reinterpret_cast<float*>(smem + q_bytes + (size_t)S * KTILE_BYTES);       // [rows_pad]
+  PoolBarriers* bars = reinterpret_cast<PoolBarriers*>(reinterpret_cast<uint8_t*>(nlse) + MAX_ROWS * 4);
+  volatile int* abort_flag = &bars->abort_flag;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+  if ((smem_base & 1023u) != 0) {
+    if (threadIdx.x == 0) report(a.status, ACTKV_E_CUDA, -2, (int32_t)smem_base);
+    return;
+  }
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < S; ++s) { mbar_init(smem_u32(&bars->k_full[s]), 1); mbar_init(smem_u32(&bars->k_empty[s]), 1); }
+    mbar_init(smem_u32(&bars->q_full), 1);
+    for (int b = 0; b < 2; ++b) {
+      mbar_init(smem_u32(&bars->tmem_full[b]), 1);
+      mbar_init(smem_u32(&bars->tmem_empty[b]), POOL_EPI_WARPS / 2);
+    }
+    mbar_init(smem_u32(&bars->part_full), POOL_EPI_WARPS / 2);
+    mbar_init(smem_u32(&bars->part_empty), POOL_EPI_WARPS / 2);
+    mbar_init(smem_u32(&bars->drained), 1);
+    bars->abort_flag = 0;
+    fence_barrier_init();
+  }
+  {
+    // -lse of every row in log2 units; padding rows get -inf so that s*c + nlse drops out of the max
+    const float* lse_base = a.lse + ((int64_t)slab * a.sum_win + w0) * a.n_q_heads + h * G;
+    for (int n = threadIdx.x; n < rows_pad; n += blockDim.x)
+      nlse[n] = (n < rows) ? -lse_base[(int64_t)(n / G) * a.n_q_heads + (n % G)] * kLog2e : -INFINITY;
+  }
+  if (warp == 1) {
+    tmem_alloc(smem_u32(&bars->tmem_base), 512);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = bars->tmem_base;
+
+  if (warp == 0) {
+    // ---------------- TMA producer ----------------
+    const int n_lp = (L + a.pool.page_size - 1) / a.pool.page_size;
+    const int layer = a.layer_begin + slab;
+    if (lane == 0) {
+      mbar_expect_tx(smem_u32(&bars->q_full), (uint32_t)n_qblk * QBLK_BYTES);
+      const int wrow = slab * a.sum_win + w0;
+      for (int qb = 0; qb < n_qblk; ++qb)
+        for (int hf = 0; hf < 2; ++hf)
+          tma_load_3d(q_smem + (qb >> 1) * 2 * QBLK_BYTES + hf * QBLK_BYTES + (qb & 1) * HALF_BYTES, &qmap,
+                      smem_u32(&bars->q_full), hf * 64, h * G, wrow + qb * (128 / G));
+    }
+    int32_t pid = (lane < 8) ? page_for_tile(a.tab, a.pool.n_pages, r, t_begin * 8 + lane, n_lp, a.status) : 0;
+    for (int it = 0; it < n_tiles; ++it) {
+      const int s = it % S;
+      const uint32_t ph = (uint32_t)(it / S) & 1u;
+      int32_t pid_next = 0;
+      if (lane < 8 && it + 1 < n_tiles)
+        pid_next = page_for_tile(a.tab, a.pool.n_pages, r, (t_begin + it + 1) * 8 + lane, n_lp, a.status);
+      int ok = 1;
+      if (lane == 0) {
+        ok = mbar_wait(smem_u32(&bars->k_empty[s]), ph ^ 1u, abort_flag) ? 1 : 0;
+        if (ok) mbar_expect_tx(smem_u32(&bars->k_full[s]), KTILE_BYTES);
+      }
+      ok = __shfl_sync(0xffffffffu, ok, 0);
+      if (!ok) break;
+      if (lane < 8) {
+        const uint32_t dst = k_smem + s * KTILE_BYTES + lane * 2048;
+        tma_load_4d(dst, &kmap, smem_u32(&bars->k_full[s]), 0, h, pid * 16, layer);
+        tma_load_4d(dst + HALF_BYTES, &kmap, smem_u32(&bars->k_full[s]), 64, h, pid * 16, layer);
+      }
+      pid = pid_next;
+    }
+  } else if (warp == 1) {
+    // ---------------- MMA issuer: D[key, row] = K Q^T ----------------
+    if (lane == 0) {
+      bool ok = mbar_wait(smem_u32(&bars->q_full), 0, abort_flag);
+      int job = 0;
+      for (int it = 0; ok && it < n_tiles; ++it) {
+        const int s = it % S;
+        ok = mbar_wait(smem_u32(&bars->k_full[s]), (uint32_t)(it / S) & 1u, abort_flag);
+        for (int rc = 0; ok && rc < n_rc; ++rc, ++job) {
+          const int b = job & 1;
+          ok = mbar_wait(smem_u32(&bars->tmem_empty[b]), ((uint32_t)(job >> 1) & 1u) ^ 1u, abort_flag);
+          if (!ok) break;
+          tc_fence_after();
+          const int ncols = min(256, rows_pad - rc * 256);
+          const uint32_t idesc = idesc_bf16(128, ncols);
+#pragma unroll
+          for (int kk = 0; kk < 8; ++kk) {
+            const uint64_t adesc = smem_desc_sw128(k_smem + s * KTILE_BYTES + (kk >> 2) * HALF_BYTES + (kk & 3) * 32);
+            const uint64_t bdesc = smem_desc_sw128(q_smem + rc * 2 * QBLK_BYTES + (kk >> 2) * QBLK_BYTES + (kk & 3) * 32);
+            umma_bf16(tmem_base + b * 256, adesc, bdesc, idesc, kk > 0 ? 1u : 0u);
+          }
+          umma_commit(smem_u32(&bars->tmem_full[b]));
+        }
+        if (ok) umma_commit(smem_u32(&bars->k_empty[s]));
+      }
+      umma_commit(smem_u32(&bars->drained));
+      mbar_wait(smem_u32(&bars->drained), 0, abort_flag, ok ? WAIT_LIMIT_NS : DRAIN_LIMIT_NS);
+    }
+    __syncwarp();                                  // lanes 1..31 wait here for the issuing lane
+  } else {
+    // ---------------- epilogue: one key per thread, jobs of this warpgroup's parity ----------------
+    const int wg = (warp - 2) >> 2;               // 0 or 1 = accumulator it drains
+    const int quarter = warp & 3;                 // TMEM lane quarter this warp may read
+    const float c = a.scale_log2;
+    const float inv_w = 1.0f / (float)W;
+    float* out = a.score_out + ((int64_t)slab * Hkv + h) * a.sum_tok + a.tok_indptr[r];
+    const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + wg * 256;
+    for (int job = wg; job < n_jobs; job += 2) {
+      const int it = (n_rc == 2) ? (job >> 1) : job;
+      const int rc = (n_rc == 2) ? (job & 1) : 0;
+      const int key = (t_begin + it) * TK + quarter * 32 + lane;
+      // causal: row w sees key j iff j <= L - W + w  <=>  w >= j - (L - W)
+      const int w_min = a.causal ? max(0, key - (L - W)) : 0;
+      if (!mbar_wait(smem_u32(&bars->tmem_full[wg]), (uint32_t)(job >> 1) & 1u, abort_flag)) break;
+      tc_fence_after();
+      const int n_cg = (min(rows, rc * 256 + 256) - rc * 256 + 31) / 32;      // 32-column groups with live rows
+      float acc = 0.f;
+      pool_job<G>(taddr, nlse + rc * 256, n_cg, (rc * 256) / G, w_min, c, acc);
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(smem_u32(&bars->tmem_empty[wg]));
+      if (n_rc == 1) {
+        if (key < L) out[key] = acc * inv_w;
+      } else if (wg == 1) {
+        // partial over the second row chunk: hand it to warpgroup 0 once it has read the previous tile's
+        if (!mbar_wait(smem_u32(&bars->part_empty), ((uint32_t)it & 1u) ^ 1u, abort_flag)) break;
+        bars->exch[quarter * 32 + lane] = acc;
+        __syncwarp();
+        if (lane == 0) mbar_arrive(smem_u32(&bars->part_full));
+      } else {
+        if (!mbar_wait(smem_u32(&bars->part_full), (uint32_t)it & 1u, abort_flag)) break;
+        acc += bars->exch[quarter * 32 + lane];
+        __syncwarp();
+        if (lane == 0) mbar_arrive(smem_u32(&bars->part_empty));
+        if (key < L) out[key] = acc * inv_w;
+      }
+    }
+  }
+  // ---------------- teardown ----------------
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 0 && lane == 0 && *abort_flag) {
+    report(a.status, ACTKV_E_TIMEOUT, u, kchunk);
+    for (int s = 0; s < S; ++s) mbar_wait(smem_u32(&bars->k_full[s]), 0, abort_flag, DRAIN_LIMIT_NS / 8);
+  }
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, 512);
+  }
+}
+
+}  // namespace tc
+}  // namespace actkv

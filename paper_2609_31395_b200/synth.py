@@ -258,3 +258,109 @@ def table1_case(n_req: int, L: int, B: int) -> Workload:
     """Shapes of the paper's kernel table: page 16, 8 KV heads, head_dim 128 (G = 4, W = 32 assumed)."""
     return Workload(f"t1_r{n_req}_{L}_{B}", 1, 8, 4, [L] * n_req, [32] * n_req, [B] * n_req,
                     table_style="fragmented", seed=10 + n_req)
+
+
+def config4(n_layers: int = 48, n_req: int = 64, seed: int = 4) -> Workload:
+    """Serving mix on the Qwen3-30B-A3B shape: lengths log-uniform in 8K-64K, shared fragmented pool.
+    Budgets are placeholders (20% of length): the workload's budgets come from actkv_budget."""
+    g = torch.Generator()
+    g.manual_seed(5000 + seed)
+    u = torch.rand(n_req, generator=g)
+    lens = [int(math.exp(math.log(8192) + float(x) * (math.log(65536) - math.log(8192)))) for x in u]
+    return Workload("c4_serving_mix_x64", n_layers, 4, 8, lens, [64] * n_req, [L // 5 for L in lens],
+                    table_style="fragmented", pool_slack=1.05, n_topics=64, seed=seed)
+
+
+class AgentTrace:
+    """Iterative agent trace (Qwen3-8B attention shape): every round appends an observation, a
+    reasoning segment and an action to each request's paged cache; the action tokens are the window
+    (causal: the last W cached tokens) and the budget is 25% of the uncompressed tokens so far.
+
+    The owner of pool / tables between compression steps: `next_round()` pops pages from the free
+    list for the new tokens and writes their K/V (host-side integer work + torch fills, no method
+    arithmetic); the compression step itself is run by the caller on the tensors held here.
+    """
+
+    def __init__(self, n_layers=36, n_kv_heads=8, group=4, n_req=16, n_rounds=25, head_dim=128, page_size=16,
+                 seed=5, device="cpu", prompt=(8192, 16384), obs=(1024, 2048), reason=(200, 800), action=(32, 96),
+                 budget_frac=0.25, plant_frac=0.02, max_tokens_per_req=24576):
+        self.NL, self.Hkv, self.G, self.R, self.D, self.P = n_layers, n_kv_heads, group, n_req, head_dim, page_size
+        self.n_rounds, self.rng_ranges = n_rounds, dict(prompt=prompt, obs=obs, reason=reason, action=action)
+        self.budget_frac, self.plant_frac = budget_frac, plant_frac
+        self.dev = torch.device(device)
+        self.g = torch.Generator(device=self.dev)
+        self.g.manual_seed(6000 + seed)
+        self.g_cpu = torch.Generator()
+        self.g_cpu.manual_seed(7000 + seed)
+        self.max_pages = -(-max_tokens_per_req // page_size)
+        # every request may hold max_tokens_per_req tokens plus the fresh pages of one compaction
+        self.n_pages = int(n_req * self.max_pages * 1.6) + 8
+        self.pool = torch.zeros((n_layers, 2, self.n_pages, page_size, n_kv_heads, head_dim), dtype=torch.bfloat16,
+                                device=self.dev)
+        self.page_table = torch.full((n_req, self.max_pages), -1, dtype=torch.int32, device=self.dev)
+        self.seq_len = torch.zeros(n_req, dtype=torch.int32, device=self.dev)
+        perm = torch.randperm(self.n_pages, generator=self.g_cpu).to(torch.int32)
+        self.free_list = perm.to(self.dev)
+        self.free_count = torch.tensor([self.n_pages], dtype=torch.int32, device=self.dev)
+        self.uncompressed = [0] * n_req
+        self.round = 0
+        # the shared direction of each (layer, request, KV head)'s action queries persists over rounds
+        self.mu = torch.randn((n_layers, n_req, n_kv_heads, 1, head_dim), generator=self.g, device=self.dev)
+
+    def _draw(self, key):
+        lo, hi = self.rng_ranges[key]
+        return int(torch.randint(lo, hi + 1, (1,), generator=self.g_cpu))
+
+    def next_round(self):
+        """Appends this round's tokens; returns (q, win_indptr, tok_indptr, budget, windows, seq_lens)."""
+        NL, Hkv, G, R, D, P = self.NL, self.Hkv, self.G, self.R, self.D, self.P
+        seq = self.seq_len.cpu().tolist()
+        table = self.page_table.cpu()
+        free = self.free_list.cpu()
+        fc = int(self.free_count.cpu())
+        windows, new_lens = [], []
+        for r in range(R):
+            n_new = self._draw("obs") + self._draw("reason")
+            if self.round == 0:
+                n_new += self._draw("prompt")
+            W = self._draw("action")
+            windows.append(W)
+            new_lens.append(n_new + W)
+        sum_win = sum(windows)
+        q = torch.empty((NL, sum_win, Hkv * G, D), dtype=torch.bfloat16, device=self.dev)
+        w0 = 0
+        for r in range(R):
+            L0, n_new, W = seq[r], new_lens[r], windows[r]
+            L1 = L0 + n_new
+            assert -(-L1 // P) <= self.max_pages, "request outgrew max_tokens_per_req"
+            for lp in range(-(-L0 // P), -(-L1 // P)):              # pop pages for the new tokens
+                fc -= 1
+                table[r, lp] = free[fc]
+            j = torch.arange(L0, L1, dtype=torch.int64)
+            slots = (table[r].to(torch.int64)[j // P] * P + j % P).to(self.dev)
+            n_pl = int(round(self.plant_frac * (n_new - W)))
+            pl = torch.randperm(n_new - W, generator=self.g_cpu)[:n_pl].to(self.dev)
+            for l in range(NL):
+                eps = torch.randn((W, Hkv, G, D), generator=self.g, device=self.dev)
+                q_r = ((self.mu[l, r][None] + eps) / math.sqrt(2.0)).to(torch.bfloat16)     # [W, Hkv, G, D]
+                q[l, w0:w0 + W] = q_r.view(W, Hkv * G, D)
+                for kv in range(2):
+                    vals = torch.randn((n_new, Hkv, D), generator=self.g, device=self.dev)
+                    if kv == 0 and n_pl:
+                        q_mean = q_r.float().mean(dim=(0, 2))
+                        vals[pl] = 0.5 * q_mean[None] + 0.1 * torch.randn((n_pl, Hkv, D), generator=self.g, device=self.dev)
+                    self.pool[l, kv].view(self.n_pages * P, Hkv, D)[slots] = vals.to(torch.bfloat16)
+            seq[r] = L1
+            self.uncompressed[r] += n_new
+            w0 += W
+        self.page_table.copy_(table)
+        self.free_count.fill_(fc)
+        self.seq_len.copy_(torch.tensor(seq, dtype=torch.int32))
+        budget = [int(math.ceil(self.budget_frac * u)) for u in self.uncompressed]
+        win_indptr = torch.zeros(R + 1, dtype=torch.int32)
+        win_indptr[1:] = torch.cumsum(torch.tensor(windows, dtype=torch.int32), 0)
+        tok_indptr = torch.zeros(R + 1, dtype=torch.int32)
+        tok_indptr[1:] = torch.cumsum(torch.tensor(seq, dtype=torch.int32), 0)
+        self.round += 1
+        return (q, win_indptr.to(self.dev), tok_indptr.to(self.dev),
+                torch.tensor(budget, dtype=torch.int32, device=self.dev), windows, seq)

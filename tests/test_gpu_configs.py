@@ -1,0 +1,222 @@
+"""GPU parity at the benchmark configurations' full sizes (through the C ABI, in the launch
+configuration bench.py times), on sampled units the oracle can compute one by one, plus properties
+that hold for every unit:
+
+  * scores of sampled (layer, head, request) units against the oracle, max-rel <= 2e-3;
+  * TopK of EVERY unit against the oracle's TopK of the GPU's own float32 scores (bit-exact);
+  * compaction of whole sampled layers against the oracle's compaction of the GPU's index lists
+    (bit-exact, including "nothing else changed"); tables, free list and counts exact;
+  * planted action-critical keys retained in every unit.
+"""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import actkv_oracle as O
+from paper_2609_31395_b200 import binding as B
+from paper_2609_31395_b200 import harness as H
+from paper_2609_31395_b200 import synth
+
+import parity_util as U
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+
+def _check_sampled_scores(pool, page_table_before, seq_len_before, q, win_indptr, tok_indptr, wl_like, score, units,
+                          layer_of_slab=None):
+    """score: GPU tensor [NLs, Hkv, sum_tok]; units: (slab, head, request)."""
+    Hkv, G, D, P, causal, sm_scale = wl_like
+    pt = page_table_before.cpu().numpy()
+    sl = seq_len_before.cpu().numpy()
+    wi = win_indptr.cpu().numpy()
+    ti = tok_indptr.cpu().numpy()
+    worst = 0.0
+    for (a, h, r) in units:
+        layer = a if layer_of_slab is None else layer_of_slab[a]
+        L = int(sl[r])
+        slots = torch.from_numpy(O.slot_map(pt[r], L, P)).to(pool.device)
+        k_bits = U.bits(pool[layer, 0].view(-1, Hkv, D)[slots, h])
+        q_bits = U.bits(q[a, wi[r]:wi[r + 1], h * G:(h + 1) * G])
+        want, _ = O.score_unit(O.bf16_bits_to_f64(q_bits), O.bf16_bits_to_f64(k_bits), sm_scale, causal)
+        got = score[a, h, ti[r]:ti[r + 1]].cpu().numpy()
+        assert np.isfinite(got).all()
+        err = U.max_rel(got, want)
+        assert err <= U.SCORE_RTOL, f"unit {(a, h, r)}: score max-rel {err:.3e}"
+        worst = max(worst, err)
+    return worst
+
+
+def _check_all_select(score, tok_indptr, budgets, sel_idx, keep_indptr):
+    sc = score.cpu().numpy().reshape(-1, score.shape[-1])
+    U.check_select_exact(sc, tok_indptr.cpu().numpy(), budgets, sel_idx.cpu().numpy(), keep_indptr.cpu().numpy())
+
+
+def _check_layer_compaction(layer_before, layer_after, tables_before, sel_idx, keep_indptr, budgets, Hkv, slab):
+    """One pool layer [2, n_pages, P, Hkv, D] before / after against the oracle's compaction."""
+    ki = keep_indptr.cpu().numpy()
+    sel_np = sel_idx.cpu().numpy()
+    R = len(budgets)
+    sel = [[[sel_np[slab * Hkv + h, ki[r]:ki[r + 1]] for r in range(R)] for h in range(Hkv)]]
+    want_pool, want_t = O.compact(U.bits(layer_before)[None], tables_before, sel, budgets, layers=[0])
+    assert np.array_equal(U.bits(layer_after)[None], want_pool)
+    return want_t
+
+
+def _check_tables(inst_like, want_t):
+    page_table, seq_len, free_list, free_count = inst_like
+    fc = int(free_count.cpu())
+    assert np.array_equal(page_table.cpu().numpy(), want_t.page_table)
+    assert np.array_equal(seq_len.cpu().numpy(), want_t.seq_len)
+    assert fc == want_t.free_count
+    assert np.array_equal(free_list.cpu().numpy()[:fc], want_t.free_list[:fc])
+
+
+def _run_fixed_workload(wl, score_units, compaction_slabs):
+    inst = synth.generate(wl, DEV)
+    tables_before = U.oracle_tables(inst)
+    pt_before, sl_before = inst.page_table.clone(), inst.seq_len.clone()
+    snap = {a: inst.pool[a].clone() for a in compaction_slabs}
+    comp = U.run_step(inst)
+    comp.check_status()
+    wl_like = (wl.n_kv_heads, wl.group, wl.head_dim, wl.page_size, wl.causal, wl.sm_scale)
+    worst = _check_sampled_scores(inst.pool, pt_before, sl_before, inst.q, inst.win_indptr, inst.tok_indptr, wl_like,
+                                  comp.score, score_units)
+    _check_all_select(comp.score, inst.tok_indptr, wl.budgets, comp.sel_idx, comp.keep_indptr)
+    want_t = None
+    for a in compaction_slabs:
+        want_t = _check_layer_compaction(snap[a], inst.pool[a], tables_before, comp.sel_idx, comp.keep_indptr,
+                                         wl.budgets, wl.n_kv_heads, a)
+    _check_tables((inst.page_table, inst.seq_len, inst.free_list, inst.free_count), want_t)
+    # planted keys survive in every unit
+    sel = comp.sel_idx.cpu().numpy()
+    ki = comp.keep_indptr.cpu().numpy()
+    for r in range(wl.n_req):
+        planted = inst.planted[r].numpy()
+        for o in range(sel.shape[0]):
+            kept = sel[o, ki[r]:ki[r + 1]]
+            assert np.isin(planted, kept).all(), f"planted key evicted in unit ({o},{r})"
+    return worst
+
+
+def test_config2_qwen3_8b_32k():
+    """36 layers, 32 q / 8 KV heads, 32768 tokens, window 64, B = 25%: every head of 4 layers
+    (first and last included) against the oracle."""
+    wl = synth.config2()
+    units = [(a, h, 0) for a in (0, 11, 24, 35) for h in range(wl.n_kv_heads)]
+    _run_fixed_workload(wl, units, compaction_slabs=[0, 35])
+
+
+def test_config3_qwen3_30b_35k_x8_bench_shape():
+    """The benchmark workload at full size (48 layers, 8 x 35000 tokens): sampled units of three
+    layers covering every request and every head, TopK of all 1536 units, two whole layers of the
+    compaction, tables."""
+    wl = synth.config3()
+    units = [(0, 0, 0), (0, 1, 3), (0, 2, 5), (0, 3, 7), (23, 0, 1), (23, 1, 2), (23, 2, 4), (23, 3, 6),
+             (47, 0, 7), (47, 1, 0), (47, 2, 1), (47, 3, 2)]
+    _run_fixed_workload(wl, units, compaction_slabs=[0, 47])
+
+
+def test_config4_serving_mix_budgets_from_monitor():
+    """64 requests, lengths log-uniform in 8K-64K; budgets produced on the device by actkv_budget
+    from 256 action-token logit rows per request (V = 151936), clamped to 15-40% of length.  Two of
+    the 48 layers are resident (all 48 would need 159 GiB); layers are independent repetitions."""
+    wl = synth.config4(n_layers=2)
+    R = wl.n_req
+    inst = synth.generate(wl, DEV)
+    rows = 256
+    # logits in request batches through one reused buffer (64 x 256 x 151936 fp32 = 10 GB at once otherwise)
+    hist_cap = 512
+    conf_hist = torch.zeros((R, hist_cap), dtype=torch.float32, device=DEV)
+    hist_len = torch.zeros(R, dtype=torch.int32, device=DEV)
+    budget_in = torch.tensor([L // 5 for L in wl.seq_lens], dtype=torch.int32, device=DEV)
+    budget_out = torch.zeros(R, dtype=torch.int32, device=DEV)
+    slopes = torch.zeros(R, dtype=torch.float64, device=DEV)
+    status = torch.zeros(4, dtype=torch.int32, device=DEV)
+    params = B.BudgetParams.paper_defaults(clamp_lo_ppm=150000, clamp_hi_ppm=400000)
+    batch = 16
+    ws = torch.empty(B.actkv_budget_workspace_bytes(batch * rows, batch, hist_cap) + 256, dtype=torch.uint8, device=DEV)
+    sampled_T = {}
+    for b0 in range(0, R, batch):
+        logits, ltok = synth.confidence_logits(batch, rows, 151936, seed=40 + b0, device=DEV)
+        B.actkv_budget(logits, ltok, batch * rows, 151936, conf_hist[b0:b0 + batch], hist_len[b0:b0 + batch], hist_cap,
+                       params, inst.seq_len[b0:b0 + batch], budget_in[b0:b0 + batch], budget_out[b0:b0 + batch],
+                       slopes[b0:b0 + batch], batch, ws, status)
+        if b0 == 0:                                       # oracle token confidences for two requests
+            torch.cuda.synchronize()
+            for r in (0, 5):
+                sampled_T[r] = O.token_confidence(logits[r * rows:(r + 1) * rows].cpu().numpy(), 20)
+    torch.cuda.synchronize()
+    assert status.cpu().tolist()[0] == 0
+    hist = conf_hist.cpu().numpy()
+    for r, T in sampled_T.items():
+        assert np.abs(hist[r, :rows] - T).max() <= 2e-5
+    op = O.BudgetParams(clamp_lo_ppm=150000, clamp_hi_ppm=400000)
+    got_B = budget_out.cpu().numpy()
+    n_scaled = 0
+    for r in range(R):                                   # decision on the GPU's own history: exact
+        a = O.fit_slope(O.trace_confidence(hist[r, :rows], op.w, op.s, op.b_percent))
+        assert abs(a - slopes.cpu().numpy()[r]) <= 1e-12 * max(1.0, abs(a))
+        want = O.budget_update(int(budget_in[r]), a, op, wl.seq_lens[r])
+        assert got_B[r] == want
+        assert -(-wl.seq_lens[r] * 150000 // 1000000) <= got_B[r] <= wl.seq_lens[r] * 400000 // 1000000
+        n_scaled += a < 0
+    assert 0 < n_scaled < R                               # the drift gives both outcomes
+    # compression with those budgets
+    wl.budgets = [int(b) for b in got_B]
+    inst.budget = budget_out
+    tables_before = U.oracle_tables(inst)
+    pt_before, sl_before = inst.page_table.clone(), inst.seq_len.clone()
+    snap = inst.pool[1].clone()
+    comp = U.run_step(inst)
+    comp.check_status()
+    order = np.argsort(wl.seq_lens)
+    longest, shortest, median = int(order[-1]), int(order[0]), int(order[R // 2])
+    units = [(0, 0, longest), (1, 3, longest), (0, 1, shortest), (1, 2, shortest), (0, 2, median), (1, 0, median)]
+    wl_like = (wl.n_kv_heads, wl.group, wl.head_dim, wl.page_size, wl.causal, wl.sm_scale)
+    _check_sampled_scores(inst.pool, pt_before, sl_before, inst.q, inst.win_indptr, inst.tok_indptr, wl_like,
+                          comp.score, units)
+    _check_all_select(comp.score, inst.tok_indptr, wl.budgets, comp.sel_idx, comp.keep_indptr)
+    want_t = _check_layer_compaction(snap, inst.pool[1], tables_before, comp.sel_idx, comp.keep_indptr, wl.budgets,
+                                     wl.n_kv_heads, 1)
+    _check_tables((inst.page_table, inst.seq_len, inst.free_list, inst.free_count), want_t)
+
+
+def test_config5_agent_trace_25_rounds():
+    """16 requests x 25 rounds on the Qwen3-8B shape (2 of the 36 layers resident): each round appends
+    observation + reasoning + action tokens, then compresses the already-compressed cache with the
+    action tokens as a causal, ragged window and budget 25% of the uncompressed length."""
+    tr = synth.AgentTrace(n_layers=2, device=DEV)
+    rng = np.random.default_rng(0)
+    wl_like = (tr.Hkv, tr.G, tr.D, tr.P, True, 1.0 / math.sqrt(tr.D))
+    final_uncompressed = None
+    for rnd in range(tr.n_rounds):
+        q, win_indptr, tok_indptr, budget, windows, seq = tr.next_round()
+        budgets = budget.cpu().tolist()
+        keep = [min(b, L) for b, L in zip(budgets, seq)]
+        sz = H.StepSizes(tr.R, sum(windows), max(windows), sum(seq), max(seq), max(1, sum(keep)), max(keep))
+        comp = H.Compressor(tr.pool, tr.page_table, tr.seq_len, tr.free_list, tr.free_count, tr.Hkv * tr.G, sz)
+        tables_before = O.Tables(tr.page_table.cpu().numpy().copy(), tr.seq_len.cpu().numpy().copy(),
+                                 tr.free_list.cpu().numpy().copy(), int(tr.free_count.cpu()))
+        pt_before, sl_before = tr.page_table.clone(), tr.seq_len.clone()
+        full_pool_check = rnd in (0, 12, 24)
+        snap = tr.pool[1].clone() if full_pool_check else None
+        comp.step(q, win_indptr, tok_indptr, budget, wl_like[5], True)
+        torch.cuda.synchronize()
+        comp.check_status()
+        units = [(int(rng.integers(0, 2)), int(rng.integers(0, tr.Hkv)), int(rng.integers(0, tr.R))) for _ in range(3)]
+        _check_sampled_scores(tr.pool, pt_before, sl_before, q, win_indptr, tok_indptr, wl_like, comp.score, units)
+        _check_all_select(comp.score, tok_indptr, budgets, comp.sel_idx, comp.keep_indptr)
+        if full_pool_check:
+            want_t = _check_layer_compaction(snap, tr.pool[1], tables_before, comp.sel_idx, comp.keep_indptr, budgets,
+                                             tr.Hkv, 1)
+        else:                                             # tables only
+            empty_pool = np.zeros((0, 2, tr.n_pages, tr.P, tr.Hkv, tr.D), dtype=np.uint16)
+            _, want_t = O.compact(empty_pool, tables_before, [], budgets, layers=[])
+        _check_tables((tr.page_table, tr.seq_len, tr.free_list, tr.free_count), want_t)
+        # the newest tokens (this round's action) were visible to few rows; the kept set is still n_r long
+        assert tr.seq_len.cpu().tolist() == keep
+        final_uncompressed = list(tr.uncompressed)
+    assert 40000 <= min(final_uncompressed) and max(final_uncompressed) <= 90000
