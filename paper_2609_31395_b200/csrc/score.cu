@@ -84,7 +84,20 @@ static int score_impl(int mode, const actkv_pool_t* pool, const actkv_tables_t* 
   a.sum_win = sum_win;
   a.sum_tok = sum_tok;
   a.rows_max = lay.rows_max;
-  a.n_chunks = lay.n_chunks;
+  // Keys per LSE partial.  A CTA pays a fixed cost (operand set-up, pipeline fill and drain), so chunks
+  // are as long as they can be while there are still several CTAs per SM: the largest multiple of the
+  // minimum chunk that leaves at least 6 x 148 work items (never more chunks than the workspace holds).
+  {
+    const int64_t units_ = (int64_t)(layer_end - layer_begin) * Hkv * R;
+    const int64_t row_groups = (lay.rows_max + 255) / 256;
+    int n_chunks = (int)((6 * 148 + units_ * row_groups - 1) / (units_ * row_groups));
+    if (n_chunks < 1) n_chunks = 1;
+    if (n_chunks > lay.n_chunks) n_chunks = lay.n_chunks;
+    int chunk = (max_tok + n_chunks - 1) / n_chunks;
+    chunk = (chunk + LSE_CHUNK - 1) / LSE_CHUNK * LSE_CHUNK;
+    a.lse_chunk = chunk;
+    a.n_chunks = (max_tok + chunk - 1) / chunk;
+  }
   a.n_tiles = (max_tok + FMA_TK - 1) / FMA_TK;
   a.scale_log2 = sm_scale * kLog2e;
   a.causal = causal;
@@ -98,7 +111,7 @@ static int score_impl(int mode, const actkv_pool_t* pool, const actkv_tables_t* 
       int rc = score_tc_launch_lse(a, pool, max_tok, max_win, s);
       if (rc != ACTKV_OK) return rc;
     } else {
-      const int64_t grid1 = units * lay.n_chunks;
+      const int64_t grid1 = units * a.n_chunks;
       if (grid1 > 0x7fffffffLL) return ACTKV_E_INVALID;
       const size_t sm1 = score_fma_smem_bytes(D, lay.rows_max, 1);
       if (sm1 > 200 * 1024) return ACTKV_E_INVALID;

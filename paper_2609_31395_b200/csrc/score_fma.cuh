@@ -28,6 +28,7 @@ struct ScoreArgs {
   int32_t* status;
   int32_t layer_begin, n_layers_sub, n_q_heads, group;
   int32_t sum_win, sum_tok, rows_max, n_chunks, n_tiles;
+  int32_t lse_chunk;             // keys per LSE partial of this launch (multiple of 128, >= LSE_CHUNK)
   float scale_log2;              // sm_scale * log2(e)
   int32_t causal;
 };
@@ -66,13 +67,13 @@ __global__ void __launch_bounds__(FMA_NT) score_fma_kernel(const ScoreArgs a) {
   const int r = u % R, h = (u / R) % Hkv, slab = u / (R * Hkv);
   const int L = a.tab.seq_len[r];
   const int w0 = a.win_indptr[r], W = a.win_indptr[r + 1] - w0;
-  const int key_begin = part * ((PASS == 1) ? LSE_CHUNK : FMA_TK);
+  const int key_begin = part * ((PASS == 1) ? a.lse_chunk : FMA_TK);
   if (key_begin >= L) return;
   if (W <= 0 || (a.causal && W > L)) {               // no window, or a window longer than the cache
     if (threadIdx.x == 0 && part == 0) report(a.status, ACTKV_E_INVALID, r, W);
     return;
   }
-  const int key_end = min(L, key_begin + ((PASS == 1) ? LSE_CHUNK : FMA_TK));
+  const int key_end = min(L, key_begin + ((PASS == 1) ? a.lse_chunk : FMA_TK));
   const int rows = W * G;
   const int wpc = FMA_RQ / G;                          // window rows per chunk
   const int n_rc = (W + wpc - 1) / wpc;
@@ -211,7 +212,7 @@ __global__ void lse_combine_kernel(const ScoreArgs a, float* lse_out, float* lse
   const int L = a.tab.seq_len[r];
   const int w0 = a.win_indptr[r], W = a.win_indptr[r + 1] - w0;
   if (row >= W * G || L <= 0) return;
-  const int n_chunks = (L + LSE_CHUNK - 1) / LSE_CHUNK;
+  const int n_chunks = (L + a.lse_chunk - 1) / a.lse_chunk;
   const float2* p = a.partials + (int64_t)u * a.n_chunks * a.rows_max + row;
   float M = -INFINITY;
   for (int c = 0; c < n_chunks; ++c) M = fmaxf(M, p[(int64_t)c * a.rows_max].x);

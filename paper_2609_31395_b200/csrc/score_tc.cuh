@@ -95,6 +95,17 @@ inline bool score_tc_supported(const actkv_pool_t* p, int G, int max_win, float 
   return tc::encode_fn() != nullptr;
 }
 
+template <int POLY>
+inline int score_tc_launch_lse_p(const CUtensorMap& kmap, const CUtensorMap& qmap, const tc::TcArgs& ta, unsigned grid,
+                                 size_t smem, cudaStream_t s) {
+  (void)qmap;
+  if (cudaFuncSetAttribute(tc::score_tc_lse_kernel<POLY>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+    return ACTKV_E_CUDA;
+  tc::score_tc_lse_kernel<POLY><<<grid, tc::LSE_THREADS, smem, s>>>(kmap, ta);
+  ACTKV_CHECK_LAUNCH();
+  return ACTKV_OK;
+}
+
 inline int score_tc_launch_lse(ScoreArgs& a, const actkv_pool_t* pool, int max_tok, int max_win, cudaStream_t s) {
   (void)max_tok;
   CUtensorMap kmap, qmap;
@@ -103,18 +114,24 @@ inline int score_tc_launch_lse(ScoreArgs& a, const actkv_pool_t* pool, int max_t
   ta.a = a;
   const int rows_pad = (max_win * a.group + 127) & ~127;
   ta.n_rg = (rows_pad + 255) / 256;
-  ta.n_stages = 4;
+  ta.n_stages = 6;
   ta.tiles_per_cta = 0;
   ta.n_kchunks = 0;
   const int64_t units = (int64_t)a.n_layers_sub * a.pool.n_kv_heads * a.tab.n_req;
   const int64_t grid = units * ta.n_rg * a.n_chunks;
   if (grid > 0x7fffffffLL) return ACTKV_E_INVALID;
-  const size_t smem = 2 * tc::QBLK_BYTES + (size_t)ta.n_stages * tc::KTILE_BYTES + sizeof(tc::Barriers);
-  if (cudaFuncSetAttribute(tc::score_tc_lse_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
-    return ACTKV_E_CUDA;
-  tc::score_tc_lse_kernel<<<(unsigned)grid, tc::LSE_THREADS, smem, s>>>(kmap, qmap, ta);
-  ACTKV_CHECK_LAUNCH();
-  return ACTKV_OK;
+  const size_t smem = (size_t)ta.n_stages * tc::KTILE_BYTES + sizeof(tc::LseBarriers);
+  // share of the exps evaluated by the polynomial (tuning knob; the default is what the bench uses)
+  int poly = tc::LSE_POLY_PAIRS_DEFAULT;
+  if (const char* e = getenv("ACTKV_LSE_POLY")) poly = atoi(e);
+  switch (poly) {
+    case 0: return score_tc_launch_lse_p<0>(kmap, qmap, ta, (unsigned)grid, smem, s);
+    case 1: return score_tc_launch_lse_p<1>(kmap, qmap, ta, (unsigned)grid, smem, s);
+    case 2: return score_tc_launch_lse_p<2>(kmap, qmap, ta, (unsigned)grid, smem, s);
+    case 4: return score_tc_launch_lse_p<4>(kmap, qmap, ta, (unsigned)grid, smem, s);
+    case 5: return score_tc_launch_lse_p<5>(kmap, qmap, ta, (unsigned)grid, smem, s);
+    default: return score_tc_launch_lse_p<3>(kmap, qmap, ta, (unsigned)grid, smem, s);
+  }
 }
 
 template <int G>
@@ -144,9 +161,9 @@ inline int score_tc_launch_score(ScoreArgs& a, const actkv_pool_t* pool, int max
   const int64_t units = (int64_t)a.n_layers_sub * a.pool.n_kv_heads * a.tab.n_req;
   const int max_tiles = (max_tok + tc::TK - 1) / tc::TK;
   // enough CTAs to fill the 148 SMs a few times over, few enough that the Q load is amortised
-  int64_t tpc = (units * max_tiles) / (148 * 8);
+  int64_t tpc = (units * max_tiles) / (148 * 6);
   if (tpc < 4) tpc = 4;
-  if (tpc > 64) tpc = 64;
+  if (tpc > max_tiles) tpc = max_tiles;
   ta.tiles_per_cta = (int)tpc;
   ta.n_kchunks = (max_tiles + ta.tiles_per_cta - 1) / ta.tiles_per_cta;
   const int64_t grid = units * ta.n_kchunks;

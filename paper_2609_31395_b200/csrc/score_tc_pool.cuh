@@ -15,7 +15,7 @@ namespace actkv {
 namespace tc {
 
 constexpr int POOL_EPI_WARPS = 8;
-constexpr int POOL_THREADS = (2 + POOL_EPI_WARPS) * 32;
+constexpr int POOL_THREADS = (2 + POOL_EPI_WARPS) * 32;     // producer, MMA issuer, epilogue
 
 struct PoolBarriers {
   uint64_t k_full[8];
@@ -48,7 +48,11 @@ __device__ __forceinline__ void pool_job(uint32_t taddr, const float* nlse, int 
       const float4* l4 = reinterpret_cast<const float4*>(nlse + cg * 32);
 #pragma unroll
       for (int q4 = 0; q4 < 8; ++q4) {
+#ifdef ACTKV_EXP_NO_NLSE
+        const float4 l = make_float4(-1.f, -1.f, -1.f, -1.f + (float)(l4 == nullptr));
+#else
         const float4 l = l4[q4];
+#endif
         ffma2(x[q4 * 4 + 0], x[q4 * 4 + 1], x[q4 * 4 + 0], x[q4 * 4 + 1], c, l.x, l.y);
         ffma2(x[q4 * 4 + 2], x[q4 * 4 + 3], x[q4 * 4 + 2], x[q4 * 4 + 3], c, l.z, l.w);
       }
@@ -96,7 +100,7 @@ score_tc_pool_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_cons
   float* nlse = reinterpret_cast<float*>(smem + q_bytes + (size_t)S * KTILE_BYTES);       // [rows_pad]
   PoolBarriers* bars = reinterpret_cast<PoolBarriers*>(reinterpret_cast<uint8_t*>(nlse) + MAX_ROWS * 4);
   volatile int* abort_flag = &bars->abort_flag;
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int warp = __shfl_sync(0xffffffffu, (int)(threadIdx.x >> 5), 0), lane = threadIdx.x & 31;   // warp-uniform
 
   if ((smem_base & 1023u) != 0) {
     if (threadIdx.x == 0) report(a.status, ACTKV_E_CUDA, -2, (int32_t)smem_base);
@@ -142,13 +146,15 @@ score_tc_pool_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_cons
           tma_load_3d(q_smem + (qb >> 1) * 2 * QBLK_BYTES + hf * QBLK_BYTES + (qb & 1) * HALF_BYTES, &qmap,
                       smem_u32(&bars->q_full), hf * 64, h * G, wrow + qb * (128 / G));
     }
-    int32_t pid = (lane < 8) ? page_for_tile(a.tab, a.pool.n_pages, r, t_begin * 8 + lane, n_lp, a.status) : 0;
+    // page ids of four tiles at a time, one per lane (lane / 8 = tile within the group, lane % 8 = page);
+    // the next group's ids are loaded while the current four tiles are being issued
+    int32_t pid = page_for_tile(a.tab, a.pool.n_pages, r, t_begin * 8 + lane, n_lp, a.status);
+    int32_t pid_next = 0;
     for (int it = 0; it < n_tiles; ++it) {
       const int s = it % S;
       const uint32_t ph = (uint32_t)(it / S) & 1u;
-      int32_t pid_next = 0;
-      if (lane < 8 && it + 1 < n_tiles)
-        pid_next = page_for_tile(a.tab, a.pool.n_pages, r, (t_begin + it + 1) * 8 + lane, n_lp, a.status);
+      if ((it & 3) == 0 && it + 4 < n_tiles)
+        pid_next = page_for_tile(a.tab, a.pool.n_pages, r, (t_begin + it + 4) * 8 + lane, n_lp, a.status);
       int ok = 1;
       if (lane == 0) {
         ok = mbar_wait(smem_u32(&bars->k_empty[s]), ph ^ 1u, abort_flag) ? 1 : 0;
@@ -156,42 +162,62 @@ score_tc_pool_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_cons
       }
       ok = __shfl_sync(0xffffffffu, ok, 0);
       if (!ok) break;
-      if (lane < 8) {
-        const uint32_t dst = k_smem + s * KTILE_BYTES + lane * 2048;
+      if ((lane >> 3) == (it & 3)) {
+        const uint32_t dst = k_smem + s * KTILE_BYTES + (lane & 7) * 2048;
         tma_load_4d(dst, &kmap, smem_u32(&bars->k_full[s]), 0, h, pid * 16, layer);
         tma_load_4d(dst + HALF_BYTES, &kmap, smem_u32(&bars->k_full[s]), 64, h, pid * 16, layer);
       }
-      pid = pid_next;
+      if ((it & 3) == 3) pid = pid_next;
     }
   } else if (warp == 1) {
     // ---------------- MMA issuer: D[key, row] = K Q^T ----------------
-    if (lane == 0) {
-      bool ok = mbar_wait(smem_u32(&bars->q_full), 0, abort_flag);
-      int job = 0;
-      for (int it = 0; ok && it < n_tiles; ++it) {
-        const int s = it % S;
-        ok = mbar_wait(smem_u32(&bars->k_full[s]), (uint32_t)(it / S) & 1u, abort_flag);
-        for (int rc = 0; ok && rc < n_rc; ++rc, ++job) {
-          const int b = job & 1;
-          ok = mbar_wait(smem_u32(&bars->tmem_empty[b]), ((uint32_t)(job >> 1) & 1u) ^ 1u, abort_flag);
-          if (!ok) break;
-          tc_fence_after();
-          const int ncols = min(256, rows_pad - rc * 256);
-          const uint32_t idesc = idesc_bf16(128, ncols);
-#pragma unroll
-          for (int kk = 0; kk < 8; ++kk) {
-            const uint64_t adesc = smem_desc_sw128(k_smem + s * KTILE_BYTES + (kk >> 2) * HALF_BYTES + (kk & 3) * 32);
-            const uint64_t bdesc = smem_desc_sw128(q_smem + rc * 2 * QBLK_BYTES + (kk >> 2) * QBLK_BYTES + (kk & 3) * 32);
-            umma_bf16(tmem_base + b * 256, adesc, bdesc, idesc, kk > 0 ? 1u : 0u);
-          }
-          umma_commit(smem_u32(&bars->tmem_full[b]));
-        }
-        if (ok) umma_commit(smem_u32(&bars->k_empty[s]));
+    // The whole warp runs the loop (waits and descriptor arithmetic stay warp-uniform, so they can
+    // live in uniform registers); one elected lane issues the tcgen05 instructions.
+    // The tensor pipe's queue is shallow: whatever the issuing warp spends between two jobs (a successful
+    // barrier wait costs 100-200 cycles) is idle time of the pipe.  So the barriers of job j+1 are polled
+    // (mbarrier.test_wait, non-blocking) BEFORE the MMAs of job j are issued and the answers are only read
+    // afterwards; the blocking wait is the fallback when they were not ready yet.
+    const uint64_t kdesc0 = smem_desc_sw128(k_smem);
+    const uint64_t qdesc0 = smem_desc_sw128(q_smem);
+    bool ok = mbar_wait(smem_u32(&bars->q_full), 0, abort_flag);
+    if (ok) ok = mbar_wait(smem_u32(&bars->k_full[0]), 0, abort_flag);               // job 0: stage 0, accumulator 0
+    for (int job = 0; ok && job < n_jobs; ++job) {
+      const int it = (n_rc == 2) ? (job >> 1) : job;
+      const int rc = (n_rc == 2) ? (job & 1) : 0;
+      const int s = it % S, b = job & 1;
+      const int jn = job + 1;
+      const int itn = (n_rc == 2) ? (jn >> 1) : jn;
+      const int sn = itn % S;
+      const uint32_t kfull_n = smem_u32(&bars->k_full[sn]), kpar_n = (uint32_t)(itn / S) & 1u;
+      const uint32_t empty_n = smem_u32(&bars->tmem_empty[jn & 1]), epar_n = ((uint32_t)(jn >> 1) & 1u) ^ 1u;
+      bool kready = true, eready = true;
+      if (jn < n_jobs) {
+        kready = (itn == it) || mbar_test_wait(kfull_n, kpar_n);
+        eready = mbar_test_wait(empty_n, epar_n);
       }
-      umma_commit(smem_u32(&bars->drained));
-      mbar_wait(smem_u32(&bars->drained), 0, abort_flag, ok ? WAIT_LIMIT_NS : DRAIN_LIMIT_NS);
+      tc_fence_after();
+      const int ncols = min(256, rows_pad - rc * 256);
+      const uint32_t idesc = idesc_bf16(128, ncols);
+      const uint64_t adesc_s = kdesc0 + (uint64_t)((s * KTILE_BYTES) >> 4);
+      const uint64_t bdesc_c = qdesc0 + (uint64_t)((rc * 2 * QBLK_BYTES) >> 4);
+      if (elect_one()) {
+#pragma unroll
+        for (int kk = 0; kk < 8; ++kk)
+          umma_bf16(tmem_base + b * 256, adesc_s + (uint64_t)(((kk >> 2) * HALF_BYTES + (kk & 3) * 32) >> 4),
+                    bdesc_c + (uint64_t)(((kk >> 2) * QBLK_BYTES + (kk & 3) * 32) >> 4), idesc, kk > 0 ? 1u : 0u);
+        umma_commit(smem_u32(&bars->tmem_full[b]));
+        if (rc == n_rc - 1) umma_commit(smem_u32(&bars->k_empty[s]));
+      }
+      __syncwarp();
+      if (jn < n_jobs) {
+        if (!kready) ok = mbar_wait(kfull_n, kpar_n, abort_flag);
+        if (ok && !eready) ok = mbar_wait(empty_n, epar_n, abort_flag);
+      }
     }
-    __syncwarp();                                  // lanes 1..31 wait here for the issuing lane
+    if (elect_one()) umma_commit(smem_u32(&bars->drained));
+    __syncwarp();
+    mbar_wait(smem_u32(&bars->drained), 0, abort_flag, ok ? WAIT_LIMIT_NS : DRAIN_LIMIT_NS);
+    __syncwarp();
   } else {
     // ---------------- epilogue: one key per thread, jobs of this warpgroup's parity ----------------
     const int wg = (warp - 2) >> 2;               // 0 or 1 = accumulator it drains
@@ -210,7 +236,13 @@ score_tc_pool_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_cons
       tc_fence_after();
       const int n_cg = (min(rows, rc * 256 + 256) - rc * 256 + 31) / 32;      // 32-column groups with live rows
       float acc = 0.f;
+#ifndef ACTKV_EXP_NO_EPI
+#ifdef ACTKV_EXP_NO_NLSE
+      pool_job<G>(taddr, nlse, 0 * n_cg + n_cg, (rc * 256) / G, w_min, c, acc);
+#else
       pool_job<G>(taddr, nlse + rc * 256, n_cg, (rc * 256) / G, w_min, c, acc);
+#endif
+#endif
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(smem_u32(&bars->tmem_empty[wg]));
