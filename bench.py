@@ -213,7 +213,8 @@ def run_ours(args):
     inst = synth.generate(wl, dev)
     sz = H.sizes_of(inst)
     comp = H.Compressor(inst.pool, inst.page_table, inst.seq_len, inst.free_list, inst.free_count, wl.n_q_heads, sz,
-                        layers_per_call=args.layers_per_call, want_lse=True)
+                        layers_per_call=args.layers_per_call if args.layers_per_call else (8 if args.overlap else None),
+                        want_lse=True)
     # budget inputs: LOGIT_ROWS action-token logit rows per request
     logits, ltok = synth.confidence_logits(R, LOGIT_ROWS, VOCAB, seed=wl.seed, device=dev)
     n_rows = logits.shape[0]
@@ -240,18 +241,26 @@ def run_ours(args):
     stage_names = ["budget", "lse", "score", "select", "compact"]
 
     def one_step(events=None):
-        def mark(name):
+        # events: list of (name, event); stage time = time since the previous event on the SAME stream
+        # ("begin" / "begin_aux" only open an interval).  Main stream: budget, lse, score; second
+        # stream (overlapped mode): select, compact.
+        def mark(name, stream=None):
             if events is not None:
                 e = torch.cuda.Event(enable_timing=True)
-                e.record()
+                e.record(stream if stream is not None else torch.cuda.current_stream())
                 events.append((name, e))
         mark("start")
         B.actkv_budget(logits, ltok, n_rows, VOCAB, conf_hist, hist_len, hist_cap, bparams, inst.seq_len, budget_in,
                        budget_dev, None, R, ws_budget, comp.status)
         bud = budget_dev if args.workload == "c3" else inst.budget
         mark("budget")
-        n = comp.step(inst.q, inst.win_indptr, inst.tok_indptr, bud, wl.sm_scale, wl.causal,
-                      lse_in=lse_supplied, marks=(lambda nm: mark(nm)) if events is not None else (lambda nm: None))
+        if args.overlap:
+            n = comp.step_overlapped(inst.q, inst.win_indptr, inst.tok_indptr, bud, wl.sm_scale, wl.causal,
+                                     lse_in=lse_supplied, marks=mark)
+        else:
+            n = comp.step(inst.q, inst.win_indptr, inst.tok_indptr, bud, wl.sm_scale, wl.causal,
+                          lse_in=lse_supplied, marks=(lambda nm: mark(nm)))
+        mark("end")
         return n + 2
 
     for _ in range(args.warmup):
@@ -283,14 +292,19 @@ def run_ours(args):
 
     stage_ms = {k: 0.0 for k in stage_names}
     total_ms = 0.0
+    aux_names = ("begin_aux", "select", "compact") if args.overlap else ()
     for ev in all_events:
         total_ms += ev[0][1].elapsed_time(ev[-1][1])
-        prev = ev[0][1]
+        prev_main, prev_aux = ev[0][1], None
         for name, e in ev[1:]:
-            if name == "begin":
-                continue
-            stage_ms[name] += prev.elapsed_time(e)
-            prev = e
+            if name in aux_names:
+                if name != "begin_aux":
+                    stage_ms[name] += prev_aux.elapsed_time(e)
+                prev_aux = e
+            else:
+                if name not in ("begin", "end"):
+                    stage_ms[name] += prev_main.elapsed_time(e)
+                prev_main = e
     ms_per_step = total_ms / args.steps
     stage_ms = {k: v / args.steps for k, v in stage_ms.items()}
     t = torch.tensor([ms_per_step], dtype=torch.float64, device=dev)
@@ -327,43 +341,31 @@ def run_ours(args):
     # ---- end to end: host buffers in, host results out, every step -------------------------------
     e2e = None
     if not args.no_e2e:
-        q_host = inst.q.cpu().pin_memory()
-        logits_host = logits.cpu().pin_memory()
-        tabs_host = [t.cpu().pin_memory() for t in saved]
-        bin_host = budget_in.cpu().pin_memory()
-        out_host = [torch.empty_like(t).pin_memory() for t in tabs_host[:2]] + \
-                   [torch.empty(1, dtype=torch.int32).pin_memory(), torch.empty(4, dtype=torch.int32).pin_memory(),
-                    torch.empty(R, dtype=torch.int32).pin_memory()]
-        h2d = q_host.numel() * 2 + logits_host.numel() * 4 + sum(t.numel() * 4 for t in tabs_host) + bin_host.numel() * 4
-        d2h = sum(t.numel() * 4 for t in out_host)
+        # restore the device tables first: the runner snapshots them as the host-side state of the engine
+        restore()
+        torch.cuda.synchronize()
+        runner = H.HostStepRunner(comp, inst.q, inst.win_indptr, inst.tok_indptr, budget_in, wl.sm_scale, wl.causal,
+                                  logits=logits, logit_indptr=ltok, hist_cap=hist_cap, params=bparams)
+        h2d, d2h = runner.h2d_bytes, runner.d2h_bytes
         e2e_ms = []
-        for it in range(1 + min(args.steps, 3)):
-            hist_len.zero_(); comp.status.zero_()
+        for it in range(1 + min(args.steps, 5)):
             torch.cuda.synchronize()
             if dist is not None:
                 dist.barrier()
             t0 = time.perf_counter()
-            inst.q.copy_(q_host, non_blocking=True)
-            logits.copy_(logits_host, non_blocking=True)
-            for dst, src in zip((inst.page_table, inst.seq_len, inst.free_list, inst.free_count), tabs_host):
-                dst.copy_(src, non_blocking=True)
-            budget_in.copy_(bin_host, non_blocking=True)
-            one_step()
-            out_host[0].copy_(inst.page_table, non_blocking=True)
-            out_host[1].copy_(inst.seq_len, non_blocking=True)
-            out_host[2].copy_(inst.free_count, non_blocking=True)
-            out_host[3].copy_(comp.status, non_blocking=True)
-            out_host[4].copy_(budget_dev, non_blocking=True)
-            torch.cuda.synchronize()
+            out = runner.run()                 # one C-ABI call: H2D copies, the whole path, D2H copies, stream sync
             if it > 0:
                 e2e_ms.append((time.perf_counter() - t0) * 1e3)
+            if out["st"].tolist()[0] != 0:
+                raise SystemExit(f"actkv_step_host: device status {out['st'].tolist()}")
         te = torch.tensor([sum(e2e_ms) / len(e2e_ms)], dtype=torch.float64, device=dev)
         if dist is not None:
             dist.all_reduce(te, op=dist.ReduceOp.MAX)
         e2e = {"value": world * tokens / (float(te.item()) * 1e-3), "unit": UNIT, "ms_per_step": float(te.item()),
                "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h),
-               "note": "KV pool stays resident in HBM (it is the cache being compressed); queries, logits, tables "
-                       "and budgets come from pinned host memory, new tables / budgets / status go back"}
+               "note": "one actkv_step_host call per step: queries, logits, index arrays, tables and budgets come from "
+                       "pinned host memory, new tables / free list / budgets / status go back; the KV pool stays "
+                       "resident in HBM (it is the cache being compressed)"}
 
     # ---- the oracle on the host cores (rank 0, single GPU only) ----------------------------------
     cpu_baseline = None
@@ -382,6 +384,8 @@ def run_ours(args):
                        "kv_heads": Hkv, "q_heads": wl.n_q_heads, "head_dim": D, "page": wl.page_size,
                        "window": wl.windows[0], "budget": wl.budgets[0], "lse": args.lse,
                        "layers_per_call": comp.lpc, "replicas": world,
+                       "overlap": "select+compact of a layer group on a second stream under the score kernels "
+                                  "of the next group" if args.overlap else "none (one stream)",
                        "l2": "inputs (KV pool %.1f GB) far larger than the 126 MB L2" % (inst.pool.numel() * 2 / 1e9)},
             "stage_ms": stage_ms, "hbm_roofline_frac_whole_step": hbm_frac_whole,
             "algorithmic_bytes_per_step": alg_bytes, "k_bytes_per_pass": bytes_k,
@@ -401,7 +405,11 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="c3", choices=["c1", "c2", "c3"])
     ap.add_argument("--layers", type=int, default=None, help="override the layer count (debugging only)")
-    ap.add_argument("--layers-per-call", type=int, default=None)
+    ap.add_argument("--layers-per-call", type=int, default=None,
+                    help="layers per score/select/compact call (default: 8 when overlapped, else all)")
+    ap.add_argument("--overlap", action="store_true",
+                    help="run select + compact of a layer group on a second stream under the score kernels of the "
+                         "next group (measured: no gain, the score CTAs fill the register file of every SM)")
     ap.add_argument("--lse", default="internal", choices=["internal", "supplied"])
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")

@@ -226,6 +226,54 @@ int actkv_compact(const actkv_pool_t* pool /* host */, const actkv_tables_t* tab
                   void* ws, size_t ws_bytes, int32_t* status, actkv_stream_t stream);
 
 /* ---------------------------------------------------------------------------------------
+ * actkv_step_host — one whole compression step (Algorithm 1 steps 1, 5, 6 with Algorithm 2 in
+ * front) for a caller whose per-step inputs live in HOST memory.
+ *
+ * Copies this step's queries, action-token logits, index arrays, budgets and tables from the host
+ * (pinned memory recommended) into the caller's device staging buffers on `stream`, runs
+ * actkv_budget (when logits are given) -> actkv_keep_indptr -> per group of `layers_per_call`
+ * layers: actkv_score_lse, actkv_score, actkv_select, actkv_compact, copies the new page table,
+ * seq_len, free list, free count, budgets and the status words back to the host, and
+ * SYNCHRONISES the stream before returning (the one entry point that does: its outputs are host
+ * memory).  The KV pool stays in device memory — it is the cache being compressed.
+ * Every pointer named *_host is host memory, every other pointer device memory owned by the caller
+ * and sized as the corresponding argument of the per-stage calls (score_dev:
+ * [layers_per_call, n_kv_heads, sum_tok]; sel_idx_dev: [layers_per_call*n_kv_heads, sel_stride];
+ * lse_dev: [n_layers, sum_win, n_q_heads]; q_dev: [n_layers, sum_win, n_q_heads, head_dim]).
+ * `tables` holds the DEVICE copies of the tables; they are overwritten from the *_host inputs.
+ * Output host pointers may be NULL to skip that copy.  budget_dev holds budget_in on entry of the
+ * path and the budget that was applied on exit.
+ */
+typedef struct {
+  const void*    q_host;
+  const float*   logits_host;          /* [n_rows, vocab] or NULL: no budget update */
+  const int32_t* win_indptr_host;      /* [n_req+1] */
+  const int32_t* tok_indptr_host;      /* [n_req+1] */
+  const int32_t* logit_indptr_host;    /* [n_req+1] (with logits) */
+  const int32_t* budget_in_host;       /* [n_req] */
+  const int32_t* page_table_host;      /* [n_req, max_pages] */
+  const int32_t* seq_len_host;         /* [n_req] */
+  const int32_t* free_list_host;       /* [n_pages] */
+  const int32_t* free_count_host;      /* [1] */
+  int32_t* page_table_out_host; int32_t* seq_len_out_host; int32_t* free_list_out_host;
+  int32_t* free_count_out_host; int32_t* budget_out_host; int32_t* status_out_host /* [4] */;
+  int32_t n_q_heads, sum_win, max_win, sum_tok, max_tok, n_rows, vocab, hist_cap, max_keep;
+  int32_t causal, layers_per_call;
+  float   sm_scale;
+  int64_t sel_stride;
+  void* q_dev; float* logits_dev;
+  int32_t* win_indptr_dev; int32_t* tok_indptr_dev; int32_t* logit_indptr_dev;
+  int32_t* budget_dev; int32_t* keep_indptr_dev;
+  float* conf_hist_dev; int32_t* hist_len_dev; float* lse_dev; float* score_dev; int32_t* sel_idx_dev;
+  void* ws_budget; size_t ws_budget_bytes; void* ws_score; size_t ws_score_bytes;
+  void* ws_compact; size_t ws_compact_bytes;
+  int32_t* status_dev;                 /* [4] */
+} actkv_host_step_t;
+int actkv_step_host(const actkv_pool_t* pool /* host */, const actkv_tables_t* tables /* host */,
+                    const actkv_budget_params_t* params /* host, may be NULL without logits */,
+                    const actkv_host_step_t* io /* host */, actkv_stream_t stream);
+
+/* ---------------------------------------------------------------------------------------
  * actkv_compact_noalloc — actkv_compact without a caller-supplied workspace.
  * (The paper has no counterpart; this is a convenience of the library.)
  *

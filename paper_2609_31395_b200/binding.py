@@ -25,7 +25,7 @@ EXPORTS = ["actkv_budget_workspace_bytes", "actkv_budget", "actkv_score_workspac
            "actkv_score_lse",
            "actkv_keep_indptr", "actkv_select_workspace_bytes", "actkv_select",
            "actkv_compact_workspace_bytes", "actkv_compact", "actkv_compact_noalloc",
-           "actkv_compact_noalloc_max_bytes", "actkv_version"]
+           "actkv_compact_noalloc_max_bytes", "actkv_step_host", "actkv_version"]
 
 
 class ActKVError(RuntimeError):
@@ -59,6 +59,25 @@ class BudgetParams(C.Structure):
 class TieReport(C.Structure):
     _fields_ = [("threshold", C.c_float), ("n_equal_kept", C.c_int32), ("n_equal_total", C.c_int32),
                 ("n_keep", C.c_int32)]
+
+
+class HostStep(C.Structure):
+    """actkv_host_step_t: host inputs / outputs, sizes, device staging and scratch of actkv_step_host."""
+    _fields_ = ([(n, C.c_void_p) for n in
+                 ("q_host", "logits_host", "win_indptr_host", "tok_indptr_host", "logit_indptr_host", "budget_in_host",
+                  "page_table_host", "seq_len_host", "free_list_host", "free_count_host",
+                  "page_table_out_host", "seq_len_out_host", "free_list_out_host", "free_count_out_host",
+                  "budget_out_host", "status_out_host")] +
+                [(n, C.c_int32) for n in
+                 ("n_q_heads", "sum_win", "max_win", "sum_tok", "max_tok", "n_rows", "vocab", "hist_cap", "max_keep",
+                  "causal", "layers_per_call")] +
+                [("sm_scale", C.c_float), ("sel_stride", C.c_int64)] +
+                [(n, C.c_void_p) for n in
+                 ("q_dev", "logits_dev", "win_indptr_dev", "tok_indptr_dev", "logit_indptr_dev", "budget_dev",
+                  "keep_indptr_dev", "conf_hist_dev", "hist_len_dev", "lse_dev", "score_dev", "sel_idx_dev")] +
+                [("ws_budget", C.c_void_p), ("ws_budget_bytes", C.c_size_t), ("ws_score", C.c_void_p),
+                 ("ws_score_bytes", C.c_size_t), ("ws_compact", C.c_void_p), ("ws_compact_bytes", C.c_size_t),
+                 ("status_dev", C.c_void_p)])
 
 
 _lib = None
@@ -105,6 +124,9 @@ def load():
     lib.actkv_compact.restype = i32
     lib.actkv_compact.argtypes = [C.POINTER(PoolDesc), C.POINTER(TablesDesc), i32, i32, vp, i64, vp, vp, i32,
                                   vp, sz, vp, vp]
+    lib.actkv_step_host.restype = i32
+    lib.actkv_step_host.argtypes = [C.POINTER(PoolDesc), C.POINTER(TablesDesc), C.POINTER(BudgetParams),
+                                    C.POINTER(HostStep), vp]
     lib.actkv_compact_noalloc_max_bytes.restype = sz
     lib.actkv_compact_noalloc_max_bytes.argtypes = []
     lib.actkv_compact_noalloc.restype = i32
@@ -242,6 +264,13 @@ def actkv_compact(pool: PoolDesc, tables: TablesDesc, layer_begin, layer_end, se
                               max_keep, _ptr(ws, None, "ws"), ws.numel() * ws.element_size(),
                               _ptr(status, torch.int32, "status"), _stream(stream))
     _check("actkv_compact", rc)
+
+
+def actkv_step_host(pool: PoolDesc, tables: TablesDesc, params: Optional[BudgetParams], io: HostStep, stream=None):
+    """One whole step with host-resident per-step inputs and outputs (synchronises `stream`)."""
+    rc = load().actkv_step_host(C.byref(pool), C.byref(tables), None if params is None else C.byref(params),
+                                C.byref(io), _stream(stream))
+    _check("actkv_step_host", rc)
 
 
 def actkv_compact_noalloc_max_bytes() -> int:

@@ -127,10 +127,9 @@ inline int score_tc_launch_lse(ScoreArgs& a, const actkv_pool_t* pool, int max_t
   switch (poly) {
     case 0: return score_tc_launch_lse_p<0>(kmap, qmap, ta, (unsigned)grid, smem, s);
     case 1: return score_tc_launch_lse_p<1>(kmap, qmap, ta, (unsigned)grid, smem, s);
-    case 2: return score_tc_launch_lse_p<2>(kmap, qmap, ta, (unsigned)grid, smem, s);
+    case 3: return score_tc_launch_lse_p<3>(kmap, qmap, ta, (unsigned)grid, smem, s);
     case 4: return score_tc_launch_lse_p<4>(kmap, qmap, ta, (unsigned)grid, smem, s);
-    case 5: return score_tc_launch_lse_p<5>(kmap, qmap, ta, (unsigned)grid, smem, s);
-    default: return score_tc_launch_lse_p<3>(kmap, qmap, ta, (unsigned)grid, smem, s);
+    default: return score_tc_launch_lse_p<2>(kmap, qmap, ta, (unsigned)grid, smem, s);
   }
 }
 

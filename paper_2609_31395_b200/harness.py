@@ -118,10 +118,128 @@ class Compressor:
             launches += (3 if lse_in is None else 1) + 1 + 2 + (1 if l1 == NL else 0)
         return launches
 
+    def step_overlapped(self, q, win_indptr, tok_indptr, budget, sm_scale, causal, lse_in=None, marks=None):
+        """The same step with select + compact of layer group g running on a second stream while
+        the score kernels of group g+1 run on the current one (the score kernels are bound by the
+        tensor / MUFU pipes, compaction by HBM).  Score and index buffers are double-buffered by
+        group parity.  Tables are still rewritten only by the last compact call, so every score
+        call reads the old tables; compaction writes fresh pages only.
+        `marks`: optional callable(name, stream).  Returns the number of kernels launched."""
+        NL, Hkv, s = self.pd.n_layers, self.pd.n_kv_heads, self.sz
+        main = torch.cuda.current_stream()
+        if not hasattr(self, "_aux"):
+            self._aux = torch.cuda.Stream(device=self.dev)
+            self._score2 = [self.score, torch.empty_like(self.score)]
+            self._sel2 = [self.sel_idx, torch.empty_like(self.sel_idx)]
+            self._ev_score = [torch.cuda.Event(), torch.cuda.Event()]
+            self._ev_sel = [torch.cuda.Event(), torch.cuda.Event()]
+            self._ev_done = torch.cuda.Event()
+            if self.lse is None and lse_in is None:
+                self.lse = torch.empty((NL, s.sum_win, self.n_q_heads), dtype=torch.float32, device=self.dev)
+        aux = self._aux
+        mark = marks if marks is not None else (lambda name, stream: None)
+        B.actkv_keep_indptr(self.seq_len, budget, s.n_req, self.keep_indptr, main)
+        launches = 1
+        for gi, l0 in enumerate(range(0, NL, self.lpc)):
+            l1 = min(NL, l0 + self.lpc)
+            buf = gi & 1
+            score, sel = self._score2[buf], self._sel2[buf]
+            if gi >= 2:
+                main.wait_event(self._ev_sel[buf])          # select of group gi-2 has read this score buffer
+            mark("begin", main)
+            if lse_in is None:
+                self.run_lse(q, win_indptr, tok_indptr, sm_scale, causal, l0, l1, self.lse[l0:l1], main)
+                mark("lse", main)
+                lse = self.lse
+            else:
+                lse = lse_in
+            B.actkv_score(self.pd, self.td, l0, l1, q[l0:l1], win_indptr, self.n_q_heads, lse[l0:l1], sm_scale,
+                          causal, tok_indptr, score[: l1 - l0], None, s.sum_win, s.max_win, s.sum_tok, s.max_tok,
+                          self.ws_score, self.status, main)
+            mark("score", main)
+            self._ev_score[buf].record(main)
+            aux.wait_event(self._ev_score[buf])
+            mark("begin_aux", aux)
+            B.actkv_select(score, tok_indptr, s.sum_tok, budget, (l1 - l0) * Hkv, s.n_req, self.keep_indptr, sel,
+                           s.sel_stride, None, None, self.ws_select, self.status, aux)
+            self._ev_sel[buf].record(aux)
+            mark("select", aux)
+            B.actkv_compact(self.pd, self.td, l0, l1, sel, s.sel_stride, self.keep_indptr, budget, s.max_keep,
+                            self.ws_compact, self.status, aux)
+            mark("compact", aux)
+            launches += (3 if lse_in is None else 1) + 1 + 2 + (1 if l1 == NL else 0)
+        self._ev_done.record(aux)
+        main.wait_event(self._ev_done)
+        return launches
+
     def check_status(self):
         st = self.status.cpu().tolist()
         if st[0] != 0:
             raise B.ActKVError(f"device status {st}", st[0])
+
+
+class HostStepRunner:
+    """Pinned host buffers + device staging for actkv_step_host, the host-buffer form of the step.
+
+    `comp` supplies the device scratch (score, index lists, workspaces, status); this class adds the
+    host side: pinned copies of the per-step inputs and pinned result buffers."""
+
+    def __init__(self, comp: Compressor, q: torch.Tensor, win_indptr, tok_indptr, budget_in, sm_scale: float,
+                 causal: bool, logits: Optional[torch.Tensor] = None, logit_indptr=None, hist_cap: int = 4096,
+                 params: Optional[B.BudgetParams] = None):
+        self.comp, self.params = comp, params
+        dev, s, R = comp.dev, comp.sz, comp.sz.n_req
+        pin = lambda t: t.detach().cpu().contiguous().pin_memory()
+        self.h_in = {"q": pin(q), "win": pin(win_indptr), "tok": pin(tok_indptr), "bud": pin(budget_in),
+                     "pt": pin(comp.page_table), "sl": pin(comp.seq_len), "fl": pin(comp.free_list),
+                     "fc": pin(comp.free_count)}
+        self.h_out = {"pt": torch.empty_like(self.h_in["pt"]).pin_memory(),
+                      "sl": torch.empty_like(self.h_in["sl"]).pin_memory(),
+                      "fl": torch.empty_like(self.h_in["fl"]).pin_memory(),
+                      "fc": torch.empty(1, dtype=torch.int32).pin_memory(),
+                      "bud": torch.empty(R, dtype=torch.int32).pin_memory(),
+                      "st": torch.empty(4, dtype=torch.int32).pin_memory()}
+        self.d = {"q": torch.empty_like(q), "win": torch.empty_like(win_indptr), "tok": torch.empty_like(tok_indptr),
+                  "bud": torch.empty(R, dtype=torch.int32, device=dev)}
+        if comp.lse is None:
+            comp.lse = torch.empty((comp.pd.n_layers, s.sum_win, comp.n_q_heads), dtype=torch.float32, device=dev)
+        n_rows = vocab = 0
+        if logits is not None:
+            n_rows, vocab = logits.shape
+            self.h_in["lg"], self.h_in["lgi"] = pin(logits), pin(logit_indptr)
+            self.d["lg"], self.d["lgi"] = torch.empty_like(logits), torch.empty_like(logit_indptr)
+            self.d["hist"] = torch.zeros((R, hist_cap), dtype=torch.float32, device=dev)
+            self.d["hlen"] = torch.zeros(R, dtype=torch.int32, device=dev)
+            self.d["wsb"] = _ws(B.actkv_budget_workspace_bytes(n_rows, R, hist_cap), dev)
+        io = B.HostStep()
+        hp = lambda k: self.h_in[k].data_ptr() if k in self.h_in else None
+        io.q_host, io.logits_host, io.win_indptr_host, io.tok_indptr_host = hp("q"), hp("lg"), hp("win"), hp("tok")
+        io.logit_indptr_host, io.budget_in_host, io.page_table_host = hp("lgi"), hp("bud"), hp("pt")
+        io.seq_len_host, io.free_list_host, io.free_count_host = hp("sl"), hp("fl"), hp("fc")
+        io.page_table_out_host, io.seq_len_out_host = self.h_out["pt"].data_ptr(), self.h_out["sl"].data_ptr()
+        io.free_list_out_host, io.free_count_out_host = self.h_out["fl"].data_ptr(), self.h_out["fc"].data_ptr()
+        io.budget_out_host, io.status_out_host = self.h_out["bud"].data_ptr(), self.h_out["st"].data_ptr()
+        io.n_q_heads, io.sum_win, io.max_win, io.sum_tok, io.max_tok = comp.n_q_heads, s.sum_win, s.max_win, s.sum_tok, s.max_tok
+        io.n_rows, io.vocab, io.hist_cap, io.max_keep = n_rows, vocab, hist_cap, s.max_keep
+        io.causal, io.layers_per_call, io.sm_scale, io.sel_stride = int(bool(causal)), comp.lpc, float(sm_scale), s.sel_stride
+        dp = lambda k: self.d[k].data_ptr() if k in self.d else None
+        io.q_dev, io.logits_dev, io.win_indptr_dev, io.tok_indptr_dev = dp("q"), dp("lg"), dp("win"), dp("tok")
+        io.logit_indptr_dev, io.budget_dev, io.keep_indptr_dev = dp("lgi"), dp("bud"), comp.keep_indptr.data_ptr()
+        io.conf_hist_dev, io.hist_len_dev, io.lse_dev = dp("hist"), dp("hlen"), comp.lse.data_ptr()
+        io.score_dev, io.sel_idx_dev = comp.score.data_ptr(), comp.sel_idx.data_ptr()
+        io.ws_budget, io.ws_budget_bytes = dp("wsb"), (self.d["wsb"].numel() if "wsb" in self.d else 0)
+        io.ws_score, io.ws_score_bytes = comp.ws_score.data_ptr(), comp.ws_score.numel()
+        io.ws_compact, io.ws_compact_bytes = comp.ws_compact.data_ptr(), comp.ws_compact.numel()
+        io.status_dev = comp.status.data_ptr()
+        self.io = io
+        self.h2d_bytes = sum(t.numel() * t.element_size() for t in self.h_in.values())
+        self.d2h_bytes = sum(t.numel() * t.element_size() for t in self.h_out.values())
+
+    def run(self, stream=None):
+        if "hlen" in self.d:
+            self.d["hlen"].zero_()
+        B.actkv_step_host(self.comp.pd, self.comp.td, self.params, self.io, stream)
+        return self.h_out
 
 
 def sizes_of(inst, sel_stride: Optional[int] = None) -> StepSizes:

@@ -83,6 +83,48 @@ def test_layer_sub_ranges_give_the_same_result():
     assert torch.equal(a.free_list, b.free_list) and torch.equal(a.free_count, b.free_count)
 
 
+def test_overlapped_step_gives_the_same_result():
+    """select + compact of layer group g on a second stream under the score of group g+1."""
+    wl = synth.Workload("ovl", 5, 2, 8, [1200, 333, 700], [32, 16, 64], [300, 100, 200],
+                        table_style="fragmented", seed=12, poison_tail=True)
+    a = synth.generate(wl, DEV)
+    b = synth.generate(wl, DEV)
+    _full_check(a)
+    sz = H.sizes_of(b)
+    comp = H.Compressor(b.pool, b.page_table, b.seq_len, b.free_list, b.free_count, wl.n_q_heads, sz,
+                        layers_per_call=2)
+    comp.step_overlapped(b.q, b.win_indptr, b.tok_indptr, b.budget, wl.sm_scale, wl.causal)
+    torch.cuda.synchronize()
+    comp.check_status()
+    assert torch.equal(a.pool.view(torch.int16), b.pool.view(torch.int16))
+    assert torch.equal(a.page_table, b.page_table) and torch.equal(a.seq_len, b.seq_len)
+    assert torch.equal(a.free_list, b.free_list) and torch.equal(a.free_count, b.free_count)
+
+
+def test_step_host_matches_device_step():
+    """actkv_step_host (host buffers in, host results out) gives what the per-stage calls give."""
+    wl = synth.Workload("host", 3, 2, 4, [900, 333, 500], [16, 8, 32], [250, 100, 125],
+                        table_style="fragmented", seed=14, poison_tail=True)
+    a = synth.generate(wl, DEV)
+    b = synth.generate(wl, DEV)
+    _full_check(a)
+    comp = H.Compressor(b.pool, b.page_table, b.seq_len, b.free_list, b.free_count, wl.n_q_heads, H.sizes_of(b),
+                        layers_per_call=2)
+    runner = H.HostStepRunner(comp, b.q, b.win_indptr, b.tok_indptr, b.budget, wl.sm_scale, wl.causal)
+    # scribble over the device copies: the call must bring everything from the host buffers
+    b.page_table.fill_(-7)
+    b.seq_len.zero_()
+    out = runner.run()
+    assert out["st"].tolist()[0] == 0
+    assert torch.equal(out["pt"], a.page_table.cpu()) and torch.equal(out["sl"], a.seq_len.cpu())
+    assert int(out["fc"]) == int(a.free_count.cpu())
+    fc = int(out["fc"])
+    assert torch.equal(out["fl"][:fc], a.free_list.cpu()[:fc])
+    assert out["bud"].tolist() == wl.budgets
+    assert torch.equal(a.pool.view(torch.int16), b.pool.view(torch.int16))
+    assert runner.h2d_bytes > b.q.numel() * 2 and runner.d2h_bytes > 0
+
+
 def test_config1_all_units_and_planted_keys():
     inst = synth.generate(synth.config1(), DEV)
     res = _full_check(inst)
