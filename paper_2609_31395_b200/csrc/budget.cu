@@ -77,7 +77,9 @@ __device__ __forceinline__ void pick_digit(const uint32_t* hist, int nbins, uint
 __global__ void __launch_bounds__(TC_NT) token_conf_kernel(
     const float* __restrict__ logits, const int32_t* __restrict__ tok_indptr, int32_t vocab,
     int32_t n_req, int32_t k_top, float* __restrict__ conf_hist, const int32_t* __restrict__ hist_len,
-    int32_t hist_cap, float* __restrict__ conf_new, int32_t* status) {
+    int32_t hist_cap, const int32_t* __restrict__ redo, int32_t* status) {
+  // three-sweep form: runs only for the rows the single-sweep kernel gave up on
+  if (redo != nullptr && redo[blockIdx.x] == 0) return;
   __shared__ uint32_t hist[2048];
   __shared__ uint32_t warp_tot[TC_NT / 32];
   __shared__ uint32_t s_pick[3];
@@ -169,11 +171,156 @@ __global__ void __launch_bounds__(TC_NT) token_conf_kernel(
     top += (double)need * (double)okey_inv((prefix22 << 10) | d3);
     const float lse = mx + logf((float)se);
     const float T = lse - (float)(top / (double)k);
-    conf_new[row] = T;
     // request of this row: last r with tok_indptr[r] <= row
     int lo = 0, hi = n_req;
     while (hi - lo > 1) {
       int mid = (lo + hi) >> 1;
+      if (tok_indptr[mid] <= row) lo = mid; else hi = mid;
+    }
+    const int pos = hist_len[lo] + (row - tok_indptr[lo]);
+    if (pos < hist_cap) conf_hist[(int64_t)lo * hist_cap + pos] = T;
+    else report(status, ACTKV_E_INVALID, lo, pos);
+  }
+}
+
+// -----------------------------------------------------------------------------------------------
+// Single-sweep token confidence.  The k-th largest of any subset of a row is a lower bound of the
+// k-th largest of the row, so: (A) take the first SW_HEAD logits into shared memory and find their
+// k-th largest tau exactly; (B) stream the rest of the row ONCE from HBM with an online
+// (max, sum of exp) per thread, appending the few logits >= tau to a shared candidate list;
+// (C) the top k of head-candidates + list are the top k of the row.  Rows whose list overflows
+// (adversarial order, e.g. ascending logits) are flagged and redone by the three-sweep kernel.
+constexpr int SW_HEAD = 8192;
+constexpr int SW_CAP = 4096;
+
+struct SweepSmem {
+  float head[SW_HEAD];
+  float cand[SW_CAP];
+  uint32_t hist[2048];
+  uint32_t warp_tot[TC_NT / 32];
+  uint32_t pick[3];
+  uint32_t n_cand;
+  float red_f[TC_NT / 32];
+  double red_d[TC_NT / 32];
+};
+
+// k-th largest (k >= 1) of vals[0..n) by three radix digits; all threads call it.  Returns the key of
+// that element and the number of elements equal to it that belong to the top k.
+__device__ __forceinline__ void smem_kth_largest(const float* vals, int n, uint32_t k, SweepSmem* sm,
+                                                 uint32_t& key_out, uint32_t& need_out) {
+  const int tid = threadIdx.x;
+  uint32_t prefix = 0, remaining = k;
+  for (int pass = 0; pass < 3; ++pass) {
+    const int nb = pass == 2 ? 1024 : 2048;
+    const int shift = pass == 0 ? 21 : (pass == 1 ? 10 : 0);
+    for (int i = tid; i < nb; i += TC_NT) sm->hist[i] = 0;
+    __syncthreads();
+    for (int i = tid; i < n; i += TC_NT) {
+      const uint32_t key = okey(vals[i]);
+      const bool in = pass == 0 || (pass == 1 ? (key >> 21) == prefix : (key >> 10) == prefix);
+      if (in) atomicAdd(&sm->hist[(key >> shift) & (uint32_t)(nb - 1)], 1u);
+    }
+    __syncthreads();
+    pick_digit(sm->hist, nb, remaining, sm->warp_tot, sm->pick);
+    prefix = (pass == 0) ? sm->pick[0] : ((prefix << (pass == 1 ? 11 : 10)) | sm->pick[0]);
+    remaining = sm->pick[1];
+    __syncthreads();
+  }
+  key_out = prefix;
+  need_out = remaining;
+}
+
+__global__ void __launch_bounds__(TC_NT, 1) token_conf_sweep_kernel(
+    const float* __restrict__ logits, const int32_t* __restrict__ tok_indptr, int32_t vocab, int32_t n_req,
+    int32_t k_top, float* __restrict__ conf_hist, const int32_t* __restrict__ hist_len, int32_t hist_cap,
+    int32_t* __restrict__ redo, int32_t* status) {
+  extern __shared__ __align__(16) uint8_t sweep_raw[];
+  SweepSmem* sm = reinterpret_cast<SweepSmem*>(sweep_raw);
+  const int row = blockIdx.x, tid = threadIdx.x;
+  const float* z = logits + (int64_t)row * vocab;
+  const int k = min(k_top, vocab);
+  const int n_head = min(vocab, SW_HEAD);
+
+  // ---- (A) head of the row -> shared memory, its k-th largest is the candidate threshold ----
+  for (int i = tid; i < n_head; i += TC_NT) sm->head[i] = z[i];
+  if (tid == 0) sm->n_cand = 0;
+  __syncthreads();
+  uint32_t tau_key, need;
+  smem_kth_largest(sm->head, n_head, (uint32_t)k, sm, tau_key, need);
+  const float tau = okey_inv(tau_key);
+
+  // ---- (B) one sweep: online (max, sum exp2) per thread, candidates >= tau ----
+  float m = -INFINITY, s = 0.f;
+  auto visit = [&](float x, bool collect) {
+    if (x > m) { s *= exp2f((m - x) * kLog2e); m = x; }      // m = -inf: s is 0 and stays 0
+    s += exp2f((x - m) * kLog2e);
+    if (collect && x >= tau) {
+      const uint32_t pos = atomicAdd(&sm->n_cand, 1u);
+      if (pos < SW_CAP) sm->cand[pos] = x;
+    }
+  };
+  for (int i = tid; i < n_head; i += TC_NT) visit(sm->head[i], false);
+  const bool vec = (vocab % 4 == 0) && ((reinterpret_cast<uintptr_t>(z) & 15) == 0) && (SW_HEAD % 4 == 0);
+  if (vec) {
+    const float4* z4 = reinterpret_cast<const float4*>(z);
+    const int n4 = vocab / 4;
+    int i = SW_HEAD / 4 + tid;
+    for (; i + 3 * TC_NT < n4; i += 4 * TC_NT) {               // four 16-byte loads in flight per thread
+      const float4 a = z4[i], b = z4[i + TC_NT], c = z4[i + 2 * TC_NT], d = z4[i + 3 * TC_NT];
+      visit(a.x, true); visit(a.y, true); visit(a.z, true); visit(a.w, true);
+      visit(b.x, true); visit(b.y, true); visit(b.z, true); visit(b.w, true);
+      visit(c.x, true); visit(c.y, true); visit(c.z, true); visit(c.w, true);
+      visit(d.x, true); visit(d.y, true); visit(d.z, true); visit(d.w, true);
+    }
+    for (; i < n4; i += TC_NT) {
+      const float4 a = z4[i];
+      visit(a.x, true); visit(a.y, true); visit(a.z, true); visit(a.w, true);
+    }
+  } else {
+    for (int i = SW_HEAD + tid; i < vocab; i += TC_NT) visit(z[i], true);
+  }
+  // block (max, sum): fixed-order trees
+  const float M = block_reduce_max(m, sm->red_f);
+  const double S = block_reduce_sum((m > -INFINITY) ? (double)s * (double)exp2f((m - M) * kLog2e) : 0.0, sm->red_d);
+  __syncthreads();
+  const uint32_t n_cand = sm->n_cand;
+  if (n_cand > SW_CAP) {                                     // adversarial order: leave the row to the fallback
+    if (tid == 0) redo[row] = 1;
+    return;
+  }
+  // ---- (C) top k of {head elements >= tau} U candidates ----
+  // move the head's own candidates behind the streamed ones (at most k + ties of them; ties could be many,
+  // so the count is checked again)
+  for (int i = tid; i < n_head; i += TC_NT) {
+    const float x = sm->head[i];
+    if (x >= tau) {
+      const uint32_t pos = atomicAdd(&sm->n_cand, 1u);
+      if (pos < SW_CAP) sm->cand[pos] = x;
+    }
+  }
+  __syncthreads();
+  const uint32_t n_all = sm->n_cand;
+  if (n_all > SW_CAP) {
+    if (tid == 0) redo[row] = 1;
+    return;
+  }
+  uint32_t kth_key, need_k;
+  smem_kth_largest(sm->cand, (int)n_all, (uint32_t)k, sm, kth_key, need_k);
+  const float kth = okey_inv(kth_key);
+  double top = 0.0;
+  for (int i = tid; i < (int)n_all; i += TC_NT) {
+    const float x = sm->cand[i];
+    if (okey(x) > kth_key) top += (double)x;
+  }
+  top = block_reduce_sum(top, sm->red_d);
+  if (tid == 0) {
+    redo[row] = 0;
+    top += (double)need_k * (double)kth;
+    const float lse = M + logf((float)S);
+    const float T = lse - (float)(top / (double)k);
+    int lo = 0, hi = n_req;
+    while (hi - lo > 1) {
+      const int mid = (lo + hi) >> 1;
       if (tok_indptr[mid] <= row) lo = mid; else hi = mid;
     }
     const int pos = hist_len[lo] + (row - tok_indptr[lo]);
@@ -285,11 +432,18 @@ int actkv_budget(const float* logits, const int32_t* tok_indptr, int32_t n_rows,
   if (params->clamp_hi_ppm > 0 && !seq_len) return ACTKV_E_INVALID;
   if (ws_bytes < actkv_budget_workspace_bytes(n_rows, n_req, hist_cap)) return ACTKV_E_WORKSPACE;
   cudaStream_t s = (cudaStream_t)stream;
-  float* conf_new = (float*)ws;
+  int32_t* redo = (int32_t*)ws;                 // per row: 1 = the single-sweep kernel gave up, redo in three sweeps
   float* pooled = (float*)((char*)ws + actkv::align_up((size_t)n_rows * 4, 256));
   if (n_rows > 0) {
+    const size_t sm = sizeof(actkv::SweepSmem);
+    if (cudaFuncSetAttribute(actkv::token_conf_sweep_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm) !=
+        cudaSuccess)
+      return ACTKV_E_CUDA;
+    actkv::token_conf_sweep_kernel<<<(unsigned)n_rows, actkv::TC_NT, sm, s>>>(
+        logits, tok_indptr, vocab, n_req, params->k, conf_hist, hist_len, hist_cap, redo, status);
+    ACTKV_CHECK_LAUNCH();
     actkv::token_conf_kernel<<<(unsigned)n_rows, actkv::TC_NT, 0, s>>>(
-        logits, tok_indptr, vocab, n_req, params->k, conf_hist, hist_len, hist_cap, conf_new, status);
+        logits, tok_indptr, vocab, n_req, params->k, conf_hist, hist_len, hist_cap, redo, status);
     ACTKV_CHECK_LAUNCH();
   }
   actkv::BudgetParamsDev p{params->w, params->s, params->b_percent, params->scale_up,

@@ -93,6 +93,23 @@ def test_against_oracle_gaussian_logits(vocab, R, T):
             assert got_B[r] == min(int(budget_in[r] * 1.75), 30000)
 
 
+def test_sorted_rows_overflow_the_candidate_list_and_are_redone():
+    """Ascending rows make every later logit a top-k candidate: the single-sweep kernel gives them up
+    and the three-sweep kernel redoes them; descending and shuffled rows stay on the fast path."""
+    R, T, V = 3, 70, 151936
+    g = torch.Generator(device=DEV)
+    g.manual_seed(77)
+    base = torch.randn((R * T, V), generator=g, device=DEV) * 2.0
+    logits = base.clone()
+    logits[:T] = torch.sort(base[:T], dim=1).values                       # ascending
+    logits[T:2 * T] = torch.sort(base[T:2 * T], dim=1, descending=True).values
+    tok = torch.arange(0, (R + 1) * T, T, dtype=torch.int32, device=DEV)
+    hist0 = torch.zeros((R, 128), dtype=torch.float32)
+    len0 = torch.zeros(R, dtype=torch.int32)
+    _compare(logits, tok, hist0, len0, torch.tensor([512, 512, 512], dtype=torch.int32),
+             B.BudgetParams.paper_defaults())
+
+
 def test_history_accumulates_across_calls_and_clamp():
     R, T, V = 4, 40, 2048
     p = B.BudgetParams.paper_defaults(clamp_lo_ppm=150000, clamp_hi_ppm=400000)
