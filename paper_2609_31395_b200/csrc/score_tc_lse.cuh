@@ -196,41 +196,46 @@ score_tc_lse_kernel(const __grid_constant__ CUtensorMap kmap, const TcArgs ta) {
     bool ok = mbar_wait(smem_u32(&bars->q_ready), 0, abort_flag);
     tc_fence_after();
     if (ok) ok = mbar_wait(smem_u32(&bars->k_full[0]), 0, abort_flag);               // job 0: stage 0, slot 0
+    // All indices are carried incrementally (no divisions in the loop): any cycle the issuer spends
+    // between two MMAs beyond the queue's depth is a bubble in the tensor pipe.
+    int s = 0, b = 0, slot = 0;
+    uint32_t kpar = 0, epar = 7u;                  // bit i: parity to wait for on tmem_empty[i] (fresh barriers pass with 1)
+    const bool leader = elect_one();
     for (int job = 0; ok && job < n_jobs; ++job) {
-      const int it = (n_mb == 2) ? (job >> 1) : job;
-      const int b = (n_mb == 2) ? (job & 1) : 0;
-      const int s = it % S;
-      const int slot = job % LSE_SLOTS;
-      // poll the next job's barriers
-      const int jn = job + 1;
-      const int itn = (n_mb == 2) ? (jn >> 1) : jn;
-      const int sn = itn % S, slotn = jn % LSE_SLOTS;
-      const uint32_t kfull_n = smem_u32(&bars->k_full[sn]), kpar_n = (uint32_t)(itn / S) & 1u;
-      const uint32_t empty_n = smem_u32(&bars->tmem_empty[slotn]), epar_n = ((uint32_t)(jn / LSE_SLOTS) & 1u) ^ 1u;
+      int bn = b + 1, sn = s;
+      uint32_t kparn = kpar;
+      if (bn == n_mb) { bn = 0; sn = s + 1; if (sn == S) { sn = 0; kparn ^= 1u; } }
+      const int slotn = slot == LSE_SLOTS - 1 ? 0 : slot + 1;
+      const bool has_next = job + 1 < n_jobs;
+      const uint32_t kfull_n = smem_u32(&bars->k_full[sn]);
+      const uint32_t empty_n = smem_u32(&bars->tmem_empty[slotn]);
+      const uint32_t epar_n = (epar >> slotn) & 1u;
       bool kready = true, eready = true;
-      if (jn < n_jobs) {
-        kready = (itn == it) || mbar_test_wait(kfull_n, kpar_n);
+      if (has_next) {
+        kready = (sn == s) || mbar_test_wait(kfull_n, kparn);
         eready = mbar_test_wait(empty_n, epar_n);
       }
       tc_fence_after();
-      const uint64_t desc_s = desc0 + (uint64_t)((s * KTILE_BYTES) >> 4);
-      if (elect_one()) {
+      if (leader) {
+        const uint64_t desc_s = desc0 + (uint64_t)((s * KTILE_BYTES) >> 4);
         const uint32_t d = tmem_base + LSE_A_COLS + slot * 128, at = tmem_base + b * 64;
 #pragma unroll
         for (int kk = 0; kk < 8; ++kk)
           umma_bf16_ts(d, at + kk * 8, desc_s + (uint64_t)(((kk >> 2) * HALF_BYTES + (kk & 3) * 32) >> 4), idesc,
                        kk > 0 ? 1u : 0u);
         umma_commit(smem_u32(&bars->tmem_full[slot]));
-        if (b == n_mb - 1) umma_commit(smem_u32(&bars->k_empty[s]));
+        if (bn == 0) umma_commit(smem_u32(&bars->k_empty[s]));
       }
-      __syncwarp();
-      if (jn < n_jobs) {
-        if (!kready) ok = mbar_wait(kfull_n, kpar_n, abort_flag);
+      epar ^= 1u << slot;
+      if (has_next) {
+        if (!kready) ok = mbar_wait(kfull_n, kparn, abort_flag);
         if (ok && !eready) ok = mbar_wait(empty_n, epar_n, abort_flag);
       }
+      b = bn; s = sn; kpar = kparn; slot = slotn;
     }
     // drain: every MMA issued above has completed before TMEM is freed
-    if (elect_one()) umma_commit(smem_u32(&bars->drained));
+    __syncwarp();
+    if (leader) umma_commit(smem_u32(&bars->drained));
     __syncwarp();
     mbar_wait(smem_u32(&bars->drained), 0, abort_flag, ok ? WAIT_LIMIT_NS : DRAIN_LIMIT_NS);
     __syncwarp();

@@ -177,44 +177,50 @@ score_tc_pool_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_cons
     // barrier wait costs 100-200 cycles) is idle time of the pipe.  So the barriers of job j+1 are polled
     // (mbarrier.test_wait, non-blocking) BEFORE the MMAs of job j are issued and the answers are only read
     // afterwards; the blocking wait is the fallback when they were not ready yet.
+    // All indices are carried incrementally (no divisions in the loop): any cycle the issuer spends
+    // between two MMAs beyond the queue's depth is a bubble in the tensor pipe.
     const uint64_t kdesc0 = smem_desc_sw128(k_smem);
     const uint64_t qdesc0 = smem_desc_sw128(q_smem);
+    const uint32_t idesc_c[2] = {idesc_bf16(128, min(256, rows_pad)), idesc_bf16(128, max(16, rows_pad - 256))};
     bool ok = mbar_wait(smem_u32(&bars->q_full), 0, abort_flag);
     if (ok) ok = mbar_wait(smem_u32(&bars->k_full[0]), 0, abort_flag);               // job 0: stage 0, accumulator 0
+    int s = 0, rc = 0;
+    uint32_t kpar = 0, epar0 = 1, epar1 = 1;       // parities to wait for (a fresh "empty" barrier passes with 1)
+    const bool leader = elect_one();
     for (int job = 0; ok && job < n_jobs; ++job) {
-      const int it = (n_rc == 2) ? (job >> 1) : job;
-      const int rc = (n_rc == 2) ? (job & 1) : 0;
-      const int s = it % S, b = job & 1;
-      const int jn = job + 1;
-      const int itn = (n_rc == 2) ? (jn >> 1) : jn;
-      const int sn = itn % S;
-      const uint32_t kfull_n = smem_u32(&bars->k_full[sn]), kpar_n = (uint32_t)(itn / S) & 1u;
-      const uint32_t empty_n = smem_u32(&bars->tmem_empty[jn & 1]), epar_n = ((uint32_t)(jn >> 1) & 1u) ^ 1u;
+      const int b = job & 1;
+      int rcn = rc + 1, sn = s;
+      uint32_t kparn = kpar;
+      if (rcn == n_rc) { rcn = 0; sn = s + 1; if (sn == S) { sn = 0; kparn ^= 1u; } }
+      const bool has_next = job + 1 < n_jobs;
+      const uint32_t kfull_n = smem_u32(&bars->k_full[sn]);
+      const uint32_t empty_n = smem_u32(&bars->tmem_empty[b ^ 1]);
+      const uint32_t epar_n = b ? epar0 : epar1;
       bool kready = true, eready = true;
-      if (jn < n_jobs) {
-        kready = (itn == it) || mbar_test_wait(kfull_n, kpar_n);
+      if (has_next) {
+        kready = (sn == s) || mbar_test_wait(kfull_n, kparn);
         eready = mbar_test_wait(empty_n, epar_n);
       }
       tc_fence_after();
-      const int ncols = min(256, rows_pad - rc * 256);
-      const uint32_t idesc = idesc_bf16(128, ncols);
-      const uint64_t adesc_s = kdesc0 + (uint64_t)((s * KTILE_BYTES) >> 4);
-      const uint64_t bdesc_c = qdesc0 + (uint64_t)((rc * 2 * QBLK_BYTES) >> 4);
-      if (elect_one()) {
+      if (leader) {
+        const uint64_t adesc_s = kdesc0 + (uint64_t)((s * KTILE_BYTES) >> 4);
+        const uint64_t bdesc_c = qdesc0 + (uint64_t)((rc * 2 * QBLK_BYTES) >> 4);
 #pragma unroll
         for (int kk = 0; kk < 8; ++kk)
           umma_bf16(tmem_base + b * 256, adesc_s + (uint64_t)(((kk >> 2) * HALF_BYTES + (kk & 3) * 32) >> 4),
-                    bdesc_c + (uint64_t)(((kk >> 2) * QBLK_BYTES + (kk & 3) * 32) >> 4), idesc, kk > 0 ? 1u : 0u);
+                    bdesc_c + (uint64_t)(((kk >> 2) * QBLK_BYTES + (kk & 3) * 32) >> 4), idesc_c[rc], kk > 0 ? 1u : 0u);
         umma_commit(smem_u32(&bars->tmem_full[b]));
-        if (rc == n_rc - 1) umma_commit(smem_u32(&bars->k_empty[s]));
+        if (rcn == 0) umma_commit(smem_u32(&bars->k_empty[s]));
       }
-      __syncwarp();
-      if (jn < n_jobs) {
-        if (!kready) ok = mbar_wait(kfull_n, kpar_n, abort_flag);
+      if (b) epar1 ^= 1u; else epar0 ^= 1u;
+      if (has_next) {
+        if (!kready) ok = mbar_wait(kfull_n, kparn, abort_flag);
         if (ok && !eready) ok = mbar_wait(empty_n, epar_n, abort_flag);
       }
+      rc = rcn; s = sn; kpar = kparn;
     }
-    if (elect_one()) umma_commit(smem_u32(&bars->drained));
+    __syncwarp();
+    if (leader) umma_commit(smem_u32(&bars->drained));
     __syncwarp();
     mbar_wait(smem_u32(&bars->drained), 0, abort_flag, ok ? WAIT_LIMIT_NS : DRAIN_LIMIT_NS);
     __syncwarp();

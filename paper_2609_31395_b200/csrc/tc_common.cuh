@@ -56,11 +56,11 @@ __device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity) {
 // at least half as long in wall time.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag,
                                           uint64_t limit_ns = WAIT_LIMIT_NS) {
-  // Spin on the non-blocking poll first: a thread parked in try_wait is only woken with a delay of
-  // the order of a microsecond, which is as long as a whole key tile takes.
+  // try_wait parks the thread in hardware (no polling traffic on shared memory, which the MMA operand
+  // fetch needs); measured the same or better than spinning on test_wait here.
 #pragma unroll 1
-  for (int i = 0; i < 4096; ++i)
-    if (mbar_test_wait(bar, parity)) return true;
+  for (int i = 0; i < 64; ++i)
+    if (mbar_try_wait(bar, parity)) return true;
   const long long t0 = clock64();
   const long long limit_cycles = (long long)limit_ns * 2;
   for (;;) {
