@@ -177,6 +177,61 @@ def select(score_all: np.ndarray, tok_indptr, budget) -> list:
 # Section 7.2 / Algorithm 4 — compaction (fresh-page form)
 
 
+# --------------------------------------------------------------------------------------------
+# Section 5.1, Algorithm 1 steps 2-5 — attention-aware LRFU keep-score
+
+
+MASS_BITS = 32            # scores are weighed in units of 2^-32 so that masses add exactly
+P_DENOM = 10000           # top-p is taken to 1/10000
+
+
+def hit_mask_unit(score_f32: np.ndarray, top_p: float) -> np.ndarray:
+    """GetHitMask(AttnScore, p): an entry is hit if its score falls within the top-p set
+    (Section 5.1; p = 90% in Section 8.1).
+
+    The top-p set is the shortest prefix of the entries ordered by (score descending, index
+    ascending) whose mass reaches p of the unit's total mass; the entry that crosses the mark
+    is in.  Mass is counted in exact integers: m_i = floor(score_i * 2^32), mark =
+    ceil(p_q * sum(m) / 10000) with p_q = round(p * 10000) — so the set does not depend on a
+    summation order.  Entries of zero mass are never needed and are not hits.
+    """
+    s = np.asarray(score_f32, dtype=np.float32)
+    L = s.shape[0]
+    # scores are pooled probabilities in [0, 1]; anything outside [0, 256] is clipped so that masses of
+    # up to 2^16 entries still add up in 64 bits
+    mass = [int(math.floor(min(max(float(x), 0.0), 256.0) * (1 << MASS_BITS))) for x in s]
+    total = sum(mass)
+    p_q = int(round(top_p * P_DENOM))
+    mark = -(-(p_q * total) // P_DENOM)
+    order = np.lexsort((np.arange(L), -s.astype(np.float64)))
+    hit = np.zeros(L, dtype=bool)
+    acc = 0
+    for i in order:
+        if acc >= mark:
+            break
+        hit[i] = True
+        acc += mass[i]
+    return hit
+
+
+def keep_score_update(ks_f32: np.ndarray, score_f32: np.ndarray, hit: np.ndarray, lam: float) -> np.ndarray:
+    """KS_t = lambda * KS_{t-1} + AttnScore_t * [hit at t]   (Section 5.1 equation; Algorithm 1 step 4),
+    in float32 with one rounding per operation (product, then sum).  New entries of the round
+    enter with KS = 0 (Algorithm 1 step 2)."""
+    ks = np.asarray(ks_f32, dtype=np.float32)
+    s = np.asarray(score_f32, dtype=np.float32)
+    decayed = (np.float32(lam) * ks).astype(np.float32)
+    return np.where(hit, (decayed + s).astype(np.float32), decayed).astype(np.float32)
+
+
+def rank_keys(ks_f32: np.ndarray, n_protect: int) -> np.ndarray:
+    """What TopK ranks (Algorithm 1 step 5): the keep-score, with the first n_protect entries (system
+    prompt and task description, Section 8.1) lifted to +inf so that they are always retained."""
+    out = np.array(ks_f32, dtype=np.float32, copy=True)
+    out[: int(n_protect)] = np.inf
+    return out
+
+
 @dataclass
 class Tables:
     page_table: np.ndarray   # int32 [R, max_pages], unused -1
