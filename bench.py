@@ -248,6 +248,7 @@ def run_ours(args):
         comp.status.zero_()
 
     lse_supplied = None
+    lrfu_state = None                          # set for the secondary LRFU-policy line only
     stage_names = ["budget", "lse", "score", "select", "compact"]
 
     def one_step(events=None):
@@ -269,7 +270,7 @@ def run_ours(args):
                                      lse_in=lse_supplied, marks=mark)
         else:
             n = comp.step(inst.q, inst.win_indptr, inst.tok_indptr, bud, wl.sm_scale, wl.causal,
-                          lse_in=lse_supplied, marks=(lambda nm: mark(nm)))
+                          lse_in=lse_supplied, marks=(lambda nm: mark(nm)), lrfu=lrfu_state)
         mark("end")
         return n + 2
 
@@ -402,6 +403,36 @@ def run_ours(args):
                                  alg_bytes / (float(tl.item()) * 1e-3) / 1e9 / pk["hbm_gbs"]}
         comp.check_status()
 
+    # ---- the same step ranking by the attention-aware LRFU keep-score (Section 5.1): score -> keepscore
+    # -> select -> gather keep-scores -> compact, p = 0.9, lambda = 0.5, 512 protected tokens per request
+    lrfu_line = None
+    if not args.overlap and not args.no_lrfu:
+        lrfu_state = H.LrfuState(NL * Hkv, sz, dev, 0.9, 0.5,
+                                 torch.full((R,), 512, dtype=torch.int32, device=dev))
+        lrfu_state.keep_score.uniform_(0.0, 1e-3, generator=torch.Generator(device=dev).manual_seed(wl.seed))
+        ms, ks_ms = [], []
+        for it in range(2 + min(args.steps, 5)):
+            restore()
+            ev = []
+            one_step(ev)
+            torch.cuda.synchronize()
+            if it >= 2:
+                ms.append(ev[0][1].elapsed_time(ev[-1][1]))
+                ks_ms.append(sum(ev[i - 1][1].elapsed_time(ev[i][1]) for i in range(1, len(ev))
+                                 if ev[i][0] == "keepscore"))
+        lrfu_state = None
+        tl = torch.tensor([sum(ms) / len(ms)], dtype=torch.float64, device=dev)
+        if dist is not None:
+            dist.all_reduce(tl, op=dist.ReduceOp.MAX)
+        ks = sum(ks_ms) / len(ks_ms)
+        # algorithmic bytes of the keep-score stage: score read + KS read + KS write + key write
+        ks_bytes = 16.0 * tokens * Hkv * NL
+        lrfu_line = {"ms_per_step": float(tl.item()), "value": world * tokens / (float(tl.item()) * 1e-3), "unit": UNIT,
+                     "keepscore_ms": ks, "keepscore_gbs": ks_bytes / (ks * 1e-3) / 1e9,
+                     "keepscore_frac_of_hbm_peak": ks_bytes / (ks * 1e-3) / 1e9 / pk["hbm_gbs"],
+                     "top_p": 0.9, "lambda": 0.5, "n_protect": 512}
+        comp.check_status()
+
     # ---- the oracle on the host cores (rank 0, single GPU only) ----------------------------------
     cpu_baseline = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
@@ -423,7 +454,7 @@ def run_ours(args):
                                   "of the next group" if args.overlap else "none (one stream)",
                        "l2": "inputs (KV pool %.1f GB) far larger than the 126 MB L2" % (inst.pool.numel() * 2 / 1e9)},
             "stage_ms": stage_ms, "hbm_roofline_frac_whole_step": hbm_frac_whole,
-            "with_lse_supplied": lse_supplied_line,
+            "with_lse_supplied": lse_supplied_line, "with_lrfu_policy": lrfu_line,
             "algorithmic_bytes_per_step": alg_bytes, "k_bytes_per_pass": bytes_k,
             "roofline": roofline, "roofline_stages": stages, "cpu_baseline": cpu_baseline, "e2e": e2e,
             "clocks": clocks, "gpu_launches": launches, "wall_s_timed_region": t_wall,
@@ -449,6 +480,7 @@ def main():
     ap.add_argument("--lse", default="internal", choices=["internal", "supplied"])
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-lrfu", action="store_true", help="skip the secondary LRFU-policy line")
     args = ap.parse_args()
     if args.warmup < 3 and args.impl == "ours":
         print("note: fewer than 3 warm-up steps", file=sys.stderr)

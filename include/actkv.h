@@ -182,6 +182,39 @@ int actkv_keep_indptr(const int32_t* seq_len, const int32_t* budget, int32_t n_r
                       int32_t* keep_indptr, actkv_stream_t stream);
 
 /* ---------------------------------------------------------------------------------------
+ * actkv_keepscore — attention-aware LRFU keep-score (Section 5.1 equation; Algorithm 1 steps 2-4),
+ * an optional stage between actkv_score and actkv_select.
+ *
+ * Per unit (o, r) over score[o, tok_indptr[r] .. tok_indptr[r+1]):
+ *   hit_i  = 1 iff entry i falls within the top-p set of the unit: the shortest prefix of the
+ *            entries ordered by (score descending, index ascending) whose mass reaches p of the
+ *            unit's total mass, the crossing entry included.  Mass is counted exactly:
+ *            m_i = floor(clip(score_i, 0, 256) * 2^32), mark = ceil(round(p*10000) * sum m / 10000).
+ *   KS_i   = lambda * KS_i + score_i * hit_i        (float32, one rounding per operation)
+ *   score_i is then OVERWRITTEN with the key actkv_select should rank: KS_i, or +inf for the
+ *            first n_protect[r] entries (system prompt / task description, Section 8.1), which are
+ *            therefore always retained while the budget allows.
+ * keep_score float32 [n_outer, sum_tok], same layout as score, in/out.  Entries appended since the
+ *            last compression must hold 0 (Algorithm 1 step 2).
+ * n_protect  int32 [n_req] or NULL.  hit_mask optional bitmap [n_outer, ceil(sum_tok/32)], zeroed
+ *            by the caller.  Scores are expected in [0, 1] (pooled probabilities).
+ */
+int actkv_keepscore(float* score, const int32_t* tok_indptr, int32_t sum_tok, int32_t n_outer,
+                    int32_t n_req, float top_p, float lambda, const int32_t* n_protect,
+                    float* keep_score, uint32_t* hit_mask, int32_t* status, actkv_stream_t stream);
+
+/* ---------------------------------------------------------------------------------------
+ * actkv_gather_f32 — the survivors' keep-scores move with them (Algorithm 1 step 5 returns KS'):
+ *   dst[o, keep_indptr[r] + i] = src[o, tok_indptr[r] + sel_idx[o, keep_indptr[r] + i]].
+ * src float32 [n_outer, src_stride]; dst float32 [n_outer, dst_stride]; max_total_keep: host upper
+ * bound on keep_indptr[n_req].
+ */
+int actkv_gather_f32(const float* src, int64_t src_stride, const int32_t* tok_indptr,
+                     const int32_t* sel_idx, int64_t sel_stride, const int32_t* keep_indptr,
+                     int32_t n_outer, int32_t n_req, int32_t max_total_keep,
+                     float* dst, int64_t dst_stride, actkv_stream_t stream);
+
+/* ---------------------------------------------------------------------------------------
  * actkv_select — TopK(score, k = B) per unit (Algorithm 1 step 5, applied to the pooled
  * score, independently per layer and KV head).
  *

@@ -25,7 +25,8 @@ EXPORTS = ["actkv_budget_workspace_bytes", "actkv_budget", "actkv_score_workspac
            "actkv_score_lse",
            "actkv_keep_indptr", "actkv_select_workspace_bytes", "actkv_select",
            "actkv_compact_workspace_bytes", "actkv_compact", "actkv_compact_noalloc",
-           "actkv_compact_noalloc_max_bytes", "actkv_step_host", "actkv_version"]
+           "actkv_compact_noalloc_max_bytes", "actkv_step_host", "actkv_keepscore", "actkv_gather_f32",
+           "actkv_version"]
 
 
 class ActKVError(RuntimeError):
@@ -124,6 +125,10 @@ def load():
     lib.actkv_compact.restype = i32
     lib.actkv_compact.argtypes = [C.POINTER(PoolDesc), C.POINTER(TablesDesc), i32, i32, vp, i64, vp, vp, i32,
                                   vp, sz, vp, vp]
+    lib.actkv_keepscore.restype = i32
+    lib.actkv_keepscore.argtypes = [vp, vp, i32, i32, i32, f32, f32, vp, vp, vp, vp, vp]
+    lib.actkv_gather_f32.restype = i32
+    lib.actkv_gather_f32.argtypes = [vp, i64, vp, vp, i64, vp, i32, i32, i32, vp, i64, vp]
     lib.actkv_step_host.restype = i32
     lib.actkv_step_host.argtypes = [C.POINTER(PoolDesc), C.POINTER(TablesDesc), C.POINTER(BudgetParams),
                                     C.POINTER(HostStep), vp]
@@ -264,6 +269,25 @@ def actkv_compact(pool: PoolDesc, tables: TablesDesc, layer_begin, layer_end, se
                               max_keep, _ptr(ws, None, "ws"), ws.numel() * ws.element_size(),
                               _ptr(status, torch.int32, "status"), _stream(stream))
     _check("actkv_compact", rc)
+
+
+def actkv_keepscore(score, tok_indptr, sum_tok, n_outer, n_req, top_p, lam, n_protect, keep_score, hit_mask, status,
+                    stream=None):
+    rc = load().actkv_keepscore(_ptr(score, torch.float32, "score"), _ptr(tok_indptr, torch.int32, "tok_indptr"),
+                                sum_tok, n_outer, n_req, float(top_p), float(lam),
+                                _ptr(n_protect, torch.int32, "n_protect"), _ptr(keep_score, torch.float32, "keep_score"),
+                                _ptr(hit_mask, torch.int32, "hit_mask"), _ptr(status, torch.int32, "status"),
+                                _stream(stream))
+    _check("actkv_keepscore", rc)
+
+
+def actkv_gather_f32(src, src_stride, tok_indptr, sel_idx, sel_stride, keep_indptr, n_outer, n_req, max_total_keep,
+                     dst, dst_stride, stream=None):
+    rc = load().actkv_gather_f32(_ptr(src, torch.float32, "src"), src_stride, _ptr(tok_indptr, torch.int32, "tok_indptr"),
+                                 _ptr(sel_idx, torch.int32, "sel_idx"), sel_stride,
+                                 _ptr(keep_indptr, torch.int32, "keep_indptr"), n_outer, n_req, max_total_keep,
+                                 _ptr(dst, torch.float32, "dst"), dst_stride, _stream(stream))
+    _check("actkv_gather_f32", rc)
 
 
 def actkv_step_host(pool: PoolDesc, tables: TablesDesc, params: Optional[BudgetParams], io: HostStep, stream=None):

@@ -77,6 +77,21 @@ class Compressor:
         B.actkv_select(self.score, tok_indptr, s.sum_tok, budget, n_layers_sub * Hkv, s.n_req, self.keep_indptr,
                        self.sel_idx, s.sel_stride, self.mask, self.ties, self.ws_select, self.status, stream)
 
+    def run_keepscore(self, lrfu: "LrfuState", tok_indptr, l0, l1, stream=None):
+        """Turns the pooled scores of layers [l0, l1) into ranking keys (keep-scores, protected prefix
+        lifted) and updates the persistent keep-scores of those layers."""
+        Hkv, s = self.pd.n_kv_heads, self.sz
+        hit = None if lrfu.hit_mask is None else lrfu.hit_mask[l0 * Hkv:l1 * Hkv]
+        B.actkv_keepscore(self.score[: l1 - l0], tok_indptr, s.sum_tok, (l1 - l0) * Hkv, s.n_req, lrfu.top_p, lrfu.lam,
+                          lrfu.n_protect, lrfu.keep_score[l0 * Hkv:l1 * Hkv], hit, self.status, stream)
+
+    def run_gather_ks(self, lrfu: "LrfuState", tok_indptr, l0, l1, stream=None):
+        """Keep-scores of the survivors of layers [l0, l1), packed like the index lists."""
+        Hkv, s = self.pd.n_kv_heads, self.sz
+        B.actkv_gather_f32(lrfu.keep_score[l0 * Hkv:l1 * Hkv], s.sum_tok, tok_indptr, self.sel_idx, s.sel_stride,
+                           self.keep_indptr, (l1 - l0) * Hkv, s.n_req, s.sel_stride,
+                           lrfu.kept[l0 * Hkv:l1 * Hkv], s.sel_stride, stream)
+
     def run_compact(self, budget, l0=0, l1=None, stream=None):
         l1 = self.pd.n_layers if l1 is None else l1
         B.actkv_compact(self.pd, self.td, l0, l1, self.sel_idx, self.sz.sel_stride, self.keep_indptr, budget,
@@ -89,9 +104,12 @@ class Compressor:
                           tok_indptr, lse_out, s.sum_win, s.max_win, s.sum_tok, s.max_tok, self.ws_score,
                           self.status, stream)
 
-    def step(self, q, win_indptr, tok_indptr, budget, sm_scale, causal, lse_in=None, stream=None, marks=None):
+    def step(self, q, win_indptr, tok_indptr, budget, sm_scale, causal, lse_in=None, stream=None, marks=None,
+             lrfu: Optional["LrfuState"] = None):
         """score -> select -> compact over all layers, `layers_per_call` layers at a time.
         Tables are rewritten by the last compact call; earlier calls see the old tables.
+        `lrfu`: rank by the attention-aware LRFU keep-score instead of the raw pooled score
+        (score -> keepscore -> select -> gather keep-scores -> compact).
         `marks`: optional callable(name) invoked between stages (the benchmark records CUDA events
         there); with it the LSE pass and the pooled-score pass run as two calls so that each can be
         timed on its own.  Returns the number of kernels launched."""
@@ -111,7 +129,13 @@ class Compressor:
             else:
                 self.run_score(q, win_indptr, tok_indptr, sm_scale, causal, l0, l1, lse_in, stream)
             mark("score")
+            if lrfu is not None:
+                self.run_keepscore(lrfu, tok_indptr, l0, l1, stream)
+                mark("keepscore")
             self.run_select(tok_indptr, budget, l1 - l0, stream)
+            if lrfu is not None:
+                self.run_gather_ks(lrfu, tok_indptr, l0, l1, stream)
+                launches += 2
             mark("select")
             self.run_compact(budget, l0, l1, stream)
             mark("compact")
@@ -176,6 +200,34 @@ class Compressor:
         st = self.status.cpu().tolist()
         if st[0] != 0:
             raise B.ActKVError(f"device status {st}", st[0])
+
+
+class LrfuState:
+    """Device buffers of the attention-aware LRFU policy (Section 5.1) for one pool: the persistent
+    keep-scores KS [layers * KV heads, sum_tok] in the score layout, the survivors' keep-scores
+    `kept` [layers * KV heads, sel_stride] in the index-list layout, and the policy constants."""
+
+    def __init__(self, n_outer: int, sizes: StepSizes, device, top_p: float = 0.9, lam: float = 0.9,
+                 n_protect: Optional[torch.Tensor] = None, want_hits: bool = False):
+        self.top_p, self.lam, self.n_protect = float(top_p), float(lam), n_protect
+        self.keep_score = torch.zeros((n_outer, sizes.sum_tok), dtype=torch.float32, device=device)
+        self.kept = torch.zeros((n_outer, sizes.sel_stride), dtype=torch.float32, device=device)
+        self.hit_mask = (torch.zeros((n_outer, (sizes.sum_tok + 31) // 32), dtype=torch.int32, device=device)
+                         if want_hits else None)
+
+
+def extend_keep_scores(ks_compact: torch.Tensor, keep_counts, new_seq_lens) -> torch.Tensor:
+    """Keep-score array for the next round: per request the survivors' keep-scores (as gathered by
+    actkv_gather_f32, packed by keep_indptr) followed by zeros for the tokens appended since
+    (Algorithm 1 step 2: new entries enter with keep-score 0).  Buffer bookkeeping only."""
+    n_outer = ks_compact.shape[0]
+    out = torch.zeros((n_outer, int(sum(new_seq_lens))), dtype=torch.float32, device=ks_compact.device)
+    src = dst = 0
+    for n, L in zip(keep_counts, new_seq_lens):
+        out[:, dst:dst + n] = ks_compact[:, src:src + n]
+        src += n
+        dst += L
+    return out
 
 
 class HostStepRunner:
