@@ -303,6 +303,83 @@ def compact(pool_bits: np.ndarray, tables: Tables, sel, budget, layers=None):
     return new_pool, Tables(pt, sl, fl, fc)
 
 
+def tail_region(L: int, B: int, P: int):
+    """Section 7.2 target-region equations / Algorithm 4 step 1: Y = ceil(L/BS), X = ceil(B/BS),
+    Start = (Y - X) * BS, End = Start + B.  Returns (Y, X, Start, End)."""
+    Y = -(-int(L) // P)
+    X = -(-int(B) // P)
+    start = (Y - X) * P
+    return Y, X, start, start + int(B)
+
+
+def copy_pairs_unit(kept, L: int, B: int, P: int):
+    """Algorithm 4 steps 1-5 for one keep mask, in logical slots: returns (src, dst), ascending, zipped
+    pairwise.  The mask spans every allocated slot (Y * BS of them: the region may reach past L
+    into the unused slots of the last block, which are holes)."""
+    Y, X, start, end = tail_region(L, B, P)
+    keep_mask = np.zeros(Y * P, dtype=bool)
+    keep_mask[np.asarray(kept, dtype=np.int64)] = True
+    dst_mask = np.zeros(Y * P, dtype=bool)
+    dst_mask[start:end] = ~keep_mask[start:end]                    # step 2
+    keep_mask[start:end] = False                                   # step 3
+    src_mask = keep_mask
+    dst = np.nonzero(dst_mask)[0]
+    src = np.nonzero(src_mask)[0]
+    assert src.shape[0] == dst.shape[0], "as many survivors outside the region as holes inside"
+    return src, dst                                                # step 5: Zip(src, dst)
+
+
+def compact_inplace(pool_bits: np.ndarray, tables: Tables, sel, budget, layers=None):
+    """Algorithm 4 / Section 7.2, applied per (layer, KV head) keep mask: survivors outside the last X
+    logical blocks move into the holes inside them, then the first Y - X blocks of the request go back
+    to the serving system.
+
+      requests r with B_r < L_r: region [Start, End) from `tail_region`; for every layer and head the
+      copy pairs of that unit's keep mask (`copy_pairs_unit`), translated through the slot map
+      (step 4), all copied at once (step 6; sources and destinations are disjoint);
+      then page_table[r] = its last X pages ++ -1.., seq_len[r] = B_r, and, r ascending, the dropped
+      pages are pushed on the free list in ascending logical order.
+    sel[a][h][r]: ascending kept token indices of pool layer layers[a] (the keep mask as a list).
+    Returns (new pool_bits, new Tables, order) where order[a][h][r][i] is the original token index
+    of what now sits at logical slot i (None for requests that do not compact).
+    """
+    P, Hkv = pool_bits.shape[3], pool_bits.shape[4]
+    n_pages = pool_bits.shape[2]
+    layers = list(range(pool_bits.shape[0])) if layers is None else list(layers)
+    new_pool = pool_bits.copy()
+    pt = tables.page_table.copy()
+    sl = tables.seq_len.copy()
+    fl = tables.free_list.copy()
+    fc = int(tables.free_count)
+    R = len(sl)
+    order = [[[None] * R for _ in range(Hkv)] for _ in layers]
+    for r in range(R):
+        L, B = int(sl[r]), int(budget[r])
+        if B >= L:
+            continue
+        Y, X, start, end = tail_region(L, B, P)
+        old = [int(x) for x in tables.page_table[r, :Y]]
+        slot_of = slot_map(old, Y * P, P)                          # every allocated slot, used or not
+        for a, layer in enumerate(layers):
+            before = pool_bits[layer].reshape(2, n_pages * P, Hkv, -1)
+            after = new_pool[layer].reshape(2, n_pages * P, Hkv, -1)
+            for h in range(Hkv):
+                kept = np.asarray(sel[a][h][r], dtype=np.int64)
+                assert kept.shape[0] == B
+                src, dst = copy_pairs_unit(kept, L, B, P)
+                after[:, slot_of[dst], h, :] = before[:, slot_of[src], h, :]
+                now = np.arange(start, end)
+                now[dst - start] = src
+                order[a][h][r] = now
+        pt[r, :] = -1
+        pt[r, :X] = old[Y - X:]
+        sl[r] = B
+        for p in old[:Y - X]:
+            fl[fc] = p
+            fc += 1
+    return new_pool, Tables(pt, sl, fl, fc), order
+
+
 # --------------------------------------------------------------------------------------------
 # Section 6.1, Algorithm 2 — confidence monitor and budget update
 
