@@ -119,6 +119,21 @@ def aggregate_replicas(ms_local: float, tokens_per_replica: int, world: int, dis
     return ms_max, world * tokens_per_replica / (ms_max * 1e-3)
 
 
+def count_inplace_moves(comp, wl) -> int:
+    """Rows the in-place compaction of the last call had to move: kept indices outside the tail region
+    [Start, End) of their request (counted from the index lists; reporting only)."""
+    P = wl.page_size
+    ki = comp.keep_indptr.cpu().tolist()
+    moved = 0
+    for r, (L, b) in enumerate(zip(wl.seq_lens, wl.budgets)):
+        if b >= L:
+            continue
+        start = (-(-L // P) - -(-b // P)) * P
+        seg = comp.sel_idx[:, ki[r]:ki[r + 1]]
+        moved += int(((seg < start) | (seg >= start + b)).sum())
+    return moved
+
+
 def visible_gpu_index(local_rank: int) -> int:
     vis = os.environ.get("CUDA_VISIBLE_DEVICES")
     if vis:
@@ -249,6 +264,7 @@ def run_ours(args):
 
     lse_supplied = None
     lrfu_state = None                          # set for the secondary LRFU-policy line only
+    inplace_mode = False                       # set for the secondary in-place-compaction line only
     stage_names = ["budget", "lse", "score", "select", "compact"]
 
     def one_step(events=None):
@@ -270,7 +286,7 @@ def run_ours(args):
                                      lse_in=lse_supplied, marks=mark)
         else:
             n = comp.step(inst.q, inst.win_indptr, inst.tok_indptr, bud, wl.sm_scale, wl.causal,
-                          lse_in=lse_supplied, marks=(lambda nm: mark(nm)), lrfu=lrfu_state)
+                          lse_in=lse_supplied, marks=(lambda nm: mark(nm)), lrfu=lrfu_state, inplace=inplace_mode)
         mark("end")
         return n + 2
 
@@ -433,6 +449,38 @@ def run_ours(args):
                      "top_p": 0.9, "lambda": 0.5, "n_protect": 512}
         comp.check_status()
 
+    # ---- the same step compacting in place into the tail blocks (Algorithm 4) instead of fresh pages.
+    # Run last: it overwrites evicted slots of the original layout, which the fresh-page form never does.
+    inplace_line = None
+    if not args.overlap and not args.no_inplace:
+        inplace_mode = True
+        ms, cp_ms = [], []
+        pool_backup = inst.pool.clone()        # the pool is restored (untimed) before every in-place step
+        for it in range(2 + min(args.steps, 5)):
+            inst.pool.copy_(pool_backup)
+            restore()
+            ev = []
+            one_step(ev)
+            torch.cuda.synchronize()
+            if it >= 2:
+                ms.append(ev[0][1].elapsed_time(ev[-1][1]))
+                cp_ms.append(sum(ev[i - 1][1].elapsed_time(ev[i][1]) for i in range(1, len(ev))
+                                 if ev[i][0] == "compact"))
+        inplace_mode = False
+        del pool_backup
+        comp.check_status()
+        # rows that had to move: survivors outside the tail region, counted from the last step's lists
+        moved = count_inplace_moves(comp, wl)
+        tl = torch.tensor([sum(ms) / len(ms)], dtype=torch.float64, device=dev)
+        if dist is not None:
+            dist.all_reduce(tl, op=dist.ReduceOp.MAX)
+        cp = sum(cp_ms) / len(cp_ms)
+        moved_bytes = 4.0 * D * 2 * moved * n_calls      # K and V rows, read + write, bf16; lists of the last call
+        inplace_line = {"ms_per_step": float(tl.item()), "value": world * tokens / (float(tl.item()) * 1e-3), "unit": UNIT,
+                        "compact_ms": cp, "rows_moved_fraction_of_kept": moved / max(1.0, rho * tokens * Hkv * comp.lpc),
+                        "compact_gbs": moved_bytes / (cp * 1e-3) / 1e9,
+                        "compact_frac_of_hbm_peak": moved_bytes / (cp * 1e-3) / 1e9 / pk["hbm_gbs"]}
+
     # ---- the oracle on the host cores (rank 0, single GPU only) ----------------------------------
     cpu_baseline = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
@@ -455,6 +503,7 @@ def run_ours(args):
                        "l2": "inputs (KV pool %.1f GB) far larger than the 126 MB L2" % (inst.pool.numel() * 2 / 1e9)},
             "stage_ms": stage_ms, "hbm_roofline_frac_whole_step": hbm_frac_whole,
             "with_lse_supplied": lse_supplied_line, "with_lrfu_policy": lrfu_line,
+            "with_inplace_compaction": inplace_line,
             "algorithmic_bytes_per_step": alg_bytes, "k_bytes_per_pass": bytes_k,
             "roofline": roofline, "roofline_stages": stages, "cpu_baseline": cpu_baseline, "e2e": e2e,
             "clocks": clocks, "gpu_launches": launches, "wall_s_timed_region": t_wall,
@@ -481,6 +530,7 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-lrfu", action="store_true", help="skip the secondary LRFU-policy line")
+    ap.add_argument("--no-inplace", action="store_true", help="skip the secondary in-place-compaction line")
     args = ap.parse_args()
     if args.warmup < 3 and args.impl == "ours":
         print("note: fewer than 3 warm-up steps", file=sys.stderr)

@@ -259,6 +259,33 @@ int actkv_compact(const actkv_pool_t* pool /* host */, const actkv_tables_t* tab
                   void* ws, size_t ws_bytes, int32_t* status, actkv_stream_t stream);
 
 /* ---------------------------------------------------------------------------------------
+ * actkv_compact_inplace — compaction into the last X logical blocks of each request, without
+ * fresh pages (Section 7.2 region equations; Algorithm 4 steps 1-6), one keep mask per
+ * (layer, KV head), given as the ascending index lists actkv_select writes.
+ *
+ * Requests with budget[r] >= seq_len[r] are left untouched.  For the others, with L = seq_len[r],
+ * B = budget[r], Y = ceil(L / page_size), X = ceil(B / page_size):
+ *     Start = (Y - X) * page_size,  End = Start + B        (logical slots; End may pass L inside
+ *                                                           the last block: unused slots are holes)
+ * For every layer in [layer_begin, layer_end) and head: the holes of [Start, End) (slots not in
+ * the list) in ascending order receive, pairwise, the K and V rows of the listed slots outside
+ * [Start, End) in ascending order.  Sources and destinations are disjoint, nothing else is
+ * written.  When layer_end == pool->n_layers the tables are updated after the copies, r ascending:
+ * free_list[free_count++] = page i of r for i < Y - X ascending, page_table[r] = its last X pages
+ * then -1, seq_len[r] = B.  No page is popped, so the call cannot run short of free pages.
+ * Survivors do not keep ascending order: new_order (optional, int32, same layout as sel_idx)
+ * receives at [.., keep_indptr[r] + i] the original token index of what now sits at logical slot
+ * i (for untouched requests: the list itself), e.g. for actkv_gather_f32.
+ * On a device-detected error the tables stay as they were; only holes were overwritten.
+ * max_keep: host upper bound on min(budget[r], seq_len[r]).  No workspace.
+ */
+int actkv_compact_inplace(const actkv_pool_t* pool /* host */, const actkv_tables_t* tables /* host */,
+                          int32_t layer_begin, int32_t layer_end,
+                          const int32_t* sel_idx, int64_t sel_stride, const int32_t* keep_indptr,
+                          const int32_t* budget, int32_t max_keep, int32_t* new_order,
+                          int32_t* status, actkv_stream_t stream);
+
+/* ---------------------------------------------------------------------------------------
  * actkv_step_host — one whole compression step (Algorithm 1 steps 1, 5, 6 with Algorithm 2 in
  * front) for a caller whose per-step inputs live in HOST memory.
  *

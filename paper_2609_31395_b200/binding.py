@@ -26,6 +26,7 @@ EXPORTS = ["actkv_budget_workspace_bytes", "actkv_budget", "actkv_score_workspac
            "actkv_keep_indptr", "actkv_select_workspace_bytes", "actkv_select",
            "actkv_compact_workspace_bytes", "actkv_compact", "actkv_compact_noalloc",
            "actkv_compact_noalloc_max_bytes", "actkv_step_host", "actkv_keepscore", "actkv_gather_f32",
+           "actkv_compact_inplace",
            "actkv_version"]
 
 
@@ -127,6 +128,9 @@ def load():
                                   vp, sz, vp, vp]
     lib.actkv_keepscore.restype = i32
     lib.actkv_keepscore.argtypes = [vp, vp, i32, i32, i32, f32, f32, vp, vp, vp, vp, vp]
+    lib.actkv_compact_inplace.restype = i32
+    lib.actkv_compact_inplace.argtypes = [C.POINTER(PoolDesc), C.POINTER(TablesDesc), i32, i32, vp, i64, vp, vp, i32,
+                                          vp, vp, vp]
     lib.actkv_gather_f32.restype = i32
     lib.actkv_gather_f32.argtypes = [vp, i64, vp, vp, i64, vp, i32, i32, i32, vp, i64, vp]
     lib.actkv_step_host.restype = i32
@@ -269,6 +273,17 @@ def actkv_compact(pool: PoolDesc, tables: TablesDesc, layer_begin, layer_end, se
                               max_keep, _ptr(ws, None, "ws"), ws.numel() * ws.element_size(),
                               _ptr(status, torch.int32, "status"), _stream(stream))
     _check("actkv_compact", rc)
+
+
+def actkv_compact_inplace(pool: PoolDesc, tables: TablesDesc, layer_begin, layer_end, sel_idx, sel_stride, keep_indptr,
+                          budget, max_keep, new_order, status, stream=None):
+    rc = load().actkv_compact_inplace(C.byref(pool), C.byref(tables), layer_begin, layer_end,
+                                      _ptr(sel_idx, torch.int32, "sel_idx"), sel_stride,
+                                      _ptr(keep_indptr, torch.int32, "keep_indptr"),
+                                      _ptr(budget, torch.int32, "budget"), max_keep,
+                                      _ptr(new_order, torch.int32, "new_order"),
+                                      _ptr(status, torch.int32, "status"), _stream(stream))
+    _check("actkv_compact_inplace", rc)
 
 
 def actkv_keepscore(score, tok_indptr, sum_tok, n_outer, n_req, top_p, lam, n_protect, keep_score, hit_mask, status,

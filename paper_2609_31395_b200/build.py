@@ -8,7 +8,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libactkv.so")
-SOURCES = ["score.cu", "select.cu", "compact.cu", "budget.cu", "keepscore.cu", "host_step.cu"]
+SOURCES = ["score.cu", "select.cu", "compact.cu", "compact_inplace.cu", "budget.cu", "keepscore.cu", "host_step.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-lineinfo", "-std=c++17",
               "--use_fast_math", "-Xcompiler", "-fPIC", "-cudart", "static"]
 

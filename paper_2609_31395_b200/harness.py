@@ -85,12 +85,23 @@ class Compressor:
         B.actkv_keepscore(self.score[: l1 - l0], tok_indptr, s.sum_tok, (l1 - l0) * Hkv, s.n_req, lrfu.top_p, lrfu.lam,
                           lrfu.n_protect, lrfu.keep_score[l0 * Hkv:l1 * Hkv], hit, self.status, stream)
 
-    def run_gather_ks(self, lrfu: "LrfuState", tok_indptr, l0, l1, stream=None):
-        """Keep-scores of the survivors of layers [l0, l1), packed like the index lists."""
+    def run_gather_ks(self, lrfu: "LrfuState", tok_indptr, l0, l1, stream=None, idx=None):
+        """Keep-scores of the survivors of layers [l0, l1), packed like the index lists (`idx`: the
+        lists to follow, default the ascending ones; after an in-place compaction its new order)."""
         Hkv, s = self.pd.n_kv_heads, self.sz
-        B.actkv_gather_f32(lrfu.keep_score[l0 * Hkv:l1 * Hkv], s.sum_tok, tok_indptr, self.sel_idx, s.sel_stride,
+        B.actkv_gather_f32(lrfu.keep_score[l0 * Hkv:l1 * Hkv], s.sum_tok, tok_indptr,
+                           self.sel_idx if idx is None else idx, s.sel_stride,
                            self.keep_indptr, (l1 - l0) * Hkv, s.n_req, s.sel_stride,
                            lrfu.kept[l0 * Hkv:l1 * Hkv], s.sel_stride, stream)
+
+    def run_compact_inplace(self, budget, l0=0, l1=None, stream=None, want_order=True):
+        """In-place tail compaction (Algorithm 4) of layers [l0, l1); `self.new_order` then holds, per
+        unit, the original token index at every new logical slot."""
+        l1 = self.pd.n_layers if l1 is None else l1
+        if want_order and getattr(self, "new_order", None) is None:
+            self.new_order = torch.empty_like(self.sel_idx)
+        B.actkv_compact_inplace(self.pd, self.td, l0, l1, self.sel_idx, self.sz.sel_stride, self.keep_indptr, budget,
+                                self.sz.max_keep, self.new_order if want_order else None, self.status, stream)
 
     def run_compact(self, budget, l0=0, l1=None, stream=None):
         l1 = self.pd.n_layers if l1 is None else l1
@@ -105,11 +116,12 @@ class Compressor:
                           self.status, stream)
 
     def step(self, q, win_indptr, tok_indptr, budget, sm_scale, causal, lse_in=None, stream=None, marks=None,
-             lrfu: Optional["LrfuState"] = None):
+             lrfu: Optional["LrfuState"] = None, inplace: bool = False):
         """score -> select -> compact over all layers, `layers_per_call` layers at a time.
         Tables are rewritten by the last compact call; earlier calls see the old tables.
         `lrfu`: rank by the attention-aware LRFU keep-score instead of the raw pooled score
         (score -> keepscore -> select -> gather keep-scores -> compact).
+        `inplace`: compact into the tail blocks of each request (Algorithm 4) instead of fresh pages.
         `marks`: optional callable(name) invoked between stages (the benchmark records CUDA events
         there); with it the LSE pass and the pooled-score pass run as two calls so that each can be
         timed on its own.  Returns the number of kernels launched."""
@@ -133,13 +145,18 @@ class Compressor:
                 self.run_keepscore(lrfu, tok_indptr, l0, l1, stream)
                 mark("keepscore")
             self.run_select(tok_indptr, budget, l1 - l0, stream)
-            if lrfu is not None:
+            if lrfu is not None and not inplace:
                 self.run_gather_ks(lrfu, tok_indptr, l0, l1, stream)
-                launches += 2
             mark("select")
-            self.run_compact(budget, l0, l1, stream)
+            if inplace:
+                self.run_compact_inplace(budget, l0, l1, stream, want_order=lrfu is not None)
+                if lrfu is not None:
+                    self.run_gather_ks(lrfu, tok_indptr, l0, l1, stream, idx=self.new_order)
+            else:
+                self.run_compact(budget, l0, l1, stream)
             mark("compact")
-            launches += (3 if lse_in is None else 1) + 1 + 2 + (1 if l1 == NL else 0)
+            launches += (3 if lse_in is None else 1) + 1 + (1 if inplace else 2) + (1 if l1 == NL else 0)
+            launches += 2 if lrfu is not None else 0
         return launches
 
     def step_overlapped(self, q, win_indptr, tok_indptr, budget, sm_scale, causal, lse_in=None, marks=None):

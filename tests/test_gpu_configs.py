@@ -119,6 +119,34 @@ def test_config3_qwen3_30b_35k_x8_bench_shape():
     _run_fixed_workload(wl, units, compaction_slabs=[0, 47])
 
 
+def test_config3_inplace_tail_compaction_full_size():
+    """The benchmark workload compacted in place (Algorithm 4) in the launch configuration the
+    benchmark's in-place line times: two whole layers (every byte), tables and free list against
+    the oracle run on the GPU's own index lists."""
+    wl = synth.config3()
+    inst = synth.generate(wl, DEV)
+    tables_before = U.oracle_tables(inst)
+    slabs = [0, 47]
+    snap = {a: inst.pool[a].clone() for a in slabs}
+    sz = H.sizes_of(inst)
+    comp = H.Compressor(inst.pool, inst.page_table, inst.seq_len, inst.free_list, inst.free_count, wl.n_q_heads, sz)
+    comp.step(inst.q, inst.win_indptr, inst.tok_indptr, inst.budget, wl.sm_scale, wl.causal, inplace=True)
+    torch.cuda.synchronize()
+    comp.check_status()
+    _check_all_select(comp.score, inst.tok_indptr, wl.budgets, comp.sel_idx, comp.keep_indptr)
+    ki = comp.keep_indptr.cpu().numpy()
+    sel_np = comp.sel_idx.cpu().numpy()
+    Hkv, R = wl.n_kv_heads, wl.n_req
+    want_t = None
+    for a in slabs:
+        lists = [[[sel_np[a * Hkv + h, ki[r]:ki[r + 1]] for r in range(R)] for h in range(Hkv)]]
+        want_pool, want_t, _ = O.compact_inplace(U.bits(snap[a])[None], tables_before, lists, wl.budgets, layers=[0])
+        assert np.array_equal(U.bits(inst.pool[a])[None], want_pool)
+    _check_tables((inst.page_table, inst.seq_len, inst.free_list, inst.free_count), want_t)
+    assert int(inst.free_count.cpu()) == tables_before.free_count + sum(
+        -(-L // wl.page_size) - -(-b // wl.page_size) for L, b in zip(wl.seq_lens, wl.budgets))
+
+
 def test_config4_serving_mix_budgets_from_monitor():
     """64 requests, lengths log-uniform in 8K-64K; budgets produced on the device by actkv_budget
     from 256 action-token logit rows per request (V = 151936), clamped to 15-40% of length.  Two of

@@ -138,11 +138,14 @@ def test_gather_f32_follows_the_index_lists():
         assert (got[o, ki[-1]:] == -7.0).all()
 
 
-def test_lrfu_trace_keepscores_travel_with_the_survivors():
+@pytest.mark.parametrize("inplace", [False, True])
+def test_lrfu_trace_keepscores_travel_with_the_survivors(inplace):
     """Six rounds of a small agent trace under the LRFU policy (p = 0.9, lambda = 0.5, protected
     prompt head): every round the raw scores match the oracle on sampled units, and hit masks,
     keep-scores, index lists, gathered keep-scores, pool and tables match the oracle's policy run on
-    the GPU's own float32 scores, with the oracle carrying its own keep-score state."""
+    the GPU's own float32 scores, with the oracle carrying its own keep-score state.  With
+    `inplace` the cache is compacted into the tail blocks (Algorithm 4) and the keep-scores follow
+    the new slot order."""
     tr = synth.AgentTrace(n_layers=2, n_kv_heads=2, group=4, n_req=3, n_rounds=6, device=DEV, prompt=(700, 1500),
                           obs=(150, 300), reason=(40, 120), action=(16, 48), max_tokens_per_req=4096, seed=9)
     Hkv, R, NL = tr.Hkv, tr.R, tr.NL
@@ -162,25 +165,32 @@ def test_lrfu_trace_keepscores_travel_with_the_survivors():
         keep = [min(b, L) for b, L in zip(budgets, seq)]
         sz = H.StepSizes(R, sum(windows), max(windows), sum(seq), max(seq), max(1, sum(keep)), max(keep))
         comp = H.Compressor(tr.pool, tr.page_table, tr.seq_len, tr.free_list, tr.free_count, Hkv * tr.G, sz)
-        lrfu = H.LrfuState(n_outer, sz, DEV, top_p, lam, d_protect, want_hits=True)
+        # fresh pages keep ascending order, so the protected prompt head stays the first n_protect slots;
+        # in place the order changes, so protection travels with the tokens instead: their keep-score
+        # starts at +inf (and stays there under the recurrence) and no prefix is named
+        lrfu = H.LrfuState(n_outer, sz, DEV, top_p, lam, None if inplace else d_protect, want_hits=True)
         if ks_gpu_prev is not None:
             lrfu.keep_score.copy_(H.extend_keep_scores(ks_gpu_prev, keep_prev, seq))
+        elif inplace:
+            t0 = tok_indptr.cpu().tolist()
+            for r in range(R):
+                lrfu.keep_score[:, t0[r]:t0[r] + protect[r]] = float("inf")
         tables_before = O.Tables(tr.page_table.cpu().numpy().copy(), tr.seq_len.cpu().numpy().copy(),
                                  tr.free_list.cpu().numpy().copy(), int(tr.free_count.cpu()))
         pt_before, sl_before = tr.page_table.clone(), tr.seq_len.clone()
-        snap = tr.pool[0].clone()
+        pool_snap = tr.pool.clone()
+        snap = pool_snap[0]
         raw = {}
 
         def marks(name):
             if name == "score":
                 raw["score"] = comp.score.clone()
 
-        comp.step(q, win_indptr, tok_indptr, budget, wl_like[5], True, marks=marks, lrfu=lrfu)
+        comp.step(q, win_indptr, tok_indptr, budget, wl_like[5], True, marks=marks, lrfu=lrfu, inplace=inplace)
         torch.cuda.synchronize()
         comp.check_status()
         units = [(int(rng.integers(0, NL)), int(rng.integers(0, Hkv)), int(rng.integers(0, R))) for _ in range(2)]
-        # compaction writes fresh pages only, so the old slots still hold what the scores were computed from
-        TC._check_sampled_scores(tr.pool, pt_before, sl_before, q, win_indptr, tok_indptr, wl_like, raw["score"], units)
+        TC._check_sampled_scores(pool_snap, pt_before, sl_before, q, win_indptr, tok_indptr, wl_like, raw["score"], units)
 
         tok = tok_indptr.cpu().numpy()
         ki = comp.keep_indptr.cpu().numpy()
@@ -189,6 +199,7 @@ def test_lrfu_trace_keepscores_travel_with_the_survivors():
         kept_np = lrfu.kept.cpu().numpy()
         sel_np = comp.sel_idx.cpu().numpy()
         hit_np = lrfu.hit_mask.cpu().numpy()
+        order_np = comp.new_order.cpu().numpy() if inplace else None
         ks_orc_new = [[None] * R for _ in range(n_outer)]
         for o in range(n_outer):
             for r in range(R):
@@ -196,18 +207,36 @@ def test_lrfu_trace_keepscores_travel_with_the_survivors():
                 prev = np.zeros(b - a, dtype=np.float32)
                 if ks_orc_prev is not None:
                     prev[: keep_prev[r]] = ks_orc_prev[o][r]
+                elif inplace:
+                    prev[: protect[r]] = np.inf
                 hit = O.hit_mask_unit(raw_np[o, a:b], top_p)
                 ks = O.keep_score_update(prev, raw_np[o, a:b], hit, lam)
-                sel = O.select_unit(O.rank_keys(ks, min(protect[r], b - a)), budgets[r])
+                sel = O.select_unit(O.rank_keys(ks, 0 if inplace else min(protect[r], b - a)), budgets[r])
                 assert np.array_equal(_unpack_hits(hit_np[o], a, b), hit), f"round {rnd} unit ({o},{r}): hit mask"
                 assert np.array_equal(_f32_bits(ks_np[o, a:b]), _f32_bits(ks)), f"round {rnd} unit ({o},{r}): KS"
                 assert np.array_equal(sel_np[o, ki[r]:ki[r + 1]], sel), f"round {rnd} unit ({o},{r}): TopK"
-                assert np.array_equal(_f32_bits(kept_np[o, ki[r]:ki[r + 1]]), _f32_bits(ks[sel]))
+                now = sel                                       # original token index at every new logical slot
+                if inplace and budgets[r] < b - a:
+                    src, dst = O.copy_pairs_unit(sel, b - a, budgets[r], tr.P)
+                    start = O.tail_region(b - a, budgets[r], tr.P)[2]
+                    now = np.arange(start, start + budgets[r])
+                    now[dst - start] = src
+                if inplace:
+                    assert np.array_equal(order_np[o, ki[r]:ki[r + 1]], now), f"round {rnd} unit ({o},{r}): order"
+                assert np.array_equal(_f32_bits(kept_np[o, ki[r]:ki[r + 1]]), _f32_bits(ks[now]))
                 n_prot = min(protect[r], b - a, budgets[r])
-                evicted_protected += int(n_prot - np.isin(np.arange(n_prot), sel).sum())
-                ks_orc_new[o][r] = ks[sel]
-        want_t = TC._check_layer_compaction(snap, tr.pool[0], tables_before, comp.sel_idx, comp.keep_indptr, budgets,
-                                            Hkv, 0)
+                if inplace:                                     # protected tokens are the +inf ones, wherever they sit
+                    evicted_protected += int(n_prot - np.isinf(kept_np[o, ki[r]:ki[r + 1]]).sum())
+                else:
+                    evicted_protected += int(n_prot - np.isin(np.arange(n_prot), sel).sum())
+                ks_orc_new[o][r] = ks[now]
+        if inplace:
+            lists = [[[sel_np[h, ki[r]:ki[r + 1]] for r in range(R)] for h in range(Hkv)]]
+            want_pool, want_t, _ = O.compact_inplace(U.bits(snap)[None], tables_before, lists, budgets, layers=[0])
+            assert np.array_equal(U.bits(tr.pool[0])[None], want_pool)
+        else:
+            want_t = TC._check_layer_compaction(snap, tr.pool[0], tables_before, comp.sel_idx, comp.keep_indptr,
+                                                budgets, Hkv, 0)
         TC._check_tables((tr.page_table, tr.seq_len, tr.free_list, tr.free_count), want_t)
         ks_gpu_prev = lrfu.kept[:, : int(ki[-1])].clone()
         ks_orc_prev, keep_prev = ks_orc_new, keep
