@@ -147,6 +147,47 @@ def score(pool_bits, page_table, seq_len, q_bits, win_indptr, n_q_heads, sm_scal
     return out, lse, tok_indptr
 
 
+def score_stream_step(out_prev: np.ndarray, n_prev: int, q_tok: np.ndarray, k_unit: np.ndarray,
+                      lse_tok: np.ndarray, sm_scale: float) -> np.ndarray:
+    """Algorithm 3 steps 3-5 for ONE current action query of one (request, KV head): the form in which
+    the kernel is triggered at every decode step of an action region, with the LSE handed over by the
+    attention backend (Section 7.1).
+
+    q_tok float64 [G, D]: the current query of the G q-heads of the group.  k_unit float64 [L, D]:
+    the keys cached at this step (the current token's own key included).  lse_tok float64 [G].
+    out_prev float64 [<= L]: running mean after the n_prev earlier action queries of this region
+    (entries appended since are taken as 0; n_prev = 0 at region entry: the state starts from zero).
+
+      for every q-head of the group: Logits = Q_head . K^T (scaled), Attn = exp(Logits - LSE)   (step 3)
+      AttnScore = max over the group of Attn                                                    (step 4)
+      Out <- running mean over the action queries seen so far                                   (step 5)
+    Returns the new running mean, float64 [L].
+    """
+    G = q_tok.shape[0]
+    L = k_unit.shape[0]
+    attn_score = np.zeros(L, dtype=np.float64)
+    for g in range(G):
+        logits = sm_scale * (k_unit @ q_tok[g])
+        attn = np.exp(logits - float(lse_tok[g]))
+        attn_score = np.maximum(attn_score, attn)
+    out = np.zeros(L, dtype=np.float64)
+    out[: out_prev.shape[0]] = out_prev
+    return (n_prev * out + attn_score) / (n_prev + 1)
+
+
+def score_stream(q_unit: np.ndarray, k_unit: np.ndarray, sm_scale: float, lse: np.ndarray,
+                 out_prev: np.ndarray | None = None, n_prev: int = 0) -> np.ndarray:
+    """`score_stream_step` over the W queries of q_unit [W, G, D] in decoding order: query w is issued
+    when the cache holds the first L - W + w + 1 keys of k_unit [L, D].  lse float64 [W, G].
+    Returns float64 [L] (the running mean after n_prev + W action queries)."""
+    W = q_unit.shape[0]
+    L = k_unit.shape[0]
+    out = np.zeros(0, dtype=np.float64) if out_prev is None else np.asarray(out_prev, dtype=np.float64)
+    for w in range(W):
+        out = score_stream_step(out, n_prev + w, q_unit[w], k_unit[: L - W + w + 1], lse[w], sm_scale)
+    return out
+
+
 # --------------------------------------------------------------------------------------------
 # Algorithm 1, step 5 — TopK(score, k = B)
 
