@@ -449,6 +449,35 @@ def run_ours(args):
                      "top_p": 0.9, "lambda": 0.5, "n_protect": 512}
         comp.check_status()
 
+    # ---- streaming form (Algorithm 3 as triggered per decode step): one action query per request per call,
+    # LSE supplied, running mean updated in place; all layers in one call.  Bound by the K reads.
+    stream_line = None
+    if not args.no_stream and comp.lse is not None:
+        restore()
+        first = inst.win_indptr[:-1].to(torch.int64)
+        q1 = inst.q[:, first].contiguous()
+        lse1 = comp.lse[:, first].contiguous()
+        win1 = torch.arange(R + 1, dtype=torch.int32, device=dev)
+        steps1 = torch.ones(R, dtype=torch.int32, device=dev)
+        run_io = torch.zeros((NL, Hkv, sz.sum_tok), dtype=torch.float32, device=dev)
+        ev = [torch.cuda.Event(enable_timing=True) for _ in range(2)]
+        n_it = 3 + min(args.steps, 10)
+        for it in range(n_it):
+            if it == 3:
+                ev[0].record()
+            B.actkv_score_accumulate(comp.pd, comp.td, 0, NL, q1, win1, wl.n_q_heads, lse1, wl.sm_scale, wl.causal,
+                                     inst.tok_indptr, steps1, run_io, R, 1, sz.sum_tok, sz.max_tok, comp.ws_score,
+                                     comp.status)
+        ev[1].record()
+        torch.cuda.synchronize()
+        comp.check_status()
+        ms1 = ev[0].elapsed_time(ev[1]) / (n_it - 3)
+        st_bytes = (2.0 * D + 8.0) * tokens * Hkv * NL          # K row read + running mean read and write
+        stream_line = {"ms_per_call": ms1, "value": world * tokens / (ms1 * 1e-3), "unit": "KV tokens examined/s",
+                       "gbs": st_bytes / (ms1 * 1e-3) / 1e9, "frac_of_hbm_peak": st_bytes / (ms1 * 1e-3) / 1e9 / pk["hbm_gbs"],
+                       "queries_per_request": 1, "layers_per_call": NL}
+        del run_io
+
     # ---- the same step compacting in place into the tail blocks (Algorithm 4) instead of fresh pages.
     # Run last: it overwrites evicted slots of the original layout, which the fresh-page form never does.
     inplace_line = None
@@ -503,7 +532,7 @@ def run_ours(args):
                        "l2": "inputs (KV pool %.1f GB) far larger than the 126 MB L2" % (inst.pool.numel() * 2 / 1e9)},
             "stage_ms": stage_ms, "hbm_roofline_frac_whole_step": hbm_frac_whole,
             "with_lse_supplied": lse_supplied_line, "with_lrfu_policy": lrfu_line,
-            "with_inplace_compaction": inplace_line,
+            "with_inplace_compaction": inplace_line, "streaming_update": stream_line,
             "algorithmic_bytes_per_step": alg_bytes, "k_bytes_per_pass": bytes_k,
             "roofline": roofline, "roofline_stages": stages, "cpu_baseline": cpu_baseline, "e2e": e2e,
             "clocks": clocks, "gpu_launches": launches, "wall_s_timed_region": t_wall,
@@ -531,6 +560,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-lrfu", action="store_true", help="skip the secondary LRFU-policy line")
     ap.add_argument("--no-inplace", action="store_true", help="skip the secondary in-place-compaction line")
+    ap.add_argument("--no-stream", action="store_true", help="skip the secondary streaming-update line")
     args = ap.parse_args()
     if args.warmup < 3 and args.impl == "ours":
         print("note: fewer than 3 warm-up steps", file=sys.stderr)

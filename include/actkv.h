@@ -175,6 +175,34 @@ int actkv_score_lse(const actkv_pool_t* pool /* host */, const actkv_tables_t* t
                     void* ws, size_t ws_bytes, int32_t* status, actkv_stream_t stream);
 
 /* ---------------------------------------------------------------------------------------
+ * actkv_score_accumulate — the streaming form of actkv_score: Algorithm 3 as it is triggered
+ * at every decode step of an action region, with the LSE handed over by the attention backend
+ * (Section 7.1) and the running mean over the action queries kept in score_io (Algorithm 3
+ * step 5; the state restarts from zero at region entry).
+ *
+ * Per call every request contributes its W_r newest action queries (W_r = 1 per decode step;
+ * W_r = 0: the request is outside an action region and is skipped).  With n_r = acc_steps[r]
+ * action queries already folded in, and S_j = sum_w max_g exp(s - lse_in) as in actkv_score:
+ *   score_io[l, h, tok_indptr[r]+j] <- (n_r * score_io[..] + S_j) / (n_r + W_r),   j < L_r.
+ * n_r == 0 (region entry): the old content is not read, the value is S_j / W_r.  For n_r > 0
+ * the entries of keys cached since the previous call must hold 0 (zero the request's segment at
+ * region entry).  The caller adds W_r to acc_steps[r] after the call (same stream).
+ * tok_indptr gives the OFFSET of each request's segment in score_io; segments may be longer than
+ * L_r (capacity), L_r is read from tables->seq_len.  causal as in actkv_score (within the call's
+ * W_r queries; irrelevant for W_r = 1).  lse_in and acc_steps (int32 [n_req], device) are
+ * required.  Other arguments, workspace and errors as actkv_score.
+ * After the last query of a region score_io equals actkv_score's result for the whole window
+ * (causal != 0) up to float32 rounding of the running mean.
+ */
+int actkv_score_accumulate(const actkv_pool_t* pool /* host */, const actkv_tables_t* tables /* host */,
+                           int32_t layer_begin, int32_t layer_end,
+                           const void* q, const int32_t* win_indptr, int32_t n_q_heads,
+                           const float* lse_in, float sm_scale, int32_t causal,
+                           const int32_t* tok_indptr, const int32_t* acc_steps, float* score_io,
+                           int32_t sum_win, int32_t max_win, int32_t sum_tok, int32_t max_tok,
+                           void* ws, size_t ws_bytes, int32_t* status, actkv_stream_t stream);
+
+/* ---------------------------------------------------------------------------------------
  * actkv_keep_indptr — helper: keep_indptr[r] = sum_{r'<r} min(budget[r'], seq_len[r']),
  * keep_indptr[n_req] = total (Algorithm 1 step 5 keeps min(B, L) entries).  One tiny kernel.
  */

@@ -22,7 +22,7 @@ ERROR_NAMES = {E_INVALID: "ACTKV_E_INVALID", E_WORKSPACE: "ACTKV_E_WORKSPACE", E
                E_TIMEOUT: "ACTKV_E_TIMEOUT", E_TOOBIG: "ACTKV_E_TOOBIG"}
 
 EXPORTS = ["actkv_budget_workspace_bytes", "actkv_budget", "actkv_score_workspace_bytes", "actkv_score",
-           "actkv_score_lse",
+           "actkv_score_lse", "actkv_score_accumulate",
            "actkv_keep_indptr", "actkv_select_workspace_bytes", "actkv_select",
            "actkv_compact_workspace_bytes", "actkv_compact", "actkv_compact_noalloc",
            "actkv_compact_noalloc_max_bytes", "actkv_step_host", "actkv_keepscore", "actkv_gather_f32",
@@ -115,6 +115,9 @@ def load():
     lib.actkv_score_lse.restype = i32
     lib.actkv_score_lse.argtypes = [C.POINTER(PoolDesc), C.POINTER(TablesDesc), i32, i32, vp, vp, i32, f32, i32,
                                     vp, vp, i32, i32, i32, i32, vp, sz, vp, vp]
+    lib.actkv_score_accumulate.restype = i32
+    lib.actkv_score_accumulate.argtypes = [C.POINTER(PoolDesc), C.POINTER(TablesDesc), i32, i32, vp, vp, i32, vp, f32,
+                                           i32, vp, vp, vp, i32, i32, i32, i32, vp, sz, vp, vp]
     lib.actkv_keep_indptr.restype = i32
     lib.actkv_keep_indptr.argtypes = [vp, vp, i32, vp, vp]
     lib.actkv_select_workspace_bytes.restype = sz
@@ -237,6 +240,20 @@ def actkv_score_lse(pool: PoolDesc, tables: TablesDesc, layer_begin, layer_end, 
                                 _ptr(ws, None, "ws"), ws.numel() * ws.element_size(),
                                 _ptr(status, torch.int32, "status"), _stream(stream))
     _check("actkv_score_lse", rc)
+
+
+def actkv_score_accumulate(pool: PoolDesc, tables: TablesDesc, layer_begin, layer_end, q, win_indptr, n_q_heads, lse_in,
+                           sm_scale, causal, tok_indptr, acc_steps, score_io, sum_win, max_win, sum_tok, max_tok, ws,
+                           status, stream=None):
+    rc = load().actkv_score_accumulate(C.byref(pool), C.byref(tables), layer_begin, layer_end,
+                                       _ptr(q, torch.bfloat16, "q"), _ptr(win_indptr, torch.int32, "win_indptr"),
+                                       n_q_heads, _ptr(lse_in, torch.float32, "lse_in"), float(sm_scale),
+                                       int(bool(causal)), _ptr(tok_indptr, torch.int32, "tok_indptr"),
+                                       _ptr(acc_steps, torch.int32, "acc_steps"),
+                                       _ptr(score_io, torch.float32, "score_io"), sum_win, max_win, sum_tok, max_tok,
+                                       _ptr(ws, None, "ws"), ws.numel() * ws.element_size(),
+                                       _ptr(status, torch.int32, "status"), _stream(stream))
+    _check("actkv_score_accumulate", rc)
 
 
 def actkv_keep_indptr(seq_len, budget, n_req, keep_indptr, stream=None):

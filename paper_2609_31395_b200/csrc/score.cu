@@ -1,6 +1,9 @@
 // actkv_score: host entry point and path selection.
-//   tensor-core path (score_tc.cuh): window x group rows >= 64, page 16, head_dim 128, packed pool;
+//   tensor-core path (score_tc.cuh): window x group rows >= 64 (any row count for the streaming update),
+//   page 16, head_dim 128, packed pool;
 //   FMA path (score_fma.cuh): everything else.
+// actkv_score_accumulate (streaming, Algorithm 3 per decode step) runs the pooled-score pass alone against
+// the supplied LSE and folds its result into the running mean held in the score array.
 // Both write per-chunk (max, sum) partials of the LSE pass into the caller's workspace, merge them
 // with lse_combine_kernel, then run the pooled-score pass against the merged (or supplied) LSE.
 #include "score_fma.cuh"
@@ -44,7 +47,8 @@ static int score_impl(int mode, const actkv_pool_t* pool, const actkv_tables_t* 
                       int32_t layer_end, const void* q, const int32_t* win_indptr, int32_t n_q_heads,
                       const float* lse_in, float sm_scale, int32_t causal, const int32_t* tok_indptr,
                       float* score_out, float* lse_out, int32_t sum_win, int32_t max_win, int32_t sum_tok,
-                      int32_t max_tok, void* ws, size_t ws_bytes, int32_t* status, actkv_stream_t stream) {
+                      int32_t max_tok, void* ws, size_t ws_bytes, int32_t* status, actkv_stream_t stream,
+                      const int32_t* acc_steps = nullptr) {
   using namespace actkv;
   if (!pool || !tables || !pool->base) return ACTKV_E_INVALID;
   if (layer_begin < 0 || layer_end > pool->n_layers || layer_begin > layer_end) return ACTKV_E_INVALID;
@@ -62,6 +66,7 @@ static int score_impl(int mode, const actkv_pool_t* pool, const actkv_tables_t* 
   if (!q || !win_indptr || !tok_indptr || !tables->page_table || !tables->seq_len) return ACTKV_E_INVALID;
   if ((mode & 2) && !score_out) return ACTKV_E_INVALID;
   if (mode == 1 && !lse_out) return ACTKV_E_INVALID;
+  if (acc_steps != nullptr && sum_win == 0) return ACTKV_OK;      // no request is inside an action region
   if (max_win <= 0 || sum_win <= 0) return ACTKV_E_INVALID;
   const ScoreWsLayout lay = score_ws_layout(Hkv, R, nls, n_q_heads, sum_win, max_win, max_tok);
   if (!ws || ws_bytes < lay.total) return ACTKV_E_WORKSPACE;
@@ -101,8 +106,9 @@ static int score_impl(int mode, const actkv_pool_t* pool, const actkv_tables_t* 
   a.n_tiles = (max_tok + FMA_TK - 1) / FMA_TK;
   a.scale_log2 = sm_scale * kLog2e;
   a.causal = causal;
+  a.acc_steps = acc_steps;
   const int64_t units = (int64_t)nls * Hkv * R;
-  const bool use_tc = score_tc_supported(pool, G, max_win, sm_scale, q);
+  const bool use_tc = score_tc_supported(pool, G, max_win, sm_scale, q, acc_steps ? 1 : 64);
 
   const float* lse = lse_in;
   if (mode & 1) {
@@ -159,6 +165,18 @@ int actkv_score_lse(const actkv_pool_t* pool, const actkv_tables_t* tables, int3
                     void* ws, size_t ws_bytes, int32_t* status, actkv_stream_t stream) {
   return score_impl(1, pool, tables, layer_begin, layer_end, q, win_indptr, n_q_heads, nullptr, sm_scale, causal,
                     tok_indptr, nullptr, lse_out, sum_win, max_win, sum_tok, max_tok, ws, ws_bytes, status, stream);
+}
+
+int actkv_score_accumulate(const actkv_pool_t* pool, const actkv_tables_t* tables, int32_t layer_begin,
+                           int32_t layer_end, const void* q, const int32_t* win_indptr, int32_t n_q_heads,
+                           const float* lse_in, float sm_scale, int32_t causal, const int32_t* tok_indptr,
+                           const int32_t* acc_steps, float* score_io, int32_t sum_win, int32_t max_win,
+                           int32_t sum_tok, int32_t max_tok, void* ws, size_t ws_bytes, int32_t* status,
+                           actkv_stream_t stream) {
+  if (!lse_in || !acc_steps) return ACTKV_E_INVALID;
+  return score_impl(2, pool, tables, layer_begin, layer_end, q, win_indptr, n_q_heads, lse_in, sm_scale, causal,
+                    tok_indptr, score_io, nullptr, sum_win, max_win, sum_tok, max_tok, ws, ws_bytes, status, stream,
+                    acc_steps);
 }
 
 const char* actkv_version(void) { return "actkv-b200 0.1 (sm_100a)"; }

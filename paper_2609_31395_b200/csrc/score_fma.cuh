@@ -31,7 +31,20 @@ struct ScoreArgs {
   int32_t lse_chunk;             // keys per LSE partial of this launch (multiple of 128, >= LSE_CHUNK)
   float scale_log2;              // sm_scale * log2(e)
   int32_t causal;
+  const int32_t* acc_steps;      // accumulate mode (streaming, Algorithm 3 step 5): [R] action queries already
+                                 // folded into score_out; nullptr: score_out is overwritten with this call's mean
 };
+
+// What is stored for one key: the mean over this call's W action tokens (`mean_w`), or in accumulate
+// mode the running mean over the n earlier action tokens of the region and this call's W
+// (n = 0: the old value is not read, the state restarts).
+__device__ __forceinline__ void store_pooled(const ScoreArgs& a, int r, float* slot, float sum_w, float mean_w, int W) {
+  if (a.acc_steps != nullptr) {
+    const int n = a.acc_steps[r];
+    if (n > 0) mean_w = fmaf(*slot, (float)n, sum_w) / (float)(n + W);
+  }
+  *slot = mean_w;
+}
 
 __device__ __forceinline__ float2 bf16x2_to_float2(uint32_t v) {
   return make_float2(__uint_as_float(v << 16), __uint_as_float(v & 0xffff0000u));
@@ -69,6 +82,7 @@ __global__ void __launch_bounds__(FMA_NT) score_fma_kernel(const ScoreArgs a) {
   const int w0 = a.win_indptr[r], W = a.win_indptr[r + 1] - w0;
   const int key_begin = part * ((PASS == 1) ? a.lse_chunk : FMA_TK);
   if (key_begin >= L) return;
+  if (W <= 0 && a.acc_steps != nullptr) return;      // accumulate mode: a request outside its action region
   if (W <= 0 || (a.causal && W > L)) {               // no window, or a window longer than the cache
     if (threadIdx.x == 0 && part == 0) report(a.status, ACTKV_E_INVALID, r, W);
     return;
@@ -189,7 +203,8 @@ __global__ void __launch_bounds__(FMA_NT) score_fma_kernel(const ScoreArgs a) {
   } else {
     const int j = key_begin + threadIdx.x;
     if (threadIdx.x < FMA_TK && j < L) {
-      a.score_out[((int64_t)slab * Hkv + h) * a.sum_tok + a.tok_indptr[r] + j] = pooled / (float)W;
+      store_pooled(a, r, a.score_out + ((int64_t)slab * Hkv + h) * a.sum_tok + a.tok_indptr[r] + j, pooled,
+                   pooled / (float)W, W);
     }
   }
 }

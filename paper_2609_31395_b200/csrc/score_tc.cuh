@@ -81,15 +81,18 @@ constexpr size_t SMEM_LIMIT = 232448;        // 227 KB of dynamic shared memory 
 }  // namespace tc
 
 // The tensor-core path takes: page 16, head_dim 128, packed [slot][head][dim] pages, 128-byte aligned
-// base, power-of-two group size <= 32, 64 <= window x group rows <= 512, positive softmax scale.
-inline bool score_tc_supported(const actkv_pool_t* p, int G, int max_win, float sm_scale, const void* q) {
+// base, power-of-two group size <= 32, min_rows <= window x group rows <= 512, positive softmax scale.
+// The full score (LSE + pooled pass) takes it from 64 rows up; the streaming update, which runs the
+// pooled pass alone and is bound by the K reads, from a single row.
+inline bool score_tc_supported(const actkv_pool_t* p, int G, int max_win, float sm_scale, const void* q,
+                               int min_rows = 64) {
   if (p->page_size != 16 || p->head_dim != 128) return false;
   if (p->stride_head != 128 || p->stride_slot != (int64_t)p->n_kv_heads * 128 || p->stride_page != 16 * p->stride_slot)
     return false;
   if (((uintptr_t)p->base & 127) || ((uintptr_t)q & 127) || (p->stride_layer % 8) != 0) return false;
   if (G < 1 || G > 32 || (G & (G - 1)) != 0) return false;
   const int rows = max_win * G;
-  if (rows < 64 || rows > tc::MAX_ROWS) return false;
+  if (rows < min_rows || rows > tc::MAX_ROWS) return false;
   if (!(sm_scale > 0.f)) return false;
   if (getenv("ACTKV_FORCE_FMA") != nullptr) return false;
   return tc::encode_fn() != nullptr;

@@ -81,6 +81,7 @@ score_tc_pool_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_cons
   const int rows = W * G;
   const int t_begin = kchunk * ta.tiles_per_cta;
   if (t_begin * TK >= L) return;
+  if (W <= 0 && a.acc_steps != nullptr) return;            // accumulate mode: a request outside its action region
   if (W <= 0 || (a.causal && W > L)) {
     if (threadIdx.x == 0 && kchunk == 0) report(a.status, ACTKV_E_INVALID, r, W);
     return;
@@ -253,7 +254,7 @@ score_tc_pool_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_cons
       __syncwarp();
       if (lane == 0) mbar_arrive(smem_u32(&bars->tmem_empty[wg]));
       if (n_rc == 1) {
-        if (key < L) out[key] = acc * inv_w;
+        if (key < L) store_pooled(a, r, out + key, acc, acc * inv_w, W);
       } else if (wg == 1) {
         // partial over the second row chunk: hand it to warpgroup 0 once it has read the previous tile's
         if (!mbar_wait(smem_u32(&bars->part_empty), ((uint32_t)it & 1u) ^ 1u, abort_flag)) break;
@@ -265,7 +266,7 @@ score_tc_pool_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_cons
         acc += bars->exch[quarter * 32 + lane];
         __syncwarp();
         if (lane == 0) mbar_arrive(smem_u32(&bars->part_empty));
-        if (key < L) out[key] = acc * inv_w;
+        if (key < L) store_pooled(a, r, out + key, acc, acc * inv_w, W);
       }
     }
   }
