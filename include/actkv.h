@@ -318,12 +318,19 @@ int actkv_compact_inplace(const actkv_pool_t* pool /* host */, const actkv_table
  * front) for a caller whose per-step inputs live in HOST memory.
  *
  * Copies this step's queries, action-token logits, index arrays, budgets and tables from the host
- * (pinned memory recommended) into the caller's device staging buffers on `stream`, runs
- * actkv_budget (when logits are given) -> actkv_keep_indptr -> per group of `layers_per_call`
- * layers: actkv_score_lse, actkv_score, actkv_select, actkv_compact, copies the new page table,
- * seq_len, free list, free count, budgets and the status words back to the host, and
- * SYNCHRONISES the stream before returning (the one entry point that does: its outputs are host
- * memory).  The KV pool stays in device memory — it is the cache being compressed.
+ * (pinned memory recommended) into the caller's device staging buffers, runs actkv_score_lse per
+ * group of layers, actkv_budget (when logits are given) -> actkv_keep_indptr, then per group:
+ * actkv_score, actkv_select, actkv_compact, copies the new page table, seq_len, free list, free
+ * count, budgets and the status words back to the host, and SYNCHRONISES the stream before
+ * returning (the one entry point that does: its outputs are host memory).  The KV pool stays in
+ * device memory — it is the cache being compressed.
+ * The queries and logits are copied on a stream of the library's own (created on first use, one per
+ * device), ordered after the work already queued on `stream`, so that the transfers overlap the LSE
+ * kernels; everything is joined into `stream` before the results are copied back.  Those streams
+ * are shared by all calls on a device: host threads must not run this entry point concurrently on
+ * the same device.
+ * layers_per_call: capacity of score_dev / sel_idx_dev / the score workspace in layers (0: all
+ * layers).  The library works in groups of min(layers_per_call, 16) layers.
  * Every pointer named *_host is host memory, every other pointer device memory owned by the caller
  * and sized as the corresponding argument of the per-stage calls (score_dev:
  * [layers_per_call, n_kv_heads, sum_tok]; sel_idx_dev: [layers_per_call*n_kv_heads, sel_stride];
