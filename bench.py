@@ -70,19 +70,28 @@ class ClockSampler:
     def __init__(self, index: int):
         self.index = index
         self.proc = None
-        self.lines = []
+        self.lines = []          # (host time the line was read, line)
+        self.t_begin = self.t_end = None
 
     def start(self):
+        """Starts nvidia-smi (it needs a moment to produce its first sample, so this is called before
+        the warm-up); only samples read between begin() and end() count."""
         try:
             self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
-                                          "-lms", "50", "-i", str(self.index)], stdout=subprocess.PIPE, text=True)
+                                          "-lms", "20", "-i", str(self.index)], stdout=subprocess.PIPE, text=True)
             threading.Thread(target=self._read, daemon=True).start()
         except Exception:
             self.proc = None
 
     def _read(self):
         for line in self.proc.stdout:
-            self.lines.append(line.strip())
+            self.lines.append((time.perf_counter(), line.strip()))
+
+    def begin(self):
+        self.t_begin = time.perf_counter()
+
+    def end(self):
+        self.t_end = time.perf_counter()
 
     def stop(self):
         if self.proc is None:
@@ -94,7 +103,11 @@ class ClockSampler:
             self.proc.kill()
         sm, mx, reasons = [], [], set()
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        for ln in self.lines:
+        t_lo = self.t_begin if self.t_begin is not None else -1.0
+        t_hi = (self.t_end if self.t_end is not None else float("inf")) + 0.02       # a sample covers the 20 ms before it
+        for t, ln in self.lines:
+            if not (t_lo <= t <= t_hi):
+                continue
             f = [x.strip() for x in ln.split(",")]
             if len(f) < 7:
                 continue
@@ -235,6 +248,8 @@ def run_ours(args):
     wl = make_workload(args.workload, args.layers)
     wl.seed += 100 * rank                      # every replica draws its own batch
     R, NL, Hkv, G, D = wl.n_req, wl.n_layers, wl.n_kv_heads, wl.group, wl.head_dim
+    sampler = ClockSampler(visible_gpu_index(local_rank))
+    sampler.start()                            # early: nvidia-smi takes a moment to deliver its first sample
     inst = synth.generate(wl, dev)
     sz = H.sizes_of(inst)
     comp = H.Compressor(inst.pool, inst.page_table, inst.seq_len, inst.free_list, inst.free_count, wl.n_q_heads, sz,
@@ -298,12 +313,11 @@ def run_ours(args):
     if args.lse == "supplied":
         lse_supplied = comp.lse.clone()
 
-    sampler = ClockSampler(visible_gpu_index(local_rank))
-    sampler.start()
     if dist is not None:
         dist.barrier()
     torch.cuda.synchronize()
     all_events, launches = [], 0
+    sampler.begin()
     t_wall0 = time.perf_counter()
     for _ in range(args.steps):
         restore()
@@ -314,6 +328,7 @@ def run_ours(args):
     if dist is not None:
         dist.barrier()
     t_wall = time.perf_counter() - t_wall0
+    sampler.end()
     clocks = sampler.stop()
     comp.check_status()
 

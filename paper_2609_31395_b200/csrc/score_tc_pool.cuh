@@ -34,9 +34,12 @@ struct PoolBarriers {
 // One accumulator: columns [0, 32*n_cg) hold s for rows n0 .. of this key (lane).  nlse = -lse*log2(e)
 // per row (-inf for padding rows).  Adds sum_w exp2(max_g(s*c + nlse)) over the live rows to `acc`.
 // TMEM loads are software-pipelined against the arithmetic of the previous 32 columns.
+// Action tokens outside [w_min, w_end) do not count: below w_min the key is not visible yet (causal
+// rule), from w_end on the columns are padding (with a narrow MMA they were never written and may hold
+// anything; whatever the arithmetic makes of them is discarded by the select).
 template <int G>
-__device__ __forceinline__ void pool_job(uint32_t taddr, const float* nlse, int n_cg, int w_first, int w_min, float c,
-                                         float& acc) {
+__device__ __forceinline__ void pool_job(uint32_t taddr, const float* nlse, int n_cg, int w_first, int w_min, int w_end,
+                                         float c, float& acc) {
   float v[2][32];
   tmem_ld32(taddr, v[0]);
 #pragma unroll
@@ -61,7 +64,7 @@ __device__ __forceinline__ void pool_job(uint32_t taddr, const float* nlse, int 
       for (int i = 0; i < WPG; ++i) {
         const float mx = max_of<G>(x + i * G);
         const int w = w_first + cg * WPG + i;
-        acc += (w >= w_min) ? exp2f(mx) : 0.f;    // padding rows: mx = -inf -> 0
+        acc += (w >= w_min && w < w_end) ? exp2f(mx) : 0.f;
       }
     }
   }
@@ -182,7 +185,10 @@ score_tc_pool_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_cons
     // between two MMAs beyond the queue's depth is a bubble in the tensor pipe.
     const uint64_t kdesc0 = smem_desc_sw128(k_smem);
     const uint64_t qdesc0 = smem_desc_sw128(q_smem);
-    const uint32_t idesc_c[2] = {idesc_bf16(128, min(256, rows_pad)), idesc_bf16(128, max(16, rows_pad - 256))};
+    // MMA width of each row chunk: its live rows rounded up to 16 (a decode-step update has only G)
+    const int n0 = rows <= 256 ? max(16, (rows + 15) & ~15) : 256;
+    const int n1 = max(16, (rows - 256 + 15) & ~15);
+    const uint32_t idesc_c[2] = {idesc_bf16(128, n0), idesc_bf16(128, n1)};
     bool ok = mbar_wait(smem_u32(&bars->q_full), 0, abort_flag);
     if (ok) ok = mbar_wait(smem_u32(&bars->k_full[0]), 0, abort_flag);               // job 0: stage 0, accumulator 0
     int s = 0, rc = 0;
@@ -245,9 +251,9 @@ score_tc_pool_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_cons
       float acc = 0.f;
 #ifndef ACTKV_EXP_NO_EPI
 #ifdef ACTKV_EXP_NO_NLSE
-      pool_job<G>(taddr, nlse, 0 * n_cg + n_cg, (rc * 256) / G, w_min, c, acc);
+      pool_job<G>(taddr, nlse, 0 * n_cg + n_cg, (rc * 256) / G, w_min, W, c, acc);
 #else
-      pool_job<G>(taddr, nlse + rc * 256, n_cg, (rc * 256) / G, w_min, c, acc);
+      pool_job<G>(taddr, nlse + rc * 256, n_cg, (rc * 256) / G, w_min, W, c, acc);
 #endif
 #endif
       tc_fence_before();
