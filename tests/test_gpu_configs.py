@@ -147,6 +147,92 @@ def test_config3_inplace_tail_compaction_full_size():
         -(-L // wl.page_size) - -(-b // wl.page_size) for L, b in zip(wl.seq_lens, wl.budgets))
 
 
+def test_config3_lrfu_policy_full_size():
+    """The benchmark workload under the LRFU policy (p = 0.9, lambda = 0.5, 512 protected tokens), in the
+    launch configuration of the benchmark's LRFU line: hit mask, keep-score and TopK of sampled units
+    against the oracle run on the GPU's own float32 scores; every unit keeps its protected prefix."""
+    wl = synth.config3()
+    inst = synth.generate(wl, DEV)
+    sz = H.sizes_of(inst)
+    R, Hkv, NL = wl.n_req, wl.n_kv_heads, wl.n_layers
+    comp = H.Compressor(inst.pool, inst.page_table, inst.seq_len, inst.free_list, inst.free_count, wl.n_q_heads, sz)
+    n_protect = 512
+    lrfu = H.LrfuState(NL * Hkv, sz, DEV, 0.9, 0.5, torch.full((R,), n_protect, dtype=torch.int32, device=DEV),
+                       want_hits=True)
+    g = torch.Generator(device=DEV).manual_seed(7)
+    lrfu.keep_score.uniform_(0.0, 1e-3, generator=g)                   # as if earlier rounds had run
+    ks_before = lrfu.keep_score.clone()
+    units = [(0, 0, 0), (17, 1, 3), (30, 2, 5), (47, 3, 7)]
+    raw = {}
+
+    def marks(name):
+        if name == "score":
+            raw["score"] = {u: comp.score[u[0], u[1]].clone() for u in units}
+
+    comp.step(inst.q, inst.win_indptr, inst.tok_indptr, inst.budget, wl.sm_scale, wl.causal, marks=marks, lrfu=lrfu)
+    torch.cuda.synchronize()
+    comp.check_status()
+    tok = inst.tok_indptr.cpu().numpy()
+    ki = comp.keep_indptr.cpu().numpy()
+    for (a, h, r) in units:
+        o = a * Hkv + h
+        lo, hi = int(tok[r]), int(tok[r + 1])
+        sc = raw["score"][(a, h, r)][lo:hi].cpu().numpy()
+        hit = O.hit_mask_unit(sc, 0.9)
+        ks = O.keep_score_update(ks_before[o, lo:hi].cpu().numpy(), sc, hit, 0.5)
+        sel = O.select_unit(O.rank_keys(ks, n_protect), wl.budgets[r])
+        words = lrfu.hit_mask[o].cpu().numpy().view(np.uint32)
+        idx = np.arange(lo, hi)
+        got_hit = ((words[idx >> 5] >> (idx & 31).astype(np.uint32)) & 1).astype(bool)
+        assert np.array_equal(got_hit, hit)
+        assert np.array_equal(lrfu.keep_score[o, lo:hi].cpu().numpy().view(np.uint32), ks.view(np.uint32))
+        assert np.array_equal(comp.sel_idx[o, ki[r]:ki[r + 1]].cpu().numpy(), sel)
+        assert np.array_equal(lrfu.kept[o, ki[r]:ki[r + 1]].cpu().numpy().view(np.uint32), ks[sel].view(np.uint32))
+        assert 0 < hit.sum() < hi - lo
+    # the protected prefix leads every unit's list
+    sel_all = comp.sel_idx.cpu().numpy()
+    want_prefix = np.arange(n_protect)
+    for r in range(R):
+        assert (sel_all[:, ki[r]:ki[r] + n_protect] == want_prefix[None]).all()
+
+
+def test_config3_streaming_update_full_size():
+    """One decode-step update (one query per request, LSE supplied, three queries already folded in) at
+    the benchmark shape, all 48 layers in one call as the benchmark's streaming line launches it:
+    sampled units against the oracle's step."""
+    wl = synth.config3()
+    inst = synth.generate(wl, DEV)
+    sz = H.sizes_of(inst)
+    R, Hkv, NL, G = wl.n_req, wl.n_kv_heads, wl.n_layers, wl.group
+    comp = H.Compressor(inst.pool, inst.page_table, inst.seq_len, inst.free_list, inst.free_count, wl.n_q_heads, sz,
+                        want_lse=True)
+    comp.run_lse(inst.q, inst.win_indptr, inst.tok_indptr, wl.sm_scale, wl.causal, 0, NL, comp.lse)
+    first = inst.win_indptr[:-1].to(torch.int64)
+    q1 = inst.q[:, first].contiguous()
+    lse1 = comp.lse[:, first].contiguous()
+    win1 = torch.arange(R + 1, dtype=torch.int32, device=DEV)
+    steps = torch.tensor([3, 0, 1, 3, 7, 0, 2, 3], dtype=torch.int32, device=DEV)
+    g = torch.Generator(device=DEV).manual_seed(8)
+    state = torch.rand((NL, Hkv, sz.sum_tok), generator=g, device=DEV) * 1e-4
+    before = state.clone()
+    B.actkv_score_accumulate(comp.pd, comp.td, 0, NL, q1, win1, wl.n_q_heads, lse1, wl.sm_scale, wl.causal,
+                             inst.tok_indptr, steps, state, R, 1, sz.sum_tok, sz.max_tok, comp.ws_score, comp.status)
+    torch.cuda.synchronize()
+    comp.check_status()
+    pt, tok = inst.page_table.cpu().numpy(), inst.tok_indptr.cpu().numpy()
+    n_prev = steps.cpu().tolist()
+    for (a, h, r) in [(0, 0, 0), (11, 1, 1), (23, 2, 4), (35, 3, 5), (47, 0, 7)]:
+        L = wl.seq_lens[r]
+        slots = torch.from_numpy(O.slot_map(pt[r], L, wl.page_size)).to(DEV)
+        k = O.bf16_bits_to_f64(U.bits(inst.pool[a, 0].view(-1, Hkv, wl.head_dim)[slots, h]))
+        q = O.bf16_bits_to_f64(U.bits(q1[a, r, h * G:(h + 1) * G]))
+        lse = lse1[a, r, h * G:(h + 1) * G].cpu().numpy().astype(np.float64)
+        old = before[a, h, tok[r]:tok[r + 1]].cpu().numpy().astype(np.float64)
+        want = O.score_stream_step(old, n_prev[r], q, k, lse, wl.sm_scale)
+        got = state[a, h, tok[r]:tok[r + 1]].cpu().numpy()
+        assert U.max_rel(got, want) <= U.SCORE_RTOL, f"unit {(a, h, r)}"
+
+
 def test_config4_serving_mix_budgets_from_monitor():
     """64 requests, lengths log-uniform in 8K-64K; budgets produced on the device by actkv_budget
     from 256 action-token logit rows per request (V = 151936), clamped to 15-40% of length.  Two of
