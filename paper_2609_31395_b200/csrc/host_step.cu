@@ -6,10 +6,11 @@
 //
 // The large inputs (queries, logits) cross the host link on a copy stream of the library while the
 // score kernels already run: the queries go first, one layer group at a time, and the LSE pass of a
-// group starts as soon as its queries have landed; the logits follow, the budget monitor runs on a
-// side stream when they are in, and the pooled-score / select / compact passes, which are the first
-// to need the budgets, start after the last LSE pass.  All side work is joined into the caller's
-// stream before the results are copied back.
+// group starts as soon as its queries have landed (the first group is short, so that this is soon);
+// the logits follow, the budget monitor runs on a side stream when they are in, and the first select,
+// which is the first kernel to need the budgets, comes after the last LSE pass and the first
+// pooled-score pass.  All side work is joined into the caller's stream before the results are copied
+// back.
 #include <mutex>
 
 #include "common.cuh"
@@ -76,8 +77,20 @@ static int step_enqueue(const actkv_pool_t* pool, const actkv_tables_t* tab, con
   int lpc = io->layers_per_call > 0 && io->layers_per_call < kDefaultGroupLayers ? io->layers_per_call
                                                                                  : kDefaultGroupLayers;
   if (lpc > NL) lpc = NL;
-  if ((NL + lpc - 1) / lpc > kMaxGroups) return ACTKV_E_INVALID;
-  const int n_groups = (NL + lpc - 1) / lpc;
+  if ((NL + lpc - 1) / lpc + 1 > kMaxGroups) return ACTKV_E_INVALID;
+  const int n_groups = (NL + lpc - 1) / lpc;                  // groups of the passes that follow the LSE
+  // Groups of the query copies and LSE passes: a short first group, so that the first kernel starts
+  // after a quarter of a group's transfer time, then groups of lpc layers.
+  int lse_bound[kMaxGroups + 1];
+  int n_lse_groups = 0;
+  lse_bound[0] = 0;
+  {
+    const int first = lpc >= 4 && NL > lpc / 4 ? lpc / 4 : (lpc < NL ? lpc : NL);
+    for (int l = first; ; l += lpc) {
+      lse_bound[++n_lse_groups] = l < NL ? l : NL;
+      if (l >= NL) break;
+    }
+  }
   const size_t q_layer_bytes = (size_t)io->sum_win * io->n_q_heads * pool->head_dim * 2;
   const size_t tbl_bytes = (size_t)R * tab->max_pages * 4;
 
@@ -99,8 +112,8 @@ static int step_enqueue(const actkv_pool_t* pool, const actkv_tables_t* tab, con
   if (with_budget) ACTKV_TRY(h2d(io->logit_indptr_dev, io->logit_indptr_host, (size_t)(R + 1) * 4, c));
   if (cudaMemsetAsync(io->status_dev, 0, 16, c) != cudaSuccess) return ACTKV_E_CUDA;
   ACTKV_TRY(record(st->small, c));
-  for (int g = 0; g < n_groups; ++g) {
-    const int l0 = g * lpc, l1 = l0 + lpc < NL ? l0 + lpc : NL;
+  for (int g = 0; g < n_lse_groups; ++g) {
+    const int l0 = lse_bound[g], l1 = lse_bound[g + 1];
     ACTKV_TRY(h2d((char*)io->q_dev + (size_t)l0 * q_layer_bytes, (const char*)io->q_host + (size_t)l0 * q_layer_bytes,
                   (size_t)(l1 - l0) * q_layer_bytes, st->copy));
     ACTKV_TRY(record(st->q[g], st->copy));
@@ -120,23 +133,25 @@ static int step_enqueue(const actkv_pool_t* pool, const actkv_tables_t* tab, con
   }
 
   // ---- caller's stream: LSE pass of every group while the rest of the input arrives ----
-  for (int g = 0; g < n_groups; ++g) {
-    const int l0 = g * lpc, l1 = l0 + lpc < NL ? l0 + lpc : NL;
+  for (int g = 0; g < n_lse_groups; ++g) {
+    const int l0 = lse_bound[g], l1 = lse_bound[g + 1];
     ACTKV_TRY(wait(s, st->q[g]));
     ACTKV_TRY(actkv_score_lse(pool, tab, l0, l1, (const char*)io->q_dev + (size_t)l0 * q_layer_bytes, io->win_indptr_dev,
                               io->n_q_heads, io->sm_scale, io->causal, io->tok_indptr_dev,
                               io->lse_dev + (size_t)l0 * io->sum_win * io->n_q_heads, io->sum_win, io->max_win,
                               io->sum_tok, io->max_tok, io->ws_score, io->ws_score_bytes, io->status_dev, stream));
   }
-  // ---- then the passes that need the budgets ----
-  if (with_budget) ACTKV_TRY(wait(s, st->budget));
-  ACTKV_TRY(actkv_keep_indptr(tab->seq_len, io->budget_dev, R, io->keep_indptr_dev, stream));
+  // ---- then the other passes; the budgets are first needed by the first select ----
   for (int g = 0; g < n_groups; ++g) {
     const int l0 = g * lpc, l1 = l0 + lpc < NL ? l0 + lpc : NL;
     ACTKV_TRY(actkv_score(pool, tab, l0, l1, (const char*)io->q_dev + (size_t)l0 * q_layer_bytes, io->win_indptr_dev,
                           io->n_q_heads, io->lse_dev + (size_t)l0 * io->sum_win * io->n_q_heads, io->sm_scale, io->causal,
                           io->tok_indptr_dev, io->score_dev, nullptr, io->sum_win, io->max_win, io->sum_tok,
                           io->max_tok, io->ws_score, io->ws_score_bytes, io->status_dev, stream));
+    if (g == 0) {
+      if (with_budget) ACTKV_TRY(wait(s, st->budget));
+      ACTKV_TRY(actkv_keep_indptr(tab->seq_len, io->budget_dev, R, io->keep_indptr_dev, stream));
+    }
     ACTKV_TRY(actkv_select(io->score_dev, io->tok_indptr_dev, io->sum_tok, io->budget_dev, (l1 - l0) * Hkv, R,
                            io->keep_indptr_dev, io->sel_idx_dev, io->sel_stride, nullptr, nullptr, nullptr, 0,
                            io->status_dev, stream));
