@@ -33,24 +33,34 @@ struct PoolBarriers {
 
 // One accumulator: columns [0, 32*n_cg) hold s for rows n0 .. of this key (lane).  nlse = -lse*log2(e)
 // per row (-inf for padding rows).  Adds sum_w exp2(max_g(s*c + nlse)) over the live rows to `acc`.
-// TMEM loads are software-pipelined against the arithmetic of the previous 32 columns.
 // Action tokens outside [w_min, w_end) do not count: below w_min the key is not visible yet (causal
 // rule), from w_end on the columns are padding (with a narrow MMA they were never written and may hold
 // anything; whatever the arithmetic makes of them is discarded by the select).
 template <int G>
 __device__ __forceinline__ void pool_job(uint32_t taddr, const float* nlse, int n_cg, int w_first, int w_min, int w_end,
-                                         float c, float& acc) {
-  float v[2][32];
-  tmem_ld32(taddr, v[0]);
+                                         float c, float& acc, uint32_t empty_bar, int lane) {
+  // 64 columns per load, two register buffers: the load of the next 64 columns is in flight while these
+  // are folded, so the round trip to tensor memory is paid four times per accumulator, not eight, and
+  // mostly hidden.  The accumulator is handed back to the MMA warp as soon as its last columns are in
+  // registers, before they are folded.
+  const int n_c2 = (n_cg + 1) >> 1;
+  float v[2][64];
+  tmem_ld64(taddr, v[0]);
 #pragma unroll
-  for (int cg = 0; cg < 8; ++cg) {
-    if (cg < n_cg) {
+  for (int c2 = 0; c2 < 4; ++c2) {
+    if (c2 < n_c2) {
       tmem_ld_wait();
-      if (cg + 1 < n_cg) tmem_ld32(taddr + (cg + 1) * 32, v[(cg + 1) & 1]);
-      float* x = v[cg & 1];
-      const float4* l4 = reinterpret_cast<const float4*>(nlse + cg * 32);
+      if (c2 + 1 < n_c2) {
+        tmem_ld64(taddr + (c2 + 1) * 64, v[(c2 + 1) & 1]);
+      } else {
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(empty_bar);
+      }
+      float* x = v[c2 & 1];
+      const float4* l4 = reinterpret_cast<const float4*>(nlse + c2 * 64);
 #pragma unroll
-      for (int q4 = 0; q4 < 8; ++q4) {
+      for (int q4 = 0; q4 < 16; ++q4) {
 #ifdef ACTKV_EXP_NO_NLSE
         const float4 l = make_float4(-1.f, -1.f, -1.f, -1.f + (float)(l4 == nullptr));
 #else
@@ -59,11 +69,11 @@ __device__ __forceinline__ void pool_job(uint32_t taddr, const float* nlse, int 
         ffma2(x[q4 * 4 + 0], x[q4 * 4 + 1], x[q4 * 4 + 0], x[q4 * 4 + 1], c, l.x, l.y);
         ffma2(x[q4 * 4 + 2], x[q4 * 4 + 3], x[q4 * 4 + 2], x[q4 * 4 + 3], c, l.z, l.w);
       }
-      constexpr int WPG = 32 / G;                 // action tokens per 32-column group
+      constexpr int WPG = 64 / G;                 // action tokens per 64-column group (G <= 32)
 #pragma unroll
       for (int i = 0; i < WPG; ++i) {
         const float mx = max_of<G>(x + i * G);
-        const int w = w_first + cg * WPG + i;
+        const int w = w_first + c2 * WPG + i;
         acc += (w >= w_min && w < w_end) ? exp2f(mx) : 0.f;
       }
     }
@@ -251,14 +261,15 @@ score_tc_pool_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_cons
       float acc = 0.f;
 #ifndef ACTKV_EXP_NO_EPI
 #ifdef ACTKV_EXP_NO_NLSE
-      pool_job<G>(taddr, nlse, 0 * n_cg + n_cg, (rc * 256) / G, w_min, W, c, acc);
+      pool_job<G>(taddr, nlse, 0 * n_cg + n_cg, (rc * 256) / G, w_min, W, c, acc, smem_u32(&bars->tmem_empty[wg]), lane);
 #else
-      pool_job<G>(taddr, nlse + rc * 256, n_cg, (rc * 256) / G, w_min, W, c, acc);
+      pool_job<G>(taddr, nlse + rc * 256, n_cg, (rc * 256) / G, w_min, W, c, acc, smem_u32(&bars->tmem_empty[wg]), lane);
 #endif
-#endif
+#else
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(smem_u32(&bars->tmem_empty[wg]));
+#endif
       if (n_rc == 1) {
         if (key < L) store_pooled(a, r, out + key, acc, acc * inv_w, W);
       } else if (wg == 1) {
