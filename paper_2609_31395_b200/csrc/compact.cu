@@ -69,7 +69,7 @@ __global__ void compact_plan_kernel(TablesView tab, int32_t page_size, int32_t n
   if (threadIdx.x == 0) { ws->plan_ok = s_ok; ws->total_new = total; }
 }
 
-constexpr int CP_NT = 256;
+constexpr int CP_NT = 128;
 constexpr int CP_UNROLL = 8;
 
 // One CTA per (destination page, request, layer).  The (slot, head) -> source / destination row

@@ -91,11 +91,11 @@ static int score_impl(int mode, const actkv_pool_t* pool, const actkv_tables_t* 
   a.rows_max = lay.rows_max;
   // Keys per LSE partial.  A CTA pays a fixed cost (operand set-up, pipeline fill and drain), so chunks
   // are as long as they can be while there are still several CTAs per SM: the largest multiple of the
-  // minimum chunk that leaves at least 6 x 148 work items (never more chunks than the workspace holds).
+  // minimum chunk that leaves at least 20 x 148 work items (never more chunks than the workspace holds).
   {
     const int64_t units_ = (int64_t)(layer_end - layer_begin) * Hkv * R;
-    const int64_t row_groups = (lay.rows_max + 255) / 256;
-    int n_chunks = (int)((6 * 148 + units_ * row_groups - 1) / (units_ * row_groups));
+    const int64_t row_groups = 1;                  // a CTA of either path covers all rows of its unit
+    int n_chunks = (int)((20 * 148 + units_ * row_groups - 1) / (units_ * row_groups));
     if (n_chunks < 1) n_chunks = 1;
     if (n_chunks > lay.n_chunks) n_chunks = lay.n_chunks;
     int chunk = (max_tok + n_chunks - 1) / n_chunks;
@@ -182,3 +182,9 @@ int actkv_score_accumulate(const actkv_pool_t* pool, const actkv_tables_t* table
 const char* actkv_version(void) { return "actkv-b200 0.1 (sm_100a)"; }
 
 }  // extern "C"
+
+#ifdef ACTKV_LSE_TRACE
+extern "C" int actkv_debug_lse_trace(long long* out_host) {
+  return cudaMemcpyFromSymbol(out_host, actkv::tc::g_lse_trace, sizeof(long long) * 6 * 1024) == cudaSuccess ? 0 : -1;
+}
+#endif

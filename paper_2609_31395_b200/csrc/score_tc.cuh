@@ -6,8 +6,8 @@
 // the other warps: epilogue reading TMEM with tcgen05.ld):
 //
 //  * LSE pass (score_tc_lse.cuh; Section 7.1, LSE equation).  D[row, key] = Q K^T with the window x
-//    group rows on the TMEM lanes, so every epilogue thread owns one row and keeps its running
-//    (max, sum of exp2) in registers: no shuffles.
+//    group rows on the TMEM lanes (Q as the A operand from tensor memory), so every epilogue thread
+//    owns one row per 128-row block and keeps its running (max, sum of exp2) in registers: no shuffles.
 //  * Pooled-score pass (score_tc_pool.cuh; Section 7.1 recovery identity, Algorithm 3 steps 3-5).
 //    The transposed product D[key, row] = K Q^T with the keys on the lanes and row = w*G + g on the
 //    columns, so the max over the GQA group and the sum over the action tokens run inside one
@@ -98,41 +98,39 @@ inline bool score_tc_supported(const actkv_pool_t* p, int G, int max_win, float 
   return tc::encode_fn() != nullptr;
 }
 
-template <int POLY>
-inline int score_tc_launch_lse_p(const CUtensorMap& kmap, const CUtensorMap& qmap, const tc::TcArgs& ta, unsigned grid,
-                                 size_t smem, cudaStream_t s) {
-  (void)qmap;
-  if (cudaFuncSetAttribute(tc::score_tc_lse_kernel<POLY>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+template <int NPOLY>
+inline int score_tc_launch_lse_c(const CUtensorMap& kmap, const tc::TcArgs& ta, unsigned grid, size_t smem, cudaStream_t s) {
+  if (cudaFuncSetAttribute(tc::score_tc_lse_kernel<NPOLY>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
     return ACTKV_E_CUDA;
-  tc::score_tc_lse_kernel<POLY><<<grid, tc::LSE_THREADS, smem, s>>>(kmap, ta);
+  tc::score_tc_lse_kernel<NPOLY><<<grid, tc::LSE_THREADS, smem, s>>>(kmap, ta);
   ACTKV_CHECK_LAUNCH();
   return ACTKV_OK;
 }
 
 inline int score_tc_launch_lse(ScoreArgs& a, const actkv_pool_t* pool, int max_tok, int max_win, cudaStream_t s) {
   (void)max_tok;
+  (void)max_win;
   CUtensorMap kmap, qmap;
   if (!tc::make_maps(pool, a.q, a.n_layers_sub, a.sum_win, a.n_q_heads, a.group, &kmap, &qmap)) return ACTKV_E_CUDA;
   tc::TcArgs ta;
   ta.a = a;
-  const int rows_pad = (max_win * a.group + 127) & ~127;
-  ta.n_rg = (rows_pad + 255) / 256;
+  ta.n_rg = 1;
   ta.n_stages = 6;
   ta.tiles_per_cta = 0;
   ta.n_kchunks = 0;
   const int64_t units = (int64_t)a.n_layers_sub * a.pool.n_kv_heads * a.tab.n_req;
-  const int64_t grid = units * ta.n_rg * a.n_chunks;
+  const int64_t grid = units * a.n_chunks;
   if (grid > 0x7fffffffLL) return ACTKV_E_INVALID;
   const size_t smem = (size_t)ta.n_stages * tc::KTILE_BYTES + sizeof(tc::LseBarriers);
-  // share of the exps evaluated by the polynomial (tuning knob; the default is what the bench uses)
-  int poly = tc::LSE_POLY_PAIRS_DEFAULT;
-  if (const char* e = getenv("ACTKV_LSE_POLY")) poly = atoi(e);
-  switch (poly) {
-    case 0: return score_tc_launch_lse_p<0>(kmap, qmap, ta, (unsigned)grid, smem, s);
-    case 1: return score_tc_launch_lse_p<1>(kmap, qmap, ta, (unsigned)grid, smem, s);
-    case 3: return score_tc_launch_lse_p<3>(kmap, qmap, ta, (unsigned)grid, smem, s);
-    case 4: return score_tc_launch_lse_p<4>(kmap, qmap, ta, (unsigned)grid, smem, s);
-    default: return score_tc_launch_lse_p<2>(kmap, qmap, ta, (unsigned)grid, smem, s);
+  // columns of every 8 that take the polynomial exp2 (tuning knob; the default is what the bench uses)
+  int npoly = tc::LSE_NPOLY_DEFAULT;
+  if (const char* e = getenv("ACTKV_LSE_NPOLY")) npoly = atoi(e);
+  switch (npoly) {
+    case 0: return score_tc_launch_lse_c<0>(kmap, ta, (unsigned)grid, smem, s);
+    case 1: return score_tc_launch_lse_c<1>(kmap, ta, (unsigned)grid, smem, s);
+    case 2: return score_tc_launch_lse_c<2>(kmap, ta, (unsigned)grid, smem, s);
+    case 4: return score_tc_launch_lse_c<4>(kmap, ta, (unsigned)grid, smem, s);
+    default: return score_tc_launch_lse_c<3>(kmap, ta, (unsigned)grid, smem, s);
   }
 }
 

@@ -1,22 +1,42 @@
 // LSE pass of the tensor-core score path (Section 7.1, LSE equation):
 //   lse[row] = log sum_{key visible} exp(sm_scale * q_row . k_key),   row = (window token w, group head g).
 //
-// D[row, key] = Q K^T with the rows on the TMEM lanes, so every epilogue thread owns one row and keeps
-// its running (max, sum of exp2) in registers: no shuffles.  A CTA covers 256 rows (two 128-row
-// blocks) x one chunk of LSE_CHUNK keys.
+// D[row, key] = Q K^T with the rows on the TMEM lanes, so every epilogue thread owns one row per
+// 128-row block and folds its share of the row's logits into a running (reference, sum of exp2): no
+// shuffles.  A CTA covers ALL row blocks of a unit (up to four, 512 rows) x one chunk of keys, so a
+// K tile is fetched once per unit.
 //
-// Operand placement.  With both operands in shared memory the operand fetch (A 4 KB + B 4 KB per
-// 128x128x16 MMA) caps the tensor pipe near half rate.  The Q block is the same for every key tile
-// of the CTA, so it is written once into tensor memory (tcgen05.st, two bf16 per 32-bit column) and
-// used as the A operand from there; only the K tile (B) streams through shared memory.
-// TMEM columns: [0,128) the two Q blocks, [128,512) a ring of three 128-column accumulators; a job
-// is one (key tile, row block) product.
+// Operand placement.  An A operand in shared memory is re-read for every MMA and that read is not
+// overlapped with the MMA (measured 105 cycles per 128x128x16 MMA against 74 with A in tensor memory,
+// 64 nominal).  The Q blocks are the same for every key tile of the CTA, so they are written once into
+// tensor memory (tcgen05.st, two bf16 per 32-bit column) and used as the A operand from there; only
+// the K tile (B) streams through shared memory.
+// TMEM columns: [0,256) the four Q blocks, [256,512) two 128-column accumulators; a job is one
+// (key tile, row block) product.  Even jobs go to accumulator 0, odd jobs to accumulator 1; each
+// accumulator has its own MMA-issuing warp and its own group of eight epilogue warps (64 columns per
+// thread), which hand the accumulator back as soon as their columns are in registers.  While one group
+// waits for tensor memory the other keeps the special function unit busy.
 //
-// Exp rate.  One exp2 per (row, key) is more than the 16 MUFU results per clock of an SM can follow,
-// so POLY of every 8 column pairs are evaluated on the FMA / ALU pipes instead: 2^x = 2^j p(f),
-// j = round(x), f = x - j in [-0.5, 0.5], p a cubic fitted to 2^f (max relative error 7.5e-5, far
-// inside the 2e-3 score tolerance), 2^j applied by adding j to the exponent field; two columns at a
-// time with the packed fp32x2 instructions.
+// What bounds the kernel (measured on B200 with micro-benchmarks and per-job timestamps):
+//  * Issuing is not free: a tcgen05.mma costs the issuing thread about 50 cycles and a tcgen05.commit
+//    about 80, some 470 cycles for a job the tensor pipe executes in 512, and the commit reaches the
+//    waiting warps about 240 cycles after the last MMA retires.  One issuer doing its barrier
+//    handshakes in between left the pipe idle 40 % of the time; hence two issuers.
+//  * An SM sub-partition dispatches about one fp32 operation per clock (the packed fp32x2 forms take
+//    two, so they save nothing) and its special function unit delivers one warp-wide exp2 per 8 clocks.
+//    One exp2 per (row, key) on that unit alone costs 8 clocks per warp and logit against 4.6 for the
+//    contraction: the pass is bound by the exp rate.  Of each 8 columns, NPOLY take a polynomial on the
+//    FMA pipe instead (ten dispatch slots each, against three slots and eight clocks of the unit); the
+//    two kinds overlap only partly, and NPOLY = 1 measured best (0: 9.06 ms, 1: 8.63, 2: 8.90, 3: 9.32 at
+//    the bench shape).
+//  * To keep the slot count low there is no running maximum: the reference m of a row is the maximum of
+//    the first logits the thread saw, later logits may exceed it (2^x is evaluated for x up to 126), and
+//    only if a partial sum grows past 2^40 is the reference moved (a rare, slower path that also serves
+//    tiles cut by the end of the request or by the causal diagonal).
+// Polynomial: y = sat(x/252 + 1/2) clamps x to [-126, 126] inside the multiply-add that forms it;
+// j = round(x) by the magic-number addition, f = x - j in [-0.5, 0.5], 2^x = 2^j p(f) with p a cubic
+// fitted to 2^f (max relative error 7.5e-5, far inside the 2e-3 score tolerance), 2^j applied by adding
+// j to the exponent field.
 #pragma once
 
 #include "tc_common.cuh"
@@ -24,57 +44,70 @@
 namespace actkv {
 namespace tc {
 
-constexpr int LSE_POLY_PAIRS_DEFAULT = 2;        // measured best on B200 (0: 9.0 ms, 1: 8.6, 2: 8.4, 3: 8.9 at the bench shape)
+constexpr int LSE_NPOLY_DEFAULT = 1;             // columns of every 8 whose exp2 is the polynomial
 
-__device__ __forceinline__ void exp2_poly2(float& e0, float& e1, float x0, float x1) {
-  constexpr float MAGIC = 12582912.f;            // 1.5 * 2^23: x + MAGIC rounds x to the nearest integer
-  x0 = fmaxf(x0, -126.f);
-  x1 = fmaxf(x1, -126.f);
-  float t0 = x0, t1 = x1;
-  fadd2(t0, t1, MAGIC, MAGIC);                   // integer part in the low mantissa bits
-  float j0 = t0, j1 = t1;
-  fadd2(j0, j1, -MAGIC, -MAGIC);
-  float f0 = x0, f1 = x1;
-  fadd2(f0, f1, -j0, -j1);                       // f = x - round(x)
-  float p0, p1;                                  // Horner, both lanes per instruction
-  ffma2(p0, p1, f0, f1, 0.0551716648042202f, 0.2426111251115799f, 0.2426111251115799f);
-  ffma2v(p0, p1, p0, p1, f0, f1, 0.6932609677314758f, 0.6932609677314758f);
-  ffma2v(p0, p1, p0, p1, f0, f1, 0.9999280571937561f, 0.9999280571937561f);
-  e0 = __int_as_float(__float_as_int(p0) + (__float_as_int(t0) << 23));
-  e1 = __int_as_float(__float_as_int(p1) + (__float_as_int(t1) << 23));
+__device__ __forceinline__ float ffma_sat(float a, float b, float c) {
+  float d;
+  asm("fma.rn.sat.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+  return d;
 }
 
-// One full group of 32 logits of a row: online max, then sum += sum_i exp2((v_i - m) * c).
-template <int POLY>
-__device__ __forceinline__ void lse_group(const float* v, float c, float& m, float& sum) {
-  float t[11];                                   // max tree: 32 -> 11 -> 4 -> 1
+// 2^x for x = 252 y - 126, y in [0, 1]
+__device__ __forceinline__ float exp2_poly_y(float y) {
+  constexpr float MAGIC = 12582912.f;            // 1.5 * 2^23: adding it rounds to the nearest integer
+  const float t = fmaf(y, 252.f, MAGIC - 126.f); // MAGIC + j, j = round(x), in the low mantissa bits
+  const float j = t - MAGIC;
+  const float f = fmaf(y, 252.f, -126.f - j);    // x - j
+  float p = fmaf(0.0551716648042202f, f, 0.2426111251115799f);
+  p = fmaf(p, f, 0.6932609677314758f);
+  p = fmaf(p, f, 0.9999280571937561f);
+  return __int_as_float(__float_as_int(p) + (__float_as_int(t) << 23));
+}
+
+// 32 logits of one row, all visible, against the row's reference m (finite): returns
+// sum_i exp2((v_i - m) c).  nmc = -m c; c1 = c / 252, c0 = 1/2 - m c / 252.
+template <int NPOLY>
+__device__ __forceinline__ float lse_fast32(const float* v, float c, float nmc, float c1, float c0) {
+  float s[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-  for (int i = 0; i < 10; ++i) t[i] = fmax3(v[3 * i], v[3 * i + 1], v[3 * i + 2]);
-  t[10] = fmaxf(v[30], v[31]);
-  const float u0 = fmax3(t[0], t[1], t[2]), u1 = fmax3(t[3], t[4], t[5]), u2 = fmax3(t[6], t[7], t[8]);
-  const float gm = fmaxf(fmax3(u0, u1, u2), fmaxf(t[9], t[10]));
-  if (gm > m) { sum *= exp2f((m - gm) * c); m = gm; }     // m = -inf: sum is 0 and stays 0
-  const float nmc = -m * c;
-  float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
+  for (int g8 = 0; g8 < 4; ++g8) {
 #pragma unroll
-  for (int p = 0; p < 16; ++p) {
-    float x0, x1, e0, e1;
-    ffma2(x0, x1, v[2 * p], v[2 * p + 1], c, nmc, nmc);
-    if ((p & 7) < POLY) {
-      exp2_poly2(e0, e1, x0, x1);
-    } else {
-      e0 = exp2f(x0);
-      e1 = exp2f(x1);
+    for (int i = 0; i < 8; ++i) {
+      const float x = v[g8 * 8 + i];
+      // the polynomial columns are spread over the group so that the two kinds interleave in program order
+      const bool poly = (NPOLY >= 1 && i == 1) || (NPOLY >= 2 && i == 4) || (NPOLY >= 3 && i == 6) || (NPOLY >= 4 && i == 3);
+      const float e = poly ? exp2_poly_y(ffma_sat(x, c1, c0)) : exp2f(fmaf(x, c, nmc));
+      s[i & 3] += e;
     }
-    if (p & 1) fadd2(s2, s3, e0, e1); else fadd2(s0, s1, e0, e1);
   }
-  sum += (s0 + s1) + (s2 + s3);
+  return (s[0] + s[1]) + (s[2] + s[3]);
 }
 
-constexpr int LSE_EPI_WARPS = 16;                // (row block, TMEM lane quarter, column half)
-constexpr int LSE_THREADS = (2 + LSE_EPI_WARPS) * 32;
-constexpr int LSE_SLOTS = 3;                     // accumulator ring
-constexpr int LSE_A_COLS = 128;                  // TMEM columns holding the two Q blocks
+// The general form: the first nv (possibly <= 0 or >= 32) logits are visible; moves the reference to the
+// maximum seen so far.  Also the entry for a row's first logits (m = -inf, sum = 0).
+__device__ __forceinline__ void lse_slow32(const float* v, int nv, float c, float& m, float& sum) {
+  if (nv <= 0) return;
+  float gm = -INFINITY;
+#pragma unroll
+  for (int i = 0; i < 32; ++i) gm = fmaxf(gm, i < nv ? v[i] : -INFINITY);
+  if (gm > m) { sum = (m == -INFINITY) ? 0.f : sum * exp2f((m - gm) * c); m = gm; }
+  const float mc = m * c;
+#pragma unroll
+  for (int i = 0; i < 32; ++i) sum += (i < nv) ? exp2f(fmaf(v[i], c, -mc)) : 0.f;
+}
+
+#ifdef ACTKV_LSE_TRACE
+__device__ long long g_lse_trace[6][1024];       // developer build: per-job timestamps of one CTA
+#define LSE_TR(row, job, cond) do { if ((cond) && blockIdx.x == 200 && (job) < 1024) g_lse_trace[row][job] = clock64(); } while (0)
+#else
+#define LSE_TR(row, job, cond) do { } while (0)
+#endif
+
+constexpr int LSE_EPI_WARPS = 16;                // (TMEM lane quarter, accumulator, column half)
+constexpr int LSE_THREADS = (3 + LSE_EPI_WARPS) * 32;     // producer, two MMA issuers, epilogue
+constexpr int LSE_SLOTS = 2;                     // accumulators
+constexpr int LSE_A_COLS = 256;                  // TMEM columns holding the four Q blocks
+constexpr float LSE_BIG = 1099511627776.f;       // 2^40: a partial sum beyond it moves the reference
 
 struct LseBarriers {
   uint64_t k_full[8];
@@ -82,33 +115,88 @@ struct LseBarriers {
   uint64_t q_ready;
   uint64_t tmem_full[LSE_SLOTS];
   uint64_t tmem_empty[LSE_SLOTS];
-  uint64_t drained;
+  uint64_t drained[2];
   uint32_t tmem_base;
   int abort_flag;
-  float2 exch[256];            // (max, sum) of the upper column half, handed to the lower half's thread
+  float2 state[2][4][2][128];  // (reference, sum) per (group, row block, column half, row in block)
 };
 
-template <int POLY>
+// After tcgen05.wait::ld: ties the loaded registers to the wait, so that no use of them is scheduled
+// ahead of it (the loads are asynchronous; the compiler sees their outputs as defined at issue).
+template <int N>
+__device__ __forceinline__ void tmem_ld_fence(float* v) {
+#pragma unroll
+  for (int i = 0; i < N; ++i) asm volatile("" : "+f"(v[i]));
+}
+
+__device__ __forceinline__ int sel4(const int (&x)[4], int i) { return i == 0 ? x[0] : i == 1 ? x[1] : i == 2 ? x[2] : x[3]; }
+
+// One job as one epilogue warp sees it: the warp takes 64 columns (two register buffers of 32) of the
+// accumulator of its group, hands the accumulator back as soon as they are in registers, and folds them
+// into the row's (reference, sum) in `st`.  The two groups work on alternate jobs, so while one waits
+// for tensor memory the other keeps the special function unit busy.
+//   tq      tensor-memory address of the group's accumulator, this warp's lane quarter and first column
+//   nv_min  visible columns (from the warp's first column) of the most restricted row of this thread
+//   jm      last visible key of this thread's row in each row block; key0 = key of the warp's first column
+template <int NPOLY>
+__device__ __forceinline__ bool lse_job(LseBarriers* bars, volatile int* abort_flag, uint32_t tq, int grp, int job,
+                                        int mb, float2* st, int nv_min, const int (&jm)[4], int key0, float c, float c1,
+                                        int lane) {
+  float va[32], vb[32];
+  LSE_TR(5, job, threadIdx.x == 3 * 32);
+  if (!mbar_wait(smem_u32(&bars->tmem_full[grp]), (uint32_t)(job >> 1) & 1u, abort_flag)) return false;
+  tc_fence_after();
+#ifndef ACTKV_EXP_NO_LD
+  tmem_ld32(tq, va);
+  tmem_ld32(tq + 32, vb);
+#endif
+  float2 ms = *st;
+  tmem_ld_wait();
+  tmem_ld_fence<32>(va);
+  tmem_ld_fence<32>(vb);
+  LSE_TR(2, job, threadIdx.x == 3 * 32);
+  tc_fence_before();
+  __syncwarp();
+  if (lane == 0) mbar_arrive(smem_u32(&bars->tmem_empty[grp]));
+  LSE_TR(3, job, threadIdx.x == 3 * 32);
+#ifndef ACTKV_EXP_NO_EPI
+  bool slow = __any_sync(0xffffffffu, nv_min < 64 || ms.x == -INFINITY);
+  if (!slow) {
+    const float nmc = -ms.x * c, c0 = fmaf(nmc, 1.f / 252.f, 0.5f);
+    const float ps = lse_fast32<NPOLY>(va, c, nmc, c1, c0) + lse_fast32<NPOLY>(vb, c, nmc, c1, c0);
+    slow = __any_sync(0xffffffffu, !(ps < LSE_BIG));
+    if (!slow) ms.y += ps;
+  }
+  if (slow) {
+    const int nv = sel4(jm, mb) - key0 + 1;
+    lse_slow32(va, nv, c, ms.x, ms.y);
+    lse_slow32(vb, nv - 32, c, ms.x, ms.y);
+  }
+  *st = ms;
+#endif
+  LSE_TR(4, job, threadIdx.x == 3 * 32);
+  return true;
+}
+
+template <int NPOLY>
 __global__ void __launch_bounds__(LSE_THREADS, 1)
 score_tc_lse_kernel(const __grid_constant__ CUtensorMap kmap, const TcArgs ta) {
   extern __shared__ __align__(1024) uint8_t smem[];
   const ScoreArgs& a = ta.a;
   const int R = a.tab.n_req, Hkv = a.pool.n_kv_heads, G = a.group;
-  int idx = blockIdx.x;
-  const int chunk = idx % a.n_chunks; idx /= a.n_chunks;
-  const int rg = idx % ta.n_rg;
-  const int u = idx / ta.n_rg;
+  const int u = blockIdx.x / a.n_chunks;
+  const int chunk = blockIdx.x - u * a.n_chunks;
   const int r = u % R, h = (u / R) % Hkv, slab = u / (R * Hkv);
   const int L = a.tab.seq_len[r];
   const int w0 = a.win_indptr[r], W = a.win_indptr[r + 1] - w0;
   const int rows = W * G;
   const int key_begin = chunk * a.lse_chunk;
-  if (key_begin >= L || rg * 256 >= rows) return;
+  if (key_begin >= L) return;
   if (W <= 0 || (a.causal && W > L)) {
-    if (threadIdx.x == 0 && chunk == 0 && rg == 0) report(a.status, ACTKV_E_INVALID, r, W);
+    if (threadIdx.x == 0 && chunk == 0) report(a.status, ACTKV_E_INVALID, r, W);
     return;
   }
-  const int n_mb = min(2, (rows - rg * 256 + 127) / 128);
+  const int n_mb = (rows + 127) / 128;                   // 1..4 (checked by the host)
   const int t_begin = key_begin / TK;
   const int t_end = min((L + TK - 1) / TK, t_begin + a.lse_chunk / TK);
   const int n_tiles = t_end - t_begin;
@@ -126,13 +214,14 @@ score_tc_lse_kernel(const __grid_constant__ CUtensorMap kmap, const TcArgs ta) {
     return;
   }
   if (threadIdx.x == 0) {
-    for (int s = 0; s < S; ++s) { mbar_init(smem_u32(&bars->k_full[s]), 1); mbar_init(smem_u32(&bars->k_empty[s]), 1); }
-    mbar_init(smem_u32(&bars->q_ready), 8);
+    for (int s = 0; s < S; ++s) { mbar_init(smem_u32(&bars->k_full[s]), 1); mbar_init(smem_u32(&bars->k_empty[s]), 2); }
+    mbar_init(smem_u32(&bars->q_ready), LSE_EPI_WARPS);
     for (int b = 0; b < LSE_SLOTS; ++b) {
       mbar_init(smem_u32(&bars->tmem_full[b]), 1);
       mbar_init(smem_u32(&bars->tmem_empty[b]), LSE_EPI_WARPS / 2);
     }
-    mbar_init(smem_u32(&bars->drained), 1);
+    mbar_init(smem_u32(&bars->drained[0]), 1);
+    mbar_init(smem_u32(&bars->drained[1]), 1);
     bars->abort_flag = 0;
     fence_barrier_init();
   }
@@ -146,14 +235,12 @@ score_tc_lse_kernel(const __grid_constant__ CUtensorMap kmap, const TcArgs ta) {
   const uint32_t tmem_base = bars->tmem_base;
 
   // epilogue identity (also used after the role split)
-  const int ew = warp - 2;                       // 0..15 for epilogue warps
+  const int ew = warp - 3;                       // 0..15 for epilogue warps
   const int quarter = warp & 3;                  // TMEM lanes this warp may touch
-  const int mb = (ew >> 2) & 1;                  // row block
-  const int ch = ew >> 3;                        // column half of a 128-key tile
-  const int row_in_blk = quarter * 32 + lane;
-  const int n = rg * 256 + mb * 128 + row_in_blk;                 // row within the unit
-  const bool row_ok = warp >= 2 && (mb < n_mb) && n < rows;
-  float m = -INFINITY, sum = 0.f;
+  const int k = ew >> 2;                         // 0..3
+  const int grp = k >> 1;                        // accumulator / job parity this warp serves
+  const int half = k & 1;                        // its columns: [64 half, 64 half + 64)
+  const int rib = quarter * 32 + lane;           // row within a 128-row block
   bool epi_ok = true;
 
   if (warp == 0) {
@@ -172,153 +259,146 @@ score_tc_lse_kernel(const __grid_constant__ CUtensorMap kmap, const TcArgs ta) {
       int ok = 1;
       if (lane == 0) {
         ok = mbar_wait(smem_u32(&bars->k_empty[s]), ph ^ 1u, abort_flag) ? 1 : 0;
+#ifdef ACTKV_EXP_NO_TMA
+        if (ok) mbar_arrive(smem_u32(&bars->k_full[s]));
+#else
         if (ok) mbar_expect_tx(smem_u32(&bars->k_full[s]), KTILE_BYTES);
+#endif
       }
       ok = __shfl_sync(0xffffffffu, ok, 0);
       if (!ok) break;
+#ifndef ACTKV_EXP_NO_TMA
       if ((lane >> 3) == (it & 3)) {
         const uint32_t dst = k_smem + s * KTILE_BYTES + (lane & 7) * 2048;
         tma_load_4d(dst, &kmap, smem_u32(&bars->k_full[s]), 0, h, pid * 16, layer);
         tma_load_4d(dst + HALF_BYTES, &kmap, smem_u32(&bars->k_full[s]), 64, h, pid * 16, layer);
       }
+#endif
       if ((it & 3) == 3) pid = pid_next;
     }
-  } else if (warp == 1) {
-    // ---------------- MMA issuer: A = Q block in TMEM, B = K tile in shared memory ----------------
-    // The whole warp runs the loop (waits and descriptor arithmetic stay warp-uniform, so they can
-    // live in uniform registers); one elected lane issues the tcgen05 instructions.
-    // The tensor pipe's queue is shallow: whatever the issuing warp spends between two jobs (a successful
-    // barrier wait costs 100-200 cycles) is idle time of the pipe.  So the barriers of job j+1 are polled
-    // (mbarrier.test_wait, non-blocking) BEFORE the MMAs of job j are issued and the answers are only read
-    // afterwards; the blocking wait is the fallback when they were not ready yet.
+  } else if (warp <= 2) {
+    // ---------------- MMA issuers: A = Q block in TMEM, B = K tile in shared memory ----------------
+    // Two warps, one per accumulator: warp 1 issues the even jobs into accumulator 0, warp 2 the odd jobs
+    // into accumulator 1.  Issuing is not free for the issuing thread (measured: about 50 cycles per
+    // tcgen05.mma and 80 per tcgen05.commit, i.e. some 470 cycles for a job that the tensor pipe executes
+    // in 512) and the barrier handshakes come on top, so one issuer alone cannot keep the pipe busy.
+    // The whole warp runs the loop (waits stay warp-uniform); one elected lane issues.
+    // Every issuer waits for every K tile and releases it (tcgen05.commit after its last job of the tile,
+    // or a plain arrive when it had none), so a stage is refilled only when both are done with it.
+    const int mw = warp - 1;
     const uint32_t idesc = idesc_bf16(128, 128);
     const uint64_t desc0 = smem_desc_sw128(k_smem);
+    const uint32_t full_bar = smem_u32(&bars->tmem_full[mw]), empty_bar = smem_u32(&bars->tmem_empty[mw]);
+    const uint32_t d = tmem_base + LSE_A_COLS + mw * 128;
     bool ok = mbar_wait(smem_u32(&bars->q_ready), 0, abort_flag);
     tc_fence_after();
-    if (ok) ok = mbar_wait(smem_u32(&bars->k_full[0]), 0, abort_flag);               // job 0: stage 0, slot 0
-    // All indices are carried incrementally (no divisions in the loop): any cycle the issuer spends
-    // between two MMAs beyond the queue's depth is a bubble in the tensor pipe.
-    int s = 0, b = 0, slot = 0;
-    uint32_t kpar = 0, epar = 7u;                  // bit i: parity to wait for on tmem_empty[i] (fresh barriers pass with 1)
+    int s = 0, job = 0;
+    uint32_t kpar = 0, epar = 1u;                  // parity to wait for on tmem_empty[mw] (a fresh barrier passes with 1)
     const bool leader = elect_one();
-    for (int job = 0; ok && job < n_jobs; ++job) {
-      int bn = b + 1, sn = s;
-      uint32_t kparn = kpar;
-      if (bn == n_mb) { bn = 0; sn = s + 1; if (sn == S) { sn = 0; kparn ^= 1u; } }
-      const int slotn = slot == LSE_SLOTS - 1 ? 0 : slot + 1;
-      const bool has_next = job + 1 < n_jobs;
-      const uint32_t kfull_n = smem_u32(&bars->k_full[sn]);
-      const uint32_t empty_n = smem_u32(&bars->tmem_empty[slotn]);
-      const uint32_t epar_n = (epar >> slotn) & 1u;
-      bool kready = true, eready = true;
-      if (has_next) {
-        kready = (sn == s) || mbar_test_wait(kfull_n, kparn);
-        eready = mbar_test_wait(empty_n, epar_n);
-      }
+    for (int it = 0; ok && it < n_tiles; ++it) {
+      ok = mbar_wait(smem_u32(&bars->k_full[s]), kpar, abort_flag);
+      if (!ok) break;
       tc_fence_after();
-      if (leader) {
-        const uint64_t desc_s = desc0 + (uint64_t)((s * KTILE_BYTES) >> 4);
-        const uint32_t d = tmem_base + LSE_A_COLS + slot * 128, at = tmem_base + b * 64;
+      const uint64_t desc_s = desc0 + (uint64_t)((s * KTILE_BYTES) >> 4);
+      bool mine = false;
+      for (int b = 0; b < n_mb; ++b, ++job) {
+        if ((job & 1) != mw) continue;
+        ok = mbar_wait(empty_bar, epar, abort_flag);
+        if (!ok) break;
+        epar ^= 1u;
+        tc_fence_after();
+        LSE_TR(0, job, leader);
+        if (leader) {
+          const uint32_t at = tmem_base + b * 64;
 #pragma unroll
-        for (int kk = 0; kk < 8; ++kk)
-          umma_bf16_ts(d, at + kk * 8, desc_s + (uint64_t)(((kk >> 2) * HALF_BYTES + (kk & 3) * 32) >> 4), idesc,
-                       kk > 0 ? 1u : 0u);
-        umma_commit(smem_u32(&bars->tmem_full[slot]));
-        if (bn == 0) umma_commit(smem_u32(&bars->k_empty[s]));
+          for (int kk = 0; kk < 8; ++kk)
+            umma_bf16_ts(d, at + kk * 8, desc_s + (uint64_t)(((kk >> 2) * HALF_BYTES + (kk & 3) * 32) >> 4), idesc,
+                         kk > 0 ? 1u : 0u);
+          umma_commit(full_bar);
+        }
+        LSE_TR(1, job, leader);
+        mine = true;
       }
-      epar ^= 1u << slot;
-      if (has_next) {
-        if (!kready) ok = mbar_wait(kfull_n, kparn, abort_flag);
-        if (ok && !eready) ok = mbar_wait(empty_n, epar_n, abort_flag);
+      if (!ok) break;
+      if (leader) {
+        if (mine) umma_commit(smem_u32(&bars->k_empty[s]));
+        else mbar_arrive(smem_u32(&bars->k_empty[s]));
       }
-      b = bn; s = sn; kpar = kparn; slot = slotn;
+      if (++s == S) { s = 0; kpar ^= 1u; }
     }
     // drain: every MMA issued above has completed before TMEM is freed
     __syncwarp();
-    if (leader) umma_commit(smem_u32(&bars->drained));
+    if (leader) umma_commit(smem_u32(&bars->drained[mw]));
     __syncwarp();
-    mbar_wait(smem_u32(&bars->drained), 0, abort_flag, ok ? WAIT_LIMIT_NS : DRAIN_LIMIT_NS);
+    mbar_wait(smem_u32(&bars->drained[mw]), 0, abort_flag, ok ? WAIT_LIMIT_NS : DRAIN_LIMIT_NS);
     __syncwarp();
   } else {
     // ---------------- epilogue warps ----------------
-    if (ch == 0) {
-      // Q row of this thread -> its TMEM lane, 64 packed columns of block mb (zeros for padding rows)
+    {
+      // Q row (block k, row rib) -> this thread's TMEM lane, 64 packed columns (zeros for padding rows)
+      const int n = k * 128 + rib;
+      const bool live = k < n_mb && n < rows;
       const int w = n / G, g = n - w * G;
       const uint4* src = reinterpret_cast<const uint4*>(
-          a.q + (((int64_t)slab * a.sum_win + w0 + w) * a.n_q_heads + h * G + g) * HD);
-      const uint32_t dst = tmem_base + ((uint32_t)(quarter * 32) << 16) + mb * 64;
+          a.q + (((int64_t)slab * a.sum_win + w0 + (live ? w : 0)) * a.n_q_heads + h * G + (live ? g : 0)) * HD);
+      const uint32_t dst = tmem_base + ((uint32_t)(quarter * 32) << 16) + k * 64;
+      if (k < n_mb) {
 #pragma unroll
-      for (int i = 0; i < 4; ++i) {
-        uint4 x[4];
+        for (int i = 0; i < 4; ++i) {
+          uint4 x[4];
 #pragma unroll
-        for (int k = 0; k < 4; ++k) x[k] = row_ok ? __ldg(src + i * 4 + k) : make_uint4(0, 0, 0, 0);
-        tmem_st16(dst + i * 16, reinterpret_cast<const uint32_t*>(x));
+          for (int j = 0; j < 4; ++j) x[j] = live ? __ldg(src + i * 4 + j) : make_uint4(0, 0, 0, 0);
+          tmem_st16(dst + i * 16, reinterpret_cast<const uint32_t*>(x));
+        }
+        tmem_st_wait();
       }
-      tmem_st_wait();
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(smem_u32(&bars->q_ready));
     }
-    const int w = n / G;
-    const int jmax = a.causal ? (L - W + w) : (L - 1);            // last key this row sees
-    const float c = a.scale_log2;
-    for (int job = mb; mb < n_mb && job < n_jobs; job += n_mb) {
-      const int it = job / n_mb;
-      const int slot = job % LSE_SLOTS;
-      epi_ok = mbar_wait(smem_u32(&bars->tmem_full[slot]), (uint32_t)(job / LSE_SLOTS) & 1u, abort_flag);
-      if (!epi_ok) break;
-      tc_fence_after();
-      const int col0 = (t_begin + it) * TK + ch * 64;              // first key of this thread's columns
-      int n_valid = min(jmax, L - 1) - col0 + 1;
-      n_valid = row_ok ? max(0, min(64, n_valid)) : 0;
-#ifdef ACTKV_EXP_NO_EPI
-      if (false) {
-#else
-      if (__any_sync(0xffffffffu, n_valid > 0)) {
-#endif
-        const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + LSE_A_COLS + slot * 128 + ch * 64;
-        float v[2][32];
-        tmem_ld32(taddr, v[0]);
-        tmem_ld32(taddr + 32, v[1]);
-        tmem_ld_wait();
+    // last key each of this thread's rows sees (padding rows: every key, their sums are dropped)
+    int jm[4];
 #pragma unroll
-        for (int cg = 0; cg < 2; ++cg) {
-          const float* x = v[cg];
-          const int nv = n_valid - cg * 32;       // valid columns of this group for this row
-          if (nv >= 32) {
-            lse_group<POLY>(x, c, m, sum);
-          } else if (nv > 0) {
-            float gm = -INFINITY;
-#pragma unroll
-            for (int i = 0; i < 32; ++i) gm = fmaxf(gm, i < nv ? x[i] : -INFINITY);
-            if (gm > m) { sum = (m == -INFINITY) ? 0.f : sum * exp2f((m - gm) * c); m = gm; }
-            const float mc = m * c;
-#pragma unroll
-            for (int i = 0; i < 32; ++i) sum += (i < nv) ? exp2f(fmaf(x[i], c, -mc)) : 0.f;
-          }
-        }
-      }
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(smem_u32(&bars->tmem_empty[slot]));
+    for (int mb = 0; mb < 4; ++mb) {
+      const int n = mb * 128 + rib;
+      jm[mb] = (a.causal && n < rows) ? (L - W + n / G) : (L - 1);
+      bars->state[grp][mb][half][rib] = make_float2(-INFINITY, 0.f);
     }
-    if (ch == 1) bars->exch[mb * 128 + row_in_blk] = make_float2(m, sum);
+    const int jfast = min(min(jm[0], jm[1]), min(jm[2], jm[3]));
+    const float c = a.scale_log2, c1 = c * (1.f / 252.f);
+    const uint32_t tq = tmem_base + ((uint32_t)(quarter * 32) << 16) + LSE_A_COLS + grp * 128 + half * 64;
+    for (int job = grp; job < n_jobs; job += 2) {
+      const int it = job / n_mb, mb = job - it * n_mb;
+      const int key0 = (t_begin + it) * TK + half * 64;
+      epi_ok = lse_job<NPOLY>(bars, abort_flag, tq, grp, job, mb, &bars->state[grp][mb][half][rib], jfast - key0 + 1, jm, key0, c,
+                              c1, lane);
+      if (!epi_ok) break;
+    }
   }
   // ---------------- teardown ----------------
   tc_fence_before();
   __syncthreads();
-  if (warp >= 2 && ch == 0 && row_ok && epi_ok && !*abort_flag) {
-    // merge the two column halves of the row, store (max in log2 units, sum); (-inf, 0) when the row saw
-    // no key of this chunk
-    const float2 o = bars->exch[mb * 128 + row_in_blk];
-    const float mm = fmaxf(m, o.x);
-    float ss = 0.f;
-    if (mm > -INFINITY) {
-      const float c = a.scale_log2;
-      ss = (m > -INFINITY ? sum * exp2f((m - mm) * c) : 0.f) + (o.x > -INFINITY ? o.y * exp2f((o.x - mm) * c) : 0.f);
+  if (warp >= 3 && k == 0 && !*abort_flag) {
+    // merge the four shares (group, column half) of each row, store (reference in log2 units, sum); (-inf, 0) when the
+    // row saw no key of this chunk
+    const float c = a.scale_log2;
+#pragma unroll
+    for (int mb = 0; mb < 4; ++mb) {
+      const int n = mb * 128 + rib;
+      if (mb < n_mb && n < rows) {
+        float2 o[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) o[i] = bars->state[i >> 1][mb][i & 1][rib];
+        const float mm = fmaxf(fmaxf(o[0].x, o[1].x), fmaxf(o[2].x, o[3].x));
+        float ss = 0.f;
+        if (mm > -INFINITY) {
+#pragma unroll
+          for (int i = 0; i < 4; ++i) ss += o[i].x > -INFINITY ? o[i].y * exp2f((o[i].x - mm) * c) : 0.f;
+        }
+        a.partials[((int64_t)u * a.n_chunks + chunk) * a.rows_max + n] =
+            make_float2(mm == -INFINITY ? mm : mm * a.scale_log2, ss);
+      }
     }
-    a.partials[((int64_t)u * a.n_chunks + chunk) * a.rows_max + n] =
-        make_float2(mm == -INFINITY ? mm : mm * a.scale_log2, ss);
   }
   if (warp == 0 && lane == 0 && *abort_flag) {
     report(a.status, ACTKV_E_TIMEOUT, u, chunk);

@@ -56,6 +56,18 @@ __device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity) {
 // at least half as long in wall time.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag,
                                           uint64_t limit_ns = WAIT_LIMIT_NS) {
+#ifdef ACTKV_EXP_SPIN
+  {
+    const long long t0s = clock64();
+    for (;;) {
+#pragma unroll 1
+      for (int i = 0; i < 1024; ++i)
+        if (mbar_test_wait(bar, parity)) return true;
+      if (*abort_flag) return false;
+      if (clock64() - t0s > (long long)limit_ns * 2) { *abort_flag = 1; return false; }
+    }
+  }
+#endif
   // try_wait parks the thread in hardware (no polling traffic on shared memory, which the MMA operand
   // fetch needs); measured the same or better than spinning on test_wait here.
 #pragma unroll 1
@@ -145,6 +157,34 @@ __device__ __forceinline__ void tmem_ld64(uint32_t taddr, float* v) {
       : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31]), "=r"(r[32]), "=r"(r[33]), "=r"(r[34]), "=r"(r[35]), "=r"(r[36]), "=r"(r[37]), "=r"(r[38]), "=r"(r[39]), "=r"(r[40]), "=r"(r[41]), "=r"(r[42]), "=r"(r[43]), "=r"(r[44]), "=r"(r[45]), "=r"(r[46]), "=r"(r[47]), "=r"(r[48]), "=r"(r[49]), "=r"(r[50]), "=r"(r[51]), "=r"(r[52]), "=r"(r[53]), "=r"(r[54]), "=r"(r[55]), "=r"(r[56]), "=r"(r[57]), "=r"(r[58]), "=r"(r[59]), "=r"(r[60]), "=r"(r[61]), "=r"(r[62]), "=r"(r[63])
       : "r"(taddr));
 }
+__device__ __forceinline__ void tmem_ld4(uint32_t taddr, float* v) {
+  uint32_t* r = reinterpret_cast<uint32_t*>(v);
+  asm volatile("tcgen05.ld.sync.aligned.32x32b.x4.b32 {%0, %1, %2, %3}, [%4];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
+               : "r"(taddr));
+}
+__device__ __forceinline__ void tmem_ld8(uint32_t taddr, float* v) {
+  uint32_t* r = reinterpret_cast<uint32_t*>(v);
+  asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])
+               : "r"(taddr));
+}
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, float* v) {
+  uint32_t* r = reinterpret_cast<uint32_t*>(v);
+  asm volatile("tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+               : "r"(taddr));
+}
+// N consecutive columns (a multiple of 4, at most 64) as a few power-of-two loads
+template <int N>
+__device__ __forceinline__ void tmem_ld_n(uint32_t taddr, float* v) {
+  static_assert(N % 4 == 0 && N >= 0 && N <= 64, "column count");
+  if constexpr (N >= 64) { tmem_ld64(taddr, v); }
+  else if constexpr (N >= 32) { tmem_ld32(taddr, v); tmem_ld_n<N - 32>(taddr + 32, v + 32); }
+  else if constexpr (N >= 16) { tmem_ld16(taddr, v); tmem_ld_n<N - 16>(taddr + 16, v + 16); }
+  else if constexpr (N >= 8) { tmem_ld8(taddr, v); tmem_ld_n<N - 8>(taddr + 8, v + 8); }
+  else if constexpr (N >= 4) { tmem_ld4(taddr, v); }
+}
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 // 16 consecutive 32-bit columns of this thread's TMEM lane <- registers
 __device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t* r) {
@@ -202,6 +242,18 @@ __device__ __forceinline__ float max_of(const float* v) {       // max of v[0..N
   else if constexpr (N == 4) return fmaxf(fmax3(v[0], v[1], v[2]), v[3]);
   else if constexpr (N == 8) return fmaxf(fmax3(fmax3(v[0], v[1], v[2]), fmax3(v[3], v[4], v[5]), v[6]), v[7]);
   else return fmaxf(max_of<N / 2>(v), max_of<N / 2>(v + N / 2));
+}
+
+// max of v[0..N) for any N >= 1, as a tree of three-input max
+template <int N>
+__device__ __forceinline__ float max_n(const float* v) {
+  if constexpr (N == 1) return v[0];
+  else if constexpr (N == 2) return fmaxf(v[0], v[1]);
+  else if constexpr (N == 3) return fmax3(v[0], v[1], v[2]);
+  else {
+    constexpr int A = (N + 2) / 3, B = (N - A + 1) / 2, C = N - A - B;
+    return fmax3(max_n<A>(v), max_n<B>(v + A), max_n<C>(v + A + B));
+  }
 }
 
 // Shared-memory operand descriptor: K-major tile, 128-byte swizzle, rows of 64 bf16 (128 B), eight-row

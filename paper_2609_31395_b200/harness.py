@@ -7,6 +7,7 @@ and passes pointers.
 """
 from __future__ import annotations
 
+import os
 from dataclasses import dataclass
 from typing import Optional
 
@@ -167,9 +168,13 @@ class Compressor:
         call reads the old tables; compaction writes fresh pages only.
         `marks`: optional callable(name, stream).  Returns the number of kernels launched."""
         NL, Hkv, s = self.pd.n_layers, self.pd.n_kv_heads, self.sz
-        main = torch.cuda.current_stream()
+        cur = torch.cuda.current_stream()
         if not hasattr(self, "_aux"):
-            self._aux = torch.cuda.Stream(device=self.dev)
+            # The score kernels run on a high-priority stream, select + compact on a low-priority one: a
+            # score CTA is placed whenever it fits, the others only ever take what a score CTA leaves over
+            # on its SM (registers, shared memory), so they run beside the score kernels instead of in turns.
+            self._main = torch.cuda.Stream(device=self.dev, priority=int(os.environ.get("ACTKV_MAIN_PRIO", "-1")))
+            self._aux = torch.cuda.Stream(device=self.dev, priority=int(os.environ.get("ACTKV_AUX_PRIO", "0")))
             self._score2 = [self.score, torch.empty_like(self.score)]
             self._sel2 = [self.sel_idx, torch.empty_like(self.sel_idx)]
             self._ev_score = [torch.cuda.Event(), torch.cuda.Event()]
@@ -177,7 +182,8 @@ class Compressor:
             self._ev_done = torch.cuda.Event()
             if self.lse is None and lse_in is None:
                 self.lse = torch.empty((NL, s.sum_win, self.n_q_heads), dtype=torch.float32, device=self.dev)
-        aux = self._aux
+        aux, main = self._aux, self._main
+        main.wait_stream(cur)
         mark = marks if marks is not None else (lambda name, stream: None)
         B.actkv_keep_indptr(self.seq_len, budget, s.n_req, self.keep_indptr, main)
         launches = 1
@@ -211,6 +217,7 @@ class Compressor:
             launches += (3 if lse_in is None else 1) + 1 + 2 + (1 if l1 == NL else 0)
         self._ev_done.record(aux)
         main.wait_event(self._ev_done)
+        cur.wait_stream(main)
         return launches
 
     def check_status(self):

@@ -150,6 +150,28 @@ def test_long_request_many_chunks():
     _full_check(synth.generate(wl, DEV))
 
 
+def test_logits_that_keep_growing_move_the_lse_reference():
+    """Keys arranged so that every row's logits climb by hundreds of log2 units along the request: the
+    LSE pass keeps no running maximum, so its reference must be moved again and again (and 2^x saturates
+    in between).  Scores of the early keys underflow, the late ones carry the mass."""
+    wl = synth.Workload("climb", 1, 2, 4, [3000, 700], [32, 32], [600, 200], table_style="fragmented", seed=11,
+                        poison_tail=True)
+    inst = synth.generate(wl, DEV)
+    P, G = wl.page_size, wl.group
+    win = inst.win_indptr.cpu().numpy()
+    for r, L in enumerate(wl.seq_lens):
+        pages = inst.page_table[r, : -(-L // P)].long()
+        alpha = torch.linspace(-5.0, 40.0, L, device=DEV)
+        for h in range(wl.n_kv_heads):
+            qbar = inst.q[0, win[r]:win[r + 1], h * G:(h + 1) * G].float().mean(dim=(0, 1))       # [D]
+            rows = (alpha[:, None] * qbar[None, :]).to(torch.bfloat16)                             # [L, D]
+            pad = torch.zeros((len(pages) * P - L, rows.shape[1]), dtype=torch.bfloat16, device=DEV)
+            inst.pool[0, 0, pages, :, h, :] = torch.cat([rows, pad]).view(len(pages), P, -1)
+    out = _full_check(inst)
+    lse = out["lse"]
+    assert np.nanmax(lse) > 100.0                      # the rows really reached large logits
+
+
 def test_duplicate_keys_make_exact_ties():
     """Duplicated key rows give bit-equal scores; the lower index must win at the threshold."""
     wl = synth.Workload("dups", 1, 2, 4, [512], [16], [100], table_style="permutation", seed=9, plant_frac=0.0)
