@@ -90,16 +90,17 @@ static int score_impl(int mode, const actkv_pool_t* pool, const actkv_tables_t* 
   a.sum_tok = sum_tok;
   a.rows_max = lay.rows_max;
   // Keys per LSE partial.  A CTA pays a fixed cost (operand set-up, pipeline fill and drain), so chunks
-  // are as long as they can be while there are still several CTAs per SM: the largest multiple of the
-  // minimum chunk that leaves at least 20 x 148 work items (never more chunks than the workspace holds).
+  // are as long as they can be while there are still many CTAs per SM (the last wave of a launch is
+  // partly empty): whole key tiles, about equal, at least 20 x 148 work items and never more chunks
+  // than the workspace holds.
   {
     const int64_t units_ = (int64_t)(layer_end - layer_begin) * Hkv * R;
-    const int64_t row_groups = 1;                  // a CTA of either path covers all rows of its unit
-    int n_chunks = (int)((20 * 148 + units_ * row_groups - 1) / (units_ * row_groups));
+    int n_chunks = (int)((20 * 148 + units_ - 1) / units_);       // a CTA covers all rows of its unit
     if (n_chunks < 1) n_chunks = 1;
     if (n_chunks > lay.n_chunks) n_chunks = lay.n_chunks;
     int chunk = (max_tok + n_chunks - 1) / n_chunks;
-    chunk = (chunk + LSE_CHUNK - 1) / LSE_CHUNK * LSE_CHUNK;
+    chunk = (chunk + 127) / 128 * 128;             // whole key tiles, about equal work per chunk
+    if (chunk < LSE_CHUNK) chunk = LSE_CHUNK;
     a.lse_chunk = chunk;
     a.n_chunks = (max_tok + chunk - 1) / chunk;
   }

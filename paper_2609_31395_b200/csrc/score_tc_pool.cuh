@@ -15,7 +15,7 @@ namespace actkv {
 namespace tc {
 
 constexpr int POOL_EPI_WARPS = 8;
-constexpr int POOL_THREADS = (2 + POOL_EPI_WARPS) * 32;     // producer, MMA issuer, epilogue
+constexpr int POOL_THREADS = (3 + POOL_EPI_WARPS) * 32;     // producer, two MMA issuers, epilogue
 
 struct PoolBarriers {
   uint64_t k_full[8];
@@ -25,7 +25,7 @@ struct PoolBarriers {
   uint64_t tmem_empty[2];
   uint64_t part_full;         // warpgroup 1 -> warpgroup 0: partial sums of a tile are in `exch`
   uint64_t part_empty;        // warpgroup 0 -> warpgroup 1: `exch` has been read
-  uint64_t drained;
+  uint64_t drained[2];
   uint32_t tmem_base;
   int abort_flag;
   float exch[TK];
@@ -121,7 +121,7 @@ score_tc_pool_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_cons
     return;
   }
   if (threadIdx.x == 0) {
-    for (int s = 0; s < S; ++s) { mbar_init(smem_u32(&bars->k_full[s]), 1); mbar_init(smem_u32(&bars->k_empty[s]), 1); }
+    for (int s = 0; s < S; ++s) { mbar_init(smem_u32(&bars->k_full[s]), 1); mbar_init(smem_u32(&bars->k_empty[s]), 2); }
     mbar_init(smem_u32(&bars->q_full), 1);
     for (int b = 0; b < 2; ++b) {
       mbar_init(smem_u32(&bars->tmem_full[b]), 1);
@@ -129,7 +129,8 @@ score_tc_pool_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_cons
     }
     mbar_init(smem_u32(&bars->part_full), POOL_EPI_WARPS / 2);
     mbar_init(smem_u32(&bars->part_empty), POOL_EPI_WARPS / 2);
-    mbar_init(smem_u32(&bars->drained), 1);
+    mbar_init(smem_u32(&bars->drained[0]), 1);
+    mbar_init(smem_u32(&bars->drained[1]), 1);
     bars->abort_flag = 0;
     fence_barrier_init();
   }
@@ -183,67 +184,63 @@ score_tc_pool_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_cons
       }
       if ((it & 3) == 3) pid = pid_next;
     }
-  } else if (warp == 1) {
-    // ---------------- MMA issuer: D[key, row] = K Q^T ----------------
-    // The whole warp runs the loop (waits and descriptor arithmetic stay warp-uniform, so they can
-    // live in uniform registers); one elected lane issues the tcgen05 instructions.
-    // The tensor pipe's queue is shallow: whatever the issuing warp spends between two jobs (a successful
-    // barrier wait costs 100-200 cycles) is idle time of the pipe.  So the barriers of job j+1 are polled
-    // (mbarrier.test_wait, non-blocking) BEFORE the MMAs of job j are issued and the answers are only read
-    // afterwards; the blocking wait is the fallback when they were not ready yet.
-    // All indices are carried incrementally (no divisions in the loop): any cycle the issuer spends
-    // between two MMAs beyond the queue's depth is a bubble in the tensor pipe.
+  } else if (warp <= 2) {
+    // ---------------- MMA issuers: D[key, row] = K Q^T ----------------
+    // Two warps, one per accumulator: warp 1 issues the even jobs, warp 2 the odd ones.  Issuing costs the
+    // issuing thread about 50 cycles per tcgen05.mma and 80 per tcgen05.commit, and the barrier
+    // handshakes come on top; with one issuer that time showed up as idle time of the tensor pipe.
+    // The whole warp runs the loop (waits stay warp-uniform); one elected lane issues.  Every issuer
+    // waits for every K tile and releases it (tcgen05.commit after its last job of the tile, or a plain
+    // arrive when it had none), so a stage is refilled only when both are done with it.
+    const int mw = warp - 1;
     const uint64_t kdesc0 = smem_desc_sw128(k_smem);
     const uint64_t qdesc0 = smem_desc_sw128(q_smem);
     // MMA width of each row chunk: its live rows rounded up to 16 (a decode-step update has only G)
     const int n0 = rows <= 256 ? max(16, (rows + 15) & ~15) : 256;
     const int n1 = max(16, (rows - 256 + 15) & ~15);
     const uint32_t idesc_c[2] = {idesc_bf16(128, n0), idesc_bf16(128, n1)};
+    const uint32_t full_bar = smem_u32(&bars->tmem_full[mw]), empty_bar = smem_u32(&bars->tmem_empty[mw]);
     bool ok = mbar_wait(smem_u32(&bars->q_full), 0, abort_flag);
-    if (ok) ok = mbar_wait(smem_u32(&bars->k_full[0]), 0, abort_flag);               // job 0: stage 0, accumulator 0
-    int s = 0, rc = 0;
-    uint32_t kpar = 0, epar0 = 1, epar1 = 1;       // parities to wait for (a fresh "empty" barrier passes with 1)
+    int s = 0, job = 0;
+    uint32_t kpar = 0, epar = 1u;                  // parity to wait for on tmem_empty[mw] (a fresh barrier passes with 1)
     const bool leader = elect_one();
-    for (int job = 0; ok && job < n_jobs; ++job) {
-      const int b = job & 1;
-      int rcn = rc + 1, sn = s;
-      uint32_t kparn = kpar;
-      if (rcn == n_rc) { rcn = 0; sn = s + 1; if (sn == S) { sn = 0; kparn ^= 1u; } }
-      const bool has_next = job + 1 < n_jobs;
-      const uint32_t kfull_n = smem_u32(&bars->k_full[sn]);
-      const uint32_t empty_n = smem_u32(&bars->tmem_empty[b ^ 1]);
-      const uint32_t epar_n = b ? epar0 : epar1;
-      bool kready = true, eready = true;
-      if (has_next) {
-        kready = (sn == s) || mbar_test_wait(kfull_n, kparn);
-        eready = mbar_test_wait(empty_n, epar_n);
-      }
+    for (int it = 0; ok && it < n_tiles; ++it) {
+      ok = mbar_wait(smem_u32(&bars->k_full[s]), kpar, abort_flag);
+      if (!ok) break;
       tc_fence_after();
-      if (leader) {
-        const uint64_t adesc_s = kdesc0 + (uint64_t)((s * KTILE_BYTES) >> 4);
-        const uint64_t bdesc_c = qdesc0 + (uint64_t)((rc * 2 * QBLK_BYTES) >> 4);
+      const uint64_t adesc_s = kdesc0 + (uint64_t)((s * KTILE_BYTES) >> 4);
+      bool mine = false;
+      for (int rc = 0; rc < n_rc; ++rc, ++job) {
+        if ((job & 1) != mw) continue;
+        ok = mbar_wait(empty_bar, epar, abort_flag);
+        if (!ok) break;
+        epar ^= 1u;
+        tc_fence_after();
+        if (leader) {
+          const uint64_t bdesc_c = qdesc0 + (uint64_t)((rc * 2 * QBLK_BYTES) >> 4);
 #pragma unroll
-        for (int kk = 0; kk < 8; ++kk)
-          umma_bf16(tmem_base + b * 256, adesc_s + (uint64_t)(((kk >> 2) * HALF_BYTES + (kk & 3) * 32) >> 4),
-                    bdesc_c + (uint64_t)(((kk >> 2) * QBLK_BYTES + (kk & 3) * 32) >> 4), idesc_c[rc], kk > 0 ? 1u : 0u);
-        umma_commit(smem_u32(&bars->tmem_full[b]));
-        if (rcn == 0) umma_commit(smem_u32(&bars->k_empty[s]));
+          for (int kk = 0; kk < 8; ++kk)
+            umma_bf16(tmem_base + mw * 256, adesc_s + (uint64_t)(((kk >> 2) * HALF_BYTES + (kk & 3) * 32) >> 4),
+                      bdesc_c + (uint64_t)(((kk >> 2) * QBLK_BYTES + (kk & 3) * 32) >> 4), idesc_c[rc], kk > 0 ? 1u : 0u);
+          umma_commit(full_bar);
+        }
+        mine = true;
       }
-      if (b) epar1 ^= 1u; else epar0 ^= 1u;
-      if (has_next) {
-        if (!kready) ok = mbar_wait(kfull_n, kparn, abort_flag);
-        if (ok && !eready) ok = mbar_wait(empty_n, epar_n, abort_flag);
+      if (!ok) break;
+      if (leader) {
+        if (mine) umma_commit(smem_u32(&bars->k_empty[s]));
+        else mbar_arrive(smem_u32(&bars->k_empty[s]));
       }
-      rc = rcn; s = sn; kpar = kparn;
+      if (++s == S) { s = 0; kpar ^= 1u; }
     }
     __syncwarp();
-    if (leader) umma_commit(smem_u32(&bars->drained));
+    if (leader) umma_commit(smem_u32(&bars->drained[mw]));
     __syncwarp();
-    mbar_wait(smem_u32(&bars->drained), 0, abort_flag, ok ? WAIT_LIMIT_NS : DRAIN_LIMIT_NS);
+    mbar_wait(smem_u32(&bars->drained[mw]), 0, abort_flag, ok ? WAIT_LIMIT_NS : DRAIN_LIMIT_NS);
     __syncwarp();
   } else {
     // ---------------- epilogue: one key per thread, jobs of this warpgroup's parity ----------------
-    const int wg = (warp - 2) >> 2;               // 0 or 1 = accumulator it drains
+    const int wg = (warp - 3) >> 2;               // 0 or 1 = accumulator it drains
     const int quarter = warp & 3;                 // TMEM lane quarter this warp may read
     const float c = a.scale_log2;
     const float inv_w = 1.0f / (float)W;
