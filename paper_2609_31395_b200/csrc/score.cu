@@ -109,7 +109,10 @@ static int score_impl(int mode, const actkv_pool_t* pool, const actkv_tables_t* 
   a.causal = causal;
   a.acc_steps = acc_steps;
   const int64_t units = (int64_t)nls * Hkv * R;
-  const bool use_tc = score_tc_supported(pool, G, max_win, sm_scale, q, acc_steps ? 1 : 64);
+  // (the streaming update keeps a running mean in place, which the row-group launches of a window above
+  // 512 rows would break: such calls take the FMA path)
+  const bool use_tc = score_tc_supported(pool, G, max_win, sm_scale, q, acc_steps ? 1 : 64) &&
+                      !(acc_steps != nullptr && max_win * G > tc::MAX_ROWS);
 
   const float* lse = lse_in;
   if (mode & 1) {

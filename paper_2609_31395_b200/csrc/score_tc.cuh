@@ -21,6 +21,7 @@
 // This file: tensor-map creation and launch configuration (host side).
 #pragma once
 
+#include <algorithm>
 #include <cstdlib>
 
 #include "score_tc_lse.cuh"
@@ -81,7 +82,8 @@ constexpr size_t SMEM_LIMIT = 232448;        // 227 KB of dynamic shared memory 
 }  // namespace tc
 
 // The tensor-core path takes: page 16, head_dim 128, packed [slot][head][dim] pages, 128-byte aligned
-// base, power-of-two group size <= 32, min_rows <= window x group rows <= 512, positive softmax scale.
+// base, power-of-two group size <= 32, min_rows <= window x group rows <= 4096 (a CTA handles up to 512;
+// more are taken in groups of 512 rows), positive softmax scale.
 // The full score (LSE + pooled pass) takes it from 64 rows up; the streaming update, which runs the
 // pooled pass alone and is bound by the K reads, from a single row.
 inline bool score_tc_supported(const actkv_pool_t* p, int G, int max_win, float sm_scale, const void* q,
@@ -92,7 +94,8 @@ inline bool score_tc_supported(const actkv_pool_t* p, int G, int max_win, float 
   if (((uintptr_t)p->base & 127) || ((uintptr_t)q & 127) || (p->stride_layer % 8) != 0) return false;
   if (G < 1 || G > 32 || (G & (G - 1)) != 0) return false;
   const int rows = max_win * G;
-  if (rows < min_rows || rows > tc::MAX_ROWS) return false;
+  if (rows < min_rows || rows > tc::MAX_ROWS_TOTAL) return false;
+  if (rows > tc::MAX_ROWS && tc::MAX_ROWS % G != 0) return false;
   if (!(sm_scale > 0.f)) return false;
   if (getenv("ACTKV_FORCE_FMA") != nullptr) return false;
   return tc::encode_fn() != nullptr;
@@ -109,17 +112,17 @@ inline int score_tc_launch_lse_c(const CUtensorMap& kmap, const tc::TcArgs& ta, 
 
 inline int score_tc_launch_lse(ScoreArgs& a, const actkv_pool_t* pool, int max_tok, int max_win, cudaStream_t s) {
   (void)max_tok;
-  (void)max_win;
   CUtensorMap kmap, qmap;
   if (!tc::make_maps(pool, a.q, a.n_layers_sub, a.sum_win, a.n_q_heads, a.group, &kmap, &qmap)) return ACTKV_E_CUDA;
   tc::TcArgs ta;
   ta.a = a;
-  ta.n_rg = 1;
+  ta.n_rg = (max_win * a.group + tc::MAX_ROWS - 1) / tc::MAX_ROWS;
+  ta.row_begin = 0;
   ta.n_stages = 6;
   ta.tiles_per_cta = 0;
   ta.n_kchunks = 0;
   const int64_t units = (int64_t)a.n_layers_sub * a.pool.n_kv_heads * a.tab.n_req;
-  const int64_t grid = units * a.n_chunks;
+  const int64_t grid = units * a.n_chunks * ta.n_rg;
   if (grid > 0x7fffffffLL) return ACTKV_E_INVALID;
   const size_t smem = (size_t)ta.n_stages * tc::KTILE_BYTES + sizeof(tc::LseBarriers);
   // columns of every 8 that take the polynomial exp2 (tuning knob; the default is what the bench uses)
@@ -149,7 +152,8 @@ inline int score_tc_launch_score(ScoreArgs& a, const actkv_pool_t* pool, int max
   if (!tc::make_maps(pool, a.q, a.n_layers_sub, a.sum_win, a.n_q_heads, a.group, &kmap, &qmap)) return ACTKV_E_CUDA;
   tc::TcArgs ta;
   ta.a = a;
-  const int rows_pad = (max_win * a.group + 127) & ~127;
+  const int rows_all = max_win * a.group;
+  const int rows_pad = (std::min(rows_all, tc::MAX_ROWS) + 127) & ~127;      // per launch
   const int n_rc = (rows_pad + 255) / 256;
   const size_t q_bytes = (size_t)n_rc * 2 * tc::QBLK_BYTES;
   const size_t fixed = q_bytes + tc::MAX_ROWS * 4 + sizeof(tc::PoolBarriers);
@@ -169,15 +173,23 @@ inline int score_tc_launch_score(ScoreArgs& a, const actkv_pool_t* pool, int max
   const int64_t grid = units * ta.n_kchunks;
   if (grid > 0x7fffffffLL) return ACTKV_E_INVALID;
   const size_t smem = fixed + (size_t)stages * tc::KTILE_BYTES;
-  switch (a.group) {
-    case 1: return score_tc_launch_pool_g<1>(kmap, qmap, ta, (unsigned)grid, smem, s);
-    case 2: return score_tc_launch_pool_g<2>(kmap, qmap, ta, (unsigned)grid, smem, s);
-    case 4: return score_tc_launch_pool_g<4>(kmap, qmap, ta, (unsigned)grid, smem, s);
-    case 8: return score_tc_launch_pool_g<8>(kmap, qmap, ta, (unsigned)grid, smem, s);
-    case 16: return score_tc_launch_pool_g<16>(kmap, qmap, ta, (unsigned)grid, smem, s);
-    case 32: return score_tc_launch_pool_g<32>(kmap, qmap, ta, (unsigned)grid, smem, s);
-    default: return ACTKV_E_INVALID;
+  // a window of more than MAX_ROWS rows: one launch per group of MAX_ROWS rows (whole action tokens), in
+  // stream order; the first writes the score, the others add their share of the mean
+  for (int row_begin = 0; row_begin < rows_all; row_begin += tc::MAX_ROWS) {
+    ta.row_begin = row_begin;
+    int rc = ACTKV_E_INVALID;
+    switch (a.group) {
+      case 1: rc = score_tc_launch_pool_g<1>(kmap, qmap, ta, (unsigned)grid, smem, s); break;
+      case 2: rc = score_tc_launch_pool_g<2>(kmap, qmap, ta, (unsigned)grid, smem, s); break;
+      case 4: rc = score_tc_launch_pool_g<4>(kmap, qmap, ta, (unsigned)grid, smem, s); break;
+      case 8: rc = score_tc_launch_pool_g<8>(kmap, qmap, ta, (unsigned)grid, smem, s); break;
+      case 16: rc = score_tc_launch_pool_g<16>(kmap, qmap, ta, (unsigned)grid, smem, s); break;
+      case 32: rc = score_tc_launch_pool_g<32>(kmap, qmap, ta, (unsigned)grid, smem, s); break;
+      default: break;
+    }
+    if (rc != ACTKV_OK) return rc;
   }
+  return ACTKV_OK;
 }
 
 }  // namespace actkv

@@ -184,16 +184,19 @@ score_tc_lse_kernel(const __grid_constant__ CUtensorMap kmap, const TcArgs ta) {
   extern __shared__ __align__(1024) uint8_t smem[];
   const ScoreArgs& a = ta.a;
   const int R = a.tab.n_req, Hkv = a.pool.n_kv_heads, G = a.group;
-  const int u = blockIdx.x / a.n_chunks;
-  const int chunk = blockIdx.x - u * a.n_chunks;
+  int idx = blockIdx.x;
+  const int chunk = idx % a.n_chunks; idx /= a.n_chunks;
+  const int rg = idx % ta.n_rg;                          // row group: rows [row0, row0 + MAX_ROWS) of the unit
+  const int u = idx / ta.n_rg;
   const int r = u % R, h = (u / R) % Hkv, slab = u / (R * Hkv);
   const int L = a.tab.seq_len[r];
   const int w0 = a.win_indptr[r], W = a.win_indptr[r + 1] - w0;
-  const int rows = W * G;
+  const int row0 = rg * MAX_ROWS;
+  const int rows = min(W * G - row0, MAX_ROWS);          // rows of this CTA
   const int key_begin = chunk * a.lse_chunk;
-  if (key_begin >= L) return;
+  if (key_begin >= L || (rg > 0 && rows <= 0)) return;
   if (W <= 0 || (a.causal && W > L)) {
-    if (threadIdx.x == 0 && chunk == 0) report(a.status, ACTKV_E_INVALID, r, W);
+    if (threadIdx.x == 0 && chunk == 0 && rg == 0) report(a.status, ACTKV_E_INVALID, r, W);
     return;
   }
   const int n_mb = (rows + 127) / 128;                   // 1..4 (checked by the host)
@@ -338,7 +341,7 @@ score_tc_lse_kernel(const __grid_constant__ CUtensorMap kmap, const TcArgs ta) {
       // Q row (block k, row rib) -> this thread's TMEM lane, 64 packed columns (zeros for padding rows)
       const int n = k * 128 + rib;
       const bool live = k < n_mb && n < rows;
-      const int w = n / G, g = n - w * G;
+      const int w = (row0 + n) / G, g = (row0 + n) % G;
       const uint4* src = reinterpret_cast<const uint4*>(
           a.q + (((int64_t)slab * a.sum_win + w0 + (live ? w : 0)) * a.n_q_heads + h * G + (live ? g : 0)) * HD);
       const uint32_t dst = tmem_base + ((uint32_t)(quarter * 32) << 16) + k * 64;
@@ -361,7 +364,7 @@ score_tc_lse_kernel(const __grid_constant__ CUtensorMap kmap, const TcArgs ta) {
 #pragma unroll
     for (int mb = 0; mb < 4; ++mb) {
       const int n = mb * 128 + rib;
-      jm[mb] = (a.causal && n < rows) ? (L - W + n / G) : (L - 1);
+      jm[mb] = (a.causal && n < rows) ? (L - W + (row0 + n) / G) : (L - 1);
       bars->state[grp][mb][half][rib] = make_float2(-INFINITY, 0.f);
     }
     const int jfast = min(min(jm[0], jm[1]), min(jm[2], jm[3]));
@@ -395,7 +398,7 @@ score_tc_lse_kernel(const __grid_constant__ CUtensorMap kmap, const TcArgs ta) {
 #pragma unroll
           for (int i = 0; i < 4; ++i) ss += o[i].x > -INFINITY ? o[i].y * exp2f((o[i].x - mm) * c) : 0.f;
         }
-        a.partials[((int64_t)u * a.n_chunks + chunk) * a.rows_max + n] =
+        a.partials[((int64_t)u * a.n_chunks + chunk) * a.rows_max + row0 + n] =
             make_float2(mm == -INFINITY ? mm : mm * a.scale_log2, ss);
       }
     }

@@ -91,9 +91,13 @@ score_tc_pool_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_cons
   const int r = u % R, h = (u / R) % Hkv, slab = u / (R * Hkv);
   const int L = a.tab.seq_len[r];
   const int w0 = a.win_indptr[r], W = a.win_indptr[r + 1] - w0;
-  const int rows = W * G;
+  // rows of this launch: [row_begin, row_begin + rows) of the unit's W*G; a window of more than MAX_ROWS
+  // rows is taken MAX_ROWS (a whole number of action tokens) per launch, later launches add to the score
+  const int row_begin = ta.row_begin, w_begin = row_begin / G;
+  const int rows = min(W * G - row_begin, MAX_ROWS);
   const int t_begin = kchunk * ta.tiles_per_cta;
   if (t_begin * TK >= L) return;
+  if (row_begin > 0 && rows <= 0) return;                   // this request's window ends before this row group
   if (W <= 0 && a.acc_steps != nullptr) return;            // accumulate mode: a request outside its action region
   if (W <= 0 || (a.causal && W > L)) {
     if (threadIdx.x == 0 && kchunk == 0) report(a.status, ACTKV_E_INVALID, r, W);
@@ -136,7 +140,7 @@ score_tc_pool_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_cons
   }
   {
     // -lse of every row in log2 units; padding rows get -inf so that s*c + nlse drops out of the max
-    const float* lse_base = a.lse + ((int64_t)slab * a.sum_win + w0) * a.n_q_heads + h * G;
+    const float* lse_base = a.lse + ((int64_t)slab * a.sum_win + w0 + w_begin) * a.n_q_heads + h * G;
     for (int n = threadIdx.x; n < rows_pad; n += blockDim.x)
       nlse[n] = (n < rows) ? -lse_base[(int64_t)(n / G) * a.n_q_heads + (n % G)] * kLog2e : -INFINITY;
   }
@@ -155,7 +159,7 @@ score_tc_pool_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_cons
     const int layer = a.layer_begin + slab;
     if (lane == 0) {
       mbar_expect_tx(smem_u32(&bars->q_full), (uint32_t)n_qblk * QBLK_BYTES);
-      const int wrow = slab * a.sum_win + w0;
+      const int wrow = slab * a.sum_win + w0 + w_begin;
       for (int qb = 0; qb < n_qblk; ++qb)
         for (int hf = 0; hf < 2; ++hf)
           tma_load_3d(q_smem + (qb >> 1) * 2 * QBLK_BYTES + hf * QBLK_BYTES + (qb & 1) * HALF_BYTES, &qmap,
@@ -258,9 +262,9 @@ score_tc_pool_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_cons
       float acc = 0.f;
 #ifndef ACTKV_EXP_NO_EPI
 #ifdef ACTKV_EXP_NO_NLSE
-      pool_job<G>(taddr, nlse, 0 * n_cg + n_cg, (rc * 256) / G, w_min, W, c, acc, smem_u32(&bars->tmem_empty[wg]), lane);
+      pool_job<G>(taddr, nlse, 0 * n_cg + n_cg, w_begin + (rc * 256) / G, w_min, W, c, acc, smem_u32(&bars->tmem_empty[wg]), lane);
 #else
-      pool_job<G>(taddr, nlse + rc * 256, n_cg, (rc * 256) / G, w_min, W, c, acc, smem_u32(&bars->tmem_empty[wg]), lane);
+      pool_job<G>(taddr, nlse + rc * 256, n_cg, w_begin + (rc * 256) / G, w_min, W, c, acc, smem_u32(&bars->tmem_empty[wg]), lane);
 #endif
 #else
       tc_fence_before();
@@ -268,7 +272,7 @@ score_tc_pool_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_cons
       if (lane == 0) mbar_arrive(smem_u32(&bars->tmem_empty[wg]));
 #endif
       if (n_rc == 1) {
-        if (key < L) store_pooled(a, r, out + key, acc, acc * inv_w, W);
+        if (key < L) { if (row_begin > 0) out[key] += acc * inv_w; else store_pooled(a, r, out + key, acc, acc * inv_w, W); }
       } else if (wg == 1) {
         // partial over the second row chunk: hand it to warpgroup 0 once it has read the previous tile's
         if (!mbar_wait(smem_u32(&bars->part_empty), ((uint32_t)it & 1u) ^ 1u, abort_flag)) break;
@@ -280,7 +284,7 @@ score_tc_pool_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_cons
         acc += bars->exch[quarter * 32 + lane];
         __syncwarp();
         if (lane == 0) mbar_arrive(smem_u32(&bars->part_empty));
-        if (key < L) store_pooled(a, r, out + key, acc, acc * inv_w, W);
+        if (key < L) { if (row_begin > 0) out[key] += acc * inv_w; else store_pooled(a, r, out + key, acc, acc * inv_w, W); }
       }
     }
   }

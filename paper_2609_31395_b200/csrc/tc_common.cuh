@@ -13,7 +13,8 @@ constexpr int HD = 128;                      // head dim
 constexpr uint32_t KTILE_BYTES = TK * HD * 2;        // 32 KB: [2 halves][128 keys][64 bf16]
 constexpr uint32_t HALF_BYTES = TK * 64 * 2;         // 16 KB
 constexpr uint32_t QBLK_BYTES = 128 * HD * 2;        // 32 KB per 128 rows
-constexpr int MAX_ROWS = 512;                // window x group rows (padded to 128) held in smem
+constexpr int MAX_ROWS = 512;                // window x group rows (padded to 128) one CTA handles
+constexpr int MAX_ROWS_TOTAL = 4096;         // ... per unit: more than MAX_ROWS are taken in groups of MAX_ROWS
 constexpr uint64_t WAIT_LIMIT_NS = 2000000000ull;    // bounded waits give up after 2 s
 constexpr uint64_t DRAIN_LIMIT_NS = 50000000ull;     // waits while tearing down after a give-up
 
@@ -275,7 +276,8 @@ struct TcArgs {
   ScoreArgs a;
   int32_t tiles_per_cta;     // pooled-score pass: key tiles per CTA
   int32_t n_kchunks;         // pooled-score pass: CTAs per unit
-  int32_t n_rg;              // LSE pass: 256-row groups per unit (1 or 2)
+  int32_t n_rg;              // LSE pass: groups of MAX_ROWS rows per unit (a grid dimension)
+  int32_t row_begin;         // pooled-score pass: first row of this launch's row group (multiple of MAX_ROWS)
   int32_t n_stages;          // K stages in shared memory
 };
 

@@ -144,6 +144,16 @@ def test_window_rows_at_tensor_tile_sizes():
         _full_check(synth.generate(wl, DEV))
 
 
+@pytest.mark.parametrize("causal", [False, True])
+def test_window_rows_above_one_cta(causal):
+    """window x group above 512 rows: the score kernels take the rows in groups of 512 (whole action
+    tokens); second group full, partial, and absent for the request with the short window."""
+    for W, G in [(64, 16), (100, 8), (130, 4), (40, 32)]:
+        wl = synth.Workload("rows+", 1, 2, G, [900, 300], [W, max(1, W // 3)], [300, 80], table_style="permutation",
+                            causal=causal, seed=W * 7 + G, poison_tail=True)
+        _full_check(synth.generate(wl, DEV))
+
+
 def test_long_request_many_chunks():
     """More keys than one LSE chunk and several key tiles per CTA; ragged last page."""
     wl = synth.Workload("long", 1, 1, 4, [9000 + 7], [32], [2300], table_style="fragmented", seed=5, poison_tail=True)
