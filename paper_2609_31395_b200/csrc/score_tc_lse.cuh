@@ -178,21 +178,23 @@ __device__ __forceinline__ bool lse_job(LseBarriers* bars, volatile int* abort_f
   return true;
 }
 
-template <int NPOLY>
+// ROW_GROUPS: the unit's window has more than MAX_ROWS rows and the grid has a row-group dimension (kept
+// out of the common instantiation, whose code should not change with it).
+template <int NPOLY, bool ROW_GROUPS>
 __global__ void __launch_bounds__(LSE_THREADS, 1)
 score_tc_lse_kernel(const __grid_constant__ CUtensorMap kmap, const TcArgs ta) {
   extern __shared__ __align__(1024) uint8_t smem[];
   const ScoreArgs& a = ta.a;
   const int R = a.tab.n_req, Hkv = a.pool.n_kv_heads, G = a.group;
-  int idx = blockIdx.x;
-  const int chunk = idx % a.n_chunks; idx /= a.n_chunks;
-  const int rg = idx % ta.n_rg;                          // row group: rows [row0, row0 + MAX_ROWS) of the unit
-  const int u = idx / ta.n_rg;
+  const int cu = blockIdx.x / a.n_chunks;
+  const int chunk = blockIdx.x - cu * a.n_chunks;
+  const int rg = ROW_GROUPS ? cu % ta.n_rg : 0;          // row group: rows [row0, row0 + MAX_ROWS) of the unit
+  const int u = ROW_GROUPS ? cu / ta.n_rg : cu;
   const int r = u % R, h = (u / R) % Hkv, slab = u / (R * Hkv);
   const int L = a.tab.seq_len[r];
   const int w0 = a.win_indptr[r], W = a.win_indptr[r + 1] - w0;
-  const int row0 = rg * MAX_ROWS;
-  const int rows = min(W * G - row0, MAX_ROWS);          // rows of this CTA
+  const int row0 = ROW_GROUPS ? rg * MAX_ROWS : 0;
+  const int rows = ROW_GROUPS ? min(W * G - row0, MAX_ROWS) : W * G;     // rows of this CTA
   const int key_begin = chunk * a.lse_chunk;
   if (key_begin >= L || (rg > 0 && rows <= 0)) return;
   if (W <= 0 || (a.causal && W > L)) {
@@ -273,8 +275,16 @@ score_tc_lse_kernel(const __grid_constant__ CUtensorMap kmap, const TcArgs ta) {
 #ifndef ACTKV_EXP_NO_TMA
       if ((lane >> 3) == (it & 3)) {
         const uint32_t dst = k_smem + s * KTILE_BYTES + (lane & 7) * 2048;
-        tma_load_4d(dst, &kmap, smem_u32(&bars->k_full[s]), 0, h, pid * 16, layer);
-        tma_load_4d(dst + HALF_BYTES, &kmap, smem_u32(&bars->k_full[s]), 64, h, pid * 16, layer);
+#ifndef ACTKV_EXP_NO_K5
+        if (ta.k5) {
+          tma_load_5d(dst, &kmap, smem_u32(&bars->k_full[s]), 0, 0, h, pid, layer);
+          tma_load_5d(dst + HALF_BYTES, &kmap, smem_u32(&bars->k_full[s]), 64, 0, h, pid, layer);
+        } else
+#endif
+        {
+          tma_load_4d(dst, &kmap, smem_u32(&bars->k_full[s]), 0, h, pid * 16, layer);
+          tma_load_4d(dst + HALF_BYTES, &kmap, smem_u32(&bars->k_full[s]), 64, h, pid * 16, layer);
+        }
       }
 #endif
       if ((it & 3) == 3) pid = pid_next;

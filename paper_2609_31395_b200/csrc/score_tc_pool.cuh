@@ -183,8 +183,16 @@ score_tc_pool_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_cons
       if (!ok) break;
       if ((lane >> 3) == (it & 3)) {
         const uint32_t dst = k_smem + s * KTILE_BYTES + (lane & 7) * 2048;
-        tma_load_4d(dst, &kmap, smem_u32(&bars->k_full[s]), 0, h, pid * 16, layer);
-        tma_load_4d(dst + HALF_BYTES, &kmap, smem_u32(&bars->k_full[s]), 64, h, pid * 16, layer);
+#ifndef ACTKV_EXP_NO_K5
+        if (ta.k5) {
+          tma_load_5d(dst, &kmap, smem_u32(&bars->k_full[s]), 0, 0, h, pid, layer);
+          tma_load_5d(dst + HALF_BYTES, &kmap, smem_u32(&bars->k_full[s]), 64, 0, h, pid, layer);
+        } else
+#endif
+        {
+          tma_load_4d(dst, &kmap, smem_u32(&bars->k_full[s]), 0, h, pid * 16, layer);
+          tma_load_4d(dst + HALF_BYTES, &kmap, smem_u32(&bars->k_full[s]), 64, h, pid * 16, layer);
+        }
       }
       if ((it & 3) == 3) pid = pid_next;
     }

@@ -154,6 +154,21 @@ def test_window_rows_above_one_cta(causal):
         _full_check(synth.generate(wl, DEV))
 
 
+def test_head_major_pool_layout():
+    """A pool stored [layer][K/V][page][head][slot][dim] (HND pages), described to the library by its
+    strides alone: score (FMA path and tensor-core path), select and compaction give the same results as
+    for the oracle's logical view."""
+    small = _small(G=4, seed=21, head_dim=64, page=8)                 # FMA path
+    rows = synth.Workload("hnd", 2, 2, 8, [1100, 257], [48, 17], [300, 64], table_style="fragmented", seed=22,
+                          poison_tail=True)                          # tensor-core path (384 rows)
+    for wl in (small, rows):
+        inst = synth.generate(wl, DEV)
+        hnd = inst.pool.permute(0, 1, 2, 4, 3, 5).contiguous()      # physical [NL, 2, pages, Hkv, P, D]
+        inst.pool = hnd.permute(0, 1, 2, 4, 3, 5)                    # logical [NL, 2, pages, P, Hkv, D], HND strides
+        assert inst.pool.stride(4) == wl.page_size * wl.head_dim and inst.pool.stride(3) == wl.head_dim
+        _full_check(inst)
+
+
 def test_long_request_many_chunks():
     """More keys than one LSE chunk and several key tiles per CTA; ragged last page."""
     wl = synth.Workload("long", 1, 1, 4, [9000 + 7], [32], [2300], table_style="fragmented", seed=5, poison_tail=True)
