@@ -380,6 +380,15 @@ def run_ours(args):
     roofline.update({"kernel": dom, "launches_per_step": n_calls, "ms_per_launch": stage_ms[dom] / n_calls,
                      "traffic": traffic, "traffic_unit": "bytes per launch (ncu, scaled from the 2-layer capture)", "peak_source": pk["source"] + (" sustained bf16" if stages[dom]["bound"] == "tensor" else " copy")})
     hbm_frac_whole = alg_bytes / (ms_max * 1e-3) / 1e9 / pk["hbm_gbs"]
+    # The LSE pass evaluates one exp2 per (window row, key): besides the contraction it is bound by the
+    # special function units, 16 results per clock per SM on 148 SMs at the maximum SM clock.
+    n_exp = sum(W * G * L for W, L in zip(wl.windows, wl.seq_lens)) * Hkv * NL
+    exp_peak = 148 * 16 * (clocks.get("sm_max_mhz") or 1965.0) * 1e6 / 1e9
+    lse_exp = None
+    if stage_ms["lse"]:
+        ach = n_exp / (stage_ms["lse"] * 1e-3) / 1e9
+        lse_exp = {"bound": "alu", "achieved": ach, "peak": exp_peak, "unit": "Gexp2/s", "frac": ach / exp_peak,
+                   "kernel": "lse", "peak_source": "148 SMs x 16 MUFU results per clock x the maximum SM clock"}
 
     # ---- end to end: host buffers in, host results out, every step -------------------------------
     e2e = None
@@ -549,7 +558,8 @@ def run_ours(args):
             "with_lse_supplied": lse_supplied_line, "with_lrfu_policy": lrfu_line,
             "with_inplace_compaction": inplace_line, "streaming_update": stream_line,
             "algorithmic_bytes_per_step": alg_bytes, "k_bytes_per_pass": bytes_k,
-            "roofline": roofline, "roofline_stages": stages, "cpu_baseline": cpu_baseline, "e2e": e2e,
+            "roofline": roofline, "roofline_stages": stages, "roofline_lse_exp_rate": lse_exp,
+            "cpu_baseline": cpu_baseline, "e2e": e2e,
             "clocks": clocks, "gpu_launches": launches, "wall_s_timed_region": t_wall,
         }
         print(json.dumps(out))
