@@ -61,7 +61,7 @@ inline bool make_maps(const actkv_pool_t* pool, const void* q, int nls, int sum_
     // one head, 64 dims: 16 rows of 128 B.
     CUresult res;
     if (!pool_needs_5d(pool)) {
-      cuuint64_t dims[4] = {(cuuint64_t)HD, (cuuint64_t)pool->n_kv_heads, (cuuint64_t)pool->n_pages * pool->page_size,
+      cuuint64_t dims[4] = {(cuuint64_t)pool->head_dim, (cuuint64_t)pool->n_kv_heads, (cuuint64_t)pool->n_pages * pool->page_size,
                             (cuuint64_t)pool->n_layers};
       cuuint64_t strides[3] = {(cuuint64_t)pool->stride_head * 2, (cuuint64_t)pool->stride_slot * 2,
                                (cuuint64_t)pool->stride_layer * 2};
@@ -70,7 +70,7 @@ inline bool make_maps(const actkv_pool_t* pool, const void* q, int nls, int sum_
       res = enc(kmap, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, pool->base, dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
                 CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     } else {
-      cuuint64_t dims[5] = {(cuuint64_t)HD, (cuuint64_t)pool->page_size, (cuuint64_t)pool->n_kv_heads,
+      cuuint64_t dims[5] = {(cuuint64_t)pool->head_dim, (cuuint64_t)pool->page_size, (cuuint64_t)pool->n_kv_heads,
                             (cuuint64_t)pool->n_pages, (cuuint64_t)pool->n_layers};
       cuuint64_t strides[4] = {(cuuint64_t)pool->stride_slot * 2, (cuuint64_t)pool->stride_head * 2,
                                (cuuint64_t)pool->stride_page * 2, (cuuint64_t)pool->stride_layer * 2};
@@ -83,8 +83,9 @@ inline bool make_maps(const actkv_pool_t* pool, const void* q, int nls, int sum_
   }
   {
     // q: [slab*sum_win + w][q head][128]; a box is (64 dims, the G heads of one group, 128/G window rows)
-    cuuint64_t dims[3] = {(cuuint64_t)HD, (cuuint64_t)n_q_heads, (cuuint64_t)nls * sum_win};
-    cuuint64_t strides[2] = {(cuuint64_t)HD * 2, (cuuint64_t)n_q_heads * HD * 2};
+    const cuuint64_t D = (cuuint64_t)pool->head_dim;
+    cuuint64_t dims[3] = {D, (cuuint64_t)n_q_heads, (cuuint64_t)nls * sum_win};
+    cuuint64_t strides[2] = {D * 2, (cuuint64_t)n_q_heads * D * 2};
     cuuint32_t box[3] = {64, (cuuint32_t)G, (cuuint32_t)(128 / G)};
     cuuint32_t es[3] = {1, 1, 1};
     if (enc(qmap, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(q), dims, strides, box, es,
@@ -99,7 +100,7 @@ constexpr size_t SMEM_LIMIT = 232448;        // 227 KB of dynamic shared memory 
 
 }  // namespace tc
 
-// The tensor-core path takes: page 16, head_dim 128, slot-major or head-major pages (any strides that are
+// The tensor-core path takes: page 16, head_dim 128 or 64, slot-major or head-major pages (any strides that are
 // multiples of 16 bytes), 128-byte aligned
 // base, power-of-two group size <= 32, min_rows <= window x group rows <= 4096 (a CTA handles up to 512;
 // more are taken in groups of 512 rows), positive softmax scale.
@@ -107,7 +108,7 @@ constexpr size_t SMEM_LIMIT = 232448;        // 227 KB of dynamic shared memory 
 // pooled pass alone and is bound by the K reads, from a single row.
 inline bool score_tc_supported(const actkv_pool_t* p, int G, int max_win, float sm_scale, const void* q,
                                int min_rows = 64) {
-  if (p->page_size != 16 || p->head_dim != 128) return false;
+  if (p->page_size != 16 || (p->head_dim != 128 && p->head_dim != 64)) return false;
   // TMA: every stride a positive multiple of 16 bytes (any page layout with contiguous head dimensions)
   if (p->stride_head <= 0 || p->stride_slot <= 0 || p->stride_page <= 0 || p->stride_layer <= 0) return false;
   if ((p->stride_head % 8) || (p->stride_slot % 8) || (p->stride_page % 8) || (p->stride_layer % 8)) return false;
@@ -123,7 +124,9 @@ inline bool score_tc_supported(const actkv_pool_t* p, int G, int max_win, float 
 
 template <int NPOLY>
 inline int score_tc_launch_lse_c(const CUtensorMap& kmap, const tc::TcArgs& ta, unsigned grid, size_t smem, cudaStream_t s) {
-  auto kern = ta.n_rg > 1 ? tc::score_tc_lse_kernel<NPOLY, true> : tc::score_tc_lse_kernel<NPOLY, false>;
+  const bool rgs = ta.n_rg > 1, d64 = ta.a.pool.head_dim == 64;
+  auto kern = rgs ? (d64 ? tc::score_tc_lse_kernel<NPOLY, true, 1> : tc::score_tc_lse_kernel<NPOLY, true, 2>)
+                  : (d64 ? tc::score_tc_lse_kernel<NPOLY, false, 1> : tc::score_tc_lse_kernel<NPOLY, false, 2>);
   if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return ACTKV_E_CUDA;
   kern<<<grid, tc::LSE_THREADS, smem, s>>>(kmap, ta);
   ACTKV_CHECK_LAUNCH();
@@ -151,19 +154,17 @@ inline int score_tc_launch_lse(ScoreArgs& a, const actkv_pool_t* pool, int max_t
   if (const char* e = getenv("ACTKV_LSE_NPOLY")) npoly = atoi(e);
   switch (npoly) {
     case 0: return score_tc_launch_lse_c<0>(kmap, ta, (unsigned)grid, smem, s);
-    case 1: return score_tc_launch_lse_c<1>(kmap, ta, (unsigned)grid, smem, s);
     case 2: return score_tc_launch_lse_c<2>(kmap, ta, (unsigned)grid, smem, s);
-    case 4: return score_tc_launch_lse_c<4>(kmap, ta, (unsigned)grid, smem, s);
-    default: return score_tc_launch_lse_c<3>(kmap, ta, (unsigned)grid, smem, s);
+    default: return score_tc_launch_lse_c<1>(kmap, ta, (unsigned)grid, smem, s);
   }
 }
 
 template <int G>
 inline int score_tc_launch_pool_g(const CUtensorMap& kmap, const CUtensorMap& qmap, const tc::TcArgs& ta, unsigned grid,
                                   size_t smem, cudaStream_t s) {
-  if (cudaFuncSetAttribute(tc::score_tc_pool_kernel<G>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
-    return ACTKV_E_CUDA;
-  tc::score_tc_pool_kernel<G><<<grid, tc::POOL_THREADS, smem, s>>>(kmap, qmap, ta);
+  auto kern = ta.a.pool.head_dim == 64 ? tc::score_tc_pool_kernel<G, 1> : tc::score_tc_pool_kernel<G, 2>;
+  if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return ACTKV_E_CUDA;
+  kern<<<grid, tc::POOL_THREADS, smem, s>>>(kmap, qmap, ta);
   ACTKV_CHECK_LAUNCH();
   return ACTKV_OK;
 }

@@ -180,7 +180,8 @@ __device__ __forceinline__ bool lse_job(LseBarriers* bars, volatile int* abort_f
 
 // ROW_GROUPS: the unit's window has more than MAX_ROWS rows and the grid has a row-group dimension (kept
 // out of the common instantiation, whose code should not change with it).
-template <int NPOLY, bool ROW_GROUPS>
+// NH: 64-dim halves of the head dimension (head_dim = 64 NH); a K tile is NH x [128 keys][64 bf16].
+template <int NPOLY, bool ROW_GROUPS, int NH>
 __global__ void __launch_bounds__(LSE_THREADS, 1)
 score_tc_lse_kernel(const __grid_constant__ CUtensorMap kmap, const TcArgs ta) {
   extern __shared__ __align__(1024) uint8_t smem[];
@@ -267,7 +268,7 @@ score_tc_lse_kernel(const __grid_constant__ CUtensorMap kmap, const TcArgs ta) {
 #ifdef ACTKV_EXP_NO_TMA
         if (ok) mbar_arrive(smem_u32(&bars->k_full[s]));
 #else
-        if (ok) mbar_expect_tx(smem_u32(&bars->k_full[s]), KTILE_BYTES);
+        if (ok) mbar_expect_tx(smem_u32(&bars->k_full[s]), NH * HALF_BYTES);
 #endif
       }
       ok = __shfl_sync(0xffffffffu, ok, 0);
@@ -278,12 +279,12 @@ score_tc_lse_kernel(const __grid_constant__ CUtensorMap kmap, const TcArgs ta) {
 #ifndef ACTKV_EXP_NO_K5
         if (ta.k5) {
           tma_load_5d(dst, &kmap, smem_u32(&bars->k_full[s]), 0, 0, h, pid, layer);
-          tma_load_5d(dst + HALF_BYTES, &kmap, smem_u32(&bars->k_full[s]), 64, 0, h, pid, layer);
+          if constexpr (NH == 2) tma_load_5d(dst + HALF_BYTES, &kmap, smem_u32(&bars->k_full[s]), 64, 0, h, pid, layer);
         } else
 #endif
         {
           tma_load_4d(dst, &kmap, smem_u32(&bars->k_full[s]), 0, h, pid * 16, layer);
-          tma_load_4d(dst + HALF_BYTES, &kmap, smem_u32(&bars->k_full[s]), 64, h, pid * 16, layer);
+          if constexpr (NH == 2) tma_load_4d(dst + HALF_BYTES, &kmap, smem_u32(&bars->k_full[s]), 64, h, pid * 16, layer);
         }
       }
 #endif
@@ -324,7 +325,7 @@ score_tc_lse_kernel(const __grid_constant__ CUtensorMap kmap, const TcArgs ta) {
         if (leader) {
           const uint32_t at = tmem_base + b * 64;
 #pragma unroll
-          for (int kk = 0; kk < 8; ++kk)
+          for (int kk = 0; kk < 4 * NH; ++kk)
             umma_bf16_ts(d, at + kk * 8, desc_s + (uint64_t)(((kk >> 2) * HALF_BYTES + (kk & 3) * 32) >> 4), idesc,
                          kk > 0 ? 1u : 0u);
           umma_commit(full_bar);
@@ -353,11 +354,11 @@ score_tc_lse_kernel(const __grid_constant__ CUtensorMap kmap, const TcArgs ta) {
       const bool live = k < n_mb && n < rows;
       const int w = (row0 + n) / G, g = (row0 + n) % G;
       const uint4* src = reinterpret_cast<const uint4*>(
-          a.q + (((int64_t)slab * a.sum_win + w0 + (live ? w : 0)) * a.n_q_heads + h * G + (live ? g : 0)) * HD);
+          a.q + (((int64_t)slab * a.sum_win + w0 + (live ? w : 0)) * a.n_q_heads + h * G + (live ? g : 0)) * (64 * NH));
       const uint32_t dst = tmem_base + ((uint32_t)(quarter * 32) << 16) + k * 64;
       if (k < n_mb) {
 #pragma unroll
-        for (int i = 0; i < 4; ++i) {
+        for (int i = 0; i < 2 * NH; ++i) {
           uint4 x[4];
 #pragma unroll
           for (int j = 0; j < 4; ++j) x[j] = live ? __ldg(src + i * 4 + j) : make_uint4(0, 0, 0, 0);

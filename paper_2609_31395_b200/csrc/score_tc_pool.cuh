@@ -80,7 +80,8 @@ __device__ __forceinline__ void pool_job(uint32_t taddr, const float* nlse, int 
   }
 }
 
-template <int G>
+// NH: 64-dim halves of the head dimension (head_dim = 64 NH).
+template <int G, int NH>
 __global__ void __launch_bounds__(POOL_THREADS, 1)
 score_tc_pool_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constant__ CUtensorMap qmap, const TcArgs ta) {
   extern __shared__ __align__(1024) uint8_t smem[];
@@ -158,10 +159,10 @@ score_tc_pool_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_cons
     const int n_lp = (L + a.pool.page_size - 1) / a.pool.page_size;
     const int layer = a.layer_begin + slab;
     if (lane == 0) {
-      mbar_expect_tx(smem_u32(&bars->q_full), (uint32_t)n_qblk * QBLK_BYTES);
+      mbar_expect_tx(smem_u32(&bars->q_full), (uint32_t)n_qblk * NH * HALF_BYTES);
       const int wrow = slab * a.sum_win + w0 + w_begin;
       for (int qb = 0; qb < n_qblk; ++qb)
-        for (int hf = 0; hf < 2; ++hf)
+        for (int hf = 0; hf < NH; ++hf)
           tma_load_3d(q_smem + (qb >> 1) * 2 * QBLK_BYTES + hf * QBLK_BYTES + (qb & 1) * HALF_BYTES, &qmap,
                       smem_u32(&bars->q_full), hf * 64, h * G, wrow + qb * (128 / G));
     }
@@ -177,7 +178,7 @@ score_tc_pool_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_cons
       int ok = 1;
       if (lane == 0) {
         ok = mbar_wait(smem_u32(&bars->k_empty[s]), ph ^ 1u, abort_flag) ? 1 : 0;
-        if (ok) mbar_expect_tx(smem_u32(&bars->k_full[s]), KTILE_BYTES);
+        if (ok) mbar_expect_tx(smem_u32(&bars->k_full[s]), NH * HALF_BYTES);
       }
       ok = __shfl_sync(0xffffffffu, ok, 0);
       if (!ok) break;
@@ -186,12 +187,12 @@ score_tc_pool_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_cons
 #ifndef ACTKV_EXP_NO_K5
         if (ta.k5) {
           tma_load_5d(dst, &kmap, smem_u32(&bars->k_full[s]), 0, 0, h, pid, layer);
-          tma_load_5d(dst + HALF_BYTES, &kmap, smem_u32(&bars->k_full[s]), 64, 0, h, pid, layer);
+          if constexpr (NH == 2) tma_load_5d(dst + HALF_BYTES, &kmap, smem_u32(&bars->k_full[s]), 64, 0, h, pid, layer);
         } else
 #endif
         {
           tma_load_4d(dst, &kmap, smem_u32(&bars->k_full[s]), 0, h, pid * 16, layer);
-          tma_load_4d(dst + HALF_BYTES, &kmap, smem_u32(&bars->k_full[s]), 64, h, pid * 16, layer);
+          if constexpr (NH == 2) tma_load_4d(dst + HALF_BYTES, &kmap, smem_u32(&bars->k_full[s]), 64, h, pid * 16, layer);
         }
       }
       if ((it & 3) == 3) pid = pid_next;
@@ -231,7 +232,7 @@ score_tc_pool_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_cons
         if (leader) {
           const uint64_t bdesc_c = qdesc0 + (uint64_t)((rc * 2 * QBLK_BYTES) >> 4);
 #pragma unroll
-          for (int kk = 0; kk < 8; ++kk)
+          for (int kk = 0; kk < 4 * NH; ++kk)
             umma_bf16(tmem_base + mw * 256, adesc_s + (uint64_t)(((kk >> 2) * HALF_BYTES + (kk & 3) * 32) >> 4),
                       bdesc_c + (uint64_t)(((kk >> 2) * QBLK_BYTES + (kk & 3) * 32) >> 4), idesc_c[rc], kk > 0 ? 1u : 0u);
           umma_commit(full_bar);

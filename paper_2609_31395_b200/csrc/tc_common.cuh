@@ -57,18 +57,6 @@ __device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity) {
 // at least half as long in wall time.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag,
                                           uint64_t limit_ns = WAIT_LIMIT_NS) {
-#ifdef ACTKV_EXP_SPIN
-  {
-    const long long t0s = clock64();
-    for (;;) {
-#pragma unroll 1
-      for (int i = 0; i < 1024; ++i)
-        if (mbar_test_wait(bar, parity)) return true;
-      if (*abort_flag) return false;
-      if (clock64() - t0s > (long long)limit_ns * 2) { *abort_flag = 1; return false; }
-    }
-  }
-#endif
   // try_wait parks the thread in hardware (no polling traffic on shared memory, which the MMA operand
   // fetch needs); measured the same or better than spinning on test_wait here.
 #pragma unroll 1

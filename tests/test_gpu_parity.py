@@ -154,6 +154,15 @@ def test_window_rows_above_one_cta(causal):
         _full_check(synth.generate(wl, DEV))
 
 
+@pytest.mark.parametrize("causal", [False, True])
+def test_head_dim_64_on_the_tensor_core_path(causal):
+    """head_dim 64 with 16-token pages: a K tile is one 64-dim half, four MMAs per accumulator."""
+    for W, G in [(32, 4), (64, 8), (33, 2), (40, 16)]:
+        wl = synth.Workload("d64", 2, 2, G, [1000, 300], [W, max(1, W // 2)], [260, 90], head_dim=64,
+                            table_style="fragmented", causal=causal, seed=W * 3 + G, poison_tail=True)
+        _full_check(synth.generate(wl, DEV))
+
+
 def test_head_major_pool_layout():
     """A pool stored [layer][K/V][page][head][slot][dim] (HND pages), described to the library by its
     strides alone: score (FMA path and tensor-core path), select and compaction give the same results as
