@@ -1,30 +1,38 @@
 // actkv_select: TopK(score, k = B) per (layer x KV head, request) unit — Algorithm 1, step 5,
-// applied to the pooled action-region score.  One CTA per unit: a 4 x 8-bit most-significant-
-// digit radix select over the order-preserving integer image of the float32 scores finds the
-// n-th largest value exactly; one ordered sweep with a block scan then emits the kept token
-// indices in ascending order, entries equal to the threshold being kept lowest index first.
-// Scores are 4 bytes per token and unit-local, so the five sweeps after the first read hit L2.
+// applied to the pooled action-region score.  One CTA per unit.  The unit's scores are read once and
+// kept in shared memory as order-preserving 32-bit keys (up to 53 K tokens; longer units re-read them
+// from L2); a most-significant-digit radix select with digits of 12, 12 and 8 bits (shared-memory
+// histograms, plain atomics: a warp's keys spread over many bins once the digit reaches into the
+// mantissa, and over the few dozen bins of the populated binades before) finds the n-th largest key
+// exactly; one ordered sweep with a block scan then emits the kept token indices in ascending order,
+// entries equal to the threshold being kept lowest index first.
 #include "common.cuh"
 
 namespace actkv {
 
 constexpr int SEL_NT = 1024;
 constexpr int SEL_ITEMS = 4;
+constexpr int SEL_BINS = 4096;
+constexpr size_t SEL_SMEM = 232448 - 1024;                            // (nearly) all of an SM's shared memory: one CTA per SM
+constexpr int SEL_CAP = (int)((SEL_SMEM - SEL_BINS * 4) / 4);          // keys that fit beside the histogram
 
 __device__ __forceinline__ uint32_t order_key(float x) {
   uint32_t b = __float_as_uint(x);
   return (b & 0x80000000u) ? ~b : (b | 0x80000000u);     // larger float -> larger key
 }
 
-__global__ void __launch_bounds__(SEL_NT) select_kernel(
+__global__ void __launch_bounds__(SEL_NT, 1) select_kernel(
     const float* __restrict__ score, const int32_t* __restrict__ tok_indptr, int32_t sum_tok,
     const int32_t* __restrict__ budget, int32_t n_req, const int32_t* __restrict__ keep_indptr,
     int32_t* __restrict__ sel_idx, int64_t sel_stride, uint32_t* __restrict__ keep_mask,
     actkv_tie_t* __restrict__ tie, int32_t* status) {
-  __shared__ uint32_t hist[256];
+  extern __shared__ __align__(16) uint32_t sel_smem[];
+  uint32_t* hist = sel_smem;                             // [SEL_BINS]
+  uint32_t* skeys = sel_smem + SEL_BINS;                 // [SEL_CAP]
   __shared__ uint32_t warp_tot[SEL_NT / 32];
   __shared__ uint32_t s_bin, s_remaining, s_eq_total;
   __shared__ unsigned long long s_carry;
+  __shared__ unsigned long long wsum[SEL_NT / 32];
 
   const int u = blockIdx.x;
   const int r = u % n_req, o = u / n_req;
@@ -40,52 +48,80 @@ __global__ void __launch_bounds__(SEL_NT) select_kernel(
     if (tie != nullptr && tid == 0) tie[u] = actkv_tie_t{0.f, 0, 0, 0};
     return;
   }
+  const bool resident = L <= SEL_CAP;                    // uniform over the CTA
+  auto key_at = [&](int i) -> uint32_t { return resident ? skeys[i] : order_key(sc[i]); };
+  // The one read of the scores (16-byte vectors between an unaligned head and tail) also fills the
+  // histogram of the first digit.
+  for (int i = tid; i < SEL_BINS; i += SEL_NT) hist[i] = 0;
+  __syncthreads();
+  {
+    auto take = [&](int i, float x) {
+      const uint32_t k = order_key(x);
+      if (resident) skeys[i] = k;
+      atomicAdd(&hist[k >> 20], 1u);
+    };
+    const int head = min(L, (int)((16u - ((uint32_t)(uintptr_t)sc & 15u)) & 15u) >> 2);
+    const int n_vec = (L - head) >> 2;
+    if (tid < head) take(tid, sc[tid]);
+    const float4* sc4 = reinterpret_cast<const float4*>(sc + head);
+    for (int v = tid; v < n_vec; v += SEL_NT) {
+      const float4 x = sc4[v];
+      const int i = head + 4 * v;
+      take(i, x.x); take(i + 1, x.y); take(i + 2, x.z); take(i + 3, x.w);
+    }
+    const int tail0 = head + 4 * n_vec;
+    if (tail0 + tid < L) take(tail0 + tid, sc[tail0 + tid]);
+  }
 
   // ---- radix select: n-th largest key -----------------------------------------------------
   uint32_t prefix = 0, mask = 0, remaining = (uint32_t)n;
-  for (int shift = 24; shift >= 0; shift -= 8) {
-    if (tid < 256) hist[tid] = 0;
-    __syncthreads();
-    for (int i0 = 0; i0 < L; i0 += SEL_NT) {               // warp-uniform trip count
-      const int i = i0 + tid;
-      const uint32_t k = (i < L) ? order_key(sc[i]) : 0u;
-      const bool in = (i < L) && (k & mask) == prefix;
-      const uint32_t voters = __ballot_sync(0xffffffffu, in);
-      if (in) {
-        const uint32_t bin = (k >> shift) & 255u;
-        // warp-aggregated increment: lanes with the same bin elect one to add their count
-        const uint32_t peers = __match_any_sync(voters, bin);
-        if (lane == (__ffs(peers) - 1)) atomicAdd(&hist[bin], (uint32_t)__popc(peers));
+#pragma unroll 1
+  for (int pass = 0; pass < 3; ++pass) {
+    const int shift = pass == 0 ? 20 : pass == 1 ? 8 : 0;
+    const uint32_t dmask = pass == 2 ? 255u : 4095u;
+    const int n_bins = (int)dmask + 1;
+    if (pass > 0) {
+      for (int i = tid; i < n_bins; i += SEL_NT) hist[i] = 0;
+      __syncthreads();
+      for (int i = tid; i < L; i += SEL_NT) {
+        const uint32_t k = key_at(i);
+        if ((k & mask) == prefix) atomicAdd(&hist[(k >> shift) & dmask], 1u);
       }
     }
     __syncthreads();
-    // suffix sums over the 256 bins: cum(b) = #keys with digit >= b
-    uint32_t v = 0, incl = 0;
-    if (tid < 256) {
-      v = hist[255 - tid];                               // reversed so a prefix scan is a suffix sum
-      incl = v;
+    // suffix sums over the bins, descending: thread t owns bins n_bins-1-4t .. n_bins-4-4t
+    const int per = n_bins / SEL_NT;                     // 4, or 0 for the 256-bin pass (then one bin for tid < 256)
+    uint32_t h[4] = {0, 0, 0, 0}, mine = 0;
+    if (per == 4) {
 #pragma unroll
-      for (int d = 1; d < 32; d <<= 1) {
-        uint32_t t = __shfl_up_sync(0xffffffffu, incl, d);
-        if (lane >= d) incl += t;
-      }
-      if (lane == 31) warp_tot[warp] = incl;
+      for (int j = 0; j < 4; ++j) { h[j] = hist[n_bins - 1 - 4 * tid - j]; mine += h[j]; }
+    } else if (tid < n_bins) {
+      h[0] = hist[n_bins - 1 - tid];
+      mine = h[0];
     }
+    uint32_t incl = mine;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+      const uint32_t t = __shfl_up_sync(0xffffffffu, incl, d);
+      if (lane >= d) incl += t;
+    }
+    if (lane == 31) warp_tot[warp] = incl;
     __syncthreads();
-    if (tid < 256) {
-      uint32_t add = 0;
-      for (int w = 0; w < warp; ++w) add += warp_tot[w];
-      incl += add;                                       // keys with digit >= 255 - tid
-      uint32_t excl = incl - v;                          // keys with digit >  255 - tid
-      if (incl >= remaining && excl < remaining) {
-        s_bin = 255u - (uint32_t)tid;
-        s_remaining = remaining - excl;
-        s_eq_total = v;
+    uint32_t acc = incl - mine;                          // keys with a digit above this thread's first bin
+    for (int w = 0; w < warp; ++w) acc += warp_tot[w];
+    const int first_bin = per == 4 ? n_bins - 1 - 4 * tid : n_bins - 1 - tid;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      if (acc < remaining && acc + h[j] >= remaining) {  // exactly one bin over all threads crosses
+        s_bin = (uint32_t)(first_bin - j);
+        s_remaining = remaining - acc;
+        s_eq_total = h[j];
       }
+      acc += h[j];
     }
     __syncthreads();
     prefix |= s_bin << shift;
-    mask |= 255u << shift;
+    mask |= dmask << shift;
     remaining = s_remaining;
     __syncthreads();
   }
@@ -105,7 +141,7 @@ __global__ void __launch_bounds__(SEL_NT) select_kernel(
 #pragma unroll
     for (int k = 0; k < SEL_ITEMS; ++k) {
       const int i = i0 + k;
-      uint32_t key = (i < L) ? order_key(sc[i]) : 0u;
+      uint32_t key = (i < L) ? key_at(i) : 0u;
       gt[k] = (i < L) && key > thr;
       eq[k] = (i < L) && key == thr;
       mine += ((unsigned long long)gt[k] << 32) + eq[k];
@@ -116,7 +152,6 @@ __global__ void __launch_bounds__(SEL_NT) select_kernel(
       unsigned long long t = __shfl_up_sync(0xffffffffu, incl, d);
       if (lane >= d) incl += t;
     }
-    __shared__ unsigned long long wsum[SEL_NT / 32];
     if (lane == 31) wsum[warp] = incl;
     __syncthreads();
     unsigned long long before = s_carry;
@@ -176,7 +211,9 @@ int actkv_select(const float* score, const int32_t* tok_indptr, int32_t sum_tok,
   if (!score || !tok_indptr || !budget || !keep_indptr || !sel_idx) return ACTKV_E_INVALID;
   const int64_t units = (int64_t)n_outer * n_req;
   if (units > 0x7fffffffLL) return ACTKV_E_INVALID;
-  actkv::select_kernel<<<(unsigned)units, actkv::SEL_NT, 0, (cudaStream_t)stream>>>(
+  if (cudaFuncSetAttribute(actkv::select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)actkv::SEL_SMEM) != cudaSuccess)
+    return ACTKV_E_CUDA;
+  actkv::select_kernel<<<(unsigned)units, actkv::SEL_NT, actkv::SEL_SMEM, (cudaStream_t)stream>>>(
       score, tok_indptr, sum_tok, budget, n_req, keep_indptr, sel_idx, sel_stride, keep_mask,
       tie_report, status);
   ACTKV_CHECK_LAUNCH();
