@@ -4,9 +4,10 @@
 // Per (layer x KV head, request) unit, one CTA:
 //   1. mass m_i = floor(clip(score_i, 0, 256) * 2^32) as 64-bit integers; total = sum m_i (exact,
 //      read off the first histogram);
-//   2. mark = ceil(p_q * total / 10000); a 4 x 8-bit radix search over the order-preserving image of
-//      the scores with 64-bit integer mass histograms (warp-aggregated adds) finds the threshold
-//      score T with mass(score > T) < mark <= mass(score >= T) — exact, independent of summation order;
+//   2. mark = ceil(p_q * total / 10000); a radix search (digits of 12, 12 and 8 bits) over the
+//      order-preserving image of the scores, kept in shared memory, with 64-bit integer mass histograms
+//      finds the threshold score T with mass(score > T) < mark <= mass(score >= T) — exact, independent of
+//      summation order;
 //   3. entries above T are hits; of the entries equal to T the first ceil((mark - mass_above)/m_T)
 //      by index are hits (ordered sweep with a block scan, as in select);
 //   4. KS = lambda*KS + score*[hit], one float32 rounding per operation; the score buffer is
@@ -40,12 +41,35 @@ __device__ __forceinline__ float add_ieee(float a, float b) {
   return d;
 }
 
-__global__ void __launch_bounds__(KS_NT) keepscore_kernel(
+__device__ __forceinline__ float ks_key_to_float(uint32_t k) {
+  return __uint_as_float((k & 0x80000000u) ? (k & 0x7fffffffu) : ~k);
+}
+
+constexpr int KS_BINS = 4096;
+constexpr size_t KS_SMEM = 232448 - 1024;                              // (nearly) all of an SM's shared memory
+constexpr int KS_CAP = (int)((KS_SMEM - KS_BINS * 12) / 4);            // keys that fit beside the histogram
+// (chunk sums stay below 2^32 for units of up to 2^17 entries; the total mass needs 2^16 or fewer, see below)
+
+__global__ void __launch_bounds__(KS_NT, 1) keepscore_kernel(
     float* __restrict__ score, const int32_t* __restrict__ tok_indptr, int32_t sum_tok, int32_t n_req,
     int32_t p_q, float lambda, const int32_t* __restrict__ n_protect, float* __restrict__ keep_score,
     uint32_t* __restrict__ hit_mask) {
-  __shared__ unsigned long long hist[256];
-  __shared__ unsigned long long s_above, s_carry, s_mark;
+  // A mass is below 2^41; its three 14-bit chunks are summed in three 32-bit histograms (native shared
+  // atomics; a 64-bit shared atomic is a compare-and-swap loop) and put together when the bins are scanned.
+  extern __shared__ __align__(16) uint32_t ks_smem[];
+  uint32_t* hist = ks_smem;                                            // [3][KS_BINS] mass chunks per digit
+  uint32_t* skeys = ks_smem + 3 * KS_BINS;                             // [KS_CAP] order keys of the unit
+  auto hist_add = [&](uint32_t bin, unsigned long long m) {
+    atomicAdd(&hist[bin], (uint32_t)(m & 0x3fffull));
+    atomicAdd(&hist[KS_BINS + bin], (uint32_t)((m >> 14) & 0x3fffull));
+    atomicAdd(&hist[2 * KS_BINS + bin], (uint32_t)(m >> 28));
+  };
+  auto hist_get = [&](int bin) -> unsigned long long {
+    return (unsigned long long)hist[bin] + ((unsigned long long)hist[KS_BINS + bin] << 14) +
+           ((unsigned long long)hist[2 * KS_BINS + bin] << 28);
+  };
+  __shared__ unsigned long long warp_tot[KS_NT / 32];
+  __shared__ unsigned long long s_above, s_carry;
   __shared__ uint32_t s_bin;
 
   const int u = blockIdx.x;
@@ -56,72 +80,85 @@ __global__ void __launch_bounds__(KS_NT) keepscore_kernel(
   float* sc = score + (int64_t)o * sum_tok + base;
   float* ks = keep_score + (int64_t)o * sum_tok + base;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const bool resident = L <= KS_CAP;                     // uniform over the CTA
+  auto key_at = [&](int i) -> uint32_t { return resident ? skeys[i] : ks_order_key(sc[i]); };
 
-  // ---- radix search: largest key T with mass(key >= T) >= mark ----
-  // The first pass histograms every entry, so its bins also add up to the total mass, from which
-  // mark = ceil(p_q * total / 10000)  (total < 2^57 for up to 2^16 entries, p_q <= 10000 < 2^14:
-  // the product is taken in two halves to stay inside 64 bits).
+  // ---- radix search: largest key T with mass(key >= T) >= mark; digits of 12, 12 and 8 bits ----
+  // The scores are read once (kept in shared memory as order keys; longer units re-read them from L2) and
+  // that read also fills the histogram of the first digit, whose bins add up to the total mass, from
+  // which  mark = ceil(p_q * total / 10000)  (total < 2^57 for up to 2^16 entries, p_q <= 10000 < 2^14: the
+  // product is taken in two halves to stay inside 64 bits).
+  for (int i = tid; i < 3 * KS_BINS; i += KS_NT) hist[i] = 0u;
+  __syncthreads();
+  for (int i = tid; i < L; i += KS_NT) {
+    const float x = sc[i];
+    const uint32_t k = ks_order_key(x);
+    if (resident) skeys[i] = k;
+    const unsigned long long m = ks_mass(x);
+    if (m != 0ull) hist_add(k >> 20, m);
+  }
   uint32_t prefix = 0, mask = 0;
   unsigned long long above = 0;        // mass of keys strictly above the current prefix range
   unsigned long long mark = 0;
-  for (int shift = 24; shift >= 0; shift -= 8) {
-    if (tid < 256) hist[tid] = 0;
-    __syncthreads();
-    for (int i0 = 0; i0 < L; i0 += KS_NT) {                // warp-uniform trip count
-      const int i = i0 + tid;
-      const float x = (i < L) ? sc[i] : 0.f;
-      const uint32_t k = ks_order_key(x);
-      const unsigned long long m = ks_mass(x);
-      const bool in = (i < L) && (k & mask) == prefix && m != 0ull;
-      const uint32_t voters = __ballot_sync(0xffffffffu, in);
-      if (in) {
-        // warp-aggregated add: lanes with the same bin sum their masses (<= 2^40 each, as two
-        // chunks that cannot overflow 32 bits over 32 lanes) and elect one lane to add the sum
-        const uint32_t bin = (k >> shift) & 255u;
-        const uint32_t peers = __match_any_sync(voters, bin);
-        const uint32_t lo = __reduce_add_sync(peers, (uint32_t)(m & 0x1fffffull));
-        const uint32_t hi = __reduce_add_sync(peers, (uint32_t)(m >> 21));
-        if (lane == (__ffs(peers) - 1)) atomicAdd(&hist[bin], ((unsigned long long)hi << 21) + lo);
-      }
-    }
-    __syncthreads();
-    // warp 0: suffix sums over the 256 bins, lane l owns bins 255-8l .. 248-8l (descending)
-    if (warp == 0) {
-      unsigned long long h[8], mine = 0;
-#pragma unroll
-      for (int j = 0; j < 8; ++j) {
-        h[j] = hist[255 - 8 * lane - j];
-        mine += h[j];
-      }
-      unsigned long long incl = mine;
-#pragma unroll
-      for (int d = 1; d < 32; d <<= 1) {
-        const unsigned long long t = __shfl_up_sync(0xffffffffu, incl, d);
-        if (lane >= d) incl += t;
-      }
-      if (shift == 24) {
-        const unsigned long long total = __shfl_sync(0xffffffffu, incl, 31);
-        const unsigned long long q = total / 10000ull, rem = total % 10000ull;
-        mark = q * (unsigned long long)p_q + (rem * (unsigned long long)p_q + 9999ull) / 10000ull;
-        if (lane == 0) s_mark = mark;
-      }
-      if (mark > 0) {
-        unsigned long long acc = above + incl - mine;      // mass above this lane's first bin
-#pragma unroll
-        for (int j = 0; j < 8; ++j) {
-          if (acc < mark && acc + h[j] >= mark) {          // exactly one bin over all lanes crosses the mark
-            s_bin = 255u - 8u * lane - j;
-            s_above = acc;
-          }
-          acc += h[j];
+#pragma unroll 1
+  for (int pass = 0; pass < 3; ++pass) {
+    const int shift = pass == 0 ? 20 : pass == 1 ? 8 : 0;
+    const uint32_t dmask = pass == 2 ? 255u : 4095u;
+    const int n_bins = (int)dmask + 1;
+    if (pass > 0) {
+      for (int i = tid; i < 3 * KS_BINS; i += KS_NT) hist[i] = 0u;
+      __syncthreads();
+      for (int i = tid; i < L; i += KS_NT) {
+        const uint32_t k = key_at(i);
+        if ((k & mask) == prefix) {
+          const unsigned long long m = ks_mass(ks_key_to_float(k));
+          if (m != 0ull) hist_add((k >> shift) & dmask, m);
         }
       }
     }
     __syncthreads();
-    mark = s_mark;
-    if (mark == 0) break;                                  // nothing to cover: no hits (uniform over the CTA)
+    // suffix sums over the bins, descending: thread t owns bins n_bins-1-4t .. n_bins-4-4t
+    const int per = n_bins / KS_NT;                      // 4, or 0 for the 256-bin pass (then one bin for tid < 256)
+    unsigned long long h[4] = {0ull, 0ull, 0ull, 0ull}, mine = 0ull;
+    if (per == 4) {
+#pragma unroll
+      for (int j = 0; j < 4; ++j) { h[j] = hist_get(n_bins - 1 - 4 * tid - j); mine += h[j]; }
+    } else if (tid < n_bins) {
+      h[0] = hist_get(n_bins - 1 - tid);
+      mine = h[0];
+    }
+    unsigned long long incl = mine;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+      const unsigned long long t = __shfl_up_sync(0xffffffffu, incl, d);
+      if (lane >= d) incl += t;
+    }
+    if (lane == 31) warp_tot[warp] = incl;
+    __syncthreads();
+    unsigned long long acc = above + incl - mine;        // mass above this thread's first bin
+    unsigned long long total = 0ull;
+    for (int w = 0; w < KS_NT / 32; ++w) {
+      const unsigned long long t = warp_tot[w];
+      if (w < warp) acc += t;
+      total += t;
+    }
+    if (pass == 0) {
+      const unsigned long long q = total / 10000ull, rem = total % 10000ull;
+      mark = q * (unsigned long long)p_q + (rem * (unsigned long long)p_q + 9999ull) / 10000ull;
+    }
+    if (mark == 0ull) break;                             // nothing to cover: no hits (uniform over the CTA)
+    const int first_bin = per == 4 ? n_bins - 1 - 4 * tid : n_bins - 1 - tid;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      if (acc < mark && acc + h[j] >= mark) {            // exactly one bin over all threads crosses the mark
+        s_bin = (uint32_t)(first_bin - j);
+        s_above = acc;
+      }
+      acc += h[j];
+    }
+    __syncthreads();
     prefix |= s_bin << shift;
-    mask |= 255u << shift;
+    mask |= dmask << shift;
     above = s_above;
     __syncthreads();
   }
@@ -219,7 +256,9 @@ int actkv_keepscore(float* score, const int32_t* tok_indptr, int32_t sum_tok, in
   const int64_t units = (int64_t)n_outer * n_req;
   if (units > 0x7fffffffLL) return ACTKV_E_INVALID;
   const int32_t p_q = (int32_t)lrintf(top_p * 10000.f);
-  actkv::keepscore_kernel<<<(unsigned)units, actkv::KS_NT, 0, (cudaStream_t)stream>>>(
+  if (cudaFuncSetAttribute(actkv::keepscore_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)actkv::KS_SMEM) != cudaSuccess)
+    return ACTKV_E_CUDA;
+  actkv::keepscore_kernel<<<(unsigned)units, actkv::KS_NT, actkv::KS_SMEM, (cudaStream_t)stream>>>(
       score, tok_indptr, sum_tok, n_req, p_q, lambda, n_protect, keep_score, hit_mask);
   ACTKV_CHECK_LAUNCH();
   return ACTKV_OK;
