@@ -21,7 +21,7 @@
 
 namespace actkv {
 
-constexpr int CI_NT = 256;
+constexpr int CI_NT = 128;
 constexpr int CI_UNROLL = 8;
 
 __device__ __forceinline__ int lower_bound_i32(const int32_t* __restrict__ a, int n, int32_t key) {
