@@ -156,7 +156,6 @@ score_tc_pool_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_cons
 
   if (warp == 0) {
     // ---------------- TMA producer ----------------
-    const int n_lp = (L + a.pool.page_size - 1) / a.pool.page_size;
     const int layer = a.layer_begin + slab;
     if (lane == 0) {
       mbar_expect_tx(smem_u32(&bars->q_full), (uint32_t)n_qblk * NH * HALF_BYTES);
@@ -166,37 +165,8 @@ score_tc_pool_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_cons
           tma_load_3d(q_smem + (qb >> 1) * 2 * QBLK_BYTES + hf * QBLK_BYTES + (qb & 1) * HALF_BYTES, &qmap,
                       smem_u32(&bars->q_full), hf * 64, h * G, wrow + qb * (128 / G));
     }
-    // page ids of four tiles at a time, one per lane (lane / 8 = tile within the group, lane % 8 = page);
-    // the next group's ids are loaded while the current four tiles are being issued
-    int32_t pid = page_for_tile(a.tab, a.pool.n_pages, r, t_begin * 8 + lane, n_lp, a.status);
-    int32_t pid_next = 0;
-    for (int it = 0; it < n_tiles; ++it) {
-      const int s = it % S;
-      const uint32_t ph = (uint32_t)(it / S) & 1u;
-      if ((it & 3) == 0 && it + 4 < n_tiles)
-        pid_next = page_for_tile(a.tab, a.pool.n_pages, r, (t_begin + it + 4) * 8 + lane, n_lp, a.status);
-      int ok = 1;
-      if (lane == 0) {
-        ok = mbar_wait(smem_u32(&bars->k_empty[s]), ph ^ 1u, abort_flag) ? 1 : 0;
-        if (ok) mbar_expect_tx(smem_u32(&bars->k_full[s]), NH * HALF_BYTES);
-      }
-      ok = __shfl_sync(0xffffffffu, ok, 0);
-      if (!ok) break;
-      if ((lane >> 3) == (it & 3)) {
-        const uint32_t dst = k_smem + s * KTILE_BYTES + (lane & 7) * 2048;
-#ifndef ACTKV_EXP_NO_K5
-        if (ta.k5) {
-          tma_load_5d(dst, &kmap, smem_u32(&bars->k_full[s]), 0, 0, h, pid, layer);
-          if constexpr (NH == 2) tma_load_5d(dst + HALF_BYTES, &kmap, smem_u32(&bars->k_full[s]), 64, 0, h, pid, layer);
-        } else
-#endif
-        {
-          tma_load_4d(dst, &kmap, smem_u32(&bars->k_full[s]), 0, h, pid * 16, layer);
-          if constexpr (NH == 2) tma_load_4d(dst + HALF_BYTES, &kmap, smem_u32(&bars->k_full[s]), 64, h, pid * 16, layer);
-        }
-      }
-      if ((it & 3) == 3) pid = pid_next;
-    }
+    if (ta.k5) k_tile_producer<true, NH>(&kmap, a, bars, k_smem, S, r, h, layer, L, t_begin, n_tiles, lane, abort_flag);
+    else k_tile_producer<false, NH>(&kmap, a, bars, k_smem, S, r, h, layer, L, t_begin, n_tiles, lane, abort_flag);
   } else if (warp <= 2) {
     // ---------------- MMA issuers: D[key, row] = K Q^T ----------------
     // Two warps, one per accumulator: warp 1 issues the even jobs, warp 2 the odd ones.  Issuing costs the
