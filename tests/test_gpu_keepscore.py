@@ -52,9 +52,10 @@ def _synthetic_scores(rng, n_outer, lens):
 @pytest.mark.parametrize("top_p", [0.0, 0.5, 0.9, 1.0])
 def test_keepscore_matches_oracle_bit_exact(top_p):
     rng = np.random.default_rng(11)
-    lens = [0, 5, 1500, 4096, 9001]                      # empty, tiny, one sweep, exactly one, three sweeps
+    # empty, tiny, one sweep, exactly one, three sweeps, more than shared memory holds
+    lens = [0, 5, 1500, 4096, 9001, 60001]
     n_outer, lam = 3, 0.9
-    protect = [0, 2, 100, 0, 5000]
+    protect = [0, 2, 100, 0, 5000, 7]
     sc, tok = _synthetic_scores(rng, n_outer, lens)
     ks0 = (rng.random(sc.shape) ** 4).astype(np.float32)
     ks0[:, ::5] = 0.0
