@@ -252,8 +252,9 @@ score_tc_lse_kernel(const __grid_constant__ CUtensorMap kmap, const TcArgs ta) {
   if (warp == 0) {
     // ---------------- TMA producer: K tiles through the block table ----------------
     const int layer = a.layer_begin + slab;
-    if (ta.k5) k_tile_producer<true, NH>(&kmap, a, bars, k_smem, S, r, h, layer, L, t_begin, n_tiles, lane, abort_flag);
-    else k_tile_producer<false, NH>(&kmap, a, bars, k_smem, S, r, h, layer, L, t_begin, n_tiles, lane, abort_flag);
+    // (one producer: this pass needs a K tile per four jobs, far below what one warp delivers)
+    if (ta.k5) k_tile_producer<true, NH>(&kmap, a, bars, k_smem, S, r, h, layer, L, t_begin, n_tiles, lane, abort_flag, 0, 1);
+    else k_tile_producer<false, NH>(&kmap, a, bars, k_smem, S, r, h, layer, L, t_begin, n_tiles, lane, abort_flag, 0, 1);
   } else if (warp <= 2) {
     // ---------------- MMA issuers: A = Q block in TMEM, B = K tile in shared memory ----------------
     // Two warps, one per accumulator: warp 1 issues the even jobs into accumulator 0, warp 2 the odd jobs

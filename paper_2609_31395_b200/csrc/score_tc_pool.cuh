@@ -15,7 +15,8 @@ namespace actkv {
 namespace tc {
 
 constexpr int POOL_EPI_WARPS = 8;
-constexpr int POOL_THREADS = (3 + POOL_EPI_WARPS) * 32;     // producer, two MMA issuers, epilogue
+constexpr int POOL_THREADS = (4 + POOL_EPI_WARPS) * 32;     // producer, two MMA issuers, epilogue, second producer
+constexpr int POOL_PRODUCER2 = 3 + POOL_EPI_WARPS;          // warp index of the second producer
 
 struct PoolBarriers {
   uint64_t k_full[8];
@@ -165,8 +166,12 @@ score_tc_pool_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_cons
           tma_load_3d(q_smem + (qb >> 1) * 2 * QBLK_BYTES + hf * QBLK_BYTES + (qb & 1) * HALF_BYTES, &qmap,
                       smem_u32(&bars->q_full), hf * 64, h * G, wrow + qb * (128 / G));
     }
-    if (ta.k5) k_tile_producer<true, NH>(&kmap, a, bars, k_smem, S, r, h, layer, L, t_begin, n_tiles, lane, abort_flag);
-    else k_tile_producer<false, NH>(&kmap, a, bars, k_smem, S, r, h, layer, L, t_begin, n_tiles, lane, abort_flag);
+    if (ta.k5) k_tile_producer<true, NH>(&kmap, a, bars, k_smem, S, r, h, layer, L, t_begin, n_tiles, lane, abort_flag, 0, 2);
+    else k_tile_producer<false, NH>(&kmap, a, bars, k_smem, S, r, h, layer, L, t_begin, n_tiles, lane, abort_flag, 0, 2);
+  } else if (warp == POOL_PRODUCER2) {
+    const int layer = a.layer_begin + slab;
+    if (ta.k5) k_tile_producer<true, NH>(&kmap, a, bars, k_smem, S, r, h, layer, L, t_begin, n_tiles, lane, abort_flag, 1, 2);
+    else k_tile_producer<false, NH>(&kmap, a, bars, k_smem, S, r, h, layer, L, t_begin, n_tiles, lane, abort_flag, 1, 2);
   } else if (warp <= 2) {
     // ---------------- MMA issuers: D[key, row] = K Q^T ----------------
     // Two warps, one per accumulator: warp 1 issues the even jobs, warp 2 the odd ones.  Issuing costs the
