@@ -52,9 +52,10 @@ typedef struct CUstream_st* actkv_stream_t;
  * The paged pool, Section 2.5: PagedKVCache[2, B, BS, H, D] per layer.
  * Element (layer l, kv in {0 = K, 1 = V}, page p, slot s, head h, dim d) lives at
  *   base + l*stride_layer + kv*stride_kv + p*stride_page + s*stride_slot + h*stride_head + d.
- * The tensor-core score path needs page_size 16, head_dim 128, stride_head == head_dim,
- * stride_slot == n_kv_heads*head_dim, stride_page == page_size*stride_slot and a 128-byte
- * aligned base; other layouts take the FMA path.
+ * Any strides with contiguous head dimensions describe a pool (slot-major [page][slot][head][dim]
+ * pages as well as head-major [page][head][slot][dim] ones).  The tensor-core score path needs
+ * page_size 16, 32, 64 or 128, head_dim 64 or 128, strides that are multiples of 8 elements and a
+ * 128-byte aligned base; other shapes take the (much slower) FMA path.
  */
 typedef struct {
   void*   base;                 /* device, bf16 */

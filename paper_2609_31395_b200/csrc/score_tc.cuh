@@ -58,14 +58,14 @@ inline bool make_maps(const actkv_pool_t* pool, const void* q, int nls, int sum_
     // K half of the pool.  Slot-major pages whose slots continue across pages: [layer][slot (page*16 + s)]
     // [head][dim], four dimensions (measured 13 % faster than five on the K stream).  Any other page layout
     // (head-major pages): [layer][page][head][slot][dim] with the caller's strides.  A box is one page of
-    // one head, 64 dims: 16 rows of 128 B.
+    // one head, 64 dims: page_size rows of 128 B.
     CUresult res;
     if (!pool_needs_5d(pool)) {
       cuuint64_t dims[4] = {(cuuint64_t)pool->head_dim, (cuuint64_t)pool->n_kv_heads, (cuuint64_t)pool->n_pages * pool->page_size,
                             (cuuint64_t)pool->n_layers};
       cuuint64_t strides[3] = {(cuuint64_t)pool->stride_head * 2, (cuuint64_t)pool->stride_slot * 2,
                                (cuuint64_t)pool->stride_layer * 2};
-      cuuint32_t box[4] = {64, 1, 16, 1};
+      cuuint32_t box[4] = {64, 1, (cuuint32_t)pool->page_size, 1};
       cuuint32_t es[4] = {1, 1, 1, 1};
       res = enc(kmap, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, pool->base, dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
                 CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
@@ -74,7 +74,7 @@ inline bool make_maps(const actkv_pool_t* pool, const void* q, int nls, int sum_
                             (cuuint64_t)pool->n_pages, (cuuint64_t)pool->n_layers};
       cuuint64_t strides[4] = {(cuuint64_t)pool->stride_slot * 2, (cuuint64_t)pool->stride_head * 2,
                                (cuuint64_t)pool->stride_page * 2, (cuuint64_t)pool->stride_layer * 2};
-      cuuint32_t box[5] = {64, 16, 1, 1, 1};
+      cuuint32_t box[5] = {64, (cuuint32_t)pool->page_size, 1, 1, 1};
       cuuint32_t es[5] = {1, 1, 1, 1, 1};
       res = enc(kmap, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, pool->base, dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
                 CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
@@ -100,7 +100,7 @@ constexpr size_t SMEM_LIMIT = 232448;        // 227 KB of dynamic shared memory 
 
 }  // namespace tc
 
-// The tensor-core path takes: page 16, head_dim 128 or 64, slot-major or head-major pages (any strides that are
+// The tensor-core path takes: pages of 16, 32, 64 or 128 tokens, head_dim 128 or 64, slot-major or head-major pages (any strides that are
 // multiples of 16 bytes), 128-byte aligned
 // base, power-of-two group size <= 32, min_rows <= window x group rows <= 4096 (a CTA handles up to 512;
 // more are taken in groups of 512 rows), positive softmax scale.
@@ -108,7 +108,8 @@ constexpr size_t SMEM_LIMIT = 232448;        // 227 KB of dynamic shared memory 
 // pooled pass alone and is bound by the K reads, from a single row.
 inline bool score_tc_supported(const actkv_pool_t* p, int G, int max_win, float sm_scale, const void* q,
                                int min_rows = 64) {
-  if (p->page_size != 16 || (p->head_dim != 128 && p->head_dim != 64)) return false;
+  if (p->page_size != 16 && p->page_size != 32 && p->page_size != 64 && p->page_size != 128) return false;
+  if (p->head_dim != 128 && p->head_dim != 64) return false;
   // TMA: every stride a positive multiple of 16 bytes (any page layout with contiguous head dimensions)
   if (p->stride_head <= 0 || p->stride_slot <= 0 || p->stride_page <= 0 || p->stride_layer <= 0) return false;
   if ((p->stride_head % 8) || (p->stride_slot % 8) || (p->stride_page % 8) || (p->stride_layer % 8)) return false;

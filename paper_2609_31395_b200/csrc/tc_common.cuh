@@ -295,29 +295,35 @@ __device__ __forceinline__ int32_t page_for_tile(const TablesView& tab, int32_t 
   return checked_page(tab, n_pages, r, lp, status);
 }
 
-// The K-tile producers of both score kernels (two warps): producer p of P takes tiles p, p + P, ... of
+// The K-tile producers of both score kernels: producer p of P takes tiles p, p + P, ... of
 // [t_begin, t_begin + n_tiles) of request r, head h, layer `layer` through the block table into the ring of S
-// stages, one TMA box per (page, 64-dim half), one box per lane.  Measured on B200 (boxes of 16 rows x
-// 128 B from random pages): one warp issuing a tile's 16 boxes from 8 lanes delivers a tile per 1950
-// cycles, from 16 lanes per 1570, two warps per 1235, four per 1180 (the memory system's rate).  Only the
-// streaming update is bound by this.
-// Page ids of four of the producer's tiles at a time, one per lane (lane / 8 = tile within the group,
-// lane % 8 = page); the next group's ids are loaded while the current four tiles are being issued.
+// stages, one TMA box per (page, 64-dim half), one box per lane.  Pages of 16, 32, 64 or 128 tokens: a
+// tile of 128 keys is ppt = 128 / page_size pages, a box page_size rows of 128 B.
+// Measured on B200 (boxes of 16 rows x 128 B from random pages): one warp issuing a tile's 16 boxes from
+// 8 lanes delivers a tile per 1950 cycles, from 16 lanes per 1570, two warps per 1235, four per 1180 (the
+// memory system's rate).  Only the streaming update is bound by this.
+// Page ids of four of the producer's tiles at a time, one per lane (lane / ppt = tile within the group,
+// lane % ppt = page); the next group's ids are loaded while the current four tiles are being issued.
 // K5: five-dimensional tensor map (pages that are not slot-major).
 template <bool K5, int NH, class Bars>
 __device__ __forceinline__ void k_tile_producer(const CUtensorMap* kmap, const ScoreArgs& a, Bars* bars, uint32_t k_smem,
                                                 int S, int r, int h, int layer, int L, int t_begin, int n_tiles,
                                                 int lane, volatile int* abort_flag, int p, int P) {
-  const int n_lp = (L + a.pool.page_size - 1) / a.pool.page_size;
+  const int ps = a.pool.page_size;
+  const int ppt = TK / ps;                                      // pages per tile: 8, 4, 2 or 1
+  const int lp_shift = 31 - __clz(ppt);                         // log2(ppt)
+  const uint32_t box_bytes = (uint32_t)ps * 128u;
+  const int n_lp = (L + ps - 1) / ps;
   const int n_mine = (n_tiles - p + P - 1) / P;                  // tiles p, p + P, ... below n_tiles
-  int32_t pid = page_for_tile(a.tab, a.pool.n_pages, r, (t_begin + p + (lane >> 3) * P) * 8 + (lane & 7), n_lp, a.status);
+  const int g_tile = lane >> lp_shift, g_page = lane & (ppt - 1);            // this lane's slot in a group of four tiles
+  int32_t pid = page_for_tile(a.tab, a.pool.n_pages, r, (t_begin + p + min(g_tile, 3) * P) * ppt + g_page, n_lp, a.status);
   int32_t pid_next = 0;
   for (int i = 0; i < n_mine; ++i) {
     const int it = p + i * P;
     const int s = it % S;
     const uint32_t ph = (uint32_t)(it / S) & 1u;
     if ((i & 3) == 0 && i + 4 < n_mine)
-      pid_next = page_for_tile(a.tab, a.pool.n_pages, r, (t_begin + p + (i + 4 + (lane >> 3)) * P) * 8 + (lane & 7), n_lp,
+      pid_next = page_for_tile(a.tab, a.pool.n_pages, r, (t_begin + p + (i + 4 + min(g_tile, 3)) * P) * ppt + g_page, n_lp,
                                a.status);
     int ok = 1;
     if (lane == 0) {
@@ -330,15 +336,15 @@ __device__ __forceinline__ void k_tile_producer(const CUtensorMap* kmap, const S
     }
     ok = __shfl_sync(0xffffffffu, ok, 0);
     if (!ok) break;
-    // lane j < 8 NH: page j % 8, half j / 8 of this tile
-    const int32_t my_pid = __shfl_sync(0xffffffffu, pid, ((i & 3) << 3) | (lane & 7));
+    // lane j < ppt NH: page j % ppt, half j / ppt of this tile
+    const int32_t my_pid = __shfl_sync(0xffffffffu, pid, ((i & 3) << lp_shift) | (lane & (ppt - 1)));
 #ifndef ACTKV_EXP_NO_TMA
-    if (lane < 8 * NH) {
-      const int half = lane >> 3;
-      const uint32_t dst = k_smem + s * KTILE_BYTES + half * HALF_BYTES + (lane & 7) * 2048;
+    if (lane < ppt * NH) {
+      const int half = lane >> lp_shift;
+      const uint32_t dst = k_smem + s * KTILE_BYTES + half * HALF_BYTES + (lane & (ppt - 1)) * box_bytes;
       const uint32_t bar = smem_u32(&bars->k_full[s]);
       if constexpr (K5) tma_load_5d(dst, kmap, bar, half * 64, 0, h, my_pid, layer);
-      else tma_load_4d(dst, kmap, bar, half * 64, h, my_pid * 16, layer);
+      else tma_load_4d(dst, kmap, bar, half * 64, h, my_pid * ps, layer);
     }
 #else
     (void)my_pid;

@@ -163,6 +163,16 @@ def test_head_dim_64_on_the_tensor_core_path(causal):
         _full_check(synth.generate(wl, DEV))
 
 
+@pytest.mark.parametrize("page", [32, 64, 128])
+def test_larger_pages_on_the_tensor_core_path(page):
+    """Pages of 32, 64 and 128 tokens: a key tile is 4, 2 or 1 TMA boxes per 64-dim half."""
+    for head_dim, causal in [(128, False), (64, True)]:
+        wl = synth.Workload("pages", 2, 2, 4, [1000, 333, 130], [32, 16, 20], [250, 100, 40], head_dim=head_dim,
+                            page_size=page, table_style="fragmented", causal=causal, seed=page + head_dim,
+                            poison_tail=True)
+        _full_check(synth.generate(wl, DEV))
+
+
 def test_head_major_pool_layout():
     """A pool stored [layer][K/V][page][head][slot][dim] (HND pages), described to the library by its
     strides alone: score (FMA path and tensor-core path), select and compaction give the same results as
