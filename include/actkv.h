@@ -331,7 +331,8 @@ int actkv_compact_inplace(const actkv_pool_t* pool /* host */, const actkv_table
  * are shared by all calls on a device: host threads must not run this entry point concurrently on
  * the same device.
  * layers_per_call: capacity of score_dev / sel_idx_dev / the score workspace in layers (0: all
- * layers).  The library works in groups of min(layers_per_call, 16) layers.
+ * layers).  The LSE passes run in groups of at most min(layers_per_call, 16) layers (the first one
+ * shorter) while the queries arrive; the passes after them in groups of layers_per_call layers.
  * Every pointer named *_host is host memory, every other pointer device memory owned by the caller
  * and sized as the corresponding argument of the per-stage calls (score_dev:
  * [layers_per_call, n_kv_heads, sum_tok]; sel_idx_dev: [layers_per_call*n_kv_heads, sel_stride];

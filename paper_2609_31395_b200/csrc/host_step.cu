@@ -78,7 +78,10 @@ static int step_enqueue(const actkv_pool_t* pool, const actkv_tables_t* tab, con
                                                                                  : kDefaultGroupLayers;
   if (lpc > NL) lpc = NL;
   if ((NL + lpc - 1) / lpc + 1 > kMaxGroups) return ACTKV_E_INVALID;
-  const int n_groups = (NL + lpc - 1) / lpc;                  // groups of the passes that follow the LSE
+  // The passes that follow the LSE work on resident queries: as many layers per call as the caller's score
+  // and index buffers hold (layers_per_call; all layers when it is left open).
+  const int lpc_post = io->layers_per_call > 0 && io->layers_per_call < NL ? io->layers_per_call : NL;
+  const int n_groups = (NL + lpc_post - 1) / lpc_post;
   // Groups of the query copies and LSE passes: a short first group, so that the first kernel starts
   // after a quarter of a group's transfer time, then groups of lpc layers.
   int lse_bound[kMaxGroups + 1];
@@ -143,7 +146,7 @@ static int step_enqueue(const actkv_pool_t* pool, const actkv_tables_t* tab, con
   }
   // ---- then the other passes; the budgets are first needed by the first select ----
   for (int g = 0; g < n_groups; ++g) {
-    const int l0 = g * lpc, l1 = l0 + lpc < NL ? l0 + lpc : NL;
+    const int l0 = g * lpc_post, l1 = l0 + lpc_post < NL ? l0 + lpc_post : NL;
     ACTKV_TRY(actkv_score(pool, tab, l0, l1, (const char*)io->q_dev + (size_t)l0 * q_layer_bytes, io->win_indptr_dev,
                           io->n_q_heads, io->lse_dev + (size_t)l0 * io->sum_win * io->n_q_heads, io->sm_scale, io->causal,
                           io->tok_indptr_dev, io->score_dev, nullptr, io->sum_win, io->max_win, io->sum_tok,
