@@ -502,6 +502,34 @@ def run_ours(args):
                        "queries_per_request": 1, "layers_per_call": NL}
         del run_io
 
+    # ---- the confidence monitor on a serving-mix sized batch of logit rows (64 requests x 64 action tokens,
+    # 2.5 GB): the 512 rows of the step above are too few launches to show the kernel's rate.
+    budget_line = None
+    if not args.no_stream:
+        Rb, Tb = 64, 64
+        lg, lt = synth.confidence_logits(Rb, Tb, VOCAB, seed=wl.seed + 7, device=dev)
+        ch = torch.zeros((Rb, hist_cap), dtype=torch.float32, device=dev)
+        hl = torch.zeros(Rb, dtype=torch.int32, device=dev)
+        sl = torch.full((Rb,), 35000, dtype=torch.int32, device=dev)
+        bi = torch.full((Rb,), 512, dtype=torch.int32, device=dev)
+        bo = torch.zeros(Rb, dtype=torch.int32, device=dev)
+        wsb = torch.empty(B.actkv_budget_workspace_bytes(Rb * Tb, Rb, hist_cap) + 256, dtype=torch.uint8, device=dev)
+        ev = [torch.cuda.Event(enable_timing=True) for _ in range(2)]
+        n_it = 3 + min(args.steps, 10)
+        for it in range(n_it):
+            if it == 3:
+                ev[0].record()
+            hl.zero_()
+            B.actkv_budget(lg, lt, Rb * Tb, VOCAB, ch, hl, hist_cap, B.BudgetParams.paper_defaults(), sl, bi, bo, None,
+                           Rb, wsb, comp.status)
+        ev[1].record()
+        torch.cuda.synchronize()
+        comp.check_status()
+        msb = ev[0].elapsed_time(ev[1]) / (n_it - 3)
+        gb = 4.0 * Rb * Tb * VOCAB / (msb * 1e-3) / 1e9
+        budget_line = {"ms_per_call": msb, "rows": Rb * Tb, "vocab": VOCAB, "gbs": gb, "frac_of_hbm_peak": gb / pk["hbm_gbs"]}
+        del lg, ch, wsb
+
     # ---- the same step compacting in place into the tail blocks (Algorithm 4) instead of fresh pages.
     # Run last: it overwrites evicted slots of the original layout, which the fresh-page form never does.
     inplace_line = None
@@ -559,6 +587,7 @@ def run_ours(args):
             "with_inplace_compaction": inplace_line, "streaming_update": stream_line,
             "algorithmic_bytes_per_step": alg_bytes, "k_bytes_per_pass": bytes_k,
             "roofline": roofline, "roofline_stages": stages, "roofline_lse_exp_rate": lse_exp,
+            "budget_4096_rows": budget_line,
             "cpu_baseline": cpu_baseline, "e2e": e2e,
             "clocks": clocks, "gpu_launches": launches, "wall_s_timed_region": t_wall,
         }

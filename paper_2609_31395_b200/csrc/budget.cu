@@ -53,10 +53,17 @@ __device__ __forceinline__ double block_reduce_sum(double v, double* sm) {
 __device__ __forceinline__ void pick_digit(const uint32_t* hist, int nbins, uint32_t remaining,
                                            uint32_t* warp_tot, uint32_t* s_out) {
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  // nbins <= 2048 = 2 * TC_NT: each thread owns two adjacent reversed bins
-  const int b0 = nbins - 1 - 2 * tid, b1 = b0 - 1;
-  const uint32_t v0 = (b0 >= 0) ? hist[b0] : 0u, v1 = (b1 >= 0) ? hist[b1] : 0u;
-  uint32_t incl = v0 + v1;
+  // each thread owns `per` (at most 4) adjacent bins, descending from nbins - 1 - per * tid
+  const int per = (nbins + (int)blockDim.x - 1) / (int)blockDim.x;
+  const int b0 = nbins - 1 - per * tid;
+  uint32_t v[4], mine = 0;
+#pragma unroll
+  for (int j = 0; j < 4; ++j) {
+    const int b = b0 - j;
+    v[j] = (j < per && b >= 0) ? hist[b] : 0u;
+    mine += v[j];
+  }
+  uint32_t incl = mine;
 #pragma unroll
   for (int d = 1; d < 32; d <<= 1) {
     uint32_t t = __shfl_up_sync(0xffffffffu, incl, d);
@@ -64,13 +71,16 @@ __device__ __forceinline__ void pick_digit(const uint32_t* hist, int nbins, uint
   }
   if (lane == 31) warp_tot[warp] = incl;
   __syncthreads();
-  uint32_t add = 0;
-  for (int w = 0; w < warp; ++w) add += warp_tot[w];
-  incl += add;                                   // #(digit >= b1)
-  const uint32_t ge0 = incl - v1;                // #(digit >= b0)
-  const uint32_t gt0 = ge0 - v0;                 // #(digit >  b0)
-  if (b0 >= 0 && ge0 >= remaining && gt0 < remaining) { s_out[0] = (uint32_t)b0; s_out[1] = remaining - gt0; s_out[2] = v0; }
-  if (b1 >= 0 && incl >= remaining && ge0 < remaining) { s_out[0] = (uint32_t)b1; s_out[1] = remaining - ge0; s_out[2] = v1; }
+  uint32_t acc = incl - mine;                    // #(digit > b0)
+  for (int w = 0; w < warp; ++w) acc += warp_tot[w];
+#pragma unroll
+  for (int j = 0; j < 4; ++j) {
+    const int b = b0 - j;
+    if (j < per && b >= 0 && acc < remaining && acc + v[j] >= remaining) {
+      s_out[0] = (uint32_t)b; s_out[1] = remaining - acc; s_out[2] = v[j];
+    }
+    acc += v[j];
+  }
   __syncthreads();
 }
 
@@ -184,24 +194,32 @@ __global__ void __launch_bounds__(TC_NT) token_conf_kernel(
 }
 
 // -----------------------------------------------------------------------------------------------
-// Single-sweep token confidence.  The k-th largest of any subset of a row is a lower bound of the
-// k-th largest of the row, so: (A) take the first SW_HEAD logits into shared memory and find their
-// k-th largest tau exactly; (B) stream the rest of the row ONCE from HBM with an online
-// (max, sum of exp) per thread, appending the few logits >= tau to a shared candidate list;
-// (C) the top k of head-candidates + list are the top k of the row.  Rows whose list overflows
-// (adversarial order, e.g. ascending logits) are flagged and redone by the three-sweep kernel.
-constexpr int SW_HEAD = 8192;
+// Single-sweep token confidence.  A lower bound tau of the row's k-th largest logit lets one sweep keep
+// only the few logits >= tau while it sums the exponentials:
+//  (A) the first SW_HEAD logits are split into 64 chunks; the k-th largest of the 64 chunk maxima is tau
+//      (k of the row's logits are at least that large; k <= 64), the largest of them the reference M of
+//      the exponentials;
+//  (B) the row is streamed ONCE from HBM: sum of exp(x - M) per thread, logits >= tau appended to a shared
+//      candidate list (about half a percent of the row);
+//  (C) the top k of the list are the top k of the row: exact radix select in shared memory.
+// Rows whose list overflows (adversarial order, e.g. ascending logits), whose sum overflows (M is not the
+// row's maximum) or with k > 64 are flagged and redone by the three-sweep kernel.
+// Two CTAs of 512 threads per SM: one streams while the other is in its serial phases.
+constexpr int SW_HEAD = 4096;
 constexpr int SW_CAP = 4096;
+constexpr int SW_NT = 512;
+constexpr int SW_PER = SW_HEAD / SW_NT;     // head logits per thread (8: a chunk is 8 lanes x 8 = 64 logits)
 
 struct SweepSmem {
-  float head[SW_HEAD];
   float cand[SW_CAP];
   uint32_t hist[2048];
-  uint32_t warp_tot[TC_NT / 32];
+  float chunk_max[64];
+  uint32_t warp_tot[SW_NT / 32];
   uint32_t pick[3];
   uint32_t n_cand;
-  float red_f[TC_NT / 32];
-  double red_d[TC_NT / 32];
+  float tau, ref;
+  float red_f[SW_NT / 32];
+  double red_d[SW_NT / 32];
 };
 
 // k-th largest (k >= 1) of vals[0..n) by three radix digits; all threads call it.  Returns the key of
@@ -213,9 +231,9 @@ __device__ __forceinline__ void smem_kth_largest(const float* vals, int n, uint3
   for (int pass = 0; pass < 3; ++pass) {
     const int nb = pass == 2 ? 1024 : 2048;
     const int shift = pass == 0 ? 21 : (pass == 1 ? 10 : 0);
-    for (int i = tid; i < nb; i += TC_NT) sm->hist[i] = 0;
+    for (int i = tid; i < nb; i += SW_NT) sm->hist[i] = 0;
     __syncthreads();
-    for (int i = tid; i < n; i += TC_NT) {
+    for (int i = tid; i < n; i += SW_NT) {
       const uint32_t key = okey(vals[i]);
       const bool in = pass == 0 || (pass == 1 ? (key >> 21) == prefix : (key >> 10) == prefix);
       if (in) atomicAdd(&sm->hist[(key >> shift) & (uint32_t)(nb - 1)], 1u);
@@ -230,7 +248,7 @@ __device__ __forceinline__ void smem_kth_largest(const float* vals, int n, uint3
   need_out = remaining;
 }
 
-__global__ void __launch_bounds__(TC_NT, 1) token_conf_sweep_kernel(
+__global__ void __launch_bounds__(SW_NT, 2) token_conf_sweep_kernel(
     const float* __restrict__ logits, const int32_t* __restrict__ tok_indptr, int32_t vocab, int32_t n_req,
     int32_t k_top, float* __restrict__ conf_hist, const int32_t* __restrict__ hist_len, int32_t hist_cap,
     int32_t* __restrict__ redo, int32_t* status) {
@@ -241,74 +259,87 @@ __global__ void __launch_bounds__(TC_NT, 1) token_conf_sweep_kernel(
   const int k = min(k_top, vocab);
   const int n_head = min(vocab, SW_HEAD);
 
-  // ---- (A) head of the row -> shared memory, its k-th largest is the candidate threshold ----
-  for (int i = tid; i < n_head; i += TC_NT) sm->head[i] = z[i];
+  // ---- (A) threshold and reference from the chunk maxima of the head ----
+  const bool vec = (vocab % 4 == 0) && ((reinterpret_cast<uintptr_t>(z) & 15) == 0);
+  float hv[SW_PER];
+  float hm = -INFINITY;
+#pragma unroll
+  for (int j = 0; j < SW_PER; ++j) {
+    const int i = tid * SW_PER + j;
+    hv[j] = (i < n_head) ? z[i] : -INFINITY;
+    hm = fmaxf(hm, hv[j]);
+  }
+#pragma unroll
+  for (int o = 4; o >= 1; o >>= 1) hm = fmaxf(hm, __shfl_xor_sync(0xffffffffu, hm, o));     // over 8 lanes
+  if ((tid & 7) == 0) sm->chunk_max[tid >> 3] = hm;
   if (tid == 0) sm->n_cand = 0;
   __syncthreads();
-  uint32_t tau_key, need;
-  smem_kth_largest(sm->head, n_head, (uint32_t)k, sm, tau_key, need);
-  const float tau = okey_inv(tau_key);
-
-  // ---- (B) one sweep: online (max, sum exp2) per thread, candidates >= tau ----
-  float m = -INFINITY, s = 0.f;
-  auto visit = [&](float x, bool collect) {
-    if (x > m) { s *= exp2f((m - x) * kLog2e); m = x; }      // m = -inf: s is 0 and stays 0
-    s += exp2f((x - m) * kLog2e);
-    if (collect && x >= tau) {
-      const uint32_t pos = atomicAdd(&sm->n_cand, 1u);
-      if (pos < SW_CAP) sm->cand[pos] = x;
+  if (tid < 64) {
+    const float v = sm->chunk_max[tid];
+    int rank = 0;                                            // chunk maxima that come before this one, descending
+    float top = -INFINITY;
+    for (int u = 0; u < 64; ++u) {
+      const float w = sm->chunk_max[u];
+      rank += (w > v || (w == v && u < tid)) ? 1 : 0;
+      top = fmaxf(top, w);
     }
-  };
-  for (int i = tid; i < n_head; i += TC_NT) visit(sm->head[i], false);
-  const bool vec = (vocab % 4 == 0) && ((reinterpret_cast<uintptr_t>(z) & 15) == 0) && (SW_HEAD % 4 == 0);
-  if (vec) {
-    const float4* z4 = reinterpret_cast<const float4*>(z);
-    const int n4 = vocab / 4;
-    int i = SW_HEAD / 4 + tid;
-    for (; i + 3 * TC_NT < n4; i += 4 * TC_NT) {               // four 16-byte loads in flight per thread
-      const float4 a = z4[i], b = z4[i + TC_NT], c = z4[i + 2 * TC_NT], d = z4[i + 3 * TC_NT];
-      visit(a.x, true); visit(a.y, true); visit(a.z, true); visit(a.w, true);
-      visit(b.x, true); visit(b.y, true); visit(b.z, true); visit(b.w, true);
-      visit(c.x, true); visit(c.y, true); visit(c.z, true); visit(c.w, true);
-      visit(d.x, true); visit(d.y, true); visit(d.z, true); visit(d.w, true);
-    }
-    for (; i < n4; i += TC_NT) {
-      const float4 a = z4[i];
-      visit(a.x, true); visit(a.y, true); visit(a.z, true); visit(a.w, true);
-    }
-  } else {
-    for (int i = SW_HEAD + tid; i < vocab; i += TC_NT) visit(z[i], true);
+    if (rank == k - 1) sm->tau = v;
+    if (tid == 0) sm->ref = top;
   }
-  // block (max, sum): fixed-order trees
-  const float M = block_reduce_max(m, sm->red_f);
-  const double S = block_reduce_sum((m > -INFINITY) ? (double)s * (double)exp2f((m - M) * kLog2e) : 0.0, sm->red_d);
   __syncthreads();
-  const uint32_t n_cand = sm->n_cand;
-  if (n_cand > SW_CAP) {                                     // adversarial order: leave the row to the fallback
+  const float tau = sm->tau, M = sm->ref;
+  if (k > 64 || !(M > -INFINITY)) {                          // (uniform) no bound from 64 maxima: the fallback's row
     if (tid == 0) redo[row] = 1;
     return;
   }
-  // ---- (C) top k of {head elements >= tau} U candidates ----
-  // move the head's own candidates behind the streamed ones (at most k + ties of them; ties could be many,
-  // so the count is checked again)
-  for (int i = tid; i < n_head; i += TC_NT) {
-    const float x = sm->head[i];
+
+  // ---- (B) one sweep: sum of exp(x - M) per thread, candidates >= tau.  M is the maximum of the head, not
+  //      of the row: later logits may exceed it (the sum may grow up to the float range; a row whose sum
+  //      overflows is left to the fallback) ----
+  const float nmc = -M * kLog2e;
+  float s = 0.f;
+  auto visit = [&](float x) {
+    s += exp2f(fmaf(x, kLog2e, nmc));
     if (x >= tau) {
       const uint32_t pos = atomicAdd(&sm->n_cand, 1u);
       if (pos < SW_CAP) sm->cand[pos] = x;
     }
+  };
+#pragma unroll
+  for (int j = 0; j < SW_PER; ++j)
+    if (tid * SW_PER + j < n_head) visit(hv[j]);
+  if (vec) {
+    const float4* z4 = reinterpret_cast<const float4*>(z);
+    const int n4 = vocab / 4;
+    int i = SW_HEAD / 4 + tid;
+    for (; i + 7 * SW_NT < n4; i += 8 * SW_NT) {               // eight 16-byte loads in flight per thread
+      float4 v[8];
+#pragma unroll
+      for (int j = 0; j < 8; ++j) v[j] = z4[i + j * SW_NT];
+#pragma unroll
+      for (int j = 0; j < 8; ++j) { visit(v[j].x); visit(v[j].y); visit(v[j].z); visit(v[j].w); }
+    }
+    for (; i < n4; i += SW_NT) {
+      const float4 a = z4[i];
+      visit(a.x); visit(a.y); visit(a.z); visit(a.w);
+    }
+  } else {
+    for (int i = SW_HEAD + tid; i < vocab; i += SW_NT) visit(z[i]);
   }
+  const double S = block_reduce_sum((double)s, sm->red_d);   // fixed-order tree
   __syncthreads();
-  const uint32_t n_all = sm->n_cand;
-  if (n_all > SW_CAP) {
+  const uint32_t n_cand = sm->n_cand;
+  if (n_cand > SW_CAP || !(S < 3.0e38)) {                    // adversarial order or overflow: the fallback's row
     if (tid == 0) redo[row] = 1;
     return;
   }
+  // ---- (C) the top k of the candidates are the top k of the row ----
+  const uint32_t n_all = n_cand;
   uint32_t kth_key, need_k;
   smem_kth_largest(sm->cand, (int)n_all, (uint32_t)k, sm, kth_key, need_k);
   const float kth = okey_inv(kth_key);
   double top = 0.0;
-  for (int i = tid; i < (int)n_all; i += TC_NT) {
+  for (int i = tid; i < (int)n_all; i += SW_NT) {
     const float x = sm->cand[i];
     if (okey(x) > kth_key) top += (double)x;
   }
@@ -439,7 +470,7 @@ int actkv_budget(const float* logits, const int32_t* tok_indptr, int32_t n_rows,
     if (cudaFuncSetAttribute(actkv::token_conf_sweep_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm) !=
         cudaSuccess)
       return ACTKV_E_CUDA;
-    actkv::token_conf_sweep_kernel<<<(unsigned)n_rows, actkv::TC_NT, sm, s>>>(
+    actkv::token_conf_sweep_kernel<<<(unsigned)n_rows, actkv::SW_NT, sm, s>>>(
         logits, tok_indptr, vocab, n_req, params->k, conf_hist, hist_len, hist_cap, redo, status);
     ACTKV_CHECK_LAUNCH();
     actkv::token_conf_kernel<<<(unsigned)n_rows, actkv::TC_NT, 0, s>>>(

@@ -110,6 +110,24 @@ def test_sorted_rows_overflow_the_candidate_list_and_are_redone():
              B.BudgetParams.paper_defaults())
 
 
+def test_rows_the_single_sweep_cannot_take_are_redone():
+    """The single-sweep kernel takes its exp reference from the head of the row and its threshold from 64
+    chunk maxima: rows whose later logits dwarf the head (the sum would overflow) and calls with k > 64 go
+    to the three-sweep kernel."""
+    R, T, V = 2, 70, 151936
+    g = torch.Generator(device=DEV)
+    g.manual_seed(78)
+    logits = torch.randn((R * T, V), generator=g, device=DEV)
+    logits[:T, 100000:100040] += 95.0                                      # exp(95 - head maximum) is beyond float32
+    tok = torch.arange(0, (R + 1) * T, T, dtype=torch.int32, device=DEV)
+    hist0 = torch.zeros((R, 128), dtype=torch.float32)
+    len0 = torch.zeros(R, dtype=torch.int32)
+    _compare(logits, tok, hist0, len0, torch.tensor([512, 512], dtype=torch.int32), B.BudgetParams.paper_defaults())
+    p = B.BudgetParams.paper_defaults()
+    p.k = 100
+    _compare(logits[T:], tok[:2].clone(), hist0[:1], len0[:1], torch.tensor([512], dtype=torch.int32), p)
+
+
 def test_history_accumulates_across_calls_and_clamp():
     R, T, V = 4, 40, 2048
     p = B.BudgetParams.paper_defaults(clamp_lo_ppm=150000, clamp_hi_ppm=400000)
