@@ -375,7 +375,7 @@ def run_ours(args):
     # DRAM bytes per (token, KV head, layer) measured with ncu on the 2-layer cut of this workload
     # (profiles/kernels_c3_2layers_full_set.md: dram__bytes_read.sum + dram__bytes_write.sum over
     # 280000 tokens x 4 heads x 2 layers), scaled to one launch of this run by its unit count
-    ncu_bytes_per_unit = {"lse": 588.9e6 / 2.24e6, "score": 597.6e6 / 2.24e6, "compact": 551.6e6 / 2.24e6}
+    ncu_bytes_per_unit = {"lse": 588.1e6 / 2.24e6, "score": 595.3e6 / 2.24e6, "compact": 551.6e6 / 2.24e6}
     traffic = ncu_bytes_per_unit[dom] * tokens * Hkv * NL / n_calls if args.workload == "c3" else None
     roofline.update({"kernel": dom, "launches_per_step": n_calls, "ms_per_launch": stage_ms[dom] / n_calls,
                      "traffic": traffic, "traffic_unit": "bytes per launch (ncu, scaled from the 2-layer capture)", "peak_source": pk["source"] + (" sustained bf16" if stages[dom]["bound"] == "tensor" else " copy")})
