@@ -112,7 +112,7 @@ static int score_impl(int mode, const actkv_pool_t* pool, const actkv_tables_t* 
   // (the streaming update keeps a running mean in place, which the row-group launches of a window above
   // 512 rows would break: such calls take the FMA path)
   const bool use_tc = score_tc_supported(pool, G, max_win, sm_scale, q, acc_steps ? 1 : 64) &&
-                      !(acc_steps != nullptr && max_win * G > tc::MAX_ROWS);
+                      !(acc_steps != nullptr && max_win * tc::pow2_at_least(G) > tc::MAX_ROWS);
 
   const float* lse = lse_in;
   if (mode & 1) {

@@ -50,6 +50,8 @@ inline EncodeTiledFn encode_fn() {
 // The four-dimensional K map needs the slots of consecutive pages to continue at the slot stride.
 inline bool pool_needs_5d(const actkv_pool_t* pool) { return pool->stride_page != (int64_t)pool->page_size * pool->stride_slot; }
 
+inline int pow2_at_least(int g) { int p = 1; while (p < g) p <<= 1; return p; }
+
 inline bool make_maps(const actkv_pool_t* pool, const void* q, int nls, int sum_win, int n_q_heads, int G,
                       CUtensorMap* kmap, CUtensorMap* qmap) {
   EncodeTiledFn enc = encode_fn();
@@ -86,7 +88,8 @@ inline bool make_maps(const actkv_pool_t* pool, const void* q, int nls, int sum_
     const cuuint64_t D = (cuuint64_t)pool->head_dim;
     cuuint64_t dims[3] = {D, (cuuint64_t)n_q_heads, (cuuint64_t)nls * sum_win};
     cuuint64_t strides[2] = {D * 2, (cuuint64_t)n_q_heads * D * 2};
-    cuuint32_t box[3] = {64, (cuuint32_t)G, (cuuint32_t)(128 / G)};
+    const int Gp = pow2_at_least(G);                 // the pooled-score kernel pads a group to a power of two
+    cuuint32_t box[3] = {64, (cuuint32_t)Gp, (cuuint32_t)(128 / Gp)};
     cuuint32_t es[3] = {1, 1, 1};
     if (enc(qmap, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(q), dims, strides, box, es,
             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
@@ -102,7 +105,7 @@ constexpr size_t SMEM_LIMIT = 232448;        // 227 KB of dynamic shared memory 
 
 // The tensor-core path takes: pages of 16, 32, 64 or 128 tokens, head_dim 128 or 64, slot-major or head-major pages (any strides that are
 // multiples of 16 bytes), 128-byte aligned
-// base, power-of-two group size <= 32, min_rows <= window x group rows <= 4096 (a CTA handles up to 512;
+// base, group size <= 32 (padded to a power of two in the pooled-score pass), min_rows <= window x group rows <= 4096 (a CTA handles up to 512;
 // more are taken in groups of 512 rows), positive softmax scale.
 // The full score (LSE + pooled pass) takes it from 64 rows up; the streaming update, which runs the
 // pooled pass alone and is bound by the K reads, from a single row.
@@ -114,10 +117,10 @@ inline bool score_tc_supported(const actkv_pool_t* p, int G, int max_win, float 
   if (p->stride_head <= 0 || p->stride_slot <= 0 || p->stride_page <= 0 || p->stride_layer <= 0) return false;
   if ((p->stride_head % 8) || (p->stride_slot % 8) || (p->stride_page % 8) || (p->stride_layer % 8)) return false;
   if (((uintptr_t)p->base & 127) || ((uintptr_t)q & 127)) return false;
-  if (G < 1 || G > 32 || (G & (G - 1)) != 0) return false;
-  const int rows = max_win * G;
-  if (rows < min_rows || rows > tc::MAX_ROWS_TOTAL) return false;
-  if (rows > tc::MAX_ROWS && tc::MAX_ROWS % G != 0) return false;
+  if (G < 1 || G > 32) return false;
+  if (max_win * G < min_rows) return false;
+  const int rows = max_win * tc::pow2_at_least(G);     // rows of the pooled-score pass (groups padded to a power of two)
+  if (rows > tc::MAX_ROWS_TOTAL) return false;
   if (!(sm_scale > 0.f)) return false;
   if (getenv("ACTKV_FORCE_FMA") != nullptr) return false;
   return tc::encode_fn() != nullptr;
@@ -175,7 +178,8 @@ inline int score_tc_launch_score(ScoreArgs& a, const actkv_pool_t* pool, int max
   if (!tc::make_maps(pool, a.q, a.n_layers_sub, a.sum_win, a.n_q_heads, a.group, &kmap, &qmap)) return ACTKV_E_CUDA;
   tc::TcArgs ta;
   ta.a = a;
-  const int rows_all = max_win * a.group;
+  const int Gp = tc::pow2_at_least(a.group);
+  const int rows_all = max_win * Gp;
   const int rows_pad = (std::min(rows_all, tc::MAX_ROWS) + 127) & ~127;      // per launch
   const int n_rc = (rows_pad + 255) / 256;
   const size_t q_bytes = (size_t)n_rc * 2 * tc::QBLK_BYTES;
@@ -202,7 +206,7 @@ inline int score_tc_launch_score(ScoreArgs& a, const actkv_pool_t* pool, int max
   for (int row_begin = 0; row_begin < rows_all; row_begin += tc::MAX_ROWS) {
     ta.row_begin = row_begin;
     int rc = ACTKV_E_INVALID;
-    switch (a.group) {
+    switch (Gp) {
       case 1: rc = score_tc_launch_pool_g<1>(kmap, qmap, ta, (unsigned)grid, smem, s); break;
       case 2: rc = score_tc_launch_pool_g<2>(kmap, qmap, ta, (unsigned)grid, smem, s); break;
       case 4: rc = score_tc_launch_pool_g<4>(kmap, qmap, ta, (unsigned)grid, smem, s); break;

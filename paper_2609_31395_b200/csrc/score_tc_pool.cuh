@@ -81,6 +81,9 @@ __device__ __forceinline__ void pool_job(uint32_t taddr, const float* nlse, int 
   }
 }
 
+// G: the group size rounded up to a power of two.  A group of a.group < G query heads is padded with
+// rows that drop out of the max (-lse = -inf); their queries are whatever the TMA box picks up behind
+// the group (the next group's heads, or zeros past the last head).
 // NH: 64-dim halves of the head dimension (head_dim = 64 NH).
 template <int G, int NH>
 __global__ void __launch_bounds__(POOL_THREADS, 1)
@@ -142,9 +145,10 @@ score_tc_pool_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_cons
   }
   {
     // -lse of every row in log2 units; padding rows get -inf so that s*c + nlse drops out of the max
-    const float* lse_base = a.lse + ((int64_t)slab * a.sum_win + w0 + w_begin) * a.n_q_heads + h * G;
+    const int g_real = a.group;
+    const float* lse_base = a.lse + ((int64_t)slab * a.sum_win + w0 + w_begin) * a.n_q_heads + h * g_real;
     for (int n = threadIdx.x; n < rows_pad; n += blockDim.x)
-      nlse[n] = (n < rows) ? -lse_base[(int64_t)(n / G) * a.n_q_heads + (n % G)] * kLog2e : -INFINITY;
+      nlse[n] = (n < rows && (n % G) < g_real) ? -lse_base[(int64_t)(n / G) * a.n_q_heads + (n % G)] * kLog2e : -INFINITY;
   }
   if (warp == 1) {
     tmem_alloc(smem_u32(&bars->tmem_base), 512);
@@ -164,7 +168,7 @@ score_tc_pool_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_cons
       for (int qb = 0; qb < n_qblk; ++qb)
         for (int hf = 0; hf < NH; ++hf)
           tma_load_3d(q_smem + (qb >> 1) * 2 * QBLK_BYTES + hf * QBLK_BYTES + (qb & 1) * HALF_BYTES, &qmap,
-                      smem_u32(&bars->q_full), hf * 64, h * G, wrow + qb * (128 / G));
+                      smem_u32(&bars->q_full), hf * 64, h * a.group, wrow + qb * (128 / G));
     }
     if (ta.k5) k_tile_producer<true, NH>(&kmap, a, bars, k_smem, S, r, h, layer, L, t_begin, n_tiles, lane, abort_flag, 0, 2);
     else k_tile_producer<false, NH>(&kmap, a, bars, k_smem, S, r, h, layer, L, t_begin, n_tiles, lane, abort_flag, 0, 2);

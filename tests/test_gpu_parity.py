@@ -173,6 +173,37 @@ def test_larger_pages_on_the_tensor_core_path(page):
         _full_check(synth.generate(wl, DEV))
 
 
+@pytest.mark.parametrize("causal", [False, True])
+def test_group_sizes_that_are_not_powers_of_two(causal):
+    """G = 3, 5, 6, 7 query heads per KV head on the tensor-core path: the pooled-score pass pads a group to
+    the next power of two with rows that drop out of the max; the last group's padding reads past the last
+    query head."""
+    for W, G in [(32, 3), (24, 5), (100, 6), (40, 7)]:
+        wl = synth.Workload("odd-g", 2, 2, G, [900, 300], [W, max(1, W // 3)], [300, 80], table_style="fragmented",
+                            causal=causal, seed=W * 5 + G, poison_tail=True)
+        _full_check(synth.generate(wl, DEV))
+
+
+def test_new_shapes_really_take_the_tensor_core_path(monkeypatch):
+    """The library picks the path by itself; forcing the FMA path (developer switch) must change the bits of
+    the scores for the shapes that are meant to run on tensor cores."""
+    shapes = [dict(G=7), dict(G=4, head_dim=64), dict(G=4, page_size=64), dict(G=16, windows=[64, 20])]
+    for kw in shapes:
+        G = kw.pop("G")
+        windows = kw.pop("windows", [32, 16])
+        wl = synth.Workload("path", 1, 2, G, [700, 257], windows, [200, 64], table_style="permutation", seed=31,
+                            poison_tail=True, **kw)
+        inst = synth.generate(wl, DEV)
+        monkeypatch.delenv("ACTKV_FORCE_FMA", raising=False)
+        tc_score = U.run_step(inst).score.clone()
+        inst = synth.generate(wl, DEV)
+        monkeypatch.setenv("ACTKV_FORCE_FMA", "1")
+        fma_score = U.run_step(inst).score.clone()
+        monkeypatch.delenv("ACTKV_FORCE_FMA", raising=False)
+        assert not torch.equal(tc_score, fma_score)
+        assert torch.allclose(tc_score, fma_score, rtol=2e-3, atol=0)
+
+
 def test_head_major_pool_layout():
     """A pool stored [layer][K/V][page][head][slot][dim] (HND pages), described to the library by its
     strides alone: score (FMA path and tensor-core path), select and compaction give the same results as

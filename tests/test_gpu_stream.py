@@ -94,9 +94,10 @@ def _wl(head_dim=128, page=16, G=4, NL=4):
                           table_style="fragmented", seed=21, poison_tail=True)
 
 
-@pytest.mark.parametrize("head_dim,page,G", [(128, 16, 4), (128, 16, 8), (64, 8, 2)])
+@pytest.mark.parametrize("head_dim,page,G", [(128, 16, 4), (128, 16, 8), (64, 8, 2), (128, 16, 3), (64, 32, 7)])
 def test_one_query_per_call_matches_oracle_and_batch(head_dim, page, G):
-    """(128, 16, .) runs the tensor-core pooled pass with G live rows, (64, 8, 2) the FMA path."""
+    """(., 16 or 32, .) runs the tensor-core pooled pass with G live rows (a group of 3 or 7 padded to 4 or 8),
+    (64, 8, 2) the FMA path."""
     inst = synth.generate(_wl(head_dim, page, G), DEV)
     wl = inst.wl
     pool_bits = U.bits(inst.pool)
