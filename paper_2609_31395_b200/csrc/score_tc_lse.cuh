@@ -346,12 +346,16 @@ score_tc_lse_kernel(const __grid_constant__ CUtensorMap kmap, const TcArgs ta) {
     const int jfast = min(min(jm[0], jm[1]), min(jm[2], jm[3]));
     const float c = a.scale_log2, c1 = c * (1.f / 252.f);
     const uint32_t tq = tmem_base + ((uint32_t)(quarter * 32) << 16) + LSE_A_COLS + grp * 128 + half * 64;
+    // (key tile, row block) of this group's jobs, carried along without divisions: job = tile * n_mb + mb
+    int mb = grp % n_mb, key0 = (t_begin + grp / n_mb) * TK + half * 64;
+    const int mb_step = 2 % n_mb, tile_step = 2 / n_mb;
     for (int job = grp; job < n_jobs; job += 2) {
-      const int it = job / n_mb, mb = job - it * n_mb;
-      const int key0 = (t_begin + it) * TK + half * 64;
       epi_ok = lse_job<NPOLY>(bars, abort_flag, tq, grp, job, mb, &bars->state[grp][mb][half][rib], jfast - key0 + 1, jm, key0, c,
                               c1, lane);
       if (!epi_ok) break;
+      mb += mb_step;
+      key0 += tile_step * TK;
+      if (mb >= n_mb) { mb -= n_mb; key0 += TK; }
     }
   }
   // ---------------- teardown ----------------
