@@ -142,18 +142,18 @@ template <int NPOLY>
 __device__ __forceinline__ bool lse_job(LseBarriers* bars, volatile int* abort_flag, uint32_t tq, int grp, int job,
                                         int mb, float2* st, int nv_min, const int (&jm)[4], int key0, float c, float c1,
                                         int lane) {
-  float va[32], vb[32];
+  float v[64];
+  float* va = v;
+  float* vb = v + 32;
   LSE_TR(5, job, threadIdx.x == 3 * 32);
   if (!mbar_wait(smem_u32(&bars->tmem_full[grp]), (uint32_t)(job >> 1) & 1u, abort_flag)) return false;
   tc_fence_after();
 #ifndef ACTKV_EXP_NO_LD
-  tmem_ld32(tq, va);
-  tmem_ld32(tq + 32, vb);
+  tmem_ld64(tq, v);
 #endif
   float2 ms = *st;
   tmem_ld_wait();
-  tmem_ld_fence<32>(va);
-  tmem_ld_fence<32>(vb);
+  tmem_ld_fence<64>(v);
   LSE_TR(2, job, threadIdx.x == 3 * 32);
   tc_fence_before();
   __syncwarp();
