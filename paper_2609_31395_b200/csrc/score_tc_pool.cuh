@@ -3,10 +3,10 @@
 //
 // D[key, row] = K Q^T: the 128 keys of a tile sit on the TMEM lanes, row = w*G + g on the columns,
 // 256 columns per accumulator, two accumulators in the 512 TMEM columns.  A "job" is one (key tile,
-// 256-row chunk) accumulator.  Two epilogue warpgroups take the jobs of even / odd parity, so one
-// drains accumulator 0 while the tensor pipe fills accumulator 1 and the other warpgroup drains it.
-// With two row chunks per tile the warpgroups hold partial sums over different action tokens of the
-// same keys; warpgroup 1 hands its partial to warpgroup 0 through shared memory.
+// 256-row chunk) accumulator; even jobs use accumulator 0, odd jobs accumulator 1, each with its own
+// MMA-issuing warp.  Both epilogue warpgroups work on every job, each on one half of the columns, so an
+// accumulator goes back to its MMA warp after one 64-column step; a thread adds up its half over the row
+// chunks of a tile and warpgroup 1 hands its sum to warpgroup 0 through shared memory.
 #pragma once
 
 #include "tc_common.cuh"
@@ -53,7 +53,8 @@ __device__ __forceinline__ void pool_job(uint32_t taddr, const float* nlse, int 
       tmem_ld_wait();
       if (c2 + 1 < n_c2) {
         tmem_ld64(taddr + (c2 + 1) * 64, v[(c2 + 1) & 1]);
-      } else {
+      }
+      if (c2 + 1 >= n_c2) {
         tc_fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive(empty_bar);
@@ -111,6 +112,7 @@ score_tc_pool_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_cons
   const int t_end = min((L + TK - 1) / TK, t_begin + ta.tiles_per_cta);
   const int n_tiles = t_end - t_begin;
   const int rows_pad = (rows + 127) & ~127;               // <= MAX_ROWS (checked by the host)
+  const bool split = rows > 128;                          // both epilogue warpgroups on every job (see the epilogue)
   const int n_rc = (rows_pad + 255) / 256;                // 256-row chunks per key tile: 1 or 2
   const int n_qblk = rows_pad / 128;
   const int n_jobs = n_tiles * n_rc;
@@ -134,7 +136,7 @@ score_tc_pool_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_cons
     mbar_init(smem_u32(&bars->q_full), 1);
     for (int b = 0; b < 2; ++b) {
       mbar_init(smem_u32(&bars->tmem_full[b]), 1);
-      mbar_init(smem_u32(&bars->tmem_empty[b]), POOL_EPI_WARPS / 2);
+      mbar_init(smem_u32(&bars->tmem_empty[b]), split ? POOL_EPI_WARPS : POOL_EPI_WARPS / 2);
     }
     mbar_init(smem_u32(&bars->part_full), POOL_EPI_WARPS / 2);
     mbar_init(smem_u32(&bars->part_empty), POOL_EPI_WARPS / 2);
@@ -231,49 +233,62 @@ score_tc_pool_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_cons
     mbar_wait(smem_u32(&bars->drained[mw]), 0, abort_flag, ok ? WAIT_LIMIT_NS : DRAIN_LIMIT_NS);
     __syncwarp();
   } else {
-    // ---------------- epilogue: one key per thread, jobs of this warpgroup's parity ----------------
-    const int wg = (warp - 3) >> 2;               // 0 or 1 = accumulator it drains
+    // ---------------- epilogue: one key per thread ----------------
+    // More than 128 live rows: both warpgroups work on every job, warpgroup 0 on columns [0, 128) of the
+    // accumulator, warpgroup 1 on columns [128, 256), so an accumulator is back with its MMA warp after one
+    // 64-column step instead of three (how long an accumulator is held, not the arithmetic, is what this
+    // pass waits for besides the MMAs).  A thread adds up its share over the row chunks of a key tile; at
+    // the end of the tile warpgroup 1 hands its sum to warpgroup 0 through shared memory, which stores.
+    // At most 128 live rows (a streaming update): the warpgroups take alternate jobs whole, so that two
+    // epilogues (and their read-modify-write of the running mean) are in flight.
+    const int wg = (warp - 3) >> 2;
     const int quarter = warp & 3;                 // TMEM lane quarter this warp may read
     const float c = a.scale_log2;
     const float inv_w = 1.0f / (float)W;
     float* out = a.score_out + ((int64_t)slab * Hkv + h) * a.sum_tok + a.tok_indptr[r];
-    const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + wg * 256;
-    for (int job = wg; job < n_jobs; job += 2) {
+    const int half = split ? wg : 0;              // this warp's columns: [128 half, 128 half + 128)
+    const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + half * 128;
+    float acc = 0.f;
+    for (int job = split ? 0 : wg; job < n_jobs; job += split ? 1 : 2) {
+      const int b = job & 1;
       const int it = (n_rc == 2) ? (job >> 1) : job;
       const int rc = (n_rc == 2) ? (job & 1) : 0;
       const int key = (t_begin + it) * TK + quarter * 32 + lane;
       // causal: row w sees key j iff j <= L - W + w  <=>  w >= j - (L - W)
       const int w_min = a.causal ? max(0, key - (L - W)) : 0;
-      if (!mbar_wait(smem_u32(&bars->tmem_full[wg]), (uint32_t)(job >> 1) & 1u, abort_flag)) break;
+      if (!mbar_wait(smem_u32(&bars->tmem_full[b]), (uint32_t)(job >> 1) & 1u, abort_flag)) break;
       tc_fence_after();
-      const int n_cg = (min(rows, rc * 256 + 256) - rc * 256 + 31) / 32;      // 32-column groups with live rows
-      float acc = 0.f;
+      const int n_cg_job = (min(rows, rc * 256 + 256) - rc * 256 + 31) / 32;  // 32-column groups with live rows
+      const int n_cg = min(4, n_cg_job - half * 4);                            // ... among this warp's columns
 #ifndef ACTKV_EXP_NO_EPI
-#ifdef ACTKV_EXP_NO_NLSE
-      pool_job<G>(taddr, nlse, 0 * n_cg + n_cg, w_begin + (rc * 256) / G, w_min, W, c, acc, smem_u32(&bars->tmem_empty[wg]), lane);
-#else
-      pool_job<G>(taddr, nlse + rc * 256, n_cg, w_begin + (rc * 256) / G, w_min, W, c, acc, smem_u32(&bars->tmem_empty[wg]), lane);
+      if (n_cg > 0) {
+        pool_job<G>(taddr + b * 256, nlse + rc * 256 + half * 128, n_cg, w_begin + (rc * 256 + half * 128) / G, w_min, W, c, acc,
+                    smem_u32(&bars->tmem_empty[b]), lane);
+      } else
 #endif
-#else
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(smem_u32(&bars->tmem_empty[wg]));
-#endif
-      if (n_rc == 1) {
-        if (key < L) { if (row_begin > 0) out[key] += acc * inv_w; else store_pooled(a, r, out + key, acc, acc * inv_w, W); }
-      } else if (wg == 1) {
-        // partial over the second row chunk: hand it to warpgroup 0 once it has read the previous tile's
+      {
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(smem_u32(&bars->tmem_empty[b]));
+      }
+      if (rc + 1 < n_rc) continue;
+      // the key tile is complete
+      if (split && wg == 1) {
+        // hand the sum to warpgroup 0 once it has read the previous tile's
         if (!mbar_wait(smem_u32(&bars->part_empty), ((uint32_t)it & 1u) ^ 1u, abort_flag)) break;
         bars->exch[quarter * 32 + lane] = acc;
         __syncwarp();
         if (lane == 0) mbar_arrive(smem_u32(&bars->part_full));
       } else {
-        if (!mbar_wait(smem_u32(&bars->part_full), (uint32_t)it & 1u, abort_flag)) break;
-        acc += bars->exch[quarter * 32 + lane];
-        __syncwarp();
-        if (lane == 0) mbar_arrive(smem_u32(&bars->part_empty));
+        if (split) {
+          if (!mbar_wait(smem_u32(&bars->part_full), (uint32_t)it & 1u, abort_flag)) break;
+          acc += bars->exch[quarter * 32 + lane];
+          __syncwarp();
+          if (lane == 0) mbar_arrive(smem_u32(&bars->part_empty));
+        }
         if (key < L) { if (row_begin > 0) out[key] += acc * inv_w; else store_pooled(a, r, out + key, acc, acc * inv_w, W); }
       }
+      acc = 0.f;
     }
   }
   // ---------------- teardown ----------------
