@@ -40,26 +40,20 @@ struct PoolBarriers {
 template <int G>
 __device__ __forceinline__ void pool_job(uint32_t taddr, const float* nlse, int n_cg, int w_first, int w_min, int w_end,
                                          float c, float& acc, uint32_t empty_bar, int lane) {
-  // 64 columns per load, two register buffers: the load of the next 64 columns is in flight while these
-  // are folded, so the round trip to tensor memory is paid four times per accumulator, not eight, and
-  // mostly hidden.  The accumulator is handed back to the MMA warp as soon as its last columns are in
-  // registers, before they are folded.
+  // At most 128 columns (n_cg <= 4 groups of 32): both 64-column loads are issued at once and the
+  // accumulator is handed back to the MMA warp as soon as they are in registers, before anything is folded.
   const int n_c2 = (n_cg + 1) >> 1;
   float v[2][64];
   tmem_ld64(taddr, v[0]);
+  if (n_c2 > 1) tmem_ld64(taddr + 64, v[1]);
+  tmem_ld_wait();
+  tc_fence_before();
+  __syncwarp();
+  if (lane == 0) mbar_arrive(empty_bar);
 #pragma unroll
-  for (int c2 = 0; c2 < 4; ++c2) {
+  for (int c2 = 0; c2 < 2; ++c2) {
     if (c2 < n_c2) {
-      tmem_ld_wait();
-      if (c2 + 1 < n_c2) {
-        tmem_ld64(taddr + (c2 + 1) * 64, v[(c2 + 1) & 1]);
-      }
-      if (c2 + 1 >= n_c2) {
-        tc_fence_before();
-        __syncwarp();
-        if (lane == 0) mbar_arrive(empty_bar);
-      }
-      float* x = v[c2 & 1];
+      float* x = v[c2];
       const float4* l4 = reinterpret_cast<const float4*>(nlse + c2 * 64);
 #pragma unroll
       for (int q4 = 0; q4 < 16; ++q4) {
