@@ -21,12 +21,26 @@ static ScoreWsLayout score_ws_layout(int32_t n_kv_heads, int32_t n_req, int32_t 
   ScoreWsLayout l;
   const int G = n_q_heads / (n_kv_heads > 0 ? n_kv_heads : 1);
   l.rows_max = max_win * G;
-  l.n_chunks = (max_tok + LSE_CHUNK - 1) / LSE_CHUNK;
-  if (l.n_chunks < 1) l.n_chunks = 1;
+  // Chunks per unit of a launch over `units` units: enough for LSE_ITEMS work items of at least
+  // LSE_CHUNK_LONG keys, or for LSE_ITEMS_MIN items of at least LSE_CHUNK keys when that leaves SMs idle.  units x n_chunks <= LSE_ITEMS + 2 units, and that bound grows with the unit count,
+  // so a workspace sized for a layer range also serves every call on fewer layers.
+  const int64_t units = (int64_t)nls * n_kv_heads * n_req;
+  const int64_t by_len = max_tok > 0 ? (max_tok + LSE_CHUNK - 1) / LSE_CHUNK : 1;
+  const int64_t by_len_long = max_tok > 0 ? (max_tok + LSE_CHUNK_LONG - 1) / LSE_CHUNK_LONG : 1;
+  int64_t nc = units > 0 ? (LSE_ITEMS + units - 1) / units : 1;
+  if (nc > by_len_long) nc = by_len_long;
+  if (units > 0 && units * nc < LSE_ITEMS_MIN) {   // a small problem: shorter chunks, so that every SM has work
+    nc = (LSE_ITEMS_MIN + units - 1) / units;
+    if (nc > by_len) nc = by_len;
+  }
+  if (nc < 1) nc = 1;
+  l.n_chunks = (int32_t)nc;
+  int64_t slots = units * by_len;
+  if (slots > LSE_ITEMS + 2 * units) slots = LSE_ITEMS + 2 * units;
   l.lse_off = 0;
   l.lse_bytes = align_up((size_t)nls * sum_win * n_q_heads * 4, 256);
   l.part_off = l.lse_bytes;
-  l.part_bytes = align_up((size_t)nls * n_kv_heads * n_req * l.n_chunks * l.rows_max * sizeof(float2), 256);
+  l.part_bytes = align_up((size_t)slots * l.rows_max * sizeof(float2), 256);
   l.total = l.part_off + l.part_bytes;
   return l;
 }
@@ -91,18 +105,14 @@ static int score_impl(int mode, const actkv_pool_t* pool, const actkv_tables_t* 
   a.rows_max = lay.rows_max;
   // Keys per LSE partial.  A CTA pays a fixed cost (operand set-up, pipeline fill and drain), so chunks
   // are as long as they can be while there are still many CTAs per SM (the last wave of a launch is
-  // partly empty): whole key tiles, about equal, at least 20 x 148 work items and never more chunks
-  // than the workspace holds.
+  // partly empty): whole key tiles, about equal, the chunk count of the workspace layout (a CTA covers
+  // all rows of its unit).
   {
-    const int64_t units_ = (int64_t)(layer_end - layer_begin) * Hkv * R;
-    int n_chunks = (int)((20 * 148 + units_ - 1) / units_);       // a CTA covers all rows of its unit
-    if (n_chunks < 1) n_chunks = 1;
-    if (n_chunks > lay.n_chunks) n_chunks = lay.n_chunks;
-    int chunk = (max_tok + n_chunks - 1) / n_chunks;
-    chunk = (chunk + 127) / 128 * 128;             // whole key tiles, about equal work per chunk
+    int chunk = (max_tok + lay.n_chunks - 1) / lay.n_chunks;
+    chunk = (chunk + 127) / 128 * 128;
     if (chunk < LSE_CHUNK) chunk = LSE_CHUNK;
     a.lse_chunk = chunk;
-    a.n_chunks = (max_tok + chunk - 1) / chunk;
+    a.n_chunks = (max_tok + chunk - 1) / chunk;    // <= lay.n_chunks
   }
   a.n_tiles = (max_tok + FMA_TK - 1) / FMA_TK;
   a.scale_log2 = sm_scale * kLog2e;

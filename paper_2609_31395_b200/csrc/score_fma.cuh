@@ -14,7 +14,10 @@ namespace actkv {
 constexpr int FMA_TK = 64;        // keys per tile
 constexpr int FMA_RQ = 32;        // window x group rows per chunk (at most)
 constexpr int FMA_NT = 256;       // threads per CTA
-constexpr int LSE_CHUNK = 4096;   // keys per partial (m, sum) of the LSE pass (both paths)
+constexpr int LSE_CHUNK = 512;    // fewest keys per partial (m, sum) of the LSE pass (both paths)
+constexpr int LSE_CHUNK_LONG = 4096;  // fewest keys per partial while the launch still has LSE_ITEMS_MIN work items
+constexpr int LSE_ITEMS = 20 * 148;  // work items an LSE launch aims for: 20 per SM
+constexpr int LSE_ITEMS_MIN = 4 * 148;
 
 struct ScoreArgs {
   PoolView pool;
@@ -66,7 +69,7 @@ __device__ __forceinline__ void load_rows_padded(uint32_t* dst, int n_rows, int 
   }
 }
 
-// One kernel for both passes.  PASS 1: partial (max, sum) of exp2 over a chunk of LSE_CHUNK keys
+// One kernel for both passes.  PASS 1: partial (max, sum) of exp2 over a chunk of lse_chunk keys
 // for every window row.  PASS 2: pooled score of a tile of FMA_TK keys.
 template <int PASS>
 __global__ void __launch_bounds__(FMA_NT) score_fma_kernel(const ScoreArgs a) {

@@ -225,6 +225,25 @@ def test_long_request_many_chunks():
     _full_check(synth.generate(wl, DEV))
 
 
+def test_workspace_sized_for_a_layer_range_serves_calls_on_fewer_layers():
+    """The LSE pass cuts a request into more chunks when a call has fewer units; the workspace of the
+    whole range must hold those partials too, and the scores do not depend on the cut."""
+    wl = synth.Workload("ws", 3, 1, 4, [20000 + 13], [32], [5000], table_style="fragmented", seed=6)
+    inst = synth.generate(wl, DEV)
+    sz = H.sizes_of(inst)
+    comp = H.Compressor(inst.pool, inst.page_table, inst.seq_len, inst.free_list, inst.free_count, wl.n_q_heads, sz,
+                        want_lse=True)
+    comp.run_score(inst.q, inst.win_indptr, inst.tok_indptr, wl.sm_scale, wl.causal)
+    torch.cuda.synchronize()
+    whole, whole_lse = comp.score.clone(), comp.lse.clone()
+    for l in range(3):
+        comp.run_score(inst.q, inst.win_indptr, inst.tok_indptr, wl.sm_scale, wl.causal, l0=l, l1=l + 1)
+        torch.cuda.synchronize()
+        comp.check_status()
+        assert (comp.lse[l] - whole_lse[l]).abs().max().item() < 1e-5
+        assert torch.allclose(comp.score[0], whole[l], rtol=1e-4, atol=1e-9)
+
+
 def test_logits_that_keep_growing_move_the_lse_reference():
     """Keys arranged so that every row's logits climb by hundreds of log2 units along the request: the
     LSE pass keeps no running maximum, so its reference must be moved again and again (and 2^x saturates
