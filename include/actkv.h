@@ -150,6 +150,8 @@ int actkv_budget(const float* logits, const int32_t* tok_indptr, int32_t n_rows,
  * sum_win, max_win, sum_tok, max_tok: host copies of win_indptr[n_req], max W_r,
  *            tok_indptr[n_req], max L_r (upper bounds are accepted for the two maxima).
  * W_r == 0 for a request with L_r > 0 is reported as ACTKV_E_INVALID in status.
+ * Workspace: the size for n_layers_sub layers also serves every call on fewer layers with the
+ * same other arguments.
  */
 size_t actkv_score_workspace_bytes(const actkv_pool_t* pool /* host */, int32_t n_req,
                                    int32_t n_layers_sub, int32_t n_q_heads, int32_t sum_win,
