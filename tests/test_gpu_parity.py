@@ -219,6 +219,27 @@ def test_head_major_pool_layout():
         _full_check(inst)
 
 
+def test_every_other_layer_as_a_strided_view():
+    """A model that interleaves sliding-window layers (bounded caches the method leaves alone) with
+    full-attention layers: the full-attention layers of one allocation are described to the library as a
+    pool whose layer stride skips the others.  Results match the oracle's logical view and the skipped
+    layers keep every bit."""
+    for wl in (synth.Workload("gptoss", 3, 2, 8, [1500, 300], [16, 9], [400, 80], head_dim=64,
+                              table_style="fragmented", seed=31, poison_tail=True),
+               _small(G=4, seed=32)):
+        inst = synth.generate(wl, DEV)
+        shape = list(inst.pool.shape)
+        shape[0] *= 2
+        g = torch.Generator(device=DEV).manual_seed(99)
+        big = torch.randn(shape, generator=g, device=DEV, dtype=torch.float32).to(torch.bfloat16)
+        big[0::2] = inst.pool
+        inst.pool = big[0::2]
+        assert inst.pool.stride(0) == 2 * big[0].numel()
+        others = big[1::2].clone()
+        _full_check(inst)
+        assert torch.equal(big[1::2].view(torch.int16), others.view(torch.int16))
+
+
 def test_long_request_many_chunks():
     """More keys than one LSE chunk and several key tiles per CTA; ragged last page."""
     wl = synth.Workload("long", 1, 1, 4, [9000 + 7], [32], [2300], table_style="fragmented", seed=5, poison_tail=True)
