@@ -322,13 +322,13 @@ score_tc_lse_kernel(const __grid_constant__ CUtensorMap kmap, const TcArgs ta) {
           a.q + (((int64_t)slab * a.sum_win + w0 + (live ? w : 0)) * a.n_q_heads + h * G + (live ? g : 0)) * (64 * NH));
       const uint32_t dst = tmem_base + ((uint32_t)(quarter * 32) << 16) + k * 64;
       if (k < n_mb) {
+        // (the whole row in flight at once: under load one round trip to L2 is thousands of cycles, and the
+        // MMA issuers wait for the last row)
+        uint4 x[8 * NH];
 #pragma unroll
-        for (int i = 0; i < 2 * NH; ++i) {
-          uint4 x[4];
+        for (int j = 0; j < 8 * NH; ++j) x[j] = live ? __ldg(src + j) : make_uint4(0, 0, 0, 0);
 #pragma unroll
-          for (int j = 0; j < 4; ++j) x[j] = live ? __ldg(src + i * 4 + j) : make_uint4(0, 0, 0, 0);
-          tmem_st16(dst + i * 16, reinterpret_cast<const uint32_t*>(x));
-        }
+        for (int i = 0; i < 2 * NH; ++i) tmem_st16(dst + i * 16, reinterpret_cast<const uint32_t*>(x + 4 * i));
         tmem_st_wait();
       }
       tc_fence_before();
