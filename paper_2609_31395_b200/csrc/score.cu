@@ -197,6 +197,11 @@ const char* actkv_version(void) { return "actkv-b200 0.1 (sm_100a)"; }
 
 }  // extern "C"
 
+#ifdef ACTKV_POOL_TRACE
+extern "C" int actkv_debug_pool_trace(long long* out_host) {
+  return cudaMemcpyFromSymbol(out_host, actkv::tc::g_pool_trace, sizeof(long long) * 6 * 1024) == cudaSuccess ? 0 : -1;
+}
+#endif
 #ifdef ACTKV_LSE_TRACE
 extern "C" int actkv_debug_lse_trace(long long* out_host) {
   return cudaMemcpyFromSymbol(out_host, actkv::tc::g_lse_trace, sizeof(long long) * 6 * 1024) == cudaSuccess ? 0 : -1;

@@ -18,6 +18,13 @@ constexpr int POOL_EPI_WARPS = 8;
 constexpr int POOL_THREADS = (4 + POOL_EPI_WARPS) * 32;     // producer, two MMA issuers, epilogue, second producer
 constexpr int POOL_PRODUCER2 = 3 + POOL_EPI_WARPS;          // warp index of the second producer
 
+#ifdef ACTKV_POOL_TRACE
+__device__ long long g_pool_trace[6][1024];      // developer build: per-job timestamps of one CTA
+#define POOL_TR(row, job, cond) do { if ((cond) && blockIdx.x == 200 && (job) < 1024) g_pool_trace[row][job] = clock64(); } while (0)
+#else
+#define POOL_TR(row, job, cond) do { } while (0)
+#endif
+
 struct PoolBarriers {
   uint64_t k_full[8];
   uint64_t k_empty[8];
@@ -200,10 +207,12 @@ score_tc_pool_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_cons
       bool mine = false;
       for (int rc = 0; rc < n_rc; ++rc, ++job) {
         if ((job & 1) != mw) continue;
+        POOL_TR(0, job, leader);
         ok = mbar_wait(empty_bar, epar, abort_flag);
         if (!ok) break;
         epar ^= 1u;
         tc_fence_after();
+        POOL_TR(1, job, leader);
         if (leader) {
           const uint64_t bdesc_c = qdesc0 + (uint64_t)((rc * 2 * QBLK_BYTES) >> 4);
 #pragma unroll
@@ -212,6 +221,7 @@ score_tc_pool_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_cons
                       bdesc_c + (uint64_t)(((kk >> 2) * QBLK_BYTES + (kk & 3) * 32) >> 4), idesc_c[rc], kk > 0 ? 1u : 0u);
           umma_commit(full_bar);
         }
+        POOL_TR(2, job, leader);
         mine = true;
       }
       if (!ok) break;
@@ -243,46 +253,101 @@ score_tc_pool_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_cons
     const int half = split ? wg : 0;              // this warp's columns: [128 half, 128 half + 128)
     const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + half * 128;
     float acc = 0.f;
-    for (int job = split ? 0 : wg; job < n_jobs; job += split ? 1 : 2) {
-      const int b = job & 1;
-      const int it = (n_rc == 2) ? (job >> 1) : job;
-      const int rc = (n_rc == 2) ? (job & 1) : 0;
-      const int key = (t_begin + it) * TK + quarter * 32 + lane;
-      // causal: row w sees key j iff j <= L - W + w  <=>  w >= j - (L - W)
-      const int w_min = a.causal ? max(0, key - (L - W)) : 0;
-      if (!mbar_wait(smem_u32(&bars->tmem_full[b]), (uint32_t)(job >> 1) & 1u, abort_flag)) break;
-      tc_fence_after();
-      const int n_cg_job = (min(rows, rc * 256 + 256) - rc * 256 + 31) / 32;  // 32-column groups with live rows
-      const int n_cg = min(4, n_cg_job - half * 4);                            // ... among this warp's columns
+    if (split) {
+      // what does not change from job to job, per row chunk
+      int ncg[2], wfirst[2];
+#pragma unroll
+      for (int rc = 0; rc < 2; ++rc) {
+        const int n_cg_job = (min(rows, rc * 256 + 256) - rc * 256 + 31) / 32;     // 32-column groups with live rows
+        ncg[rc] = min(4, n_cg_job - half * 4);                                      // ... among this warp's columns
+        wfirst[rc] = w_begin + (rc * 256 + half * 128) / G;
+      }
+      const int lw = L - W;
+      int key = t_begin * TK + quarter * 32 + lane;
+      int it = 0, rc = 0;
+      // Warpgroup 0 adds warpgroup 1's share of a key tile and stores one job later, when that share has
+      // long been written: neither warpgroup waits for the other at the end of a tile.
+      bool pending = false;
+      float acc_prev = 0.f;
+      int key_prev = 0;
+      uint32_t par_prev = 0;
+      bool ok = true;
+      for (int job = 0; job < n_jobs; ++job) {
+        const int b = job & 1;
+        // causal: row w sees key j iff j <= L - W + w  <=>  w >= j - (L - W)
+        const int w_min = a.causal ? max(0, key - lw) : 0;
+        POOL_TR(3, job, threadIdx.x == 3 * 32);
+        if (!mbar_wait(smem_u32(&bars->tmem_full[b]), (uint32_t)(job >> 1) & 1u, abort_flag)) { ok = false; break; }
+        tc_fence_after();
+        POOL_TR(4, job, threadIdx.x == 3 * 32);
+        const int n_cg = rc == 0 ? ncg[0] : ncg[1];
 #ifndef ACTKV_EXP_NO_EPI
-      if (n_cg > 0) {
-        pool_job<G>(taddr + b * 256, nlse + rc * 256 + half * 128, n_cg, w_begin + (rc * 256 + half * 128) / G, w_min, W, c, acc,
-                    smem_u32(&bars->tmem_empty[b]), lane);
-      } else
+        if (n_cg > 0) {
+          pool_job<G>(taddr + b * 256, nlse + rc * 256 + half * 128, n_cg, rc == 0 ? wfirst[0] : wfirst[1], w_min, W, c, acc,
+                      smem_u32(&bars->tmem_empty[b]), lane);
+        } else
 #endif
-      {
+        {
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(smem_u32(&bars->tmem_empty[b]));
+        }
+        POOL_TR(5, job, threadIdx.x == 3 * 32);
+        if (pending) {
+          if (!mbar_wait(smem_u32(&bars->part_full), par_prev, abort_flag)) { ok = false; break; }
+          acc_prev += bars->exch[quarter * 32 + lane];
+          __syncwarp();
+          if (lane == 0) mbar_arrive(smem_u32(&bars->part_empty));
+          if (key_prev < L) {
+            if (row_begin > 0) out[key_prev] += acc_prev * inv_w;
+            else store_pooled(a, r, out + key_prev, acc_prev, acc_prev * inv_w, W);
+          }
+          pending = false;
+        }
+        if (++rc < n_rc) continue;
+        // the key tile is complete
+        if (wg == 1) {
+          if (!mbar_wait(smem_u32(&bars->part_empty), ((uint32_t)it & 1u) ^ 1u, abort_flag)) { ok = false; break; }
+          bars->exch[quarter * 32 + lane] = acc;
+          __syncwarp();
+          if (lane == 0) mbar_arrive(smem_u32(&bars->part_full));
+        } else {
+          pending = true;
+          acc_prev = acc;
+          key_prev = key;
+          par_prev = (uint32_t)it & 1u;
+        }
+        acc = 0.f;
+        rc = 0;
+        ++it;
+        key += TK;
+      }
+      if (ok && pending && mbar_wait(smem_u32(&bars->part_full), par_prev, abort_flag)) {
+        acc_prev += bars->exch[quarter * 32 + lane];
+        if (key_prev < L) {
+          if (row_begin > 0) out[key_prev] += acc_prev * inv_w;
+          else store_pooled(a, r, out + key_prev, acc_prev, acc_prev * inv_w, W);
+        }
+      }
+    } else {
+      // at most 128 live rows: one row chunk per key tile, a job is a tile
+      for (int job = wg; job < n_jobs; job += 2) {
+        const int b = job & 1;
+        const int key = (t_begin + job) * TK + quarter * 32 + lane;
+        const int w_min = a.causal ? max(0, key - (L - W)) : 0;
+        if (!mbar_wait(smem_u32(&bars->tmem_full[b]), (uint32_t)(job >> 1) & 1u, abort_flag)) break;
+        tc_fence_after();
+        const int n_cg = (rows + 31) / 32;
+#ifndef ACTKV_EXP_NO_EPI
+        pool_job<G>(taddr + b * 256, nlse, n_cg, w_begin, w_min, W, c, acc, smem_u32(&bars->tmem_empty[b]), lane);
+#else
         tc_fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive(smem_u32(&bars->tmem_empty[b]));
-      }
-      if (rc + 1 < n_rc) continue;
-      // the key tile is complete
-      if (split && wg == 1) {
-        // hand the sum to warpgroup 0 once it has read the previous tile's
-        if (!mbar_wait(smem_u32(&bars->part_empty), ((uint32_t)it & 1u) ^ 1u, abort_flag)) break;
-        bars->exch[quarter * 32 + lane] = acc;
-        __syncwarp();
-        if (lane == 0) mbar_arrive(smem_u32(&bars->part_full));
-      } else {
-        if (split) {
-          if (!mbar_wait(smem_u32(&bars->part_full), (uint32_t)it & 1u, abort_flag)) break;
-          acc += bars->exch[quarter * 32 + lane];
-          __syncwarp();
-          if (lane == 0) mbar_arrive(smem_u32(&bars->part_empty));
-        }
+#endif
         if (key < L) { if (row_begin > 0) out[key] += acc * inv_w; else store_pooled(a, r, out + key, acc, acc * inv_w, W); }
+        acc = 0.f;
       }
-      acc = 0.f;
     }
   }
   // ---------------- teardown ----------------
