@@ -199,7 +199,7 @@ const char* actkv_version(void) { return "actkv-b200 0.1 (sm_100a)"; }
 
 #ifdef ACTKV_POOL_TRACE
 extern "C" int actkv_debug_pool_trace(long long* out_host) {
-  return cudaMemcpyFromSymbol(out_host, actkv::tc::g_pool_trace, sizeof(long long) * 6 * 1024) == cudaSuccess ? 0 : -1;
+  return cudaMemcpyFromSymbol(out_host, actkv::tc::g_pool_trace, sizeof(long long) * 8 * 1024) == cudaSuccess ? 0 : -1;
 }
 #endif
 #ifdef ACTKV_LSE_TRACE

@@ -52,6 +52,26 @@ inline bool pool_needs_5d(const actkv_pool_t* pool) { return pool->stride_page !
 
 inline int pow2_at_least(int g) { int p = 1; while (p < g) p <<= 1; return p; }
 
+// CTAs per unit for a launch over `units` units of `tiles` key tiles each.  One CTA is resident per SM, so a
+// launch runs in rounds of 148 CTAs and the last round is partly empty; more CTAs make that round
+// cheaper, but every CTA pays a fixed cost (operand set-up, pipeline fill and drain) of about `ovh` key
+// tiles' worth.  Returns the count in [1, n_max] with the best product of the two, preferring fewer CTAs
+// unless more are clearly better.
+inline int best_split(int64_t units, int tiles, int ovh, int n_max) {
+  int best = 1;
+  double best_eff = 0.0;
+  if (units < 1) units = 1;
+  for (int n = 1; n <= n_max; ++n) {
+    const int tpc = (tiles + n - 1) / n;
+    if (tpc < 1) break;
+    const int64_t grid = units * ((tiles + tpc - 1) / tpc);
+    const int64_t rounds = (grid + 147) / 148;
+    const double eff = (double)grid / (double)(rounds * 148) * (double)tpc / (double)(tpc + ovh);
+    if (eff > best_eff * 1.005) { best_eff = eff; best = n; }
+  }
+  return best;
+}
+
 inline bool make_maps(const actkv_pool_t* pool, const void* q, int nls, int sum_win, int n_q_heads, int G,
                       CUtensorMap* kmap, CUtensorMap* qmap) {
   EncodeTiledFn enc = encode_fn();
@@ -192,11 +212,11 @@ inline int score_tc_launch_score(ScoreArgs& a, const actkv_pool_t* pool, int max
   ta.k5 = tc::pool_needs_5d(pool) ? 1 : 0;
   const int64_t units = (int64_t)a.n_layers_sub * a.pool.n_kv_heads * a.tab.n_req;
   const int max_tiles = (max_tok + tc::TK - 1) / tc::TK;
-  // enough CTAs to fill the 148 SMs a few times over, few enough that the Q load is amortised
-  int64_t tpc = (units * max_tiles) / (148 * 6);
-  if (tpc < 4) tpc = 4;
-  if (tpc > max_tiles) tpc = max_tiles;
-  ta.tiles_per_cta = (int)tpc;
+  // CTAs per unit: one CTA per SM is resident, so the launch runs in rounds of 148 CTAs and the last round
+  // is partly empty; more CTAs make that round cheaper, but every CTA pays for its Q load and its pipeline
+  // fill (about three key tiles' worth).  Take the count with the best product of the two.
+  ta.n_kchunks = tc::best_split(units, max_tiles, 3, std::min(64, std::max(1, max_tiles / 4)));
+  ta.tiles_per_cta = (max_tiles + ta.n_kchunks - 1) / ta.n_kchunks;
   ta.n_kchunks = (max_tiles + ta.tiles_per_cta - 1) / ta.tiles_per_cta;
   const int64_t grid = units * ta.n_kchunks;
   if (grid > 0x7fffffffLL) return ACTKV_E_INVALID;

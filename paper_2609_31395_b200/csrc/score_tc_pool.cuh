@@ -19,7 +19,7 @@ constexpr int POOL_THREADS = (4 + POOL_EPI_WARPS) * 32;     // producer, two MMA
 constexpr int POOL_PRODUCER2 = 3 + POOL_EPI_WARPS;          // warp index of the second producer
 
 #ifdef ACTKV_POOL_TRACE
-__device__ long long g_pool_trace[6][1024];      // developer build: per-job timestamps of one CTA
+__device__ long long g_pool_trace[8][1024];      // developer build: per-job timestamps of one CTA
 #define POOL_TR(row, job, cond) do { if ((cond) && blockIdx.x == 200 && (job) < 1024) g_pool_trace[row][job] = clock64(); } while (0)
 #else
 #define POOL_TR(row, job, cond) do { } while (0)
@@ -46,7 +46,7 @@ struct PoolBarriers {
 // anything; whatever the arithmetic makes of them is discarded by the select).
 template <int G>
 __device__ __forceinline__ void pool_job(uint32_t taddr, const float* nlse, int n_cg, int w_first, int w_min, int w_end,
-                                         float c, float& acc, uint32_t empty_bar, int lane) {
+                                         float c, float& acc, uint32_t empty_bar, int lane, int job = 0) {
   // At most 128 columns (n_cg <= 4 groups of 32): both 64-column loads are issued at once and the
   // accumulator is handed back to the MMA warp as soon as they are in registers, before anything is folded.
   const int n_c2 = (n_cg + 1) >> 1;
@@ -57,6 +57,11 @@ __device__ __forceinline__ void pool_job(uint32_t taddr, const float* nlse, int 
   tc_fence_before();
   __syncwarp();
   if (lane == 0) mbar_arrive(empty_bar);
+  POOL_TR(6, job, threadIdx.x == 3 * 32);
+#ifdef ACTKV_EXP_NO_FOLD
+  acc += v[0][0] + v[1][0];          // developer switch: loads and hand-back only
+  return;
+#endif
 #pragma unroll
   for (int c2 = 0; c2 < 2; ++c2) {
     if (c2 < n_c2) {
@@ -284,7 +289,7 @@ score_tc_pool_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_cons
 #ifndef ACTKV_EXP_NO_EPI
         if (n_cg > 0) {
           pool_job<G>(taddr + b * 256, nlse + rc * 256 + half * 128, n_cg, rc == 0 ? wfirst[0] : wfirst[1], w_min, W, c, acc,
-                      smem_u32(&bars->tmem_empty[b]), lane);
+                      smem_u32(&bars->tmem_empty[b]), lane, job);
         } else
 #endif
         {
@@ -304,6 +309,7 @@ score_tc_pool_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_cons
           }
           pending = false;
         }
+        POOL_TR(7, job, threadIdx.x == 3 * 32);
         if (++rc < n_rc) continue;
         // the key tile is complete
         if (wg == 1) {
