@@ -99,7 +99,9 @@ __device__ __forceinline__ void lse_slow32(const float* v, int nv, float c, floa
 #ifdef ACTKV_LSE_TRACE
 __device__ long long g_lse_trace[6][1024];       // developer build: per-job timestamps of one CTA
 #define LSE_TR(row, job, cond) do { if ((cond) && blockIdx.x == 200 && (job) < 1024) g_lse_trace[row][job] = clock64(); } while (0)
+#define LSE_TR_NS(row, job, cond) do { if ((cond) && blockIdx.x == 200 && (job) < 1024) { unsigned long long t_; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t_)); g_lse_trace[row][job] = (long long)t_; } } while (0)
 #else
+#define LSE_TR_NS(row, job, cond) do { } while (0)
 #define LSE_TR(row, job, cond) do { } while (0)
 #endif
 
@@ -185,6 +187,8 @@ template <int NPOLY, bool ROW_GROUPS, int NH>
 __global__ void __launch_bounds__(LSE_THREADS, 1)
 score_tc_lse_kernel(const __grid_constant__ CUtensorMap kmap, const TcArgs ta) {
   extern __shared__ __align__(1024) uint8_t smem[];
+  LSE_TR(0, 1000, threadIdx.x == 32);
+  LSE_TR_NS(0, 1001, threadIdx.x == 32);
   const ScoreArgs& a = ta.a;
   const int R = a.tab.n_req, Hkv = a.pool.n_kv_heads, G = a.group;
   const int cu = blockIdx.x / a.n_chunks;
@@ -393,6 +397,8 @@ score_tc_lse_kernel(const __grid_constant__ CUtensorMap kmap, const TcArgs ta) {
     tc_fence_after();
     tmem_dealloc(tmem_base, 512);
   }
+  LSE_TR(0, 1002, threadIdx.x == 32);
+  LSE_TR_NS(0, 1003, threadIdx.x == 32);
 }
 
 }  // namespace tc

@@ -21,7 +21,9 @@ constexpr int POOL_PRODUCER2 = 3 + POOL_EPI_WARPS;          // warp index of the
 #ifdef ACTKV_POOL_TRACE
 __device__ long long g_pool_trace[8][1024];      // developer build: per-job timestamps of one CTA
 #define POOL_TR(row, job, cond) do { if ((cond) && blockIdx.x == 200 && (job) < 1024) g_pool_trace[row][job] = clock64(); } while (0)
+#define POOL_TR_NS(row, job, cond) do { if ((cond) && blockIdx.x == 200 && (job) < 1024) { unsigned long long t_; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t_)); g_pool_trace[row][job] = (long long)t_; } } while (0)
 #else
+#define POOL_TR_NS(row, job, cond) do { } while (0)
 #define POOL_TR(row, job, cond) do { } while (0)
 #endif
 
@@ -96,6 +98,8 @@ template <int G, int NH>
 __global__ void __launch_bounds__(POOL_THREADS, 1)
 score_tc_pool_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constant__ CUtensorMap qmap, const TcArgs ta) {
   extern __shared__ __align__(1024) uint8_t smem[];
+  POOL_TR(0, 1000, threadIdx.x == 32);
+  POOL_TR_NS(0, 1001, threadIdx.x == 32);
   const ScoreArgs& a = ta.a;
   const int R = a.tab.n_req, Hkv = a.pool.n_kv_heads;
   const int u = blockIdx.x / ta.n_kchunks;
@@ -368,6 +372,8 @@ score_tc_pool_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_cons
     tc_fence_after();
     tmem_dealloc(tmem_base, 512);
   }
+  POOL_TR(0, 1002, threadIdx.x == 32);
+  POOL_TR_NS(0, 1003, threadIdx.x == 32);
 }
 
 }  // namespace tc
