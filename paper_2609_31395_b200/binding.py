@@ -99,7 +99,8 @@ def load():
             raise
     if not os.path.exists(LIB_PATH):
         raise ActKVError("load: libactkv.so is missing; run __graft_entry__.build()", E_CUDA)
-    lib = C.CDLL(LIB_PATH)
+    # developer switch: another build of the same sources (dev_trace.py's build with per-job timestamps)
+    lib = C.CDLL(os.environ.get("ACTKV_LIB") or LIB_PATH)
     vp, i32, i64, sz, f32 = C.c_void_p, C.c_int32, C.c_int64, C.c_size_t, C.c_float
     lib.actkv_version.restype = C.c_char_p
     lib.actkv_budget_workspace_bytes.restype = sz

@@ -21,20 +21,21 @@ def _stale() -> bool:
     return any(os.path.getmtime(d) > t for d in deps)
 
 
-def build(force: bool = False, verbose: bool = False) -> str:
-    """Compile every .cu under csrc/ into libactkv.so; returns the library path."""
-    if not force and not _stale():
+def build(force: bool = False, verbose: bool = False, out: str = LIB, extra_flags=()) -> str:
+    """Compile every .cu under csrc/ into libactkv.so (or `out`, a developer build with `extra_flags`);
+    returns the library path."""
+    if out == LIB and not force and not _stale():
         return LIB
     nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
-    extra = os.environ.get("ACTKV_NVCC_FLAGS", "").split()       # developer switch: extra nvcc flags
-    cmd = [nvcc, "-shared", "-o", LIB] + NVCC_FLAGS + extra + (["-Xptxas", "-v"] if verbose else []) + \
+    extra = os.environ.get("ACTKV_NVCC_FLAGS", "").split() + list(extra_flags)   # developer switch: extra nvcc flags
+    cmd = [nvcc, "-shared", "-o", out] + NVCC_FLAGS + extra + (["-Xptxas", "-v"] if verbose else []) + \
           [os.path.join(CSRC, s) for s in SOURCES]
     res = subprocess.run(cmd, capture_output=True, text=True)
     if verbose:
         sys.stderr.write(res.stderr)
     if res.returncode != 0:
         raise RuntimeError("nvcc failed:\n" + res.stdout + res.stderr)
-    return LIB
+    return out
 
 
 if __name__ == "__main__":

@@ -147,7 +147,7 @@ __device__ __forceinline__ bool lse_job(LseBarriers* bars, volatile int* abort_f
   float v[64];
   float* va = v;
   float* vb = v + 32;
-  LSE_TR(5, job, threadIdx.x == 3 * 32);
+  LSE_TR(5, job, (threadIdx.x == 3 * 32 || threadIdx.x == 11 * 32));
   if (!mbar_wait(smem_u32(&bars->tmem_full[grp]), (uint32_t)(job >> 1) & 1u, abort_flag)) return false;
   tc_fence_after();
 #ifndef ACTKV_EXP_NO_LD
@@ -156,11 +156,11 @@ __device__ __forceinline__ bool lse_job(LseBarriers* bars, volatile int* abort_f
   float2 ms = *st;
   tmem_ld_wait();
   tmem_ld_fence<64>(v);
-  LSE_TR(2, job, threadIdx.x == 3 * 32);
+  LSE_TR(2, job, (threadIdx.x == 3 * 32 || threadIdx.x == 11 * 32));
   tc_fence_before();
   __syncwarp();
   if (lane == 0) mbar_arrive(smem_u32(&bars->tmem_empty[grp]));
-  LSE_TR(3, job, threadIdx.x == 3 * 32);
+  LSE_TR(3, job, (threadIdx.x == 3 * 32 || threadIdx.x == 11 * 32));
 #ifndef ACTKV_EXP_NO_EPI
   bool slow = __any_sync(0xffffffffu, nv_min < 64 || ms.x == -INFINITY);
   if (!slow) {
@@ -176,7 +176,7 @@ __device__ __forceinline__ bool lse_job(LseBarriers* bars, volatile int* abort_f
   }
   *st = ms;
 #endif
-  LSE_TR(4, job, threadIdx.x == 3 * 32);
+  LSE_TR(4, job, (threadIdx.x == 3 * 32 || threadIdx.x == 11 * 32));
   return true;
 }
 
