@@ -4,9 +4,8 @@
 // D[key, row] = K Q^T: the 128 keys of a tile sit on the TMEM lanes, row = w*G + g on the columns,
 // 256 columns per accumulator, two accumulators in the 512 TMEM columns.  A "job" is one (key tile,
 // 256-row chunk) accumulator; even jobs use accumulator 0, odd jobs accumulator 1, each with its own
-// MMA-issuing warp.  Both epilogue warpgroups work on every job, each on one half of the columns, so an
-// accumulator goes back to its MMA warp after one 64-column step; a thread adds up its half over the row
-// chunks of a tile and warpgroup 1 hands its sum to warpgroup 0 through shared memory.
+// MMA-issuing warp.  The two epilogue warpgroups take alternate jobs whole, one key per thread; with two
+// row chunks per key tile warpgroup 1 hands its sum of a tile to warpgroup 0 through shared memory.
 #pragma once
 
 #include "tc_common.cuh"
@@ -46,6 +45,32 @@ struct PoolBarriers {
 // Action tokens outside [w_min, w_end) do not count: below w_min the key is not visible yet (causal
 // rule), from w_end on the columns are padding (with a narrow MMA they were never written and may hold
 // anything; whatever the arithmetic makes of them is discarded by the select).
+// 64 columns of one accumulator lane: x = s for rows n .. n + 63 of this key, nlse = -lse*log2(e) of those rows
+// (-inf for padding rows).  Adds sum_w exp2(max_g(s*c + nlse)) over the action tokens w_first .. that lie
+// in [w_min, w_end) to `acc`.
+template <int G>
+__device__ __forceinline__ void pool_fold64(float* x, const float* nlse, int w_first, int w_min, int w_end, float c,
+                                            float& acc) {
+  const float4* l4 = reinterpret_cast<const float4*>(nlse);
+#pragma unroll
+  for (int q4 = 0; q4 < 16; ++q4) {
+#ifdef ACTKV_EXP_NO_NLSE
+    const float4 l = make_float4(-1.f, -1.f, -1.f, -1.f + (float)(l4 == nullptr));
+#else
+    const float4 l = l4[q4];
+#endif
+    ffma2(x[q4 * 4 + 0], x[q4 * 4 + 1], x[q4 * 4 + 0], x[q4 * 4 + 1], c, l.x, l.y);
+    ffma2(x[q4 * 4 + 2], x[q4 * 4 + 3], x[q4 * 4 + 2], x[q4 * 4 + 3], c, l.z, l.w);
+  }
+  constexpr int WPG = 64 / G;                 // action tokens per 64-column group (G <= 32)
+#pragma unroll
+  for (int i = 0; i < WPG; ++i) {
+    const float mx = max_of<G>(x + i * G);
+    const int w = w_first + i;
+    acc += (w >= w_min && w < w_end) ? exp2f(mx) : 0.f;
+  }
+}
+
 template <int G>
 __device__ __forceinline__ void pool_job(uint32_t taddr, const float* nlse, int n_cg, int w_first, int w_min, int w_end,
                                          float c, float& acc, uint32_t empty_bar, int lane, int job = 0) {
@@ -64,30 +89,8 @@ __device__ __forceinline__ void pool_job(uint32_t taddr, const float* nlse, int 
   acc += v[0][0] + v[1][0];          // developer switch: loads and hand-back only
   return;
 #endif
-#pragma unroll
-  for (int c2 = 0; c2 < 2; ++c2) {
-    if (c2 < n_c2) {
-      float* x = v[c2];
-      const float4* l4 = reinterpret_cast<const float4*>(nlse + c2 * 64);
-#pragma unroll
-      for (int q4 = 0; q4 < 16; ++q4) {
-#ifdef ACTKV_EXP_NO_NLSE
-        const float4 l = make_float4(-1.f, -1.f, -1.f, -1.f + (float)(l4 == nullptr));
-#else
-        const float4 l = l4[q4];
-#endif
-        ffma2(x[q4 * 4 + 0], x[q4 * 4 + 1], x[q4 * 4 + 0], x[q4 * 4 + 1], c, l.x, l.y);
-        ffma2(x[q4 * 4 + 2], x[q4 * 4 + 3], x[q4 * 4 + 2], x[q4 * 4 + 3], c, l.z, l.w);
-      }
-      constexpr int WPG = 64 / G;                 // action tokens per 64-column group (G <= 32)
-#pragma unroll
-      for (int i = 0; i < WPG; ++i) {
-        const float mx = max_of<G>(x + i * G);
-        const int w = w_first + c2 * WPG + i;
-        acc += (w >= w_min && w < w_end) ? exp2f(mx) : 0.f;
-      }
-    }
-  }
+  pool_fold64<G>(v[0], nlse, w_first, w_min, w_end, c, acc);
+  if (n_c2 > 1) pool_fold64<G>(v[1], nlse + 64, w_first + 64 / G, w_min, w_end, c, acc);
 }
 
 // G: the group size rounded up to a power of two.  A group of a.group < G query heads is padded with
@@ -122,7 +125,7 @@ score_tc_pool_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_cons
   const int t_end = min((L + TK - 1) / TK, t_begin + ta.tiles_per_cta);
   const int n_tiles = t_end - t_begin;
   const int rows_pad = (rows + 127) & ~127;               // <= MAX_ROWS (checked by the host)
-  const bool split = rows > 128;                          // both epilogue warpgroups on every job (see the epilogue)
+  const bool whole = rows > 128;                          // a job has up to 256 columns: two register loads (see the epilogue)
   const int n_rc = (rows_pad + 255) / 256;                // 256-row chunks per key tile: 1 or 2
   const int n_qblk = rows_pad / 128;
   const int n_jobs = n_tiles * n_rc;
@@ -146,7 +149,7 @@ score_tc_pool_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_cons
     mbar_init(smem_u32(&bars->q_full), 1);
     for (int b = 0; b < 2; ++b) {
       mbar_init(smem_u32(&bars->tmem_full[b]), 1);
-      mbar_init(smem_u32(&bars->tmem_empty[b]), split ? POOL_EPI_WARPS : POOL_EPI_WARPS / 2);
+      mbar_init(smem_u32(&bars->tmem_empty[b]), POOL_EPI_WARPS / 2);
     }
     mbar_init(smem_u32(&bars->part_full), POOL_EPI_WARPS / 2);
     mbar_init(smem_u32(&bars->part_empty), POOL_EPI_WARPS / 2);
@@ -247,90 +250,92 @@ score_tc_pool_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_cons
     __syncwarp();
   } else {
     // ---------------- epilogue: one key per thread ----------------
-    // More than 128 live rows: both warpgroups work on every job, warpgroup 0 on columns [0, 128) of the
-    // accumulator, warpgroup 1 on columns [128, 256), so an accumulator is back with its MMA warp after one
-    // 64-column step instead of three (how long an accumulator is held, not the arithmetic, is what this
-    // pass waits for besides the MMAs).  A thread adds up its share over the row chunks of a key tile; at
-    // the end of the tile warpgroup 1 hands its sum to warpgroup 0 through shared memory, which stores.
-    // At most 128 live rows (a streaming update): the warpgroups take alternate jobs whole, so that two
-    // epilogues (and their read-modify-write of the running mean) are in flight.
+    // The two warpgroups take alternate jobs whole, so they are one job apart and one folds while the other
+    // waits for tensor memory (with both on every job, half the columns each, they ran in lockstep and the
+    // sub-partitions idled through every wait: 5.25 against 5.0 ms at the bench shape, 0.57 against 0.50
+    // at 32K x 1).  A job of more than 128 live rows is taken in two steps of 128 columns, the registers a
+    // thread has for it, and the accumulator goes back to its MMA warp when the second step is in
+    // registers.  With two row chunks per key tile a warpgroup always gets the same chunk; warpgroup 1
+    // hands its sum of a tile to warpgroup 0 through shared memory, which picks it up one job later, so
+    // neither waits for the other.
     const int wg = (warp - 3) >> 2;
     const int quarter = warp & 3;                 // TMEM lane quarter this warp may read
     const float c = a.scale_log2;
     const float inv_w = 1.0f / (float)W;
     float* out = a.score_out + ((int64_t)slab * Hkv + h) * a.sum_tok + a.tok_indptr[r];
-    const int half = split ? wg : 0;              // this warp's columns: [128 half, 128 half + 128)
-    const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + half * 128;
+    const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16);
     float acc = 0.f;
-    if (split) {
-      // what does not change from job to job, per row chunk
-      int ncg[2], wfirst[2];
-#pragma unroll
-      for (int rc = 0; rc < 2; ++rc) {
-        const int n_cg_job = (min(rows, rc * 256 + 256) - rc * 256 + 31) / 32;     // 32-column groups with live rows
-        ncg[rc] = min(4, n_cg_job - half * 4);                                      // ... among this warp's columns
-        wfirst[rc] = w_begin + (rc * 256 + half * 128) / G;
-      }
+    if (whole) {
       const int lw = L - W;
-      int key = t_begin * TK + quarter * 32 + lane;
-      int it = 0, rc = 0;
-      // Warpgroup 0 adds warpgroup 1's share of a key tile and stores one job later, when that share has
-      // long been written: neither warpgroup waits for the other at the end of a tile.
       bool pending = false;
       float acc_prev = 0.f;
       int key_prev = 0;
       uint32_t par_prev = 0;
       bool ok = true;
-      for (int job = 0; job < n_jobs; ++job) {
+      const uint32_t tq = taddr;
+      for (int job = wg; job < n_jobs; job += 2) {
         const int b = job & 1;
-        // causal: row w sees key j iff j <= L - W + w  <=>  w >= j - (L - W)
+        const int it = (n_rc == 2) ? (job >> 1) : job;
+        const int rc = (n_rc == 2) ? (job & 1) : 0;
+        const int key = (t_begin + it) * TK + quarter * 32 + lane;
         const int w_min = a.causal ? max(0, key - lw) : 0;
-        POOL_TR(3, job, threadIdx.x == 3 * 32);
         if (!mbar_wait(smem_u32(&bars->tmem_full[b]), (uint32_t)(job >> 1) & 1u, abort_flag)) { ok = false; break; }
         tc_fence_after();
-        POOL_TR(4, job, threadIdx.x == 3 * 32);
-        const int n_cg = rc == 0 ? ncg[0] : ncg[1];
-#ifndef ACTKV_EXP_NO_EPI
-        if (n_cg > 0) {
-          pool_job<G>(taddr + b * 256, nlse + rc * 256 + half * 128, n_cg, rc == 0 ? wfirst[0] : wfirst[1], w_min, W, c, acc,
-                      smem_u32(&bars->tmem_empty[b]), lane, job);
-        } else
-#endif
+        const int n_cg_job = (min(rows, rc * 256 + 256) - rc * 256 + 31) / 32;     // 1..8
         {
-          tc_fence_before();
-          __syncwarp();
-          if (lane == 0) mbar_arrive(smem_u32(&bars->tmem_empty[b]));
-        }
-        POOL_TR(5, job, threadIdx.x == 3 * 32);
-        if (pending) {
-          if (!mbar_wait(smem_u32(&bars->part_full), par_prev, abort_flag)) { ok = false; break; }
-          acc_prev += bars->exch[quarter * 32 + lane];
-          __syncwarp();
-          if (lane == 0) mbar_arrive(smem_u32(&bars->part_empty));
-          if (key_prev < L) {
-            if (row_begin > 0) out[key_prev] += acc_prev * inv_w;
-            else store_pooled(a, r, out + key_prev, acc_prev, acc_prev * inv_w, W);
+          float v[2][64];
+          const float* nl = nlse + rc * 256;
+          const int wf = w_begin + (rc * 256) / G;
+          // columns [0, 128)
+          tmem_ld64(tq + b * 256, v[0]);
+          if (n_cg_job > 2) tmem_ld64(tq + b * 256 + 64, v[1]);
+          tmem_ld_wait();
+          if (n_cg_job <= 4) {
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&bars->tmem_empty[b]));
           }
-          pending = false;
+          pool_fold64<G>(v[0], nl, wf, w_min, W, c, acc);
+          if (n_cg_job > 2) pool_fold64<G>(v[1], nl + 64, wf + 64 / G, w_min, W, c, acc);
+          if (n_cg_job > 4) {
+            // columns [128, 256)
+            tmem_ld64(tq + b * 256 + 128, v[0]);
+            if (n_cg_job > 6) tmem_ld64(tq + b * 256 + 192, v[1]);
+            tmem_ld_wait();
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&bars->tmem_empty[b]));
+            pool_fold64<G>(v[0], nl + 128, wf + 128 / G, w_min, W, c, acc);
+            if (n_cg_job > 6) pool_fold64<G>(v[1], nl + 192, wf + 192 / G, w_min, W, c, acc);
+          }
         }
-        POOL_TR(7, job, threadIdx.x == 3 * 32);
-        if (++rc < n_rc) continue;
-        // the key tile is complete
+        if (n_rc == 1) {
+          if (key < L) { if (row_begin > 0) out[key] += acc * inv_w; else store_pooled(a, r, out + key, acc, acc * inv_w, W); }
+          acc = 0.f;
+          continue;
+        }
         if (wg == 1) {
           if (!mbar_wait(smem_u32(&bars->part_empty), ((uint32_t)it & 1u) ^ 1u, abort_flag)) { ok = false; break; }
           bars->exch[quarter * 32 + lane] = acc;
           __syncwarp();
           if (lane == 0) mbar_arrive(smem_u32(&bars->part_full));
         } else {
+          if (pending) {
+            if (!mbar_wait(smem_u32(&bars->part_full), par_prev, abort_flag)) { ok = false; break; }
+            acc_prev += bars->exch[quarter * 32 + lane];
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&bars->part_empty));
+            if (key_prev < L) {
+              if (row_begin > 0) out[key_prev] += acc_prev * inv_w;
+              else store_pooled(a, r, out + key_prev, acc_prev, acc_prev * inv_w, W);
+            }
+          }
           pending = true;
           acc_prev = acc;
           key_prev = key;
           par_prev = (uint32_t)it & 1u;
         }
         acc = 0.f;
-        rc = 0;
-        ++it;
-        key += TK;
       }
       if (ok && pending && mbar_wait(smem_u32(&bars->part_full), par_prev, abort_flag)) {
         acc_prev += bars->exch[quarter * 32 + lane];
