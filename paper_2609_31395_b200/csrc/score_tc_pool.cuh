@@ -279,8 +279,10 @@ score_tc_pool_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_cons
         const int rc = (n_rc == 2) ? (job & 1) : 0;
         const int key = (t_begin + it) * TK + quarter * 32 + lane;
         const int w_min = a.causal ? max(0, key - lw) : 0;
+        POOL_TR(3, job, threadIdx.x == 3 * 32 || threadIdx.x == 7 * 32);
         if (!mbar_wait(smem_u32(&bars->tmem_full[b]), (uint32_t)(job >> 1) & 1u, abort_flag)) { ok = false; break; }
         tc_fence_after();
+        POOL_TR(4, job, threadIdx.x == 3 * 32 || threadIdx.x == 7 * 32);
         const int n_cg_job = (min(rows, rc * 256 + 256) - rc * 256 + 31) / 32;     // 1..8
         {
           float v[2][64];
@@ -305,10 +307,12 @@ score_tc_pool_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_cons
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(smem_u32(&bars->tmem_empty[b]));
+            POOL_TR(6, job, threadIdx.x == 3 * 32 || threadIdx.x == 7 * 32);
             pool_fold64<G>(v[0], nl + 128, wf + 128 / G, w_min, W, c, acc);
             if (n_cg_job > 6) pool_fold64<G>(v[1], nl + 192, wf + 192 / G, w_min, W, c, acc);
           }
         }
+        POOL_TR(5, job, threadIdx.x == 3 * 32 || threadIdx.x == 7 * 32);
         if (n_rc == 1) {
           if (key < L) { if (row_begin > 0) out[key] += acc * inv_w; else store_pooled(a, r, out + key, acc, acc * inv_w, W); }
           acc = 0.f;
@@ -335,6 +339,7 @@ score_tc_pool_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_cons
           key_prev = key;
           par_prev = (uint32_t)it & 1u;
         }
+        POOL_TR(7, job, threadIdx.x == 3 * 32 || threadIdx.x == 7 * 32);
         acc = 0.f;
       }
       if (ok && pending && mbar_wait(smem_u32(&bars->part_full), par_prev, abort_flag)) {

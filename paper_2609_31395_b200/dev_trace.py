@@ -11,7 +11,8 @@ shape `--loop` times and prints, for CTA 200 of the last launch of each:
   * LSE pass (Section 7.1, LSE equation): cycles per pair of jobs of one epilogue group, its fold time and
     the time to fetch the next accumulator, and the phase between the two groups;
   * pooled-score pass (Algorithm 3 steps 4-5): cycles per job, how long the MMA issuer waits for an
-    accumulator, and where an epilogue warp spends a job (waiting, loading, folding, end-of-tile work).
+    accumulator, and where an epilogue warp spends a job (waiting, holding the accumulator, folding, end-of-tile
+    work).
 A job is one (key tile, row block) product; the stamps themselves cost the traced CTA some 40 cycles each.
 """
 from __future__ import annotations
@@ -76,10 +77,12 @@ def main():
     nj = int((t[2, :1000] != 0).sum())           # accumulator full, folded, released, end-of-tile work done
     j = np.arange(nj // 4, nj - 4)
     print(f"pooled-score pass, CTA 200: {nj} jobs in {t[0, 1002] - t[0, 1000]} cycles; per job {np.diff(t[2, j]).mean():.0f}; "
-          f"issuer waits {(t[1, j] - t[0, j]).mean():.0f} for its accumulator and issues in {(t[2, j] - t[1, j]).mean():.0f}; "
-          f"epilogue warp: waits {(t[4, j] - t[3, j]).mean():.0f}, loads {(t[6, j] - t[4, j]).mean():.0f}, "
-          f"folds {(t[5, j] - t[6, j]).mean():.0f}, exchange {(t[7, j] - t[5, j]).mean():.0f}, "
-          f"to the next wait {(t[3, j + 1] - t[7, j]).mean():.0f}")
+          f"issuer waits {(t[1, j] - t[0, j]).mean():.0f} for its accumulator and issues in {(t[2, j] - t[1, j]).mean():.0f}")
+    for wg in (0, 1):                            # warpgroup wg takes the jobs of parity wg
+        k = j[(j & 1) == wg]
+        print(f"  epilogue warpgroup {wg}, per job of its own: waits {(t[4, k] - t[3, k]).mean():.0f} for the accumulator, "
+              f"holds it {(t[6, k] - t[4, k]).mean():.0f}, folds the rest in {(t[5, k] - t[6, k]).mean():.0f}, "
+              f"end of tile {(t[7, k] - t[5, k]).mean():.0f}, to its next wait {(t[3, k + 2] - t[7, k]).mean():.0f}")
 
 
 if __name__ == "__main__":
