@@ -272,41 +272,45 @@ score_tc_pool_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_cons
       int key_prev = 0;
       uint32_t par_prev = 0;
       bool ok = true;
-      const uint32_t tq = taddr;
-      for (int job = wg; job < n_jobs; job += 2) {
-        const int b = job & 1;
-        const int it = (n_rc == 2) ? (job >> 1) : job;
-        const int rc = (n_rc == 2) ? (job & 1) : 0;
-        const int key = (t_begin + it) * TK + quarter * 32 + lane;
+      // what does not change from job to job: a warpgroup always has the same accumulator and row chunk
+      const int b = wg;
+      const int rc = (n_rc == 2) ? wg : 0;
+      const uint32_t tq = taddr + b * 256;
+      const int n_cg_job = (min(rows, rc * 256 + 256) - rc * 256 + 31) / 32;       // 32-column groups with live rows: 1..8
+      const float* nl = nlse + rc * 256;
+      const int wf = w_begin + (rc * 256) / G;
+      const uint32_t full_bar = smem_u32(&bars->tmem_full[b]), empty_bar = smem_u32(&bars->tmem_empty[b]);
+      int it = (n_rc == 2) ? 0 : wg;
+      const int it_step = (n_rc == 2) ? 1 : 2;
+      int key = (t_begin + it) * TK + quarter * 32 + lane;
+      uint32_t fpar = 0;
+      for (int job = wg; job < n_jobs; job += 2, it += it_step, key += it_step * TK, fpar ^= 1u) {
         const int w_min = a.causal ? max(0, key - lw) : 0;
         POOL_TR(3, job, threadIdx.x == 3 * 32 || threadIdx.x == 7 * 32);
-        if (!mbar_wait(smem_u32(&bars->tmem_full[b]), (uint32_t)(job >> 1) & 1u, abort_flag)) { ok = false; break; }
+        if (!mbar_wait(full_bar, fpar, abort_flag)) { ok = false; break; }
         tc_fence_after();
         POOL_TR(4, job, threadIdx.x == 3 * 32 || threadIdx.x == 7 * 32);
-        const int n_cg_job = (min(rows, rc * 256 + 256) - rc * 256 + 31) / 32;     // 1..8
         {
           float v[2][64];
-          const float* nl = nlse + rc * 256;
-          const int wf = w_begin + (rc * 256) / G;
           // columns [0, 128)
-          tmem_ld64(tq + b * 256, v[0]);
-          if (n_cg_job > 2) tmem_ld64(tq + b * 256 + 64, v[1]);
+          tmem_ld64(tq, v[0]);
+          if (n_cg_job > 2) tmem_ld64(tq + 64, v[1]);
           tmem_ld_wait();
           if (n_cg_job <= 4) {
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive(smem_u32(&bars->tmem_empty[b]));
+            if (lane == 0) mbar_arrive(empty_bar);
           }
           pool_fold64<G>(v[0], nl, wf, w_min, W, c, acc);
           if (n_cg_job > 2) pool_fold64<G>(v[1], nl + 64, wf + 64 / G, w_min, W, c, acc);
           if (n_cg_job > 4) {
             // columns [128, 256)
-            tmem_ld64(tq + b * 256 + 128, v[0]);
-            if (n_cg_job > 6) tmem_ld64(tq + b * 256 + 192, v[1]);
+            tmem_ld64(tq + 128, v[0]);
+            if (n_cg_job > 6) tmem_ld64(tq + 192, v[1]);
             tmem_ld_wait();
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive(smem_u32(&bars->tmem_empty[b]));
+            if (lane == 0) mbar_arrive(empty_bar);
             POOL_TR(6, job, threadIdx.x == 3 * 32 || threadIdx.x == 7 * 32);
             pool_fold64<G>(v[0], nl + 128, wf + 128 / G, w_min, W, c, acc);
             if (n_cg_job > 6) pool_fold64<G>(v[1], nl + 192, wf + 192 / G, w_min, W, c, acc);
