@@ -64,10 +64,22 @@ __global__ void __launch_bounds__(SEL_NT, 1) select_kernel(
     const int n_vec = (L - head) >> 2;
     if (tid < head) take(tid, sc[tid]);
     const float4* sc4 = reinterpret_cast<const float4*>(sc + head);
-    for (int v = tid; v < n_vec; v += SEL_NT) {
-      const float4 x = sc4[v];
-      const int i = head + 4 * v;
-      take(i, x.x); take(i + 1, x.y); take(i + 2, x.z); take(i + 3, x.w);
+    // (four loads in flight per thread: the read is bound by latency, not by bandwidth)
+    for (int v0 = tid; v0 < n_vec; v0 += 4 * SEL_NT) {
+      float4 x[4];
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const int v = v0 + j * SEL_NT;
+        x[j] = v < n_vec ? __ldg(sc4 + v) : make_float4(0.f, 0.f, 0.f, 0.f);
+      }
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const int v = v0 + j * SEL_NT;
+        if (v < n_vec) {
+          const int i = head + 4 * v;
+          take(i, x[j].x); take(i + 1, x[j].y); take(i + 2, x[j].z); take(i + 3, x[j].w);
+        }
+      }
     }
     const int tail0 = head + 4 * n_vec;
     if (tail0 + tid < L) take(tail0 + tid, sc[tail0 + tid]);
@@ -107,8 +119,18 @@ __global__ void __launch_bounds__(SEL_NT, 1) select_kernel(
     }
     if (lane == 31) warp_tot[warp] = incl;
     __syncthreads();
-    uint32_t acc = incl - mine;                          // keys with a digit above this thread's first bin
-    for (int w = 0; w < warp; ++w) acc += warp_tot[w];
+    if (warp == 0) {                                     // exclusive prefix over the 32 warp totals
+      const uint32_t t = warp_tot[lane];
+      uint32_t in2 = t;
+#pragma unroll
+      for (int d = 1; d < 32; d <<= 1) {
+        const uint32_t y = __shfl_up_sync(0xffffffffu, in2, d);
+        if (lane >= d) in2 += y;
+      }
+      warp_tot[lane] = in2 - t;
+    }
+    __syncthreads();
+    uint32_t acc = incl - mine + warp_tot[warp];         // keys with a digit above this thread's first bin
     const int first_bin = per == 4 ? n_bins - 1 - 4 * tid : n_bins - 1 - tid;
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
@@ -154,9 +176,18 @@ __global__ void __launch_bounds__(SEL_NT, 1) select_kernel(
     }
     if (lane == 31) wsum[warp] = incl;
     __syncthreads();
-    unsigned long long before = s_carry;
-    for (int w = 0; w < warp; ++w) before += wsum[w];
-    before += incl - mine;
+    if (warp == 0) {                                     // exclusive prefix over the 32 warp totals
+      const unsigned long long t = wsum[lane];
+      unsigned long long in2 = t;
+#pragma unroll
+      for (int d = 1; d < 32; d <<= 1) {
+        const unsigned long long y = __shfl_up_sync(0xffffffffu, in2, d);
+        if (lane >= d) in2 += y;
+      }
+      wsum[lane] = in2 - t;
+    }
+    __syncthreads();
+    unsigned long long before = s_carry + wsum[warp] + (incl - mine);
     uint32_t gt_before = (uint32_t)(before >> 32), eq_before = (uint32_t)before;
 #pragma unroll
     for (int k = 0; k < SEL_ITEMS; ++k) {
