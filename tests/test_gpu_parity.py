@@ -145,6 +145,18 @@ def test_window_rows_at_tensor_tile_sizes():
 
 
 @pytest.mark.parametrize("causal", [False, True])
+def test_row_counts_at_every_column_group_boundary(causal):
+    """The pooled-score epilogue reads an accumulator in 32-column groups, 64 and 128 at a time, and its two
+    warpgroups take alternate jobs: one more row than every multiple of 32 between 128 and 512 (G = 1, so
+    the window is the row count), a first request with an even and a second with an odd number of key
+    tiles, ragged last tiles."""
+    for W in [129, 161, 193, 225, 257, 289, 321, 353, 385, 417, 449, 481]:
+        wl = synth.Workload("cg", 1, 2, 1, [128 * 10 + 37, 128 * 5 - 20], [W, W - 64], [300, 150], table_style="permutation",
+                            causal=causal, seed=W, poison_tail=True)
+        _full_check(synth.generate(wl, DEV))
+
+
+@pytest.mark.parametrize("causal", [False, True])
 def test_window_rows_above_one_cta(causal):
     """window x group above 512 rows: the score kernels take the rows in groups of 512 (whole action
     tokens); second group full, partial, and absent for the request with the short window."""
