@@ -12,7 +12,9 @@
  *     are HOST structs (passed by pointer, read during the call) that hold device pointers.
  *   - Every call is asynchronous on `stream`, never synchronises, never allocates or frees
  *     device memory.  Scratch comes from the caller: `ws` of at least
- *     `actkv_*_workspace_bytes(...)` bytes, 256-byte aligned.
+ *     `actkv_*_workspace_bytes(...)` bytes, 256-byte aligned.  The one exception is
+ *     actkv_step_host, whose outputs are host memory: it creates two streams and a few events
+ *     per device on first use, and synchronises `stream` before it returns.
  *   - Return value: ACTKV_OK or a negative code for what the host can see (bad argument,
  *     workspace too small, launch failure).  What only the device can see (a page id out of
  *     range, a free list that is too short) is written to the caller's `status[4]` int32 words:
@@ -163,6 +165,15 @@ int actkv_score(const actkv_pool_t* pool /* host */, const actkv_tables_t* table
                 const int32_t* tok_indptr, float* score_out, float* lse_out,
                 int32_t sum_win, int32_t max_win, int32_t sum_tok, int32_t max_tok,
                 void* ws, size_t ws_bytes, int32_t* status, actkv_stream_t stream);
+
+/* ---------------------------------------------------------------------------------------
+ * actkv_score_path — which kernels actkv_score (streaming == 0) or actkv_score_accumulate
+ * (streaming != 0) would run for this pool, group size, window bound, scale and query pointer:
+ * 1 = the tensor-core kernels (tcgen05), 0 = the FMA kernels, negative = bad argument.
+ * Launches nothing.  (Section 7.1 / Algorithm 3 are the same arithmetic on both paths.)
+ */
+int actkv_score_path(const actkv_pool_t* pool /* host */, int32_t n_q_heads, int32_t max_win,
+                     float sm_scale, const void* q, int32_t streaming);
 
 /* ---------------------------------------------------------------------------------------
  * actkv_score_lse — only the log-sum-exp of actkv_score (Section 7.1, LSE equation): what a
@@ -404,6 +415,20 @@ int actkv_compact_noalloc(const actkv_pool_t* pool /* host */, const actkv_table
                           const int32_t* sel_idx, int64_t sel_stride, const int32_t* keep_indptr,
                           const int32_t* budget, int32_t max_keep,
                           int32_t* status, actkv_stream_t stream);
+
+/* ---------------------------------------------------------------------------------------
+ * actkv_debug_inject_stall — fault-injection hook for the bounded waits of the tensor-core score
+ * kernels (the paper has no counterpart).  Every wait inside those kernels (on a shared-memory
+ * barrier) has a limit, after which the kernel writes ACTKV_E_TIMEOUT to status, all its roles
+ * leave, outstanding tensor-core work is drained, tensor memory is freed and the kernel returns;
+ * later stages of the step see the status and do nothing.  This hook makes that happen without a
+ * real fault: while after_tile >= 0, the K-tile producers of every such launch of this process
+ * issue no key tile with index >= after_tile of their CTA (nothing is left in flight: the loads are
+ * simply not issued), and every wait gives up after about wait_limit_us microseconds instead of the
+ * default two seconds.  after_tile < 0 restores normal operation.  Host-side, process-wide, takes
+ * effect at the next launch; not for production use.
+ */
+int actkv_debug_inject_stall(int32_t after_tile, int32_t wait_limit_us);
 
 /* Library version string (host pointer to static storage). */
 const char* actkv_version(void);

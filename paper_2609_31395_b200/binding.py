@@ -26,7 +26,7 @@ EXPORTS = ["actkv_budget_workspace_bytes", "actkv_budget", "actkv_score_workspac
            "actkv_keep_indptr", "actkv_select_workspace_bytes", "actkv_select",
            "actkv_compact_workspace_bytes", "actkv_compact", "actkv_compact_noalloc",
            "actkv_compact_noalloc_max_bytes", "actkv_step_host", "actkv_keepscore", "actkv_gather_f32",
-           "actkv_compact_inplace",
+           "actkv_compact_inplace", "actkv_score_path", "actkv_debug_inject_stall",
            "actkv_version"]
 
 
@@ -99,8 +99,7 @@ def load():
             raise
     if not os.path.exists(LIB_PATH):
         raise ActKVError("load: libactkv.so is missing; run __graft_entry__.build()", E_CUDA)
-    # developer switch: another build of the same sources (dev_trace.py's build with per-job timestamps)
-    lib = C.CDLL(os.environ.get("ACTKV_LIB") or LIB_PATH)
+    lib = C.CDLL(LIB_PATH)
     vp, i32, i64, sz, f32 = C.c_void_p, C.c_int32, C.c_int64, C.c_size_t, C.c_float
     lib.actkv_version.restype = C.c_char_p
     lib.actkv_budget_workspace_bytes.restype = sz
@@ -145,6 +144,10 @@ def load():
     lib.actkv_compact_noalloc.restype = i32
     lib.actkv_compact_noalloc.argtypes = [C.POINTER(PoolDesc), C.POINTER(TablesDesc), i32, i32, vp, i64, vp, vp, i32,
                                           vp, vp]
+    lib.actkv_score_path.restype = i32
+    lib.actkv_score_path.argtypes = [C.POINTER(PoolDesc), i32, i32, f32, vp, i32]
+    lib.actkv_debug_inject_stall.restype = i32
+    lib.actkv_debug_inject_stall.argtypes = [i32, i32]
     _lib = lib
     return lib
 
@@ -230,6 +233,19 @@ def actkv_score(pool: PoolDesc, tables: TablesDesc, layer_begin, layer_end, q, w
                             _ptr(ws, None, "ws"), ws.numel() * ws.element_size(),
                             _ptr(status, torch.int32, "status"), _stream(stream))
     _check("actkv_score", rc)
+
+
+def actkv_score_path(pool: PoolDesc, n_q_heads, max_win, sm_scale, q, streaming=False) -> int:
+    """1: the tensor-core kernels would run, 0: the FMA kernels."""
+    rc = load().actkv_score_path(C.byref(pool), n_q_heads, max_win, float(sm_scale), _ptr(q, torch.bfloat16, "q"),
+                                 int(bool(streaming)))
+    if rc < 0:
+        raise ActKVError("actkv_score_path", rc)
+    return rc
+
+
+def actkv_debug_inject_stall(after_tile: int, wait_limit_us: int = 0):
+    _check("actkv_debug_inject_stall", load().actkv_debug_inject_stall(int(after_tile), int(wait_limit_us)))
 
 
 def actkv_score_lse(pool: PoolDesc, tables: TablesDesc, layer_begin, layer_end, q, win_indptr, n_q_heads, sm_scale,

@@ -27,8 +27,7 @@ def build(force: bool = False, verbose: bool = False, out: str = LIB, extra_flag
     if out == LIB and not force and not _stale():
         return LIB
     nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
-    extra = os.environ.get("ACTKV_NVCC_FLAGS", "").split() + list(extra_flags)   # developer switch: extra nvcc flags
-    cmd = [nvcc, "-shared", "-o", out] + NVCC_FLAGS + extra + (["-Xptxas", "-v"] if verbose else []) + \
+    cmd = [nvcc, "-shared", "-o", out] + NVCC_FLAGS + list(extra_flags) + (["-Xptxas", "-v"] if verbose else []) + \
           [os.path.join(CSRC, s) for s in SOURCES]
     res = subprocess.run(cmd, capture_output=True, text=True)
     if verbose:

@@ -72,6 +72,18 @@ __device__ __forceinline__ int32_t checked_page(const TablesView& t, int32_t n_p
   return id;
 }
 
+// The same lookup for accesses that must not be redirected (the destination of a store, pages pushed on the
+// free list): an out-of-range id is reported and -1 returned, the caller drops the access.
+__device__ __forceinline__ int32_t page_or_neg(const TablesView& t, int32_t n_pages, int32_t r, int32_t lp,
+                                               int32_t* status) {
+  const int32_t id = t.page_table[(int64_t)r * t.max_pages + lp];
+  if ((uint32_t)id >= (uint32_t)n_pages) {
+    report(status, ACTKV_E_BADPAGE, r, id);
+    return -1;
+  }
+  return id;
+}
+
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
 

@@ -52,8 +52,27 @@ __global__ void compact_plan_kernel(TablesView tab, int32_t page_size, int32_t n
     const int32_t fc = *tab.free_count;
     if (fc < 0 || fc > n_pages) { report(status, ACTKV_E_INVALID, -1, fc); ok = false; }
     else if (off > fc) { report(status, ACTKV_E_NOFREE, off, fc); ok = false; }
+    // the old pages pushed back after the pops must fit on the stack
+    else if ((int64_t)fc - off + poff > n_pages) { report(status, ACTKV_E_INVALID, -2, fc - off + poff); ok = false; }
     s_total = off;
     s_ok = ok ? 1 : 0;
+  }
+  __syncthreads();
+  // every old page that will be pushed on the free list must be a page id
+  if (s_ok) {
+    for (int r = 0; r < R; ++r) {
+      if (new_off[r] < 0) continue;
+      const int Y = (tab.seq_len[r] + page_size - 1) / page_size;
+      const int32_t* row = tab.page_table + (int64_t)r * tab.max_pages;
+      for (int i0 = threadIdx.x; i0 < Y; i0 += 4 * blockDim.x) {        // four independent loads per thread
+        int32_t id[4];
+#pragma unroll
+        for (int k = 0; k < 4; ++k) { const int i = i0 + k * blockDim.x; id[k] = i < Y ? row[i] : 0; }
+#pragma unroll
+        for (int k = 0; k < 4; ++k)
+          if ((uint32_t)id[k] >= (uint32_t)n_pages) { report(status, ACTKV_E_BADPAGE, r, id[k]); s_ok = 0; }
+      }
+    }
   }
   __syncthreads();
   const int32_t total = s_total;
@@ -105,8 +124,9 @@ __global__ void __launch_bounds__(CP_NT) compact_copy_kernel(
     if ((uint32_t)tok >= (uint32_t)L) {
       report(status, ACTKV_E_BADINDEX, r, tok);
     } else {
-      const int32_t sp = checked_page(tab, pool.n_pages, r, tok / P, status);
-      so = (int64_t)sp * pool.stride_page + (int64_t)(tok % P) * pool.stride_slot + (int64_t)h * pool.stride_head;
+      const int32_t sp = page_or_neg(tab, pool.n_pages, r, tok / P, status);
+      if (sp >= 0)
+        so = (int64_t)sp * pool.stride_page + (int64_t)(tok % P) * pool.stride_slot + (int64_t)h * pool.stride_head;
     }
     src_off[i] = so;
     dst_off[i] = (int64_t)dst_page * pool.stride_page + (int64_t)slot * pool.stride_slot + (int64_t)h * pool.stride_head;
@@ -214,7 +234,7 @@ int actkv_compact(const actkv_pool_t* pool, const actkv_tables_t* tables, int32_
   actkv::PoolView pv = actkv::make_view(pool);
   actkv::TablesView tv = actkv::make_view(tables);
   actkv::CompactWs* w = (actkv::CompactWs*)ws;
-  actkv::compact_plan_kernel<<<1, 256, 0, s>>>(tv, pool->page_size, pool->n_pages, budget, max_keep, w, status);
+  actkv::compact_plan_kernel<<<1, 1024, 0, s>>>(tv, pool->page_size, pool->n_pages, budget, max_keep, w, status);
   ACTKV_CHECK_LAUNCH();
   const int nl = layer_end - layer_begin;
   int max_x = (max_keep + pool->page_size - 1) / pool->page_size;

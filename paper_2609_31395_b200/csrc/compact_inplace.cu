@@ -103,6 +103,14 @@ __global__ void __launch_bounds__(CI_NT) compact_inplace_copy_kernel(
       }
     }
   }
+  // a move whose source or destination page id is out of range is dropped (and reported): nothing is read
+  // from or written to a page the request does not own
+  int32_t sp = -1, dp = -1;
+  if (hole) {
+    sp = page_or_neg(tab, pool.n_pages, r, src_pos / P, status);
+    dp = page_or_neg(tab, pool.n_pages, r, p / P, status);
+    if (sp < 0 || dp < 0) hole = false;
+  }
   // pack this CTA's moves (their order within the CTA does not matter)
   const uint32_t bal = __ballot_sync(0xffffffffu, hole);
   int wbase = 0;
@@ -110,8 +118,6 @@ __global__ void __launch_bounds__(CI_NT) compact_inplace_copy_kernel(
   wbase = __shfl_sync(0xffffffffu, wbase, 0);
   if (hole) {
     const int k = wbase + __popc(bal & ((1u << lane) - 1u));
-    const int32_t sp = checked_page(tab, pool.n_pages, r, src_pos / P, status);
-    const int32_t dp = checked_page(tab, pool.n_pages, r, p / P, status);
     s_src[k] = (int64_t)sp * pool.stride_page + (int64_t)(src_pos % P) * pool.stride_slot + (int64_t)h * pool.stride_head;
     s_dst[k] = (int64_t)dp * pool.stride_page + (int64_t)(p % P) * pool.stride_slot + (int64_t)h * pool.stride_head;
   }

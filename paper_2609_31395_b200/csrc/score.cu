@@ -121,8 +121,7 @@ static int score_impl(int mode, const actkv_pool_t* pool, const actkv_tables_t* 
   const int64_t units = (int64_t)nls * Hkv * R;
   // (the streaming update keeps a running mean in place, which the row-group launches of a window above
   // 512 rows would break: such calls take the FMA path)
-  const bool use_tc = score_tc_supported(pool, G, max_win, sm_scale, q, acc_steps ? 1 : 64) &&
-                      !(acc_steps != nullptr && max_win * tc::pow2_at_least(G) > tc::MAX_ROWS);
+  const bool use_tc = actkv_score_path(pool, n_q_heads, max_win, sm_scale, q, acc_steps != nullptr) == 1;
 
   const float* lse = lse_in;
   if (mode & 1) {
@@ -193,17 +192,28 @@ int actkv_score_accumulate(const actkv_pool_t* pool, const actkv_tables_t* table
                     acc_steps);
 }
 
-const char* actkv_version(void) { return "actkv-b200 0.1 (sm_100a)"; }
+int actkv_score_path(const actkv_pool_t* pool, int32_t n_q_heads, int32_t max_win, float sm_scale, const void* q,
+                     int32_t streaming) {
+  if (!pool || pool->n_kv_heads <= 0 || n_q_heads <= 0 || n_q_heads % pool->n_kv_heads != 0) return ACTKV_E_INVALID;
+  const int G = n_q_heads / pool->n_kv_heads;
+  const bool tcp = actkv::score_tc_supported(pool, G, max_win, sm_scale, q, streaming ? 1 : 64) &&
+                   !(streaming && max_win * actkv::tc::pow2_at_least(G) > actkv::tc::MAX_ROWS);
+  return tcp ? 1 : 0;
+}
+
+int actkv_debug_inject_stall(int32_t after_tile, int32_t wait_limit_us) {
+  auto& h = actkv::tc::stall_hook();
+  if (after_tile < 0) {
+    h.stall_tile.store(-1);
+    h.wait_cycles.store(actkv::tc::WAIT_LIMIT_CYCLES);
+    return ACTKV_OK;
+  }
+  if (wait_limit_us <= 0) return ACTKV_E_INVALID;
+  h.wait_cycles.store((long long)wait_limit_us * 2100ll);       // cycles at the highest SM clock
+  h.stall_tile.store(after_tile);
+  return ACTKV_OK;
+}
+
+const char* actkv_version(void) { return "actkv-b200 0.2 (sm_100a)"; }
 
 }  // extern "C"
-
-#ifdef ACTKV_POOL_TRACE
-extern "C" int actkv_debug_pool_trace(long long* out_host) {
-  return cudaMemcpyFromSymbol(out_host, actkv::tc::g_pool_trace, sizeof(long long) * 8 * 1024) == cudaSuccess ? 0 : -1;
-}
-#endif
-#ifdef ACTKV_LSE_TRACE
-extern "C" int actkv_debug_lse_trace(long long* out_host) {
-  return cudaMemcpyFromSymbol(out_host, actkv::tc::g_lse_trace, sizeof(long long) * 6 * 1024) == cudaSuccess ? 0 : -1;
-}
-#endif

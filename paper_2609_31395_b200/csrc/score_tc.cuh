@@ -22,7 +22,7 @@
 #pragma once
 
 #include <algorithm>
-#include <cstdlib>
+#include <atomic>
 
 #include "score_tc_lse.cuh"
 #include "score_tc_pool.cuh"
@@ -121,6 +121,19 @@ inline bool make_maps(const actkv_pool_t* pool, const void* q, int nls, int sum_
 
 constexpr size_t SMEM_LIMIT = 232448;        // 227 KB of dynamic shared memory per CTA
 
+// Fault-injection hook of the bounded waits (actkv_debug_inject_stall): while stall_tile >= 0 the K-tile
+// producers of every tensor-core score launch issue no tile from that one on, and every wait gives up after
+// `wait_cycles`.  Process-wide, read at launch.
+struct StallHook {
+  std::atomic<int32_t> stall_tile{-1};
+  std::atomic<long long> wait_cycles{WAIT_LIMIT_CYCLES};
+};
+inline StallHook& stall_hook() { static StallHook h; return h; }
+inline void apply_hook(TcArgs& ta) {
+  ta.stall_tile = stall_hook().stall_tile.load();
+  ta.wait_cycles = stall_hook().wait_cycles.load();
+}
+
 }  // namespace tc
 
 // The tensor-core path takes: pages of 16, 32, 64 or 128 tokens, head_dim 128 or 64, slot-major or head-major pages (any strides that are
@@ -142,12 +155,11 @@ inline bool score_tc_supported(const actkv_pool_t* p, int G, int max_win, float 
   const int rows = max_win * tc::pow2_at_least(G);     // rows of the pooled-score pass (groups padded to a power of two)
   if (rows > tc::MAX_ROWS_TOTAL) return false;
   if (!(sm_scale > 0.f)) return false;
-  if (getenv("ACTKV_FORCE_FMA") != nullptr) return false;
   return tc::encode_fn() != nullptr;
 }
 
-template <int NPOLY>
 inline int score_tc_launch_lse_c(const CUtensorMap& kmap, const tc::TcArgs& ta, unsigned grid, size_t smem, cudaStream_t s) {
+  constexpr int NPOLY = tc::LSE_NPOLY;
   const bool rgs = ta.n_rg > 1, d64 = ta.a.pool.head_dim == 64;
   auto kern = rgs ? (d64 ? tc::score_tc_lse_kernel<NPOLY, true, 1> : tc::score_tc_lse_kernel<NPOLY, true, 2>)
                   : (d64 ? tc::score_tc_lse_kernel<NPOLY, false, 1> : tc::score_tc_lse_kernel<NPOLY, false, 2>);
@@ -169,18 +181,12 @@ inline int score_tc_launch_lse(ScoreArgs& a, const actkv_pool_t* pool, int max_t
   ta.n_stages = 6;
   ta.tiles_per_cta = 0;
   ta.n_kchunks = 0;
+  tc::apply_hook(ta);
   const int64_t units = (int64_t)a.n_layers_sub * a.pool.n_kv_heads * a.tab.n_req;
   const int64_t grid = units * a.n_chunks * ta.n_rg;
   if (grid > 0x7fffffffLL) return ACTKV_E_INVALID;
   const size_t smem = (size_t)ta.n_stages * tc::KTILE_BYTES + sizeof(tc::LseBarriers);
-  // columns of every 8 that take the polynomial exp2 (tuning knob; the default is what the bench uses)
-  int npoly = tc::LSE_NPOLY_DEFAULT;
-  if (const char* e = getenv("ACTKV_LSE_NPOLY")) npoly = atoi(e);
-  switch (npoly) {
-    case 0: return score_tc_launch_lse_c<0>(kmap, ta, (unsigned)grid, smem, s);
-    case 2: return score_tc_launch_lse_c<2>(kmap, ta, (unsigned)grid, smem, s);
-    default: return score_tc_launch_lse_c<1>(kmap, ta, (unsigned)grid, smem, s);
-  }
+  return score_tc_launch_lse_c(kmap, ta, (unsigned)grid, smem, s);
 }
 
 template <int G>
@@ -210,6 +216,7 @@ inline int score_tc_launch_score(ScoreArgs& a, const actkv_pool_t* pool, int max
   ta.n_stages = stages;
   ta.n_rg = 0;
   ta.k5 = tc::pool_needs_5d(pool) ? 1 : 0;
+  tc::apply_hook(ta);
   const int64_t units = (int64_t)a.n_layers_sub * a.pool.n_kv_heads * a.tab.n_req;
   const int max_tiles = (max_tok + tc::TK - 1) / tc::TK;
   // CTAs per unit: one CTA per SM is resident, so the launch runs in rounds of 148 CTAs and the last round

@@ -44,7 +44,7 @@
 namespace actkv {
 namespace tc {
 
-constexpr int LSE_NPOLY_DEFAULT = 1;             // columns of every 8 whose exp2 is the polynomial
+constexpr int LSE_NPOLY = 1;                     // columns of every 8 whose exp2 is the polynomial
 
 __device__ __forceinline__ float ffma_sat(float a, float b, float c) {
   float d;
@@ -96,15 +96,6 @@ __device__ __forceinline__ void lse_slow32(const float* v, int nv, float c, floa
   for (int i = 0; i < 32; ++i) sum += (i < nv) ? exp2f(fmaf(v[i], c, -mc)) : 0.f;
 }
 
-#ifdef ACTKV_LSE_TRACE
-__device__ long long g_lse_trace[6][1024];       // developer build: per-job timestamps of one CTA
-#define LSE_TR(row, job, cond) do { if ((cond) && blockIdx.x == 200 && (job) < 1024) g_lse_trace[row][job] = clock64(); } while (0)
-#define LSE_TR_NS(row, job, cond) do { if ((cond) && blockIdx.x == 200 && (job) < 1024) { unsigned long long t_; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t_)); g_lse_trace[row][job] = (long long)t_; } } while (0)
-#else
-#define LSE_TR_NS(row, job, cond) do { } while (0)
-#define LSE_TR(row, job, cond) do { } while (0)
-#endif
-
 constexpr int LSE_EPI_WARPS = 16;                // (TMEM lane quarter, accumulator, column half)
 constexpr int LSE_THREADS = (3 + LSE_EPI_WARPS) * 32;     // producer, two MMA issuers, epilogue
 constexpr int LSE_SLOTS = 2;                     // accumulators
@@ -143,25 +134,19 @@ __device__ __forceinline__ int sel4(const int (&x)[4], int i) { return i == 0 ? 
 template <int NPOLY>
 __device__ __forceinline__ bool lse_job(LseBarriers* bars, volatile int* abort_flag, uint32_t tq, int grp, int job,
                                         int mb, float2* st, int nv_min, const int (&jm)[4], int key0, float c, float c1,
-                                        int lane) {
+                                        int lane, long long wait_cycles) {
   float v[64];
   float* va = v;
   float* vb = v + 32;
-  LSE_TR(5, job, (threadIdx.x == 3 * 32 || threadIdx.x == 11 * 32));
-  if (!mbar_wait(smem_u32(&bars->tmem_full[grp]), (uint32_t)(job >> 1) & 1u, abort_flag)) return false;
+  if (!mbar_wait_warp(smem_u32(&bars->tmem_full[grp]), (uint32_t)(job >> 1) & 1u, abort_flag, wait_cycles)) return false;
   tc_fence_after();
-#ifndef ACTKV_EXP_NO_LD
   tmem_ld64(tq, v);
-#endif
   float2 ms = *st;
   tmem_ld_wait();
   tmem_ld_fence<64>(v);
-  LSE_TR(2, job, (threadIdx.x == 3 * 32 || threadIdx.x == 11 * 32));
   tc_fence_before();
   __syncwarp();
   if (lane == 0) mbar_arrive(smem_u32(&bars->tmem_empty[grp]));
-  LSE_TR(3, job, (threadIdx.x == 3 * 32 || threadIdx.x == 11 * 32));
-#ifndef ACTKV_EXP_NO_EPI
   bool slow = __any_sync(0xffffffffu, nv_min < 64 || ms.x == -INFINITY);
   if (!slow) {
     const float nmc = -ms.x * c, c0 = fmaf(nmc, 1.f / 252.f, 0.5f);
@@ -175,8 +160,6 @@ __device__ __forceinline__ bool lse_job(LseBarriers* bars, volatile int* abort_f
     lse_slow32(vb, nv - 32, c, ms.x, ms.y);
   }
   *st = ms;
-#endif
-  LSE_TR(4, job, (threadIdx.x == 3 * 32 || threadIdx.x == 11 * 32));
   return true;
 }
 
@@ -187,8 +170,6 @@ template <int NPOLY, bool ROW_GROUPS, int NH>
 __global__ void __launch_bounds__(LSE_THREADS, 1)
 score_tc_lse_kernel(const __grid_constant__ CUtensorMap kmap, const TcArgs ta) {
   extern __shared__ __align__(1024) uint8_t smem[];
-  LSE_TR(0, 1000, threadIdx.x == 32);
-  LSE_TR_NS(0, 1001, threadIdx.x == 32);
   const ScoreArgs& a = ta.a;
   const int R = a.tab.n_req, Hkv = a.pool.n_kv_heads, G = a.group;
   const int cu = blockIdx.x / a.n_chunks;
@@ -206,7 +187,12 @@ score_tc_lse_kernel(const __grid_constant__ CUtensorMap kmap, const TcArgs ta) {
     if (threadIdx.x == 0 && chunk == 0 && rg == 0) report(a.status, ACTKV_E_INVALID, r, W);
     return;
   }
-  const int n_mb = (rows + 127) / 128;                   // 1..4 (checked by the host)
+  // the host sized shared memory, tensor memory and the partials from upper bounds of the window and the length
+  if (W * G > a.rows_max || L > a.n_chunks * a.lse_chunk || rows > MAX_ROWS) {
+    if (threadIdx.x == 0 && chunk == 0 && rg == 0) report(a.status, ACTKV_E_INVALID, r, W * G > a.rows_max ? W : L);
+    return;
+  }
+  const int n_mb = (rows + 127) / 128;                   // 1..4
   const int t_begin = key_begin / TK;
   const int t_end = min((L + TK - 1) / TK, t_begin + a.lse_chunk / TK);
   const int n_tiles = t_end - t_begin;
@@ -257,8 +243,8 @@ score_tc_lse_kernel(const __grid_constant__ CUtensorMap kmap, const TcArgs ta) {
     // ---------------- TMA producer: K tiles through the block table ----------------
     const int layer = a.layer_begin + slab;
     // (one producer: this pass needs a K tile per four jobs, far below what one warp delivers)
-    if (ta.k5) k_tile_producer<true, NH>(&kmap, a, bars, k_smem, S, r, h, layer, L, t_begin, n_tiles, lane, abort_flag, 0, 1);
-    else k_tile_producer<false, NH>(&kmap, a, bars, k_smem, S, r, h, layer, L, t_begin, n_tiles, lane, abort_flag, 0, 1);
+    if (ta.k5) k_tile_producer<true, NH>(&kmap, a, bars, k_smem, S, r, h, layer, L, t_begin, n_tiles, lane, abort_flag, 0, 1, ta.wait_cycles, ta.stall_tile);
+    else k_tile_producer<false, NH>(&kmap, a, bars, k_smem, S, r, h, layer, L, t_begin, n_tiles, lane, abort_flag, 0, 1, ta.wait_cycles, ta.stall_tile);
   } else if (warp <= 2) {
     // ---------------- MMA issuers: A = Q block in TMEM, B = K tile in shared memory ----------------
     // Two warps, one per accumulator: warp 1 issues the even jobs into accumulator 0, warp 2 the odd jobs
@@ -273,24 +259,23 @@ score_tc_lse_kernel(const __grid_constant__ CUtensorMap kmap, const TcArgs ta) {
     const uint64_t desc0 = smem_desc_sw128(k_smem);
     const uint32_t full_bar = smem_u32(&bars->tmem_full[mw]), empty_bar = smem_u32(&bars->tmem_empty[mw]);
     const uint32_t d = tmem_base + LSE_A_COLS + mw * 128;
-    bool ok = mbar_wait(smem_u32(&bars->q_ready), 0, abort_flag);
+    bool ok = mbar_wait_warp(smem_u32(&bars->q_ready), 0, abort_flag, ta.wait_cycles);
     tc_fence_after();
     int s = 0, job = 0;
     uint32_t kpar = 0, epar = 1u;                  // parity to wait for on tmem_empty[mw] (a fresh barrier passes with 1)
     const bool leader = elect_one();
     for (int it = 0; ok && it < n_tiles; ++it) {
-      ok = mbar_wait(smem_u32(&bars->k_full[s]), kpar, abort_flag);
+      ok = mbar_wait_warp(smem_u32(&bars->k_full[s]), kpar, abort_flag, ta.wait_cycles);
       if (!ok) break;
       tc_fence_after();
       const uint64_t desc_s = desc0 + (uint64_t)((s * KTILE_BYTES) >> 4);
       bool mine = false;
       for (int b = 0; b < n_mb; ++b, ++job) {
         if ((job & 1) != mw) continue;
-        ok = mbar_wait(empty_bar, epar, abort_flag);
+        ok = mbar_wait_warp(empty_bar, epar, abort_flag, ta.wait_cycles);
         if (!ok) break;
         epar ^= 1u;
         tc_fence_after();
-        LSE_TR(0, job, leader);
         if (leader) {
           const uint32_t at = tmem_base + b * 64;
 #pragma unroll
@@ -299,7 +284,6 @@ score_tc_lse_kernel(const __grid_constant__ CUtensorMap kmap, const TcArgs ta) {
                          kk > 0 ? 1u : 0u);
           umma_commit(full_bar);
         }
-        LSE_TR(1, job, leader);
         mine = true;
       }
       if (!ok) break;
@@ -313,7 +297,8 @@ score_tc_lse_kernel(const __grid_constant__ CUtensorMap kmap, const TcArgs ta) {
     __syncwarp();
     if (leader) umma_commit(smem_u32(&bars->drained[mw]));
     __syncwarp();
-    mbar_wait(smem_u32(&bars->drained[mw]), 0, abort_flag, ok ? WAIT_LIMIT_NS : DRAIN_LIMIT_NS);
+    // (a tear-down wait: it does not end early because another role gave up)
+    mbar_wait_warp(smem_u32(&bars->drained[mw]), 0, nullptr, ok ? ta.wait_cycles : DRAIN_LIMIT_CYCLES);
     __syncwarp();
   } else {
     // ---------------- epilogue warps ----------------
@@ -355,7 +340,7 @@ score_tc_lse_kernel(const __grid_constant__ CUtensorMap kmap, const TcArgs ta) {
     const int mb_step = 2 % n_mb, tile_step = 2 / n_mb;
     for (int job = grp; job < n_jobs; job += 2) {
       epi_ok = lse_job<NPOLY>(bars, abort_flag, tq, grp, job, mb, &bars->state[grp][mb][half][rib], jfast - key0 + 1, jm, key0, c,
-                              c1, lane);
+                              c1, lane, ta.wait_cycles);
       if (!epi_ok) break;
       mb += mb_step;
       key0 += tile_step * TK;
@@ -390,15 +375,13 @@ score_tc_lse_kernel(const __grid_constant__ CUtensorMap kmap, const TcArgs ta) {
   if (warp == 0 && lane == 0 && *abort_flag) {
     report(a.status, ACTKV_E_TIMEOUT, u, chunk);
     // loads still in flight land in this CTA's shared memory: give them a moment before exiting
-    for (int s = 0; s < S; ++s) mbar_wait(smem_u32(&bars->k_full[s]), 0, abort_flag, DRAIN_LIMIT_NS / 8);
+    for (int s = 0; s < S; ++s) mbar_wait(smem_u32(&bars->k_full[s]), 0, nullptr, DRAIN_LIMIT_CYCLES / 64);
   }
   __syncthreads();
   if (warp == 1) {
     tc_fence_after();
     tmem_dealloc(tmem_base, 512);
   }
-  LSE_TR(0, 1002, threadIdx.x == 32);
-  LSE_TR_NS(0, 1003, threadIdx.x == 32);
 }
 
 }  // namespace tc

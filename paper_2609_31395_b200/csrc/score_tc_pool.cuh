@@ -17,15 +17,6 @@ constexpr int POOL_EPI_WARPS = 8;
 constexpr int POOL_THREADS = (4 + POOL_EPI_WARPS) * 32;     // producer, two MMA issuers, epilogue, second producer
 constexpr int POOL_PRODUCER2 = 3 + POOL_EPI_WARPS;          // warp index of the second producer
 
-#ifdef ACTKV_POOL_TRACE
-__device__ long long g_pool_trace[8][1024];      // developer build: per-job timestamps of one CTA
-#define POOL_TR(row, job, cond) do { if ((cond) && blockIdx.x == 200 && (job) < 1024) g_pool_trace[row][job] = clock64(); } while (0)
-#define POOL_TR_NS(row, job, cond) do { if ((cond) && blockIdx.x == 200 && (job) < 1024) { unsigned long long t_; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t_)); g_pool_trace[row][job] = (long long)t_; } } while (0)
-#else
-#define POOL_TR_NS(row, job, cond) do { } while (0)
-#define POOL_TR(row, job, cond) do { } while (0)
-#endif
-
 struct PoolBarriers {
   uint64_t k_full[8];
   uint64_t k_empty[8];
@@ -40,25 +31,18 @@ struct PoolBarriers {
   float exch[TK];
 };
 
-// One accumulator: columns [0, 32*n_cg) hold s for rows n0 .. of this key (lane).  nlse = -lse*log2(e)
-// per row (-inf for padding rows).  Adds sum_w exp2(max_g(s*c + nlse)) over the live rows to `acc`.
-// Action tokens outside [w_min, w_end) do not count: below w_min the key is not visible yet (causal
-// rule), from w_end on the columns are padding (with a narrow MMA they were never written and may hold
-// anything; whatever the arithmetic makes of them is discarded by the select).
 // 64 columns of one accumulator lane: x = s for rows n .. n + 63 of this key, nlse = -lse*log2(e) of those rows
 // (-inf for padding rows).  Adds sum_w exp2(max_g(s*c + nlse)) over the action tokens w_first .. that lie
-// in [w_min, w_end) to `acc`.
+// in [w_min, w_end) to `acc`.  Action tokens outside [w_min, w_end) do not count: below w_min the key is
+// not visible yet (causal rule), from w_end on the columns are padding (with a narrow MMA they were never
+// written and may hold anything).
 template <int G>
 __device__ __forceinline__ void pool_fold64(float* x, const float* nlse, int w_first, int w_min, int w_end, float c,
                                             float& acc) {
   const float4* l4 = reinterpret_cast<const float4*>(nlse);
 #pragma unroll
   for (int q4 = 0; q4 < 16; ++q4) {
-#ifdef ACTKV_EXP_NO_NLSE
-    const float4 l = make_float4(-1.f, -1.f, -1.f, -1.f + (float)(l4 == nullptr));
-#else
     const float4 l = l4[q4];
-#endif
     ffma2(x[q4 * 4 + 0], x[q4 * 4 + 1], x[q4 * 4 + 0], x[q4 * 4 + 1], c, l.x, l.y);
     ffma2(x[q4 * 4 + 2], x[q4 * 4 + 3], x[q4 * 4 + 2], x[q4 * 4 + 3], c, l.z, l.w);
   }
@@ -73,7 +57,7 @@ __device__ __forceinline__ void pool_fold64(float* x, const float* nlse, int w_f
 
 template <int G>
 __device__ __forceinline__ void pool_job(uint32_t taddr, const float* nlse, int n_cg, int w_first, int w_min, int w_end,
-                                         float c, float& acc, uint32_t empty_bar, int lane, int job = 0) {
+                                         float c, float& acc, uint32_t empty_bar, int lane) {
   // At most 128 columns (n_cg <= 4 groups of 32): both 64-column loads are issued at once and the
   // accumulator is handed back to the MMA warp as soon as they are in registers, before anything is folded.
   const int n_c2 = (n_cg + 1) >> 1;
@@ -84,11 +68,6 @@ __device__ __forceinline__ void pool_job(uint32_t taddr, const float* nlse, int 
   tc_fence_before();
   __syncwarp();
   if (lane == 0) mbar_arrive(empty_bar);
-  POOL_TR(6, job, threadIdx.x == 3 * 32);
-#ifdef ACTKV_EXP_NO_FOLD
-  acc += v[0][0] + v[1][0];          // developer switch: loads and hand-back only
-  return;
-#endif
   pool_fold64<G>(v[0], nlse, w_first, w_min, w_end, c, acc);
   if (n_c2 > 1) pool_fold64<G>(v[1], nlse + 64, w_first + 64 / G, w_min, w_end, c, acc);
 }
@@ -101,8 +80,6 @@ template <int G, int NH>
 __global__ void __launch_bounds__(POOL_THREADS, 1)
 score_tc_pool_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constant__ CUtensorMap qmap, const TcArgs ta) {
   extern __shared__ __align__(1024) uint8_t smem[];
-  POOL_TR(0, 1000, threadIdx.x == 32);
-  POOL_TR_NS(0, 1001, threadIdx.x == 32);
   const ScoreArgs& a = ta.a;
   const int R = a.tab.n_req, Hkv = a.pool.n_kv_heads;
   const int u = blockIdx.x / ta.n_kchunks;
@@ -120,6 +97,11 @@ score_tc_pool_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_cons
   if (W <= 0 && a.acc_steps != nullptr) return;            // accumulate mode: a request outside its action region
   if (W <= 0 || (a.causal && W > L)) {
     if (threadIdx.x == 0 && kchunk == 0) report(a.status, ACTKV_E_INVALID, r, W);
+    return;
+  }
+  // the host sized shared memory and the launch from upper bounds of the window and the length
+  if (W * a.group > a.rows_max || L > ta.n_kchunks * ta.tiles_per_cta * TK) {
+    if (threadIdx.x == 0 && kchunk == 0) report(a.status, ACTKV_E_INVALID, r, W * a.group > a.rows_max ? W : L);
     return;
   }
   const int t_end = min((L + TK - 1) / TK, t_begin + ta.tiles_per_cta);
@@ -185,12 +167,12 @@ score_tc_pool_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_cons
           tma_load_3d(q_smem + (qb >> 1) * 2 * QBLK_BYTES + hf * QBLK_BYTES + (qb & 1) * HALF_BYTES, &qmap,
                       smem_u32(&bars->q_full), hf * 64, h * a.group, wrow + qb * (128 / G));
     }
-    if (ta.k5) k_tile_producer<true, NH>(&kmap, a, bars, k_smem, S, r, h, layer, L, t_begin, n_tiles, lane, abort_flag, 0, 2);
-    else k_tile_producer<false, NH>(&kmap, a, bars, k_smem, S, r, h, layer, L, t_begin, n_tiles, lane, abort_flag, 0, 2);
+    if (ta.k5) k_tile_producer<true, NH>(&kmap, a, bars, k_smem, S, r, h, layer, L, t_begin, n_tiles, lane, abort_flag, 0, 2, ta.wait_cycles, ta.stall_tile);
+    else k_tile_producer<false, NH>(&kmap, a, bars, k_smem, S, r, h, layer, L, t_begin, n_tiles, lane, abort_flag, 0, 2, ta.wait_cycles, ta.stall_tile);
   } else if (warp == POOL_PRODUCER2) {
     const int layer = a.layer_begin + slab;
-    if (ta.k5) k_tile_producer<true, NH>(&kmap, a, bars, k_smem, S, r, h, layer, L, t_begin, n_tiles, lane, abort_flag, 1, 2);
-    else k_tile_producer<false, NH>(&kmap, a, bars, k_smem, S, r, h, layer, L, t_begin, n_tiles, lane, abort_flag, 1, 2);
+    if (ta.k5) k_tile_producer<true, NH>(&kmap, a, bars, k_smem, S, r, h, layer, L, t_begin, n_tiles, lane, abort_flag, 1, 2, ta.wait_cycles, ta.stall_tile);
+    else k_tile_producer<false, NH>(&kmap, a, bars, k_smem, S, r, h, layer, L, t_begin, n_tiles, lane, abort_flag, 1, 2, ta.wait_cycles, ta.stall_tile);
   } else if (warp <= 2) {
     // ---------------- MMA issuers: D[key, row] = K Q^T ----------------
     // Two warps, one per accumulator: warp 1 issues the even jobs, warp 2 the odd ones.  Issuing costs the
@@ -207,24 +189,22 @@ score_tc_pool_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_cons
     const int n1 = max(16, (rows - 256 + 15) & ~15);
     const uint32_t idesc_c[2] = {idesc_bf16(128, n0), idesc_bf16(128, n1)};
     const uint32_t full_bar = smem_u32(&bars->tmem_full[mw]), empty_bar = smem_u32(&bars->tmem_empty[mw]);
-    bool ok = mbar_wait(smem_u32(&bars->q_full), 0, abort_flag);
+    bool ok = mbar_wait_warp(smem_u32(&bars->q_full), 0, abort_flag, ta.wait_cycles);
     int s = 0, job = 0;
     uint32_t kpar = 0, epar = 1u;                  // parity to wait for on tmem_empty[mw] (a fresh barrier passes with 1)
     const bool leader = elect_one();
     for (int it = 0; ok && it < n_tiles; ++it) {
-      ok = mbar_wait(smem_u32(&bars->k_full[s]), kpar, abort_flag);
+      ok = mbar_wait_warp(smem_u32(&bars->k_full[s]), kpar, abort_flag, ta.wait_cycles);
       if (!ok) break;
       tc_fence_after();
       const uint64_t adesc_s = kdesc0 + (uint64_t)((s * KTILE_BYTES) >> 4);
       bool mine = false;
       for (int rc = 0; rc < n_rc; ++rc, ++job) {
         if ((job & 1) != mw) continue;
-        POOL_TR(0, job, leader);
-        ok = mbar_wait(empty_bar, epar, abort_flag);
+        ok = mbar_wait_warp(empty_bar, epar, abort_flag, ta.wait_cycles);
         if (!ok) break;
         epar ^= 1u;
         tc_fence_after();
-        POOL_TR(1, job, leader);
         if (leader) {
           const uint64_t bdesc_c = qdesc0 + (uint64_t)((rc * 2 * QBLK_BYTES) >> 4);
 #pragma unroll
@@ -233,7 +213,6 @@ score_tc_pool_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_cons
                       bdesc_c + (uint64_t)(((kk >> 2) * QBLK_BYTES + (kk & 3) * 32) >> 4), idesc_c[rc], kk > 0 ? 1u : 0u);
           umma_commit(full_bar);
         }
-        POOL_TR(2, job, leader);
         mine = true;
       }
       if (!ok) break;
@@ -246,7 +225,8 @@ score_tc_pool_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_cons
     __syncwarp();
     if (leader) umma_commit(smem_u32(&bars->drained[mw]));
     __syncwarp();
-    mbar_wait(smem_u32(&bars->drained[mw]), 0, abort_flag, ok ? WAIT_LIMIT_NS : DRAIN_LIMIT_NS);
+    // (a tear-down wait: it does not end early because another role gave up)
+    mbar_wait_warp(smem_u32(&bars->drained[mw]), 0, nullptr, ok ? ta.wait_cycles : DRAIN_LIMIT_CYCLES);
     __syncwarp();
   } else {
     // ---------------- epilogue: one key per thread ----------------
@@ -286,10 +266,8 @@ score_tc_pool_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_cons
       uint32_t fpar = 0;
       for (int job = wg; job < n_jobs; job += 2, it += it_step, key += it_step * TK, fpar ^= 1u) {
         const int w_min = a.causal ? max(0, key - lw) : 0;
-        POOL_TR(3, job, threadIdx.x == 3 * 32 || threadIdx.x == 7 * 32);
-        if (!mbar_wait(full_bar, fpar, abort_flag)) { ok = false; break; }
+        if (!mbar_wait_warp(full_bar, fpar, abort_flag, ta.wait_cycles)) { ok = false; break; }
         tc_fence_after();
-        POOL_TR(4, job, threadIdx.x == 3 * 32 || threadIdx.x == 7 * 32);
         {
           float v[2][64];
           // columns [0, 128)
@@ -311,25 +289,23 @@ score_tc_pool_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_cons
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(empty_bar);
-            POOL_TR(6, job, threadIdx.x == 3 * 32 || threadIdx.x == 7 * 32);
             pool_fold64<G>(v[0], nl + 128, wf + 128 / G, w_min, W, c, acc);
             if (n_cg_job > 6) pool_fold64<G>(v[1], nl + 192, wf + 192 / G, w_min, W, c, acc);
           }
         }
-        POOL_TR(5, job, threadIdx.x == 3 * 32 || threadIdx.x == 7 * 32);
         if (n_rc == 1) {
           if (key < L) { if (row_begin > 0) out[key] += acc * inv_w; else store_pooled(a, r, out + key, acc, acc * inv_w, W); }
           acc = 0.f;
           continue;
         }
         if (wg == 1) {
-          if (!mbar_wait(smem_u32(&bars->part_empty), ((uint32_t)it & 1u) ^ 1u, abort_flag)) { ok = false; break; }
+          if (!mbar_wait_warp(smem_u32(&bars->part_empty), ((uint32_t)it & 1u) ^ 1u, abort_flag, ta.wait_cycles)) { ok = false; break; }
           bars->exch[quarter * 32 + lane] = acc;
           __syncwarp();
           if (lane == 0) mbar_arrive(smem_u32(&bars->part_full));
         } else {
           if (pending) {
-            if (!mbar_wait(smem_u32(&bars->part_full), par_prev, abort_flag)) { ok = false; break; }
+            if (!mbar_wait_warp(smem_u32(&bars->part_full), par_prev, abort_flag, ta.wait_cycles)) { ok = false; break; }
             acc_prev += bars->exch[quarter * 32 + lane];
             __syncwarp();
             if (lane == 0) mbar_arrive(smem_u32(&bars->part_empty));
@@ -343,10 +319,9 @@ score_tc_pool_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_cons
           key_prev = key;
           par_prev = (uint32_t)it & 1u;
         }
-        POOL_TR(7, job, threadIdx.x == 3 * 32 || threadIdx.x == 7 * 32);
         acc = 0.f;
       }
-      if (ok && pending && mbar_wait(smem_u32(&bars->part_full), par_prev, abort_flag)) {
+      if (ok && pending && mbar_wait_warp(smem_u32(&bars->part_full), par_prev, abort_flag, ta.wait_cycles)) {
         acc_prev += bars->exch[quarter * 32 + lane];
         if (key_prev < L) {
           if (row_begin > 0) out[key_prev] += acc_prev * inv_w;
@@ -359,16 +334,10 @@ score_tc_pool_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_cons
         const int b = job & 1;
         const int key = (t_begin + job) * TK + quarter * 32 + lane;
         const int w_min = a.causal ? max(0, key - (L - W)) : 0;
-        if (!mbar_wait(smem_u32(&bars->tmem_full[b]), (uint32_t)(job >> 1) & 1u, abort_flag)) break;
+        if (!mbar_wait_warp(smem_u32(&bars->tmem_full[b]), (uint32_t)(job >> 1) & 1u, abort_flag, ta.wait_cycles)) break;
         tc_fence_after();
         const int n_cg = (rows + 31) / 32;
-#ifndef ACTKV_EXP_NO_EPI
         pool_job<G>(taddr + b * 256, nlse, n_cg, w_begin, w_min, W, c, acc, smem_u32(&bars->tmem_empty[b]), lane);
-#else
-        tc_fence_before();
-        __syncwarp();
-        if (lane == 0) mbar_arrive(smem_u32(&bars->tmem_empty[b]));
-#endif
         if (key < L) { if (row_begin > 0) out[key] += acc * inv_w; else store_pooled(a, r, out + key, acc, acc * inv_w, W); }
         acc = 0.f;
       }
@@ -379,15 +348,13 @@ score_tc_pool_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_cons
   __syncthreads();
   if (warp == 0 && lane == 0 && *abort_flag) {
     report(a.status, ACTKV_E_TIMEOUT, u, kchunk);
-    for (int s = 0; s < S; ++s) mbar_wait(smem_u32(&bars->k_full[s]), 0, abort_flag, DRAIN_LIMIT_NS / 8);
+    for (int s = 0; s < S; ++s) mbar_wait(smem_u32(&bars->k_full[s]), 0, nullptr, DRAIN_LIMIT_CYCLES / 64);
   }
   __syncthreads();
   if (warp == 1) {
     tc_fence_after();
     tmem_dealloc(tmem_base, 512);
   }
-  POOL_TR(0, 1002, threadIdx.x == 32);
-  POOL_TR_NS(0, 1003, threadIdx.x == 32);
 }
 
 }  // namespace tc

@@ -44,6 +44,14 @@ __global__ void __launch_bounds__(SEL_NT, 1) select_kernel(
   const float* sc = score + (int64_t)o * sum_tok + base;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
 
+  // An earlier stage of the step failed (a score kernel that gave up, a bad table): its scores are not
+  // consumed.  A budget the host did not size the index buffer for (the budgets are device data, e.g.
+  // straight from actkv_budget) is reported before anything is stored.
+  if (status_set(status)) return;
+  if ((int64_t)keep_indptr[r] + n > sel_stride) {
+    if (tid == 0) report(status, ACTKV_E_INVALID, r, n);
+    return;
+  }
   if (n == 0) {
     if (tie != nullptr && tid == 0) tie[u] = actkv_tie_t{0.f, 0, 0, 0};
     return;
@@ -209,7 +217,6 @@ __global__ void __launch_bounds__(SEL_NT, 1) select_kernel(
     uint32_t b = (thr & 0x80000000u) ? (thr & 0x7fffffffu) : ~thr;
     tie[u] = actkv_tie_t{__uint_as_float(b), (int32_t)need_eq, (int32_t)eq_total, n};
   }
-  (void)status;
 }
 
 __global__ void keep_indptr_kernel(const int32_t* seq_len, const int32_t* budget, int32_t n_req,

@@ -15,8 +15,10 @@ constexpr uint32_t HALF_BYTES = TK * 64 * 2;         // 16 KB
 constexpr uint32_t QBLK_BYTES = 128 * HD * 2;        // 32 KB per 128 rows
 constexpr int MAX_ROWS = 512;                // window x group rows (padded to 128) one CTA handles
 constexpr int MAX_ROWS_TOTAL = 4096;         // ... per unit: more than MAX_ROWS are taken in groups of MAX_ROWS
-constexpr uint64_t WAIT_LIMIT_NS = 2000000000ull;    // bounded waits give up after 2 s
-constexpr uint64_t DRAIN_LIMIT_NS = 50000000ull;     // waits while tearing down after a give-up
+// Bounded waits are counted on the SM cycle counter (cheap to read, unlike the global nanosecond timer).  The
+// counter runs at 2.1 GHz at most, so a limit of n cycles lasts at least n / 2.1 ns.
+constexpr long long WAIT_LIMIT_CYCLES = 4000000000ll;      // default limit of a wait: about two seconds
+constexpr long long DRAIN_LIMIT_CYCLES = 100000000ll;      // waits while tearing down after a give-up: about 50 ms
 
 // ---------------------------------------------------------------------------------------------
 // PTX wrappers
@@ -51,29 +53,33 @@ __device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity) {
       : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
   return ok != 0;
 }
-// Bounded wait.  Returns false when another role already gave up or the limit passed (then the
-// abort flag is raised so that every role stops).  The limit is counted on the SM cycle counter
-// (cheap to read, unlike the global nanosecond timer): at most 2.1 GHz, so `limit_ns` of cycles is
-// at least half as long in wall time.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag,
-                                          uint64_t limit_ns = WAIT_LIMIT_NS) {
+// Bounded wait of ONE thread.  Returns false when another role already gave up or the limit passed (then the
+// abort flag is raised so that every role stops).  abort_flag == nullptr: a wait of the tear-down path, which
+// neither looks at the flag nor raises it and only ends on success or on its own limit.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, long long limit_cycles) {
   // try_wait parks the thread in hardware (no polling traffic on shared memory, which the MMA operand
   // fetch needs); measured the same or better than spinning on test_wait here.
 #pragma unroll 1
   for (int i = 0; i < 64; ++i)
     if (mbar_try_wait(bar, parity)) return true;
   const long long t0 = clock64();
-  const long long limit_cycles = (long long)limit_ns * 2;
   for (;;) {
 #pragma unroll 1
     for (int i = 0; i < 256; ++i)
       if (mbar_try_wait(bar, parity)) return true;
-    if (*abort_flag) return false;
+    if (abort_flag != nullptr && *abort_flag) return false;
     if (clock64() - t0 > limit_cycles) {
-      *abort_flag = 1;
+      if (abort_flag != nullptr) *abort_flag = 1;
       return false;
     }
   }
+}
+// The same wait called by all 32 lanes of a converged warp, with ONE verdict for the warp: the callers go on
+// to warp-collective instructions (tcgen05.ld, elect, __syncwarp) and must not split on a wait that some
+// lanes saw complete and others gave up on.
+__device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, volatile int* abort_flag, long long limit_cycles) {
+  const bool ok = mbar_wait(bar, parity, abort_flag, limit_cycles);
+  return __all_sync(0xffffffffu, ok);
 }
 // One lane of a converged warp (always the same one for a full mask).
 __device__ __forceinline__ bool elect_one() {
@@ -274,6 +280,8 @@ struct TcArgs {
   int32_t row_begin;         // pooled-score pass: first row of this launch's row group (multiple of MAX_ROWS)
   int32_t n_stages;          // K stages in shared memory
   int32_t k5;                // K tensor map has five dimensions (pages that are not slot-major), else four
+  int32_t stall_tile;        // fault-injection hook: the K-tile producers issue no tile from this one on (< 0: off)
+  long long wait_cycles;     // limit of every bounded wait, in SM cycles
 };
 
 // Barrier block at the tail of dynamic shared memory.
@@ -308,7 +316,8 @@ __device__ __forceinline__ int32_t page_for_tile(const TablesView& tab, int32_t 
 template <bool K5, int NH, class Bars>
 __device__ __forceinline__ void k_tile_producer(const CUtensorMap* kmap, const ScoreArgs& a, Bars* bars, uint32_t k_smem,
                                                 int S, int r, int h, int layer, int L, int t_begin, int n_tiles,
-                                                int lane, volatile int* abort_flag, int p, int P) {
+                                                int lane, volatile int* abort_flag, int p, int P, long long wait_cycles,
+                                                int stall_tile) {
   const int ps = a.pool.page_size;
   const int ppt = TK / ps;                                      // pages per tile: 8, 4, 2 or 1
   const int lp_shift = 31 - __clz(ppt);                         // log2(ppt)
@@ -320,6 +329,7 @@ __device__ __forceinline__ void k_tile_producer(const CUtensorMap* kmap, const S
   int32_t pid_next = 0;
   for (int i = 0; i < n_mine; ++i) {
     const int it = p + i * P;
+    if (stall_tile >= 0 && it >= stall_tile) break;       // injected fault: this and all later tiles never arrive
     const int s = it % S;
     const uint32_t ph = (uint32_t)(it / S) & 1u;
     if ((i & 3) == 0 && i + 4 < n_mine)
@@ -327,18 +337,13 @@ __device__ __forceinline__ void k_tile_producer(const CUtensorMap* kmap, const S
                                a.status);
     int ok = 1;
     if (lane == 0) {
-      ok = mbar_wait(smem_u32(&bars->k_empty[s]), ph ^ 1u, abort_flag) ? 1 : 0;
-#ifdef ACTKV_EXP_NO_TMA
-      if (ok) mbar_arrive(smem_u32(&bars->k_full[s]));
-#else
+      ok = mbar_wait(smem_u32(&bars->k_empty[s]), ph ^ 1u, abort_flag, wait_cycles) ? 1 : 0;
       if (ok) mbar_expect_tx(smem_u32(&bars->k_full[s]), NH * HALF_BYTES);
-#endif
     }
     ok = __shfl_sync(0xffffffffu, ok, 0);
     if (!ok) break;
     // lane j < ppt NH: page j % ppt, half j / ppt of this tile
     const int32_t my_pid = __shfl_sync(0xffffffffu, pid, ((i & 3) << lp_shift) | (lane & (ppt - 1)));
-#ifndef ACTKV_EXP_NO_TMA
     if (lane < ppt * NH) {
       const int half = lane >> lp_shift;
       const uint32_t dst = k_smem + s * KTILE_BYTES + half * HALF_BYTES + (lane & (ppt - 1)) * box_bytes;
@@ -346,9 +351,6 @@ __device__ __forceinline__ void k_tile_producer(const CUtensorMap* kmap, const S
       if constexpr (K5) tma_load_5d(dst, kmap, bar, half * 64, 0, h, my_pid, layer);
       else tma_load_4d(dst, kmap, bar, half * 64, h, my_pid * ps, layer);
     }
-#else
-    (void)my_pid;
-#endif
     if ((i & 3) == 3) pid = pid_next;
   }
 }

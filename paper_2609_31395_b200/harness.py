@@ -7,7 +7,6 @@ and passes pointers.
 """
 from __future__ import annotations
 
-import os
 from dataclasses import dataclass
 from typing import Optional
 
@@ -173,8 +172,8 @@ class Compressor:
             # The score kernels run on a high-priority stream, select + compact on a low-priority one: a
             # score CTA is placed whenever it fits, the others only ever take what a score CTA leaves over
             # on its SM (registers, shared memory), so they run beside the score kernels instead of in turns.
-            self._main = torch.cuda.Stream(device=self.dev, priority=int(os.environ.get("ACTKV_MAIN_PRIO", "-1")))
-            self._aux = torch.cuda.Stream(device=self.dev, priority=int(os.environ.get("ACTKV_AUX_PRIO", "0")))
+            self._main = torch.cuda.Stream(device=self.dev, priority=-1)
+            self._aux = torch.cuda.Stream(device=self.dev, priority=0)
             self._score2 = [self.score, torch.empty_like(self.score)]
             self._sel2 = [self.sel_idx, torch.empty_like(self.sel_idx)]
             self._ev_score = [torch.cuda.Event(), torch.cuda.Event()]

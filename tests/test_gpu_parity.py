@@ -196,24 +196,22 @@ def test_group_sizes_that_are_not_powers_of_two(causal):
         _full_check(synth.generate(wl, DEV))
 
 
-def test_new_shapes_really_take_the_tensor_core_path(monkeypatch):
-    """The library picks the path by itself; forcing the FMA path (developer switch) must change the bits of
-    the scores for the shapes that are meant to run on tensor cores."""
-    shapes = [dict(G=7), dict(G=4, head_dim=64), dict(G=4, page_size=64), dict(G=16, windows=[64, 20])]
-    for kw in shapes:
+def test_new_shapes_really_take_the_tensor_core_path():
+    """The library picks the path by itself and says which (actkv_score_path): the shapes that are meant to
+    run on tensor cores do, shapes outside them (head_dim 96, pages of 8 tokens, fewer than 64 rows) take the
+    FMA kernels."""
+    from paper_2609_31395_b200 import binding as B
+    shapes = [(dict(G=7), 1), (dict(G=4, head_dim=64), 1), (dict(G=4, page_size=64), 1), (dict(G=16, windows=[64, 20]), 1),
+              (dict(G=4, head_dim=96), 0), (dict(G=4, page_size=8), 0), (dict(G=2, windows=[16, 8]), 0)]
+    for kw, want in shapes:
         G = kw.pop("G")
         windows = kw.pop("windows", [32, 16])
         wl = synth.Workload("path", 1, 2, G, [700, 257], windows, [200, 64], table_style="permutation", seed=31,
                             poison_tail=True, **kw)
         inst = synth.generate(wl, DEV)
-        monkeypatch.delenv("ACTKV_FORCE_FMA", raising=False)
-        tc_score = U.run_step(inst).score.clone()
-        inst = synth.generate(wl, DEV)
-        monkeypatch.setenv("ACTKV_FORCE_FMA", "1")
-        fma_score = U.run_step(inst).score.clone()
-        monkeypatch.delenv("ACTKV_FORCE_FMA", raising=False)
-        assert not torch.equal(tc_score, fma_score)
-        assert torch.allclose(tc_score, fma_score, rtol=2e-3, atol=0)
+        got = B.actkv_score_path(B.pool_desc(inst.pool), wl.n_q_heads, max(windows), wl.sm_scale, inst.q)
+        assert got == want, (kw, G, windows, got)
+        _full_check(inst)
 
 
 def test_head_major_pool_layout():
