@@ -252,6 +252,13 @@ def run_ours(args):
     sampler.start()                            # early: nvidia-smi takes a moment to deliver its first sample
     inst = synth.generate(wl, dev)
     sz = H.sizes_of(inst)
+    pipe_groups = None
+    if args.pipeline and args.pipeline != "none":
+        sizes = [NL // 3, NL // 3, NL - 2 * (NL // 3)] if args.pipeline == "auto" else [int(x) for x in args.pipeline.split(",")]
+        sizes = [x for x in sizes if x > 0]
+        if sum(sizes) != NL:
+            raise SystemExit(f"--pipeline: group sizes must add up to {NL} layers")
+        pipe_groups = [(sum(sizes[:i]), sum(sizes[:i + 1])) for i in range(len(sizes))]
     comp = H.Compressor(inst.pool, inst.page_table, inst.seq_len, inst.free_list, inst.free_count, wl.n_q_heads, sz,
                         layers_per_call=args.layers_per_call if args.layers_per_call else (8 if args.overlap else None),
                         want_lse=True)
@@ -278,6 +285,9 @@ def run_ours(args):
         comp.status.zero_()
 
     lse_supplied = None
+    pipelined = False                          # set for the secondary pipelined-compaction lines only
+    pipe_stats = torch.zeros((len(pipe_groups) if pipe_groups else 1, 2), dtype=torch.int32, device=dev)
+    pipe_comp = None
     lrfu_state = None                          # set for the secondary LRFU-policy line only
     inplace_mode = False                       # set for the secondary in-place-compaction line only
     stage_names = ["budget", "lse", "score", "select", "compact"]
@@ -299,6 +309,10 @@ def run_ours(args):
         if args.overlap:
             n = comp.step_overlapped(inst.q, inst.win_indptr, inst.tok_indptr, bud, wl.sm_scale, wl.causal,
                                      lse_in=lse_supplied, marks=mark)
+        elif pipelined:
+            n = pipe_comp.step_pipelined(inst.q, inst.win_indptr, inst.tok_indptr, bud, wl.sm_scale, wl.causal,
+                                         lse_in=lse_supplied, marks=(lambda nm: mark(nm)), groups=pipe_groups,
+                                         stats=pipe_stats)
         else:
             n = comp.step(inst.q, inst.win_indptr, inst.tok_indptr, bud, wl.sm_scale, wl.causal,
                           lse_in=lse_supplied, marks=(lambda nm: mark(nm)), lrfu=lrfu_state, inplace=inplace_mode)
@@ -443,6 +457,42 @@ def run_ours(args):
                                  alg_bytes / (float(tl.item()) * 1e-3) / 1e9 / pk["hbm_gbs"]}
         comp.check_status()
 
+    # ---- the same step with the compaction of a layer group hidden under the score kernels of the next group
+    # (actkv_compact_begin / actkv_score_overlap / actkv_compact_end), both LSE modes
+    pipelined_line = None
+    if pipe_groups is not None and not args.overlap:
+        lpc_p = max(l1 - l0 for l0, l1 in pipe_groups)
+        pipe_comp = H.Compressor(inst.pool, inst.page_table, inst.seq_len, inst.free_list, inst.free_count, wl.n_q_heads, sz,
+                                 layers_per_call=lpc_p, want_lse=False)
+        pipelined = True
+        pipelined_line = {"groups": [l1 - l0 for l0, l1 in pipe_groups]}
+        for mode in ("internal", "supplied"):
+            lse_supplied = comp.lse.clone() if mode == "supplied" else None
+            ms, sc_ms, cp_ms = [], [], []
+            for it in range(2 + min(args.steps, 5)):
+                restore()
+                pipe_comp.status.zero_()
+                ev = []
+                one_step(ev)
+                torch.cuda.synchronize()
+                if it >= 2:
+                    ms.append(ev[0][1].elapsed_time(ev[-1][1]))
+                    sc_ms.append(sum(ev[i - 1][1].elapsed_time(ev[i][1]) for i in range(1, len(ev)) if ev[i][0] == "score"))
+                    cp_ms.append(sum(ev[i - 1][1].elapsed_time(ev[i][1]) for i in range(1, len(ev)) if ev[i][0] == "compact"))
+            pipe_comp.check_status()
+            tl = torch.tensor([sum(ms) / len(ms)], dtype=torch.float64, device=dev)
+            if dist is not None:
+                dist.all_reduce(tl, op=dist.ReduceOp.MAX)
+            st = pipe_stats.cpu().tolist()
+            pipelined_line[mode] = {
+                "ms_per_step": float(tl.item()), "value": world * tokens / (float(tl.item()) * 1e-3), "unit": UNIT,
+                "hbm_roofline_frac_whole_step": alg_bytes / (float(tl.item()) * 1e-3) / 1e9 / pk["hbm_gbs"],
+                "score_ms_with_copies_inside": sum(sc_ms) / len(sc_ms), "exposed_compact_ms": sum(cp_ms) / len(cp_ms),
+                "copy_items_taken_by_score_kernels": [round(b / a, 3) if a else None for a, b in st]}
+        lse_supplied = None
+        pipelined = False
+        del pipe_comp
+
     # ---- the same step ranking by the attention-aware LRFU keep-score (Section 5.1): score -> keepscore
     # -> select -> gather keep-scores -> compact, p = 0.9, lambda = 0.5, 512 protected tokens per request
     lrfu_line = None
@@ -583,7 +633,8 @@ def run_ours(args):
                                   "of the next group" if args.overlap else "none (one stream)",
                        "l2": "inputs (KV pool %.1f GB) far larger than the 126 MB L2" % (inst.pool.numel() * 2 / 1e9)},
             "stage_ms": stage_ms, "hbm_roofline_frac_whole_step": hbm_frac_whole,
-            "with_lse_supplied": lse_supplied_line, "with_lrfu_policy": lrfu_line,
+            "with_lse_supplied": lse_supplied_line, "with_pipelined_compaction": pipelined_line,
+            "with_lrfu_policy": lrfu_line,
             "with_inplace_compaction": inplace_line, "streaming_update": stream_line,
             "algorithmic_bytes_per_step": alg_bytes, "k_bytes_per_pass": bytes_k,
             "roofline": roofline, "roofline_stages": stages, "roofline_lse_exp_rate": lse_exp,
@@ -609,6 +660,9 @@ def main():
     ap.add_argument("--overlap", action="store_true",
                     help="run select + compact of a layer group on a second stream under the score kernels of the "
                          "next group (measured: no gain, the score CTAs fill the register file of every SM)")
+    ap.add_argument("--pipeline", default="auto",
+                    help="layer groups of the secondary pipelined-compaction lines: 'auto' (three equal groups), "
+                         "comma-separated group sizes, or 'none'")
     ap.add_argument("--lse", default="internal", choices=["internal", "supplied"])
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")

@@ -301,6 +301,67 @@ int actkv_compact(const actkv_pool_t* pool /* host */, const actkv_tables_t* tab
                   void* ws, size_t ws_bytes, int32_t* status, actkv_stream_t stream);
 
 /* ---------------------------------------------------------------------------------------
+ * actkv_compact_begin / actkv_score_overlap / actkv_compact_end — the compaction of one layer
+ * group hidden under the score kernels of the next one.
+ * (Section 3.3: the three primitives are independent per layer; Section 7.2 / Algorithm 4: the
+ *  copies of a planned compaction are order-free, their sources and destinations disjoint.)
+ *
+ * The score kernels are bound by the tensor pipe and leave most of the HBM bandwidth idle; the
+ * copy of a compaction is bound by HBM and needs no tensor pipe.  A step over many layers can
+ * therefore run, for layer groups g = 0, 1, ...:
+ *     actkv_score_overlap(group g, pending = ws)   score of g; spare warps of its kernels copy rows of g-1
+ *     actkv_compact_end(group g-1, ws)             copies whatever is left of g-1 (+ tables after the last layer)
+ *     actkv_select(group g)
+ *     actkv_compact_begin(group g, ws)             plan of g, published as a work queue in ws; copies nothing
+ * and after the last group actkv_compact_end for it.  All calls on one stream; one workspace and
+ * one index buffer suffice, because actkv_compact_end(g-1) precedes actkv_select(g).
+ *
+ * actkv_compact_begin: arguments as actkv_compact.  Runs the plan (fresh pages for
+ *   [layer_begin, layer_end), errors as actkv_compact), resolves the source of every row once into a
+ *   table and records the job in `ws`, which must stay untouched, like sel_idx / keep_indptr /
+ *   budget / the tables, until the matching actkv_compact_end has run.  `ws` must have
+ *   actkv_compact_deferred_workspace_bytes(pool, n_req, max_pages, layer_end - layer_begin, max_keep)
+ *   bytes for the copies to be deferred; with only actkv_compact_workspace_bytes nothing is deferred
+ *   and actkv_compact_end copies everything.  reuse_plan != 0: `ws` still holds the plan of an earlier
+ *   actkv_compact_begin of the same step (same tables, budgets and max_keep, nothing finalized in
+ *   between; the plan does not depend on the layers), so only the job of this layer range is recorded.
+ * actkv_score_overlap: actkv_score with one more argument, pending_compact_ws: the workspace of a
+ *   begun compaction of OTHER layers of the same pool, or NULL (then it is actkv_score).  The
+ *   result of the score does not depend on it.  On the tensor-core path four spare warps per CTA take
+ *   items (one destination page of one request and layer) of the pending job from a queue for as
+ *   long as their CTA is scoring; the FMA path ignores the argument.
+ * actkv_compact_end: the same arguments as the actkv_compact_begin it closes.  Copies every item
+ *   not yet taken, then, when layer_end == pool->n_layers, updates the tables as actkv_compact does.
+ * begin + end without a score call in between equals actkv_compact.  Pools the item copy does not
+ * take (head_dim other than 64 / 128 / 256, more than 128 (slot, head) pairs per page) are copied
+ * entirely by actkv_compact_end.
+ */
+size_t actkv_compact_deferred_workspace_bytes(const actkv_pool_t* pool /* host */, int32_t n_req, int32_t max_pages,
+                                              int32_t n_layers_sub, int32_t max_keep);
+int actkv_compact_begin(const actkv_pool_t* pool /* host */, const actkv_tables_t* tables /* host */,
+                        int32_t layer_begin, int32_t layer_end,
+                        const int32_t* sel_idx, int64_t sel_stride, const int32_t* keep_indptr,
+                        const int32_t* budget, int32_t max_keep, int32_t reuse_plan,
+                        void* ws, size_t ws_bytes, int32_t* status, actkv_stream_t stream);
+int actkv_compact_end(const actkv_pool_t* pool /* host */, const actkv_tables_t* tables /* host */,
+                      int32_t layer_begin, int32_t layer_end,
+                      const int32_t* sel_idx, int64_t sel_stride, const int32_t* keep_indptr,
+                      const int32_t* budget, int32_t max_keep,
+                      void* ws, size_t ws_bytes, int32_t* status, actkv_stream_t stream);
+/* stats (device, int32[2]) <- { items of the job begun in ws, items that score kernels executed };
+ * an item is 32 (slot, head) pairs of one destination page.  Valid from actkv_compact_begin until
+ * the next one on the same ws. */
+int actkv_compact_stats(const void* ws, int32_t* stats, actkv_stream_t stream);
+int actkv_score_overlap(const actkv_pool_t* pool /* host */, const actkv_tables_t* tables /* host */,
+                        int32_t layer_begin, int32_t layer_end,
+                        const void* q, const int32_t* win_indptr, int32_t n_q_heads,
+                        const float* lse_in, float sm_scale, int32_t causal,
+                        const int32_t* tok_indptr, float* score_out, float* lse_out,
+                        int32_t sum_win, int32_t max_win, int32_t sum_tok, int32_t max_tok,
+                        void* ws, size_t ws_bytes, void* pending_compact_ws,
+                        int32_t* status, actkv_stream_t stream);
+
+/* ---------------------------------------------------------------------------------------
  * actkv_compact_inplace — compaction into the last X logical blocks of each request, without
  * fresh pages (Section 7.2 region equations; Algorithm 4 steps 1-6), one keep mask per
  * (layer, KV head), given as the ascending index lists actkv_select writes.

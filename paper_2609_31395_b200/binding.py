@@ -27,6 +27,7 @@ EXPORTS = ["actkv_budget_workspace_bytes", "actkv_budget", "actkv_score_workspac
            "actkv_compact_workspace_bytes", "actkv_compact", "actkv_compact_noalloc",
            "actkv_compact_noalloc_max_bytes", "actkv_step_host", "actkv_keepscore", "actkv_gather_f32",
            "actkv_compact_inplace", "actkv_score_path", "actkv_debug_inject_stall",
+           "actkv_compact_deferred_workspace_bytes", "actkv_compact_begin", "actkv_compact_end", "actkv_score_overlap", "actkv_compact_stats",
            "actkv_version"]
 
 
@@ -144,6 +145,19 @@ def load():
     lib.actkv_compact_noalloc.restype = i32
     lib.actkv_compact_noalloc.argtypes = [C.POINTER(PoolDesc), C.POINTER(TablesDesc), i32, i32, vp, i64, vp, vp, i32,
                                           vp, vp]
+    lib.actkv_compact_begin.restype = i32
+    lib.actkv_compact_begin.argtypes = [C.POINTER(PoolDesc), C.POINTER(TablesDesc), i32, i32, vp, i64, vp, vp, i32, i32, vp,
+                                        sz, vp, vp]
+    lib.actkv_compact_end.restype = i32
+    lib.actkv_compact_end.argtypes = [C.POINTER(PoolDesc), C.POINTER(TablesDesc), i32, i32, vp, i64, vp, vp, i32, vp, sz,
+                                      vp, vp]
+    lib.actkv_score_overlap.restype = i32
+    lib.actkv_score_overlap.argtypes = [C.POINTER(PoolDesc), C.POINTER(TablesDesc), i32, i32, vp, vp, i32, vp, f32, i32,
+                                        vp, vp, vp, i32, i32, i32, i32, vp, sz, vp, vp, vp]
+    lib.actkv_compact_deferred_workspace_bytes.restype = sz
+    lib.actkv_compact_deferred_workspace_bytes.argtypes = [C.POINTER(PoolDesc), i32, i32, i32, i32]
+    lib.actkv_compact_stats.restype = i32
+    lib.actkv_compact_stats.argtypes = [vp, vp, vp]
     lib.actkv_score_path.restype = i32
     lib.actkv_score_path.argtypes = [C.POINTER(PoolDesc), i32, i32, f32, vp, i32]
     lib.actkv_debug_inject_stall.restype = i32
@@ -233,6 +247,49 @@ def actkv_score(pool: PoolDesc, tables: TablesDesc, layer_begin, layer_end, q, w
                             _ptr(ws, None, "ws"), ws.numel() * ws.element_size(),
                             _ptr(status, torch.int32, "status"), _stream(stream))
     _check("actkv_score", rc)
+
+
+def actkv_score_overlap(pool: PoolDesc, tables: TablesDesc, layer_begin, layer_end, q, win_indptr, n_q_heads, lse_in,
+                        sm_scale, causal, tok_indptr, score_out, lse_out, sum_win, max_win, sum_tok, max_tok, ws,
+                        pending_compact_ws, status, stream=None):
+    rc = load().actkv_score_overlap(C.byref(pool), C.byref(tables), layer_begin, layer_end, _ptr(q, torch.bfloat16, "q"),
+                                    _ptr(win_indptr, torch.int32, "win_indptr"), n_q_heads,
+                                    _ptr(lse_in, torch.float32, "lse_in"), float(sm_scale), int(bool(causal)),
+                                    _ptr(tok_indptr, torch.int32, "tok_indptr"),
+                                    _ptr(score_out, torch.float32, "score_out"), _ptr(lse_out, torch.float32, "lse_out"),
+                                    sum_win, max_win, sum_tok, max_tok, _ptr(ws, None, "ws"),
+                                    ws.numel() * ws.element_size(), _ptr(pending_compact_ws, None, "pending_compact_ws"),
+                                    _ptr(status, torch.int32, "status"), _stream(stream))
+    _check("actkv_score_overlap", rc)
+
+
+def actkv_compact_begin(pool: PoolDesc, tables: TablesDesc, layer_begin, layer_end, sel_idx, sel_stride, keep_indptr,
+                        budget, max_keep, ws, status, stream=None, reuse_plan=False):
+    rc = load().actkv_compact_begin(C.byref(pool), C.byref(tables), layer_begin, layer_end,
+                                    _ptr(sel_idx, torch.int32, "sel_idx"), sel_stride,
+                                    _ptr(keep_indptr, torch.int32, "keep_indptr"), _ptr(budget, torch.int32, "budget"),
+                                    max_keep, int(bool(reuse_plan)), _ptr(ws, None, "ws"), ws.numel() * ws.element_size(),
+                                    _ptr(status, torch.int32, "status"), _stream(stream))
+    _check("actkv_compact_begin", rc)
+
+
+def actkv_compact_end(pool: PoolDesc, tables: TablesDesc, layer_begin, layer_end, sel_idx, sel_stride, keep_indptr,
+                      budget, max_keep, ws, status, stream=None):
+    rc = load().actkv_compact_end(C.byref(pool), C.byref(tables), layer_begin, layer_end,
+                                  _ptr(sel_idx, torch.int32, "sel_idx"), sel_stride,
+                                  _ptr(keep_indptr, torch.int32, "keep_indptr"), _ptr(budget, torch.int32, "budget"),
+                                  max_keep, _ptr(ws, None, "ws"), ws.numel() * ws.element_size(),
+                                  _ptr(status, torch.int32, "status"), _stream(stream))
+    _check("actkv_compact_end", rc)
+
+
+def actkv_compact_deferred_workspace_bytes(pool: PoolDesc, n_req, max_pages, n_layers_sub, max_keep) -> int:
+    return load().actkv_compact_deferred_workspace_bytes(C.byref(pool), n_req, max_pages, n_layers_sub, max_keep)
+
+
+def actkv_compact_stats(ws, stats, stream=None):
+    _check("actkv_compact_stats", load().actkv_compact_stats(_ptr(ws, None, "ws"), _ptr(stats, torch.int32, "stats"),
+                                                             _stream(stream)))
 
 
 def actkv_score_path(pool: PoolDesc, n_q_heads, max_win, sm_scale, q, streaming=False) -> int:

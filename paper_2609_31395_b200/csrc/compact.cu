@@ -8,27 +8,32 @@
 //              written whole and coalesced, sources are 256-byte row gathers;
 //   finalize : new page table / seq_len, pop and push on the free list (only on the call whose
 //              layer range ends at the pool's last layer).
-#include "common.cuh"
+#include <algorithm>
+
+#include "compact_job.cuh"
 
 namespace actkv {
 
-struct CompactWs {
-  int32_t plan_ok;       // 1 when the copy / finalize kernels may run
-  int32_t total_new;     // pages popped
-  int32_t pad[2];
-  // followed by int32 new_off[R], push_off[R], new_pages[R * max_pages]
+// What the host knows of a compaction call, handed to the plan kernel, which records it in the workspace.
+struct CompactJobArgs {
+  PoolView pool;
+  const int32_t* sel_idx;
+  int64_t sel_stride;
+  const int32_t* keep_indptr;
+  int32_t layer_begin, n_layers;
+  int32_t vpr_shift;     // >= 0: the copies may be deferred to a work queue (actkv_compact_begin)
+  int32_t deferred;
+  uint32_t* src_tab;     // deferred: room for the resolved sources of every item
+  int64_t src_tab_items; // ... in items (32 entries each)
 };
-
-__device__ __forceinline__ int32_t* ws_new_off(CompactWs* w) { return reinterpret_cast<int32_t*>(w + 1); }
-__device__ __forceinline__ int32_t* ws_push_off(CompactWs* w, int R) { return ws_new_off(w) + R; }
-__device__ __forceinline__ int32_t* ws_new_pages(CompactWs* w, int R) { return ws_new_off(w) + 2 * R; }
 
 __global__ void compact_plan_kernel(TablesView tab, int32_t page_size, int32_t n_pages,
                                     const int32_t* __restrict__ budget, int32_t max_keep,
-                                    CompactWs* ws, int32_t* status) {
+                                    CompactWs* ws, int32_t* status, CompactJobArgs job) {
   const int R = tab.n_req;
   int32_t* new_off = ws_new_off(ws);
   int32_t* push_off = ws_push_off(ws, R);
+  int32_t* item_off = ws_item_off(ws, R);
   int32_t* new_pages = ws_new_pages(ws, R);
   __shared__ int32_t s_total, s_ok;
   if (threadIdx.x == 0) {
@@ -37,6 +42,7 @@ __global__ void compact_plan_kernel(TablesView tab, int32_t page_size, int32_t n
     for (int r = 0; r < R; ++r) {
       const int32_t L = tab.seq_len[r];
       int32_t B = budget[r] < 0 ? 0 : budget[r];
+      item_off[r] = off;
       if (B < L) {
         new_off[r] = off;
         push_off[r] = poff;
@@ -54,6 +60,7 @@ __global__ void compact_plan_kernel(TablesView tab, int32_t page_size, int32_t n
     else if (off > fc) { report(status, ACTKV_E_NOFREE, off, fc); ok = false; }
     // the old pages pushed back after the pops must fit on the stack
     else if ((int64_t)fc - off + poff > n_pages) { report(status, ACTKV_E_INVALID, -2, fc - off + poff); ok = false; }
+    item_off[R] = off;
     s_total = off;
     s_ok = ok ? 1 : 0;
   }
@@ -85,7 +92,76 @@ __global__ void compact_plan_kernel(TablesView tab, int32_t page_size, int32_t n
     }
   }
   __syncthreads();
-  if (threadIdx.x == 0) { ws->plan_ok = s_ok; ws->total_new = total; }
+  if (threadIdx.x == 0) {
+    ws->plan_ok = s_ok;
+    ws->total_new = total;
+    ws->next_item = 0u;
+    const int32_t jp = (page_size * job.pool.n_kv_heads + 31) / 32;
+    const int64_t items = (int64_t)total * job.n_layers * jp;
+    ws->n_items = (s_ok && job.deferred && job.vpr_shift >= 0 && items <= 0x7fffffff && items <= job.src_tab_items)
+                      ? (int32_t)items : 0;
+    ws->src_tab = job.src_tab;
+    ws->pool = job.pool;
+    ws->tab = tab;
+    ws->sel_idx = job.sel_idx;
+    ws->sel_stride = job.sel_stride;
+    ws->keep_indptr = job.keep_indptr;
+    ws->budget = budget;
+    ws->status = status;
+    ws->layer_begin = job.layer_begin;
+    ws->n_layers = job.n_layers;
+    ws->vpr_shift = job.deferred ? job.vpr_shift : -1;
+    ws->parts_per_page = jp;
+    ws->role_items = 0;
+    ws->pad = 0;
+  }
+}
+
+__global__ void compact_stats_kernel(const CompactWs* ws, int32_t* out) {
+  out[0] = ws->n_items;
+  out[1] = ws->role_items;
+}
+
+// A further layer range of a step whose plan is already in the workspace (the plan depends on the tables and
+// the budgets only, not on the layers): only the job is recorded anew.
+__global__ void compact_rejob_kernel(CompactWs* ws, CompactJobArgs job, int32_t* status) {
+  const bool ok = ws->plan_ok && !status_set(status);
+  if (!ok) ws->plan_ok = 0;
+  const int64_t items = (int64_t)ws->total_new * job.n_layers * ws->parts_per_page;
+  ws->next_item = 0u;
+  ws->role_items = 0;
+  ws->n_items = (ok && job.deferred && job.vpr_shift >= 0 && items <= 0x7fffffff && items <= job.src_tab_items)
+                    ? (int32_t)items : 0;
+  ws->src_tab = job.src_tab;
+  ws->sel_idx = job.sel_idx;
+  ws->sel_stride = job.sel_stride;
+  ws->keep_indptr = job.keep_indptr;
+  ws->layer_begin = job.layer_begin;
+  ws->n_layers = job.n_layers;
+  ws->vpr_shift = job.deferred ? job.vpr_shift : -1;
+}
+
+// Resolves the sources of every item of a deferred copy (one warp per item).
+__global__ void __launch_bounds__(128) compact_resolve_kernel(CompactWs* ws) {
+  const int lane = threadIdx.x & 31;
+  const int64_t n = cj_count(ws);
+  for (int64_t item = (int64_t)blockIdx.x * 4 + (threadIdx.x >> 5); item < n; item += (int64_t)gridDim.x * 4)
+    cj_resolve_item(ws, (int)item, lane);
+}
+
+// What is left of a deferred copy: every warp takes items until the queue is empty.
+template <int VPR_SHIFT>
+__global__ void __launch_bounds__(128) compact_drain_kernel(CompactWs* ws) {
+  const int lane = threadIdx.x & 31;
+  if (ws->vpr_shift != VPR_SHIFT) return;
+  const uint32_t n = cj_count(ws);
+  if (n == 0) return;
+  uint32_t item = cj_pop(ws, lane);
+  while (item < n) {
+    const uint32_t next = cj_pop(ws, lane);              // asked for now, looked at after this item's copies
+    cj_copy_item<VPR_SHIFT, 16>(ws, (int)item, lane);
+    item = next;
+  }
 }
 
 constexpr int CP_NT = 128;
@@ -207,13 +283,26 @@ extern "C" {
 
 size_t actkv_compact_workspace_bytes(int32_t n_req, int32_t max_pages) {
   if (n_req < 0 || max_pages < 0) return 0;
-  return actkv::align_up(sizeof(actkv::CompactWs) + sizeof(int32_t) * ((size_t)2 * n_req + (size_t)n_req * max_pages), 256);
+  return actkv::align_up(sizeof(actkv::CompactWs) +
+                         sizeof(int32_t) * ((size_t)3 * n_req + 1 + (size_t)n_req * max_pages), 256);
 }
 
-int actkv_compact(const actkv_pool_t* pool, const actkv_tables_t* tables, int32_t layer_begin,
-                  int32_t layer_end, const int32_t* sel_idx, int64_t sel_stride,
-                  const int32_t* keep_indptr, const int32_t* budget, int32_t max_keep,
-                  void* ws, size_t ws_bytes, int32_t* status, actkv_stream_t stream) {
+size_t actkv_compact_deferred_workspace_bytes(const actkv_pool_t* pool, int32_t n_req, int32_t max_pages,
+                                              int32_t n_layers_sub, int32_t max_keep) {
+  if (!pool || n_req < 0 || max_pages < 0 || n_layers_sub < 0 || max_keep < 0 || pool->page_size <= 0) return 0;
+  const size_t base = actkv_compact_workspace_bytes(n_req, max_pages);
+  int64_t max_x = ((int64_t)max_keep + pool->page_size - 1) / pool->page_size;
+  if (max_x > max_pages) max_x = max_pages;
+  const int64_t jp = ((int64_t)pool->page_size * pool->n_kv_heads + 31) / 32;
+  return base + actkv::align_up((size_t)(max_x * n_req * n_layers_sub * jp) * 32 * sizeof(uint32_t), 256);
+}
+
+}  // extern "C"
+
+namespace actkv {
+
+static int compact_check(const actkv_pool_t* pool, const actkv_tables_t* tables, int32_t layer_begin, int32_t layer_end,
+                         const int32_t* budget, int32_t max_keep, int64_t sel_stride, void* ws, size_t ws_bytes) {
   if (!pool || !tables || !pool->base) return ACTKV_E_INVALID;
   if (layer_begin < 0 || layer_end > pool->n_layers || layer_begin > layer_end) return ACTKV_E_INVALID;
   if (pool->page_size <= 0 || pool->head_dim <= 0 || pool->head_dim % 8 != 0 || pool->n_kv_heads <= 0)
@@ -225,44 +314,168 @@ int actkv_compact(const actkv_pool_t* pool, const actkv_tables_t* tables, int32_
   const int R = tables->n_req;
   if (R < 0 || tables->max_pages < 0 || max_keep < 0 || sel_stride < 0) return ACTKV_E_INVALID;
   if (R == 0) return ACTKV_OK;
-  if (!tables->page_table || !tables->seq_len || !tables->free_list || !tables->free_count || !budget ||
-      !keep_indptr || !sel_idx || !ws)
+  if (!tables->page_table || !tables->seq_len || !tables->free_list || !tables->free_count || !budget || !ws)
     return ACTKV_E_INVALID;
   if (ws_bytes < actkv_compact_workspace_bytes(R, tables->max_pages)) return ACTKV_E_WORKSPACE;
   if (R > 65535 || layer_end - layer_begin > 65535) return ACTKV_E_INVALID;
-  cudaStream_t s = (cudaStream_t)stream;
-  actkv::PoolView pv = actkv::make_view(pool);
-  actkv::TablesView tv = actkv::make_view(tables);
-  actkv::CompactWs* w = (actkv::CompactWs*)ws;
-  actkv::compact_plan_kernel<<<1, 1024, 0, s>>>(tv, pool->page_size, pool->n_pages, budget, max_keep, w, status);
+  return ACTKV_OK;
+}
+
+// log2 of the 16-byte vectors per row when the warp-level item copy takes this pool: head_dim 64, 128 or 256,
+// a layer (K and V) within 2^32 16-byte units; else -1.
+static int deferrable_shift(const actkv_pool_t* pool) {
+  const int vpr = pool->head_dim / 8;
+  const int shift = vpr == 8 ? 3 : vpr == 16 ? 4 : vpr == 32 ? 5 : -1;
+  if (shift < 0) return -1;
+  const int64_t extent = pool->stride_kv + (int64_t)pool->n_pages * pool->stride_page;       // elements, upper bound
+  if (pool->stride_kv < 0 || pool->stride_page < 0 || pool->stride_slot < 0 || pool->stride_head < 0) return -1;
+  if (extent / 8 >= 0xffffffffLL) return -1;
+  return shift;
+}
+
+static int compact_plan(const actkv_pool_t* pool, const actkv_tables_t* tables, int32_t layer_begin, int32_t layer_end,
+                        const int32_t* sel_idx, int64_t sel_stride, const int32_t* keep_indptr, const int32_t* budget,
+                        int32_t max_keep, void* ws, size_t ws_bytes, int32_t* status, cudaStream_t s, bool deferred,
+                        bool reuse_plan = false) {
+  CompactJobArgs job;
+  const size_t base = actkv_compact_workspace_bytes(tables->n_req, tables->max_pages);
+  // the copies are deferred only when the workspace has room for the resolved sources of the largest job these
+  // arguments allow (the same rule decides in actkv_compact_end who copies)
+  deferred = deferred && ws_bytes >= actkv_compact_deferred_workspace_bytes(pool, tables->n_req, tables->max_pages,
+                                                                             layer_end - layer_begin, max_keep);
+  job.src_tab = (uint32_t*)((char*)ws + base);
+  job.src_tab_items = deferred ? (int64_t)((ws_bytes - base) / (32 * sizeof(uint32_t))) : 0;
+  job.pool = make_view(pool);
+  job.sel_idx = sel_idx;
+  job.sel_stride = sel_stride;
+  job.keep_indptr = keep_indptr;
+  job.layer_begin = layer_begin;
+  job.n_layers = layer_end - layer_begin;
+  job.vpr_shift = deferrable_shift(pool);
+  job.deferred = deferred ? 1 : 0;
+  if (reuse_plan)
+    compact_rejob_kernel<<<1, 1, 0, s>>>((CompactWs*)ws, job, status);
+  else
+    compact_plan_kernel<<<1, 1024, 0, s>>>(make_view(tables), pool->page_size, pool->n_pages, budget, max_keep,
+                                           (CompactWs*)ws, status, job);
   ACTKV_CHECK_LAUNCH();
-  const int nl = layer_end - layer_begin;
-  int max_x = (max_keep + pool->page_size - 1) / pool->page_size;
-  if (max_x > tables->max_pages) max_x = tables->max_pages;
-  if (nl > 0 && max_x > 0) {
-    dim3 grid((unsigned)max_x, (unsigned)R, (unsigned)nl);
-    const size_t sm = (size_t)2 * pool->page_size * pool->n_kv_heads * sizeof(int64_t);
-    if (sm > 48 * 1024) return ACTKV_E_INVALID;
-    const int vpr = pool->head_dim / 8;
-    if (vpr == 16)
-      actkv::compact_copy_kernel<4><<<grid, actkv::CP_NT, sm, s>>>(pv, tv, layer_begin, sel_idx, sel_stride,
-                                                                    keep_indptr, budget, w, status);
-    else if (vpr == 8)
-      actkv::compact_copy_kernel<3><<<grid, actkv::CP_NT, sm, s>>>(pv, tv, layer_begin, sel_idx, sel_stride,
-                                                                    keep_indptr, budget, w, status);
-    else if (vpr == 32)
-      actkv::compact_copy_kernel<5><<<grid, actkv::CP_NT, sm, s>>>(pv, tv, layer_begin, sel_idx, sel_stride,
-                                                                    keep_indptr, budget, w, status);
-    else
-      actkv::compact_copy_kernel<-1><<<grid, actkv::CP_NT, sm, s>>>(pv, tv, layer_begin, sel_idx, sel_stride,
-                                                                     keep_indptr, budget, w, status);
-    ACTKV_CHECK_LAUNCH();
-  }
-  if (layer_end == pool->n_layers) {
-    actkv::compact_finalize_kernel<<<1, 1024, 0, s>>>(tv, pool->page_size, budget, w, status);
+  if (deferred && job.vpr_shift >= 0 && job.src_tab_items > 0) {
+    // one warp per item of the largest job these arguments allow (short, independent chains of lookups)
+    int64_t max_x = ((int64_t)max_keep + pool->page_size - 1) / pool->page_size;
+    if (max_x > tables->max_pages) max_x = tables->max_pages;
+    const int64_t jp = ((int64_t)pool->page_size * pool->n_kv_heads + 31) / 32;
+    const int64_t items_max = std::min<int64_t>(max_x * tables->n_req * job.n_layers * jp, job.src_tab_items);
+    const int64_t ctas = std::min<int64_t>(std::max<int64_t>(1, (items_max + 3) / 4), 1 << 20);
+    compact_resolve_kernel<<<(unsigned)ctas, 128, 0, s>>>((CompactWs*)ws);
     ACTKV_CHECK_LAUNCH();
   }
   return ACTKV_OK;
+}
+
+// One CTA per (destination page, request, layer): the whole copy of a call in one launch.
+static int compact_copy_all(const actkv_pool_t* pool, const actkv_tables_t* tables, int32_t layer_begin, int32_t layer_end,
+                            const int32_t* sel_idx, int64_t sel_stride, const int32_t* keep_indptr, const int32_t* budget,
+                            int32_t max_keep, void* ws, int32_t* status, cudaStream_t s) {
+  PoolView pv = make_view(pool);
+  TablesView tv = make_view(tables);
+  CompactWs* w = (CompactWs*)ws;
+  const int nl = layer_end - layer_begin, R = tables->n_req;
+  int max_x = (max_keep + pool->page_size - 1) / pool->page_size;
+  if (max_x > tables->max_pages) max_x = tables->max_pages;
+  if (nl <= 0 || max_x <= 0) return ACTKV_OK;
+  dim3 grid((unsigned)max_x, (unsigned)R, (unsigned)nl);
+  const size_t sm = (size_t)2 * pool->page_size * pool->n_kv_heads * sizeof(int64_t);
+  if (sm > 48 * 1024) return ACTKV_E_INVALID;
+  const int vpr = pool->head_dim / 8;
+  if (vpr == 16)
+    compact_copy_kernel<4><<<grid, CP_NT, sm, s>>>(pv, tv, layer_begin, sel_idx, sel_stride, keep_indptr, budget, w, status);
+  else if (vpr == 8)
+    compact_copy_kernel<3><<<grid, CP_NT, sm, s>>>(pv, tv, layer_begin, sel_idx, sel_stride, keep_indptr, budget, w, status);
+  else if (vpr == 32)
+    compact_copy_kernel<5><<<grid, CP_NT, sm, s>>>(pv, tv, layer_begin, sel_idx, sel_stride, keep_indptr, budget, w, status);
+  else
+    compact_copy_kernel<-1><<<grid, CP_NT, sm, s>>>(pv, tv, layer_begin, sel_idx, sel_stride, keep_indptr, budget, w, status);
+  ACTKV_CHECK_LAUNCH();
+  return ACTKV_OK;
+}
+
+static int compact_finalize(const actkv_pool_t* pool, const actkv_tables_t* tables, int32_t layer_end, const int32_t* budget,
+                            void* ws, int32_t* status, cudaStream_t s) {
+  if (layer_end != pool->n_layers) return ACTKV_OK;
+  compact_finalize_kernel<<<1, 1024, 0, s>>>(make_view(tables), pool->page_size, budget, (CompactWs*)ws, status);
+  ACTKV_CHECK_LAUNCH();
+  return ACTKV_OK;
+}
+
+}  // namespace actkv
+
+extern "C" {
+
+int actkv_compact(const actkv_pool_t* pool, const actkv_tables_t* tables, int32_t layer_begin,
+                  int32_t layer_end, const int32_t* sel_idx, int64_t sel_stride,
+                  const int32_t* keep_indptr, const int32_t* budget, int32_t max_keep,
+                  void* ws, size_t ws_bytes, int32_t* status, actkv_stream_t stream) {
+  using namespace actkv;
+  int rc = compact_check(pool, tables, layer_begin, layer_end, budget, max_keep, sel_stride, ws, ws_bytes);
+  if (rc != ACTKV_OK || tables->n_req == 0) return rc;
+  if (!keep_indptr || !sel_idx) return ACTKV_E_INVALID;
+  cudaStream_t s = (cudaStream_t)stream;
+  rc = compact_plan(pool, tables, layer_begin, layer_end, sel_idx, sel_stride, keep_indptr, budget, max_keep, ws, ws_bytes,
+                    status, s, false);
+  if (rc != ACTKV_OK) return rc;
+  rc = compact_copy_all(pool, tables, layer_begin, layer_end, sel_idx, sel_stride, keep_indptr, budget, max_keep, ws, status, s);
+  if (rc != ACTKV_OK) return rc;
+  return compact_finalize(pool, tables, layer_end, budget, ws, status, s);
+}
+
+int actkv_compact_begin(const actkv_pool_t* pool, const actkv_tables_t* tables, int32_t layer_begin,
+                        int32_t layer_end, const int32_t* sel_idx, int64_t sel_stride,
+                        const int32_t* keep_indptr, const int32_t* budget, int32_t max_keep, int32_t reuse_plan,
+                        void* ws, size_t ws_bytes, int32_t* status, actkv_stream_t stream) {
+  using namespace actkv;
+  int rc = compact_check(pool, tables, layer_begin, layer_end, budget, max_keep, sel_stride, ws, ws_bytes);
+  if (rc != ACTKV_OK || tables->n_req == 0) return rc;
+  if (!keep_indptr || !sel_idx) return ACTKV_E_INVALID;
+  return compact_plan(pool, tables, layer_begin, layer_end, sel_idx, sel_stride, keep_indptr, budget, max_keep, ws, ws_bytes,
+                      status, (cudaStream_t)stream, true, reuse_plan != 0);
+}
+
+int actkv_compact_stats(const void* ws, int32_t* stats, actkv_stream_t stream) {
+  if (!ws || !stats) return ACTKV_E_INVALID;
+  actkv::compact_stats_kernel<<<1, 1, 0, (cudaStream_t)stream>>>((const actkv::CompactWs*)ws, stats);
+  ACTKV_CHECK_LAUNCH();
+  return ACTKV_OK;
+}
+
+int actkv_compact_end(const actkv_pool_t* pool, const actkv_tables_t* tables, int32_t layer_begin,
+                      int32_t layer_end, const int32_t* sel_idx, int64_t sel_stride,
+                      const int32_t* keep_indptr, const int32_t* budget, int32_t max_keep,
+                      void* ws, size_t ws_bytes, int32_t* status, actkv_stream_t stream) {
+  using namespace actkv;
+  int rc = compact_check(pool, tables, layer_begin, layer_end, budget, max_keep, sel_stride, ws, ws_bytes);
+  if (rc != ACTKV_OK || tables->n_req == 0) return rc;
+  if (!keep_indptr || !sel_idx) return ACTKV_E_INVALID;
+  cudaStream_t s = (cudaStream_t)stream;
+  const int shift = deferrable_shift(pool);
+  const size_t need = actkv_compact_deferred_workspace_bytes(pool, tables->n_req, tables->max_pages, layer_end - layer_begin,
+                                                             max_keep);
+  if (shift < 0 || ws_bytes < need) {
+    // a pool shape the item copy does not take: nothing was deferred (the queue is empty), the copy runs here
+    rc = compact_copy_all(pool, tables, layer_begin, layer_end, sel_idx, sel_stride, keep_indptr, budget, max_keep, ws, status, s);
+    if (rc != ACTKV_OK) return rc;
+  } else {
+    // every warp takes items until the queue is empty; at most eight CTAs of four warps per SM
+    const int64_t max_x = std::min<int64_t>((max_keep + pool->page_size - 1) / pool->page_size, tables->max_pages);
+    const int64_t jp = ((int64_t)pool->page_size * pool->n_kv_heads + 31) / 32;
+    const int64_t items_max = max_x * tables->n_req * (layer_end - layer_begin) * jp;
+    const unsigned grid = (unsigned)std::max<int64_t>(1, std::min<int64_t>((items_max + 3) / 4, 148 * 8));
+    CompactWs* w = (CompactWs*)ws;
+    if (shift == 3) compact_drain_kernel<3><<<grid, 128, 0, s>>>(w);
+    else if (shift == 4) compact_drain_kernel<4><<<grid, 128, 0, s>>>(w);
+    else compact_drain_kernel<5><<<grid, 128, 0, s>>>(w);
+    ACTKV_CHECK_LAUNCH();
+  }
+  return compact_finalize(pool, tables, layer_end, budget, ws, status, s);
 }
 
 }  // extern "C"

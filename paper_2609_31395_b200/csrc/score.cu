@@ -62,7 +62,7 @@ static int score_impl(int mode, const actkv_pool_t* pool, const actkv_tables_t* 
                       const float* lse_in, float sm_scale, int32_t causal, const int32_t* tok_indptr,
                       float* score_out, float* lse_out, int32_t sum_win, int32_t max_win, int32_t sum_tok,
                       int32_t max_tok, void* ws, size_t ws_bytes, int32_t* status, actkv_stream_t stream,
-                      const int32_t* acc_steps = nullptr) {
+                      const int32_t* acc_steps = nullptr, void* copy_ws = nullptr) {
   using namespace actkv;
   if (!pool || !tables || !pool->base) return ACTKV_E_INVALID;
   if (layer_begin < 0 || layer_end > pool->n_layers || layer_begin > layer_end) return ACTKV_E_INVALID;
@@ -107,8 +107,15 @@ static int score_impl(int mode, const actkv_pool_t* pool, const actkv_tables_t* 
   // are as long as they can be while there are still many CTAs per SM (the last wave of a launch is
   // partly empty): whole key tiles, about equal, the chunk count of the workspace layout (a CTA covers
   // all rows of its unit).
+  const bool use_tc = actkv_score_path(pool, n_q_heads, max_win, sm_scale, q, acc_steps != nullptr) == 1;
   {
-    int chunk = (max_tok + lay.n_chunks - 1) / lay.n_chunks;
+    int n_chunks = lay.n_chunks;
+    // tensor-core kernel: one CTA per SM is resident, so the launch runs in rounds of 148 CTAs; of the chunk
+    // counts the workspace allows, take the one that wastes least (partly empty last round against a fixed
+    // cost per CTA of about four key tiles: the Q blocks go to tensor memory, the pipeline fills and drains)
+    if (use_tc && (mode & 1))
+      n_chunks = tc::best_split((int64_t)nls * Hkv * R, (max_tok + tc::TK - 1) / tc::TK, 4, lay.n_chunks);
+    int chunk = (max_tok + n_chunks - 1) / n_chunks;
     chunk = (chunk + 127) / 128 * 128;
     if (chunk < LSE_CHUNK) chunk = LSE_CHUNK;
     a.lse_chunk = chunk;
@@ -121,13 +128,12 @@ static int score_impl(int mode, const actkv_pool_t* pool, const actkv_tables_t* 
   const int64_t units = (int64_t)nls * Hkv * R;
   // (the streaming update keeps a running mean in place, which the row-group launches of a window above
   // 512 rows would break: such calls take the FMA path)
-  const bool use_tc = actkv_score_path(pool, n_q_heads, max_win, sm_scale, q, acc_steps != nullptr) == 1;
 
   const float* lse = lse_in;
   if (mode & 1) {
     float* lse_buf = lse_out ? lse_out : (float*)((char*)ws + lay.lse_off);
     if (use_tc) {
-      int rc = score_tc_launch_lse(a, pool, max_tok, max_win, s);
+      int rc = score_tc_launch_lse(a, pool, max_tok, max_win, s, (CompactWs*)copy_ws);
       if (rc != ACTKV_OK) return rc;
     } else {
       const int64_t grid1 = units * a.n_chunks;
@@ -150,7 +156,7 @@ static int score_impl(int mode, const actkv_pool_t* pool, const actkv_tables_t* 
   if (!(mode & 2)) return ACTKV_OK;
   if (!lse) return ACTKV_E_INVALID;
   a.lse = lse;
-  if (use_tc) return score_tc_launch_score(a, pool, max_tok, max_win, s);
+  if (use_tc) return score_tc_launch_score(a, pool, max_tok, max_win, s, (CompactWs*)copy_ws);
   const int64_t grid2 = units * a.n_tiles;
   if (grid2 > 0x7fffffffLL) return ACTKV_E_INVALID;
   const size_t sm2 = score_fma_smem_bytes(D, lay.rows_max, 2);
@@ -169,6 +175,17 @@ int actkv_score(const actkv_pool_t* pool, const actkv_tables_t* tables, int32_t 
   return score_impl(lse_in ? 2 : 3, pool, tables, layer_begin, layer_end, q, win_indptr, n_q_heads, lse_in, sm_scale,
                     causal, tok_indptr, score_out, lse_out, sum_win, max_win, sum_tok, max_tok, ws, ws_bytes, status,
                     stream);
+}
+
+int actkv_score_overlap(const actkv_pool_t* pool, const actkv_tables_t* tables, int32_t layer_begin,
+                        int32_t layer_end, const void* q, const int32_t* win_indptr, int32_t n_q_heads,
+                        const float* lse_in, float sm_scale, int32_t causal, const int32_t* tok_indptr,
+                        float* score_out, float* lse_out, int32_t sum_win, int32_t max_win, int32_t sum_tok,
+                        int32_t max_tok, void* ws, size_t ws_bytes, void* pending_compact_ws, int32_t* status,
+                        actkv_stream_t stream) {
+  return score_impl(lse_in ? 2 : 3, pool, tables, layer_begin, layer_end, q, win_indptr, n_q_heads, lse_in, sm_scale,
+                    causal, tok_indptr, score_out, lse_out, sum_win, max_win, sum_tok, max_tok, ws, ws_bytes, status,
+                    stream, nullptr, pending_compact_ws);
 }
 
 int actkv_score_lse(const actkv_pool_t* pool, const actkv_tables_t* tables, int32_t layer_begin,

@@ -169,7 +169,8 @@ inline int score_tc_launch_lse_c(const CUtensorMap& kmap, const tc::TcArgs& ta, 
   return ACTKV_OK;
 }
 
-inline int score_tc_launch_lse(ScoreArgs& a, const actkv_pool_t* pool, int max_tok, int max_win, cudaStream_t s) {
+inline int score_tc_launch_lse(ScoreArgs& a, const actkv_pool_t* pool, int max_tok, int max_win, cudaStream_t s,
+                               CompactWs* copy_ws) {
   (void)max_tok;
   CUtensorMap kmap, qmap;
   if (!tc::make_maps(pool, a.q, a.n_layers_sub, a.sum_win, a.n_q_heads, a.group, &kmap, &qmap)) return ACTKV_E_CUDA;
@@ -181,6 +182,7 @@ inline int score_tc_launch_lse(ScoreArgs& a, const actkv_pool_t* pool, int max_t
   ta.n_stages = 6;
   ta.tiles_per_cta = 0;
   ta.n_kchunks = 0;
+  ta.copy_ws = copy_ws;
   tc::apply_hook(ta);
   const int64_t units = (int64_t)a.n_layers_sub * a.pool.n_kv_heads * a.tab.n_req;
   const int64_t grid = units * a.n_chunks * ta.n_rg;
@@ -193,13 +195,18 @@ template <int G>
 inline int score_tc_launch_pool_g(const CUtensorMap& kmap, const CUtensorMap& qmap, const tc::TcArgs& ta, unsigned grid,
                                   size_t smem, cudaStream_t s) {
   auto kern = ta.a.pool.head_dim == 64 ? tc::score_tc_pool_kernel<G, 1> : tc::score_tc_pool_kernel<G, 2>;
+  // The warpgroups of this kernel re-divide the registers the launch allocates; the epilogue warpgroups would
+  // wait for ever for registers that a smaller allocation does not have, so the allocation is checked first.
+  cudaFuncAttributes fa;
+  if (cudaFuncGetAttributes(&fa, kern) != cudaSuccess || fa.numRegs < tc::POOL_REGS_ENTRY) return ACTKV_E_CUDA;
   if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return ACTKV_E_CUDA;
   kern<<<grid, tc::POOL_THREADS, smem, s>>>(kmap, qmap, ta);
   ACTKV_CHECK_LAUNCH();
   return ACTKV_OK;
 }
 
-inline int score_tc_launch_score(ScoreArgs& a, const actkv_pool_t* pool, int max_tok, int max_win, cudaStream_t s) {
+inline int score_tc_launch_score(ScoreArgs& a, const actkv_pool_t* pool, int max_tok, int max_win, cudaStream_t s,
+                                 CompactWs* copy_ws) {
   CUtensorMap kmap, qmap;
   if (!tc::make_maps(pool, a.q, a.n_layers_sub, a.sum_win, a.n_q_heads, a.group, &kmap, &qmap)) return ACTKV_E_CUDA;
   tc::TcArgs ta;
@@ -216,6 +223,7 @@ inline int score_tc_launch_score(ScoreArgs& a, const actkv_pool_t* pool, int max
   ta.n_stages = stages;
   ta.n_rg = 0;
   ta.k5 = tc::pool_needs_5d(pool) ? 1 : 0;
+  ta.copy_ws = copy_ws;
   tc::apply_hook(ta);
   const int64_t units = (int64_t)a.n_layers_sub * a.pool.n_kv_heads * a.tab.n_req;
   const int max_tiles = (max_tok + tc::TK - 1) / tc::TK;

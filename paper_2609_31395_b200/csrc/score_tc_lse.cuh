@@ -97,7 +97,10 @@ __device__ __forceinline__ void lse_slow32(const float* v, int nv, float c, floa
 }
 
 constexpr int LSE_EPI_WARPS = 16;                // (TMEM lane quarter, accumulator, column half)
-constexpr int LSE_THREADS = (3 + LSE_EPI_WARPS) * 32;     // producer, two MMA issuers, epilogue
+constexpr int LSE_COPY_WARPS = 1;                // copy role (items of a pending compaction, when the launch carries one);
+                                                 // 20 warps of 96 registers are what the register file holds
+constexpr int LSE_COPY_WARP0 = 3 + LSE_EPI_WARPS;
+constexpr int LSE_THREADS = (3 + LSE_EPI_WARPS + LSE_COPY_WARPS) * 32;     // producer, two MMA issuers, epilogue, copy
 constexpr int LSE_SLOTS = 2;                     // accumulators
 constexpr int LSE_A_COLS = 256;                  // TMEM columns holding the four Q blocks
 constexpr float LSE_BIG = 1099511627776.f;       // 2^40: a partial sum beyond it moves the reference
@@ -111,6 +114,8 @@ struct LseBarriers {
   uint64_t drained[2];
   uint32_t tmem_base;
   int abort_flag;
+  int prod_done;               // the producer has issued its last key tile: the copy role takes no more items
+  int pad;
   float2 state[2][4][2][128];  // (reference, sum) per (group, row block, column half, row in block)
 };
 
@@ -219,6 +224,7 @@ score_tc_lse_kernel(const __grid_constant__ CUtensorMap kmap, const TcArgs ta) {
     mbar_init(smem_u32(&bars->drained[0]), 1);
     mbar_init(smem_u32(&bars->drained[1]), 1);
     bars->abort_flag = 0;
+    bars->prod_done = 0;
     fence_barrier_init();
   }
   if (warp == 1) {
@@ -245,6 +251,17 @@ score_tc_lse_kernel(const __grid_constant__ CUtensorMap kmap, const TcArgs ta) {
     // (one producer: this pass needs a K tile per four jobs, far below what one warp delivers)
     if (ta.k5) k_tile_producer<true, NH>(&kmap, a, bars, k_smem, S, r, h, layer, L, t_begin, n_tiles, lane, abort_flag, 0, 1, ta.wait_cycles, ta.stall_tile);
     else k_tile_producer<false, NH>(&kmap, a, bars, k_smem, S, r, h, layer, L, t_begin, n_tiles, lane, abort_flag, 0, 1, ta.wait_cycles, ta.stall_tile);
+    if (lane == 0) bars->prod_done = 1;
+  } else if (warp >= LSE_COPY_WARP0) {
+    // ---------------- copy role: items of the pending compaction of another layer group ----------------
+    // Order-free copies between pages this kernel neither reads nor writes (Section 7.2), on the HBM
+    // bandwidth this pass leaves idle.  Items are taken until the producer has issued the CTA's last key tile.
+    volatile int* done = &bars->prod_done;
+    cj_copy_role<NH + 2, 16>(ta.copy_ws, lane, [&]() {
+      int go = 0;
+      if (lane == 0) go = (!*done && !*abort_flag) ? 1 : 0;
+      return __shfl_sync(0xffffffffu, go, 0) != 0;
+    });
   } else if (warp <= 2) {
     // ---------------- MMA issuers: A = Q block in TMEM, B = K tile in shared memory ----------------
     // Two warps, one per accumulator: warp 1 issues the even jobs into accumulator 0, warp 2 the odd jobs
@@ -350,7 +367,7 @@ score_tc_lse_kernel(const __grid_constant__ CUtensorMap kmap, const TcArgs ta) {
   // ---------------- teardown ----------------
   tc_fence_before();
   __syncthreads();
-  if (warp >= 3 && k == 0 && !*abort_flag) {
+  if (warp >= 3 && warp < LSE_COPY_WARP0 && k == 0 && !*abort_flag) {
     // merge the four shares (group, column half) of each row, store (reference in log2 units, sum); (-inf, 0) when the
     // row saw no key of this chunk
     const float c = a.scale_log2;

@@ -13,9 +13,18 @@
 namespace actkv {
 namespace tc {
 
+// Warps: 0 producer, 1-2 MMA issuers, 3 second producer (the control warpgroup); 4-11 epilogue (two
+// warpgroups); 12-15 copy role (items of a pending compaction, when the launch carries one).
+// Registers: the kernel starts with 128 per thread (512 threads); the control warpgroup drops to 64 and the copy
+// warpgroup to 112, the two epilogue warpgroups rise to 168: 128 x (64 + 2 x 168 + 112) = 65536.
 constexpr int POOL_EPI_WARPS = 8;
-constexpr int POOL_THREADS = (4 + POOL_EPI_WARPS) * 32;     // producer, two MMA issuers, epilogue, second producer
-constexpr int POOL_PRODUCER2 = 3 + POOL_EPI_WARPS;          // warp index of the second producer
+constexpr int POOL_EPI_WARP0 = 4;                           // first epilogue warp
+constexpr int POOL_COPY_WARP0 = POOL_EPI_WARP0 + POOL_EPI_WARPS;
+constexpr int POOL_THREADS = (POOL_COPY_WARP0 + 4) * 32;
+constexpr int POOL_PRODUCER2 = 3;                           // warp index of the second producer
+constexpr uint32_t POOL_REGS_CTRL = 64, POOL_REGS_EPI = 168, POOL_REGS_COPY = 112;
+constexpr int POOL_REGS_ENTRY = 128;                        // what the launch must have allocated per thread
+static_assert(128 * (POOL_REGS_CTRL + 2 * POOL_REGS_EPI + POOL_REGS_COPY) <= POOL_THREADS * POOL_REGS_ENTRY, "register budget");
 
 struct PoolBarriers {
   uint64_t k_full[8];
@@ -28,6 +37,7 @@ struct PoolBarriers {
   uint64_t drained[2];
   uint32_t tmem_base;
   int abort_flag;
+  int prod_done;              // the first producer has issued its last key tile: the copy role takes no more items
   float exch[TK];
 };
 
@@ -138,6 +148,7 @@ score_tc_pool_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_cons
     mbar_init(smem_u32(&bars->drained[0]), 1);
     mbar_init(smem_u32(&bars->drained[1]), 1);
     bars->abort_flag = 0;
+    bars->prod_done = 0;
     fence_barrier_init();
   }
   {
@@ -156,6 +167,21 @@ score_tc_pool_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_cons
   tc_fence_after();
   const uint32_t tmem_base = bars->tmem_base;
 
+  if (warp >= POOL_COPY_WARP0) {
+    // ---------------- copy role: items of the pending compaction of another layer group ----------------
+    // Order-free copies between pages this kernel neither reads nor writes (Section 7.2); they use the HBM
+    // bandwidth the contraction leaves idle.  Items are taken until the producer has issued the CTA's last
+    // key tile: the last item then ends about when the last tiles have been scored, and the CTA retires with
+    // its main work.
+    reg_dec<POOL_REGS_COPY>();
+    volatile int* done = &bars->prod_done;
+    cj_copy_role<NH + 2, 16>(ta.copy_ws, lane, [&]() {
+      int go = 0;
+      if (lane == 0) go = (!*done && !*abort_flag) ? 1 : 0;
+      return __shfl_sync(0xffffffffu, go, 0) != 0;
+    });
+  } else if (warp < POOL_EPI_WARP0) {
+    reg_dec<POOL_REGS_CTRL>();
   if (warp == 0) {
     // ---------------- TMA producer ----------------
     const int layer = a.layer_begin + slab;
@@ -169,11 +195,12 @@ score_tc_pool_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_cons
     }
     if (ta.k5) k_tile_producer<true, NH>(&kmap, a, bars, k_smem, S, r, h, layer, L, t_begin, n_tiles, lane, abort_flag, 0, 2, ta.wait_cycles, ta.stall_tile);
     else k_tile_producer<false, NH>(&kmap, a, bars, k_smem, S, r, h, layer, L, t_begin, n_tiles, lane, abort_flag, 0, 2, ta.wait_cycles, ta.stall_tile);
+    if (lane == 0) bars->prod_done = 1;
   } else if (warp == POOL_PRODUCER2) {
     const int layer = a.layer_begin + slab;
     if (ta.k5) k_tile_producer<true, NH>(&kmap, a, bars, k_smem, S, r, h, layer, L, t_begin, n_tiles, lane, abort_flag, 1, 2, ta.wait_cycles, ta.stall_tile);
     else k_tile_producer<false, NH>(&kmap, a, bars, k_smem, S, r, h, layer, L, t_begin, n_tiles, lane, abort_flag, 1, 2, ta.wait_cycles, ta.stall_tile);
-  } else if (warp <= 2) {
+  } else {
     // ---------------- MMA issuers: D[key, row] = K Q^T ----------------
     // Two warps, one per accumulator: warp 1 issues the even jobs, warp 2 the odd ones.  Issuing costs the
     // issuing thread about 50 cycles per tcgen05.mma and 80 per tcgen05.commit, and the barrier
@@ -228,8 +255,10 @@ score_tc_pool_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_cons
     // (a tear-down wait: it does not end early because another role gave up)
     mbar_wait_warp(smem_u32(&bars->drained[mw]), 0, nullptr, ok ? ta.wait_cycles : DRAIN_LIMIT_CYCLES);
     __syncwarp();
+  }
   } else {
     // ---------------- epilogue: one key per thread ----------------
+    reg_inc<POOL_REGS_EPI>();
     // The two warpgroups take alternate jobs whole, so they are one job apart and one folds while the other
     // waits for tensor memory (with both on every job, half the columns each, they ran in lockstep and the
     // sub-partitions idled through every wait: 5.25 against 5.0 ms at the bench shape, 0.57 against 0.50
@@ -238,7 +267,7 @@ score_tc_pool_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_cons
     // registers.  With two row chunks per key tile a warpgroup always gets the same chunk; warpgroup 1
     // hands its sum of a tile to warpgroup 0 through shared memory, which picks it up one job later, so
     // neither waits for the other.
-    const int wg = (warp - 3) >> 2;
+    const int wg = (warp - POOL_EPI_WARP0) >> 2;
     const int quarter = warp & 3;                 // TMEM lane quarter this warp may read
     const float c = a.scale_log2;
     const float inv_w = 1.0f / (float)W;

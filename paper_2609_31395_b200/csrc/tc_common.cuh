@@ -3,6 +3,7 @@
 
 #include <cuda.h>
 
+#include "compact_job.cuh"
 #include "score_fma.cuh"
 
 namespace actkv {
@@ -207,6 +208,13 @@ __device__ __forceinline__ void umma_bf16_ts(uint32_t d_tmem, uint32_t a_tmem, u
       ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
 }
 
+// Register budget of a warpgroup (four consecutive warps, all of whose threads execute the instruction): the
+// control and copy warpgroups hand registers back, the epilogue warpgroups take them.
+template <uint32_t N>
+__device__ __forceinline__ void reg_dec() { asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(N)); }
+template <uint32_t N>
+__device__ __forceinline__ void reg_inc() { asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(N)); }
+
 // sm_100 arithmetic the epilogues lean on: packed two-lane fp32 FMA / add, three-input max.
 __device__ __forceinline__ void ffma2(float& x0, float& x1, float a0, float a1, float b, float c0, float c1) {
   uint64_t ra, rb, rc, rd;                      // (x0, x1) = (a0, a1) * b + (c0, c1)
@@ -280,6 +288,8 @@ struct TcArgs {
   int32_t row_begin;         // pooled-score pass: first row of this launch's row group (multiple of MAX_ROWS)
   int32_t n_stages;          // K stages in shared memory
   int32_t k5;                // K tensor map has five dimensions (pages that are not slot-major), else four
+  CompactWs* copy_ws;        // pending compaction of another layer group whose copies this launch's spare warps
+                             // take on (nullptr: none)
   int32_t stall_tile;        // fault-injection hook: the K-tile producers issue no tile from this one on (< 0: off)
   long long wait_cycles;     // limit of every bounded wait, in SM cycles
 };

@@ -58,7 +58,10 @@ class Compressor:
         self.ws_score = _ws(B.actkv_score_workspace_bytes(self.pd, s.n_req, self.lpc, n_q_heads, s.sum_win, s.max_win,
                                                           s.max_tok), self.dev)
         self.ws_select = _ws(B.actkv_select_workspace_bytes(self.lpc * Hkv, s.n_req, s.max_tok), self.dev)
-        self.ws_compact = _ws(B.actkv_compact_workspace_bytes(s.n_req, self.td.max_pages), self.dev)
+        # (sized for the pipelined step as well: room for the resolved sources of one layer group)
+        self.ws_compact = _ws(max(B.actkv_compact_workspace_bytes(s.n_req, self.td.max_pages),
+                                  B.actkv_compact_deferred_workspace_bytes(self.pd, s.n_req, self.td.max_pages, self.lpc,
+                                                                           s.max_keep)), self.dev)
 
     # -- single stages (whole layer range unless given) ------------------------------------------
     def run_score(self, q, win_indptr, tok_indptr, sm_scale, causal, l0=0, l1=None, lse_in=None, stream=None):
@@ -158,6 +161,50 @@ class Compressor:
             launches += (3 if lse_in is None else 1) + 1 + (1 if inplace else 2) + (1 if l1 == NL else 0)
             launches += 2 if lrfu is not None else 0
         return launches
+
+    def step_pipelined(self, q, win_indptr, tok_indptr, budget, sm_scale, causal, lse_in=None, stream=None, marks=None,
+                       groups=None, stats=None):
+        """score -> select -> compact over all layers with the copies of layer group g running inside the
+        score kernels of group g+1 (actkv_compact_begin / actkv_score_overlap / actkv_compact_end), all on one
+        stream.  `groups`: list of (l0, l1) layer ranges, each at most `layers_per_call` long (default: equal
+        groups of `layers_per_call`); the copies of the last group are not hidden, so a short last group
+        exposes less.  Results are those of step().  Returns the number of kernels launched."""
+        NL, Hkv, s = self.pd.n_layers, self.pd.n_kv_heads, self.sz
+        if groups is None:
+            groups = [(l0, min(NL, l0 + self.lpc)) for l0 in range(0, NL, self.lpc)]
+        assert groups[0][0] == 0 and groups[-1][1] == NL and all(a[1] == b[0] for a, b in zip(groups, groups[1:]))
+        assert all(0 < l1 - l0 <= self.lpc for l0, l1 in groups)
+        mark = marks if marks is not None else (lambda name: None)
+        B.actkv_keep_indptr(self.seq_len, budget, s.n_req, self.keep_indptr, stream)
+        launches = 1
+        prev = None
+        done = []               # groups whose statistics have been written to `stats` ([n_groups, 2] int32, optional)
+        for l0, l1 in groups:
+            mark("begin")
+            lse_g = None if lse_in is None else lse_in[l0:l1]
+            lse_out = None if self.lse is None else self.lse[l0:l1]
+            B.actkv_score_overlap(self.pd, self.td, l0, l1, q[l0:l1], win_indptr, self.n_q_heads, lse_g, sm_scale, causal,
+                                  tok_indptr, self.score[: l1 - l0], lse_out, s.sum_win, s.max_win, s.sum_tok, s.max_tok,
+                                  self.ws_score, None if prev is None else self.ws_compact, self.status, stream)
+            mark("score")
+            if prev is not None:
+                if stats is not None:
+                    B.actkv_compact_stats(self.ws_compact, stats[len(done)], stream)
+                    done.append(prev)
+                B.actkv_compact_end(self.pd, self.td, prev[0], prev[1], self.sel_idx, s.sel_stride, self.keep_indptr,
+                                    budget, s.max_keep, self.ws_compact, self.status, stream)
+                mark("compact")
+            self.run_select(tok_indptr, budget, l1 - l0, stream)
+            mark("select")
+            B.actkv_compact_begin(self.pd, self.td, l0, l1, self.sel_idx, s.sel_stride, self.keep_indptr, budget,
+                                  s.max_keep, self.ws_compact, self.status, stream, reuse_plan=prev is not None)
+            prev = (l0, l1)
+            launches += (3 if lse_in is None else 1) + 1 + 1 + 1
+        mark("begin")
+        B.actkv_compact_end(self.pd, self.td, prev[0], prev[1], self.sel_idx, s.sel_stride, self.keep_indptr, budget,
+                            s.max_keep, self.ws_compact, self.status, stream)
+        mark("compact")
+        return launches + 2
 
     def step_overlapped(self, q, win_indptr, tok_indptr, budget, sm_scale, causal, lse_in=None, marks=None):
         """The same step with select + compact of layer group g running on a second stream while

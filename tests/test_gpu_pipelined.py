@@ -1,0 +1,114 @@
+"""The compaction of a layer group hidden under the score kernels of the next group
+(actkv_compact_begin / actkv_score_overlap / actkv_compact_end): the copies are taken from a work
+queue by spare warps of the tensor-core score kernels and by a drain kernel.  Whoever executes an
+item, the result must be exactly what actkv_compact gives, which the other tests hold against the
+oracle; here the one-call step is checked against the oracle first and the pipelined step against
+it bit for bit.
+"""
+import numpy as np
+import pytest
+import torch
+
+from paper_2609_31395_b200 import binding as B
+from paper_2609_31395_b200 import harness as H
+from paper_2609_31395_b200 import synth
+
+import parity_util as U
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+
+def _same_state(a, b):
+    assert torch.equal(a.pool.view(torch.int16), b.pool.view(torch.int16))
+    assert torch.equal(a.page_table, b.page_table) and torch.equal(a.seq_len, b.seq_len)
+    assert torch.equal(a.free_list, b.free_list) and torch.equal(a.free_count, b.free_count)
+
+
+def _reference(wl):
+    """One-call step, checked against the oracle (scores, index lists, every byte of the pool, tables)."""
+    a = synth.generate(wl, DEV)
+    pool_before, tables_before = U.bits(a.pool), U.oracle_tables(a)
+    comp = U.run_step(a)
+    comp.check_status()
+    want, lse, tok, err = U.check_scores(a, comp, pool_before, tables_before)
+    sel, ki = comp.sel_idx.cpu().numpy(), comp.keep_indptr.cpu().numpy()
+    U.check_select_exact(comp.score.cpu().numpy().reshape(-1, want.shape[-1]), tok, wl.budgets, sel, ki)
+    U.check_compaction(a, pool_before, tables_before, sel, ki, wl.budgets)
+    return a, comp
+
+
+def _pipelined(wl, lpc, groups=None, lse_in=None):
+    b = synth.generate(wl, DEV)
+    comp = H.Compressor(b.pool, b.page_table, b.seq_len, b.free_list, b.free_count, wl.n_q_heads, H.sizes_of(b),
+                        layers_per_call=lpc, want_lse=True)
+    comp.step_pipelined(b.q, b.win_indptr, b.tok_indptr, b.budget, wl.sm_scale, wl.causal, lse_in=lse_in, groups=groups)
+    torch.cuda.synchronize()
+    comp.check_status()
+    return b, comp
+
+
+@pytest.mark.parametrize("causal", [False, True])
+def test_pipelined_step_equals_the_one_call_step(causal):
+    # 7 layers in groups of 2, 2, 2, 1; 256 window rows (tensor-core path), ragged last pages, one request that
+    # keeps everything (B >= L) and one that is emptied (B = 0)
+    wl = synth.Workload("pipe", 7, 2, 8, [1500, 333, 700, 90, 260], [32, 16, 24, 8, 32], [400, 100, 200, 90, 0],
+                        table_style="fragmented", causal=causal, seed=51, poison_tail=True)
+    a, comp_a = _reference(wl)
+    b, comp_b = _pipelined(wl, 2)
+    _same_state(a, b)
+    # (the LSE pass cuts the keys into chunks by the size of the launch, so its last bits depend on the grouping)
+    assert torch.allclose(comp_a.lse, comp_b.lse, rtol=0, atol=1e-5)
+    # with the LSE supplied (no LSE kernel: all copies ride on the pooled-score kernel or the drain)
+    c, _ = _pipelined(wl, 2, lse_in=comp_a.lse)
+    _same_state(a, c)
+
+
+def test_uneven_groups_and_other_shapes():
+    # head_dim 64 (8 vectors per row), 4 heads x pages of 32 tokens = 128 (slot, head) pairs per page
+    wl = synth.Workload("pipe64", 5, 4, 4, [1100, 257, 64], [32, 16, 16], [300, 64, 10], head_dim=64, page_size=32,
+                        table_style="permutation", seed=52, poison_tail=True)
+    a, _ = _reference(wl)
+    b, _ = _pipelined(wl, 3, groups=[(0, 3), (3, 4), (4, 5)])
+    _same_state(a, b)
+    # a window below 64 rows: the FMA score kernels, which carry no copy role: the drain kernel copies everything
+    wl2 = synth.Workload("pipefma", 4, 2, 2, [500, 130], [8, 4], [120, 40], table_style="fragmented", seed=53,
+                         poison_tail=True)
+    a2, _ = _reference(wl2)
+    b2, _ = _pipelined(wl2, 1)
+    _same_state(a2, b2)
+
+
+def test_begin_plus_end_is_compact_and_errors_leave_everything_untouched():
+    wl = synth.Workload("be", 2, 2, 4, [900, 333, 130], [16, 8, 16], [250, 100, 130], table_style="fragmented", seed=54,
+                        poison_tail=True)
+    a, comp_a = _reference(wl)
+    b = synth.generate(wl, DEV)
+    comp = H.Compressor(b.pool, b.page_table, b.seq_len, b.free_list, b.free_count, wl.n_q_heads, H.sizes_of(b))
+    B.actkv_keep_indptr(b.seq_len, b.budget, wl.n_req, comp.keep_indptr)
+    comp.run_score(b.q, b.win_indptr, b.tok_indptr, wl.sm_scale, wl.causal)
+    comp.run_select(b.tok_indptr, b.budget, wl.n_layers)
+    args = (comp.pd, comp.td, 0, wl.n_layers, comp.sel_idx, comp.sz.sel_stride, comp.keep_indptr, b.budget,
+            comp.sz.max_keep, comp.ws_compact, comp.status)
+    assert comp.ws_compact.numel() >= B.actkv_compact_deferred_workspace_bytes(comp.pd, wl.n_req, comp.td.max_pages,
+                                                                                wl.n_layers, comp.sz.max_keep)
+    # a free list that is too short: reported by the plan, nothing is copied by anyone, tables stay
+    snap = [U.bits(b.pool).copy()] + [t.clone() for t in (b.page_table, b.seq_len, b.free_list, b.free_count)]
+    fc = b.free_count.clone()
+    b.free_count.fill_(3)
+    snap[4] = b.free_count.clone()
+    B.actkv_compact_begin(*args)
+    B.actkv_compact_end(*args)
+    torch.cuda.synchronize()
+    assert comp.status.cpu().tolist()[0] == B.E_NOFREE
+    assert np.array_equal(U.bits(b.pool), snap[0])
+    for t, s0 in zip((b.page_table, b.seq_len, b.free_list, b.free_count), snap[1:]):
+        assert torch.equal(t, s0)
+    # the real thing
+    b.free_count.copy_(fc)
+    comp.status.zero_()
+    B.actkv_compact_begin(*args)
+    B.actkv_compact_end(*args)
+    torch.cuda.synchronize()
+    comp.check_status()
+    _same_state(a, b)
