@@ -161,46 +161,82 @@ def visible_gpu_index(local_rank: int) -> int:
 # the CPU oracle on a bounded sample (cpu_baseline and --impl reference)
 
 
-def oracle_sample(wl, n_heads_sample: int = 2):
-    """Draws a one-layer, one-request instance of `wl`'s shape on the CPU and returns a closure that
-    runs the oracle's budget + score + select + compact on it, plus the scaling to the metric."""
+_UNIT_CACHE = {}
+
+
+def _oracle_unit(task):
+    """Worker (one process per host core): the oracle's budget + score + select + compact on ONE unit of the
+    workload's shape, i.e. one request x one KV head x one layer, drawn on the CPU from the unit's own seed.
+    Returns the CPU seconds the call took.  The instance is built on the first call and kept."""
+    (name, group, L, W, Bud, head_dim, page, causal, n_topics, seed), timed = task
+    os.environ.setdefault("OMP_NUM_THREADS", "1")
     from oracle import actkv_oracle as O
-    small = synth.Workload(wl.name + "_sample", 1, n_heads_sample, wl.group, wl.seq_lens[:1], wl.windows[:1],
-                           wl.budgets[:1], head_dim=wl.head_dim, page_size=wl.page_size, causal=wl.causal,
-                           table_style="permutation", n_topics=wl.n_topics, seed=wl.seed)
-    inst = synth.generate(small, "cpu")
-    bits = lambda t: t.contiguous().view(torch.int16).numpy().view(np.uint16)
-    pool_b, q_b = bits(inst.pool), bits(inst.q)
+    key = (name, seed)
+    if key not in _UNIT_CACHE:
+        torch.set_num_threads(1)
+        small = synth.Workload(name + "_sample", 1, 1, group, [L], [W], [Bud], head_dim=head_dim, page_size=page,
+                               causal=causal, table_style="permutation", n_topics=n_topics, seed=seed)
+        inst = synth.generate(small, "cpu")
+        bits = lambda t: t.contiguous().view(torch.int16).numpy().view(np.uint16)
+        logits, tind = synth.confidence_logits(1, LOGIT_ROWS, VOCAB, seed=seed, device="cpu")
+        _UNIT_CACHE[key] = (small, inst, bits(inst.pool), bits(inst.q), logits.numpy(), tind.numpy())
+    small, inst, pool_b, q_b, logits_np, tind = _UNIT_CACHE[key]
+    if not timed:
+        return 0.0
+    c0 = time.process_time()
     pt, sl = inst.page_table.numpy(), inst.seq_len.numpy()
-    logits, tind = synth.confidence_logits(1, LOGIT_ROWS, VOCAB, seed=wl.seed, device="cpu")
-    logits_np = logits.numpy()
     bp = O.BudgetParams(clamp_lo_ppm=BUDGET_PPM, clamp_hi_ppm=BUDGET_PPM)
-
-    def run():
-        hist = np.zeros((1, 4096), dtype=np.float32)
-        _, _, bud, _, _ = O.budget(logits_np, tind.numpy(), hist, [0], small.budgets, bp, sl)
-        sc, _, tok = O.score(pool_b, pt, sl, q_b, inst.win_indptr.numpy(), small.n_q_heads, small.sm_scale,
-                             small.causal)
-        sel = [[[O.select_unit(sc[0, h], int(bud[0]))] for h in range(n_heads_sample)]]
-        tables = O.Tables(pt.copy(), sl.copy(), inst.free_list.numpy().copy(), int(inst.free_count))
-        O.compact(pool_b, tables, sel, bud)
-
-    # the sample covers 1 request x n_heads_sample heads x 1 layer of the (R x Hkv x NL) workload
-    frac = (1.0 / wl.n_req) * (n_heads_sample / wl.n_kv_heads) * (1.0 / wl.n_layers)
-    tokens_equiv = sum(wl.seq_lens) * frac
-    desc = (f"1 request x {n_heads_sample} of {wl.n_kv_heads} KV heads x 1 of {wl.n_layers} layers "
-            f"({wl.seq_lens[0]} tokens, window {wl.windows[0]}, budget {wl.budgets[0]}) + {LOGIT_ROWS} logit rows; "
-            f"tokens/s scaled by the unit count")
-    return run, tokens_equiv, desc
+    hist = np.zeros((1, 4096), dtype=np.float32)
+    _, _, bud, _, _ = O.budget(logits_np, tind, hist, [0], small.budgets, bp, sl)
+    sc, _, tok = O.score(pool_b, pt, sl, q_b, inst.win_indptr.numpy(), small.n_q_heads, small.sm_scale, small.causal)
+    sel = [[[O.select_unit(sc[0, 0], int(bud[0]))]]]
+    tables = O.Tables(pt.copy(), sl.copy(), inst.free_list.numpy().copy(), int(inst.free_count))
+    O.compact(pool_b, tables, sel, bud)
+    return time.process_time() - c0
 
 
-def timed_cpu(fn, reps: int = 1):
-    """Runs fn `reps` times; returns (seconds per run, threads actually busy = CPU time / wall time)."""
-    w0, c0 = time.perf_counter(), time.process_time()
-    for _ in range(reps):
-        fn()
-    w, c = time.perf_counter() - w0, time.process_time() - c0
-    return w / reps, max(1, int(round(c / max(w, 1e-9))))
+class OracleSample:
+    """The oracle, as it stands, on a bounded sample of the workload spread over ALL host cores: one unit
+    (request x KV head x layer) per core and step, each in its own process.  Used by the cpu_baseline leg and by
+    --impl reference alike (the same sample)."""
+
+    def __init__(self, wl):
+        import multiprocessing as mp
+        self.wl = wl
+        self.cores = os.cpu_count() or 1
+        n_units_all = wl.n_req * wl.n_kv_heads * wl.n_layers
+        # (at most one layer's worth of units, and at most 32 worker processes: each holds its own interpreter)
+        self.n_units = max(1, min(self.cores, n_units_all, wl.n_req * wl.n_kv_heads, 32))
+        # unit u: request u % R (its length, window and budget), a seed of its own
+        R = wl.n_req
+        self.tasks = [(wl.name, wl.group, wl.seq_lens[u % R], wl.windows[u % R], wl.budgets[u % R], wl.head_dim,
+                       wl.page_size, wl.causal, wl.n_topics, wl.seed * 1000 + u) for u in range(self.n_units)]
+        self.pool = mp.get_context("spawn").Pool(self.n_units)
+        self.pool.map(_oracle_unit, [(t, False) for t in self.tasks], chunksize=1)      # build the instances (untimed)
+        tok_units = sum(wl.seq_lens[u % R] for u in range(self.n_units))
+        # a unit covers 1 / (KV heads x layers) of its request's tokens
+        self.tokens_equiv = tok_units / (wl.n_kv_heads * wl.n_layers)
+        self.desc = (f"{self.n_units} units (request x KV head x layer) of {n_units_all}, one per host core, each "
+                     f"{wl.seq_lens[0]} tokens, window {wl.windows[0]}, budget {wl.budgets[0]}, + {LOGIT_ROWS} logit rows "
+                     f"per unit's request; tokens/s scaled by the unit count")
+
+    def step(self):
+        """One step: every worker runs its unit once.  Returns (wall seconds, CPU seconds summed over workers)."""
+        w0 = time.perf_counter()
+        cpu = self.pool.map(_oracle_unit, [(t, True) for t in self.tasks], chunksize=1)
+        return time.perf_counter() - w0, float(sum(cpu))
+
+    def timed(self, steps):
+        wall = cpu = 0.0
+        for _ in range(steps):
+            w, c = self.step()
+            wall += w
+            cpu += c
+        return wall / steps, max(1, int(round(cpu / max(wall, 1e-9))))
+
+    def close(self):
+        self.pool.close()
+        self.pool.join()
 
 
 def run_reference(args):
@@ -208,17 +244,19 @@ def run_reference(args):
     if rank != 0:
         return
     wl = make_workload(args.workload, args.layers)
-    run, tokens_equiv, desc = oracle_sample(wl)
-    for _ in range(args.warmup):
-        run()
-    dt, cores = timed_cpu(run, args.steps)
-    v = tokens_equiv / dt
+    smp = OracleSample(wl)
+    for _ in range(min(args.warmup, 1)):
+        smp.step()
+    dt, cores = smp.timed(args.steps)
+    smp.close()
+    v = smp.tokens_equiv / dt
     print(json.dumps({
         "impl": "reference", "metric": METRIC, "value": v, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": wl.name, "note": "CPU oracle on a bounded sample per step: " + desc},
-        "cpu_baseline": {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": desc},
+        "config": {"workload": wl.name, "note": "CPU oracle on a bounded sample per step: " + smp.desc},
+        "cpu_baseline": {"value": v, "unit": UNIT, "cores": cores, "host_cores": smp.cores, "kind": "oracle",
+                         "sample": smp.desc},
         "e2e": {"value": v, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0}))
 
@@ -261,7 +299,7 @@ def run_ours(args):
         pipe_groups = [(sum(sizes[:i]), sum(sizes[:i + 1])) for i in range(len(sizes))]
     comp = H.Compressor(inst.pool, inst.page_table, inst.seq_len, inst.free_list, inst.free_count, wl.n_q_heads, sz,
                         layers_per_call=args.layers_per_call if args.layers_per_call else (8 if args.overlap else None),
-                        want_lse=True)
+                        want_lse=True, want_ties=True)
     # budget inputs: LOGIT_ROWS action-token logit rows per request
     logits, ltok = synth.confidence_logits(R, LOGIT_ROWS, VOCAB, seed=wl.seed, device=dev)
     n_rows = logits.shape[0]
@@ -285,9 +323,16 @@ def run_ours(args):
         comp.status.zero_()
 
     lse_supplied = None
-    pipelined = False                          # set for the secondary pipelined-compaction lines only
+    # The timed step hides the compaction of a layer group under the score kernels of the next group
+    # (actkv_compact_begin / actkv_score_overlap / actkv_compact_end) unless --pipeline none; the other form
+    # (one score, one select and one compact call over all layers) is timed as a secondary line.
+    pipelined = pipe_groups is not None and not args.overlap
     pipe_stats = torch.zeros((len(pipe_groups) if pipe_groups else 1, 2), dtype=torch.int32, device=dev)
     pipe_comp = None
+    if pipelined:
+        pipe_comp = H.Compressor(inst.pool, inst.page_table, inst.seq_len, inst.free_list, inst.free_count, wl.n_q_heads,
+                                 sz, layers_per_call=max(l1 - l0 for l0, l1 in pipe_groups), want_lse=False, want_ties=True)
+        pipe_comp.lse, pipe_comp.status = comp.lse, comp.status
     lrfu_state = None                          # set for the secondary LRFU-policy line only
     inplace_mode = False                       # set for the secondary in-place-compaction line only
     stage_names = ["budget", "lse", "score", "select", "compact"]
@@ -309,7 +354,7 @@ def run_ours(args):
         if args.overlap:
             n = comp.step_overlapped(inst.q, inst.win_indptr, inst.tok_indptr, bud, wl.sm_scale, wl.causal,
                                      lse_in=lse_supplied, marks=mark)
-        elif pipelined:
+        elif pipelined and lrfu_state is None and not inplace_mode:
             n = pipe_comp.step_pipelined(inst.q, inst.win_indptr, inst.tok_indptr, bud, wl.sm_scale, wl.causal,
                                          lse_in=lse_supplied, marks=(lambda nm: mark(nm)), groups=pipe_groups,
                                          stats=pipe_stats)
@@ -346,6 +391,11 @@ def run_ours(args):
     clocks = sampler.stop()
     comp.check_status()
 
+    # ties at the k-th threshold, as actkv_select reported them for the units of the last call of the timed step
+    tie_t = (pipe_comp if pipelined else comp).ties.cpu()
+    n_eq_total, n_eq_kept = tie_t[:, 2], tie_t[:, 1]
+    ties_line = {"units_reported": int(tie_t.shape[0]), "units_with_a_tie_at_the_threshold": int((n_eq_total > n_eq_kept).sum()),
+                 "entries_equal_to_the_threshold": int(n_eq_total.sum()), "of_them_kept": int(n_eq_kept.sum())}
     stage_ms = {k: 0.0 for k in stage_names}
     total_ms = 0.0
     aux_names = ("begin_aux", "select", "compact") if args.overlap else ()
@@ -371,7 +421,7 @@ def run_ours(args):
     flops_pass = 2.0 * sum(W * G * L for W, L in zip(wl.windows, wl.seq_lens)) * D * Hkv * NL
     bytes_k = 2.0 * D * tokens * Hkv * NL
     alg_bytes = (264.0 + 1032.0 * rho) * tokens * Hkv * NL
-    n_calls = -(-NL // comp.lpc)
+    n_calls = len(pipe_groups) if pipelined else -(-NL // comp.lpc)
     stages = {
         "lse": {"bound": "tensor", "achieved": flops_pass / (stage_ms["lse"] * 1e-3) / 1e12 if stage_ms["lse"] else None,
                 "peak": pk["tf_sustained"], "unit": "TFLOP/s"},
@@ -382,17 +432,32 @@ def run_ours(args):
         "budget": {"bound": "hbm", "achieved": 4.0 * n_rows * VOCAB / (stage_ms["budget"] * 1e-3) / 1e9,
                    "peak": pk["hbm_gbs"], "unit": "GB/s"},
     }
+    if pipelined:
+        # the copies run inside the pooled-score kernels; "compact" times only what was left for the drain kernel
+        stages["compact"].update({"achieved": None, "note": "hidden under the pooled-score kernels of the next layer group; "
+                                                             "stage_ms.compact is the part that was not"})
+        stages["score"]["note"] = "with the copies of the previous layer group inside"
     for s in stages.values():
         s["frac"] = None if s["achieved"] is None else s["achieved"] / s["peak"]
     dom = max(("lse", "score", "compact"), key=lambda k: stage_ms[k])
     roofline = dict(stages[dom])
-    # DRAM bytes per (token, KV head, layer) measured with ncu on the 2-layer cut of this workload
-    # (profiles/kernels_c3_2layers_full_set.md: dram__bytes_read.sum + dram__bytes_write.sum over
-    # 280000 tokens x 4 heads x 2 layers), scaled to one launch of this run by its unit count
-    ncu_bytes_per_unit = {"lse": 588.1e6 / 2.24e6, "score": 595.3e6 / 2.24e6, "compact": 551.6e6 / 2.24e6}
-    traffic = ncu_bytes_per_unit[dom] * tokens * Hkv * NL / n_calls if args.workload == "c3" else None
-    roofline.update({"kernel": dom, "launches_per_step": n_calls, "ms_per_launch": stage_ms[dom] / n_calls,
-                     "traffic": traffic, "traffic_unit": "bytes per launch (ncu, scaled from the 2-layer capture)", "peak_source": pk["source"] + (" sustained bf16" if stages[dom]["bound"] == "tensor" else " copy")})
+    # DRAM bytes per (token, KV head, layer) of each kernel, measured with ncu on a small cut of the workload and kept
+    # in a data file beside the capture's summary; scaled to one launch of this run by its unit count (traffic grows
+    # in proportion to the units processed).  null when the file has no entry for the kernel this run launched.
+    traffic, traffic_src = None, None
+    kernel_of = {"lse": "score_tc_lse_kernel", "score": "score_tc_pool_kernel", "compact": "compact_copy_kernel"}
+    tpath = os.path.join(ROOT, "profiles", f"traffic_{args.workload}.json")
+    if os.path.exists(tpath):
+        tj = json.load(open(tpath))
+        ent = tj.get("kernels", {}).get(kernel_of[dom])
+        if ent is not None and tj.get("library_version") == B.actkv_version():
+            traffic = ent["dram_bytes_per_unit"] * tokens * Hkv * NL / n_calls
+            traffic_src = tj.get("capture")
+    roofline.update({"kernel": dom, "kernel_name": kernel_of[dom], "launches_per_step": n_calls,
+                     "ms_per_launch": stage_ms[dom] / n_calls,
+                     "traffic": traffic, "traffic_unit": "bytes per launch (ncu dram__bytes_read.sum + dram__bytes_write.sum of a "
+                                                         "small capture, scaled by the units processed)",
+                     "traffic_capture": traffic_src, "peak_source": pk["source"] + (" sustained bf16" if stages[dom]["bound"] == "tensor" else " copy")})
     hbm_frac_whole = alg_bytes / (ms_max * 1e-3) / 1e9 / pk["hbm_gbs"]
     # The LSE pass evaluates one exp2 per (window row, key): besides the contraction it is bound by the
     # special function units, 16 results per clock per SM on 148 SMs at the maximum SM clock.
@@ -410,7 +475,7 @@ def run_ours(args):
         # restore the device tables first: the runner snapshots them as the host-side state of the engine
         restore()
         torch.cuda.synchronize()
-        runner = H.HostStepRunner(comp, inst.q, inst.win_indptr, inst.tok_indptr, budget_in, wl.sm_scale, wl.causal,
+        runner = H.HostStepRunner(pipe_comp if pipelined else comp, inst.q, inst.win_indptr, inst.tok_indptr, budget_in, wl.sm_scale, wl.causal,
                                   logits=logits, logit_indptr=ltok, hist_cap=hist_cap, params=bparams)
         h2d, d2h = runner.h2d_bytes, runner.d2h_bytes
         e2e_ms = []
@@ -457,41 +522,34 @@ def run_ours(args):
                                  alg_bytes / (float(tl.item()) * 1e-3) / 1e9 / pk["hbm_gbs"]}
         comp.check_status()
 
-    # ---- the same step with the compaction of a layer group hidden under the score kernels of the next group
-    # (actkv_compact_begin / actkv_score_overlap / actkv_compact_end), both LSE modes
-    pipelined_line = None
+    # ---- the other form of the step (one score / select / compact call over all layers when the timed step is the
+    # pipelined one, and the other way round), both LSE modes
+    other_line = None
     if pipe_groups is not None and not args.overlap:
-        lpc_p = max(l1 - l0 for l0, l1 in pipe_groups)
-        pipe_comp = H.Compressor(inst.pool, inst.page_table, inst.seq_len, inst.free_list, inst.free_count, wl.n_q_heads, sz,
-                                 layers_per_call=lpc_p, want_lse=False)
-        pipelined = True
-        pipelined_line = {"groups": [l1 - l0 for l0, l1 in pipe_groups]}
+        was = pipelined
+        pipelined = not was
+        other_line = {"form": "one call per stage over all layers" if was else "pipelined",
+                      "groups": None if was else [l1 - l0 for l0, l1 in pipe_groups]}
         for mode in ("internal", "supplied"):
             lse_supplied = comp.lse.clone() if mode == "supplied" else None
-            ms, sc_ms, cp_ms = [], [], []
+            ms = []
             for it in range(2 + min(args.steps, 5)):
                 restore()
-                pipe_comp.status.zero_()
-                ev = []
-                one_step(ev)
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record()
+                one_step()
+                e1.record()
                 torch.cuda.synchronize()
                 if it >= 2:
-                    ms.append(ev[0][1].elapsed_time(ev[-1][1]))
-                    sc_ms.append(sum(ev[i - 1][1].elapsed_time(ev[i][1]) for i in range(1, len(ev)) if ev[i][0] == "score"))
-                    cp_ms.append(sum(ev[i - 1][1].elapsed_time(ev[i][1]) for i in range(1, len(ev)) if ev[i][0] == "compact"))
-            pipe_comp.check_status()
+                    ms.append(e0.elapsed_time(e1))
+            comp.check_status()
             tl = torch.tensor([sum(ms) / len(ms)], dtype=torch.float64, device=dev)
             if dist is not None:
                 dist.all_reduce(tl, op=dist.ReduceOp.MAX)
-            st = pipe_stats.cpu().tolist()
-            pipelined_line[mode] = {
-                "ms_per_step": float(tl.item()), "value": world * tokens / (float(tl.item()) * 1e-3), "unit": UNIT,
-                "hbm_roofline_frac_whole_step": alg_bytes / (float(tl.item()) * 1e-3) / 1e9 / pk["hbm_gbs"],
-                "score_ms_with_copies_inside": sum(sc_ms) / len(sc_ms), "exposed_compact_ms": sum(cp_ms) / len(cp_ms),
-                "copy_items_taken_by_score_kernels": [round(b / a, 3) if a else None for a, b in st]}
+            other_line[mode] = {"ms_per_step": float(tl.item()), "value": world * tokens / (float(tl.item()) * 1e-3), "unit": UNIT,
+                                "hbm_roofline_frac_whole_step": alg_bytes / (float(tl.item()) * 1e-3) / 1e9 / pk["hbm_gbs"]}
         lse_supplied = None
-        pipelined = False
-        del pipe_comp
+        pipelined = was
 
     # ---- the same step ranking by the attention-aware LRFU keep-score (Section 5.1): score -> keepscore
     # -> select -> gather keep-scores -> compact, p = 0.9, lambda = 0.5, 512 protected tokens per request
@@ -615,10 +673,12 @@ def run_ours(args):
     # ---- the oracle on the host cores (rank 0, single GPU only) ----------------------------------
     cpu_baseline = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        run, tokens_equiv, desc = oracle_sample(wl, n_heads_sample=wl.n_kv_heads)
-        dt, cores = timed_cpu(run, 2)
-        cpu_baseline = {"value": tokens_equiv / dt, "unit": UNIT, "cores": cores, "kind": "oracle",
-                        "sample": desc, "seconds": 2 * dt}
+        smp = OracleSample(make_workload(args.workload, args.layers))
+        n_rep = 3
+        dt, cores = smp.timed(n_rep)
+        smp.close()
+        cpu_baseline = {"value": smp.tokens_equiv / dt, "unit": UNIT, "cores": cores, "host_cores": smp.cores,
+                        "kind": "oracle", "sample": smp.desc, "seconds": n_rep * dt}
 
     if rank == 0:
         out = {
@@ -628,18 +688,24 @@ def run_ours(args):
             "config": {"workload": wl.name, "requests": R, "tokens_per_request": wl.seq_lens[0], "layers": NL,
                        "kv_heads": Hkv, "q_heads": wl.n_q_heads, "head_dim": D, "page": wl.page_size,
                        "window": wl.windows[0], "budget": wl.budgets[0], "lse": args.lse,
-                       "layers_per_call": comp.lpc, "replicas": world,
+                       "layers_per_call": pipe_comp.lpc if pipelined else comp.lpc, "replicas": world,
                        "overlap": "select+compact of a layer group on a second stream under the score kernels "
-                                  "of the next group" if args.overlap else "none (one stream)",
+                                  "of the next group" if args.overlap else
+                                  ("copies of a layer group inside the score kernels of the next one, groups of "
+                                   + "+".join(str(l1 - l0) for l0, l1 in pipe_groups) + " layers (one stream)"
+                                   if pipelined else "none (one stream)"),
                        "l2": "inputs (KV pool %.1f GB) far larger than the 126 MB L2" % (inst.pool.numel() * 2 / 1e9)},
             "stage_ms": stage_ms, "hbm_roofline_frac_whole_step": hbm_frac_whole,
-            "with_lse_supplied": lse_supplied_line, "with_pipelined_compaction": pipelined_line,
+            "with_lse_supplied": lse_supplied_line, "other_step_form": other_line,
+            "copy_items_taken_by_score_kernels": ([round(b / a, 3) if a else None for a, b in pipe_stats.cpu().tolist()]
+                                                  if pipelined else None),
             "with_lrfu_policy": lrfu_line,
             "with_inplace_compaction": inplace_line, "streaming_update": stream_line,
             "algorithmic_bytes_per_step": alg_bytes, "k_bytes_per_pass": bytes_k,
             "roofline": roofline, "roofline_stages": stages, "roofline_lse_exp_rate": lse_exp,
             "budget_4096_rows": budget_line,
             "cpu_baseline": cpu_baseline, "e2e": e2e,
+            "ties_at_threshold": ties_line,
             "clocks": clocks, "gpu_launches": launches, "wall_s_timed_region": t_wall,
         }
         print(json.dumps(out))
@@ -661,8 +727,8 @@ def main():
                     help="run select + compact of a layer group on a second stream under the score kernels of the "
                          "next group (measured: no gain, the score CTAs fill the register file of every SM)")
     ap.add_argument("--pipeline", default="auto",
-                    help="layer groups of the secondary pipelined-compaction lines: 'auto' (three equal groups), "
-                         "comma-separated group sizes, or 'none'")
+                    help="layer groups of the timed step, whose copies run inside the score kernels of the next group: "
+                         "'auto' (three equal groups), comma-separated group sizes, or 'none' (one call per stage)")
     ap.add_argument("--lse", default="internal", choices=["internal", "supplied"])
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")

@@ -395,7 +395,9 @@ int actkv_compact_inplace(const actkv_pool_t* pool /* host */, const actkv_table
  * Copies this step's queries, action-token logits, index arrays, budgets and tables from the host
  * (pinned memory recommended) into the caller's device staging buffers, runs actkv_score_lse per
  * group of layers, actkv_budget (when logits are given) -> actkv_keep_indptr, then per group:
- * actkv_score, actkv_select, actkv_compact, copies the new page table, seq_len, free list, free
+ * actkv_score_overlap, actkv_select, actkv_compact_begin / _end (the copies of a group run inside the
+ * score kernels of the next one when ws_compact has actkv_compact_deferred_workspace_bytes for
+ * layers_per_call layers), copies the new page table, seq_len, free list, free
  * count, budgets and the status words back to the host, and SYNCHRONISES the stream before
  * returning (the one entry point that does: its outputs are host memory).  The KV pool stays in
  * device memory — it is the cache being compressed.

@@ -144,13 +144,20 @@ static int step_enqueue(const actkv_pool_t* pool, const actkv_tables_t* tab, con
                               io->lse_dev + (size_t)l0 * io->sum_win * io->n_q_heads, io->sum_win, io->max_win,
                               io->sum_tok, io->max_tok, io->ws_score, io->ws_score_bytes, io->status_dev, stream));
   }
-  // ---- then the other passes; the budgets are first needed by the first select ----
+  // ---- then the other passes; the budgets are first needed by the first select.  With several layer groups the
+  // copies of group g run inside the pooled-score kernels of group g + 1 (actkv_compact_begin / actkv_score_overlap /
+  // actkv_compact_end); one index buffer suffices because the copies of g are closed before the select of g + 1. ----
+  int pl0 = -1, pl1 = -1;                      // the group whose compaction is pending
   for (int g = 0; g < n_groups; ++g) {
     const int l0 = g * lpc_post, l1 = l0 + lpc_post < NL ? l0 + lpc_post : NL;
-    ACTKV_TRY(actkv_score(pool, tab, l0, l1, (const char*)io->q_dev + (size_t)l0 * q_layer_bytes, io->win_indptr_dev,
-                          io->n_q_heads, io->lse_dev + (size_t)l0 * io->sum_win * io->n_q_heads, io->sm_scale, io->causal,
-                          io->tok_indptr_dev, io->score_dev, nullptr, io->sum_win, io->max_win, io->sum_tok,
-                          io->max_tok, io->ws_score, io->ws_score_bytes, io->status_dev, stream));
+    ACTKV_TRY(actkv_score_overlap(pool, tab, l0, l1, (const char*)io->q_dev + (size_t)l0 * q_layer_bytes, io->win_indptr_dev,
+                                  io->n_q_heads, io->lse_dev + (size_t)l0 * io->sum_win * io->n_q_heads, io->sm_scale,
+                                  io->causal, io->tok_indptr_dev, io->score_dev, nullptr, io->sum_win, io->max_win,
+                                  io->sum_tok, io->max_tok, io->ws_score, io->ws_score_bytes,
+                                  pl0 >= 0 ? io->ws_compact : nullptr, io->status_dev, stream));
+    if (pl0 >= 0)
+      ACTKV_TRY(actkv_compact_end(pool, tab, pl0, pl1, io->sel_idx_dev, io->sel_stride, io->keep_indptr_dev, io->budget_dev,
+                                  io->max_keep, io->ws_compact, io->ws_compact_bytes, io->status_dev, stream));
     if (g == 0) {
       if (with_budget) ACTKV_TRY(wait(s, st->budget));
       ACTKV_TRY(actkv_keep_indptr(tab->seq_len, io->budget_dev, R, io->keep_indptr_dev, stream));
@@ -158,9 +165,14 @@ static int step_enqueue(const actkv_pool_t* pool, const actkv_tables_t* tab, con
     ACTKV_TRY(actkv_select(io->score_dev, io->tok_indptr_dev, io->sum_tok, io->budget_dev, (l1 - l0) * Hkv, R,
                            io->keep_indptr_dev, io->sel_idx_dev, io->sel_stride, nullptr, nullptr, nullptr, 0,
                            io->status_dev, stream));
-    ACTKV_TRY(actkv_compact(pool, tab, l0, l1, io->sel_idx_dev, io->sel_stride, io->keep_indptr_dev, io->budget_dev,
-                            io->max_keep, io->ws_compact, io->ws_compact_bytes, io->status_dev, stream));
+    ACTKV_TRY(actkv_compact_begin(pool, tab, l0, l1, io->sel_idx_dev, io->sel_stride, io->keep_indptr_dev, io->budget_dev,
+                                  io->max_keep, g > 0 ? 1 : 0, io->ws_compact, io->ws_compact_bytes, io->status_dev, stream));
+    pl0 = l0;
+    pl1 = l1;
   }
+  if (pl0 >= 0)
+    ACTKV_TRY(actkv_compact_end(pool, tab, pl0, pl1, io->sel_idx_dev, io->sel_stride, io->keep_indptr_dev, io->budget_dev,
+                                io->max_keep, io->ws_compact, io->ws_compact_bytes, io->status_dev, stream));
 
   // ---- device -> host: the step's results ----
   ACTKV_TRY(d2h(io->page_table_out_host, tab->page_table, tbl_bytes, s));

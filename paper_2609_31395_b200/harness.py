@@ -183,6 +183,14 @@ class Compressor:
             mark("begin")
             lse_g = None if lse_in is None else lse_in[l0:l1]
             lse_out = None if self.lse is None else self.lse[l0:l1]
+            if marks is not None and lse_in is None:
+                # timed per kernel: the LSE pass as a call of its own (without a copy role), then the pooled-score
+                # pass with the copies inside
+                if self.lse is None:
+                    self.lse = torch.empty((NL, s.sum_win, self.n_q_heads), dtype=torch.float32, device=self.dev)
+                self.run_lse(q, win_indptr, tok_indptr, sm_scale, causal, l0, l1, self.lse[l0:l1], stream)
+                mark("lse")
+                lse_g, lse_out = self.lse[l0:l1], None
             B.actkv_score_overlap(self.pd, self.td, l0, l1, q[l0:l1], win_indptr, self.n_q_heads, lse_g, sm_scale, causal,
                                   tok_indptr, self.score[: l1 - l0], lse_out, s.sum_win, s.max_win, s.sum_tok, s.max_tok,
                                   self.ws_score, None if prev is None else self.ws_compact, self.status, stream)
