@@ -331,7 +331,8 @@ def run_ours(args):
     pipe_comp = None
     if pipelined:
         pipe_comp = H.Compressor(inst.pool, inst.page_table, inst.seq_len, inst.free_list, inst.free_count, wl.n_q_heads,
-                                 sz, layers_per_call=max(l1 - l0 for l0, l1 in pipe_groups), want_lse=False, want_ties=True)
+                                 sz, layers_per_call=max(l1 - l0 for l0, l1 in pipe_groups), want_lse=False, want_ties=True,
+                                 lse_layers_per_call=NL)
         pipe_comp.lse, pipe_comp.status = comp.lse, comp.status
     lrfu_state = None                          # set for the secondary LRFU-policy line only
     inplace_mode = False                       # set for the secondary in-place-compaction line only
@@ -655,8 +656,6 @@ def run_ours(args):
                 ms.append(ev[0][1].elapsed_time(ev[-1][1]))
                 cp_ms.append(sum(ev[i - 1][1].elapsed_time(ev[i][1]) for i in range(1, len(ev))
                                  if ev[i][0] == "compact"))
-        inplace_mode = False
-        del pool_backup
         comp.check_status()
         # rows that had to move: survivors outside the tail region, counted from the last step's lists
         moved = count_inplace_moves(comp, wl)
@@ -664,8 +663,31 @@ def run_ours(args):
         if dist is not None:
             dist.all_reduce(tl, op=dist.ReduceOp.MAX)
         cp = sum(cp_ms) / len(cp_ms)
-        moved_bytes = 4.0 * D * 2 * moved * n_calls      # K and V rows, read + write, bf16; lists of the last call
+        moved_bytes = 4.0 * D * 2 * moved * (-(-NL // comp.lpc))      # K and V rows, read + write, bf16; lists of the last call
+        # ... and with the LSE supplied as well: the paper's own mode (Section 7.1) with the paper's own compaction
+        # (Algorithm 4), the cheapest step the library has
+        lse_supplied = comp.lse.clone()
+        ms2 = []
+        for it in range(2 + min(args.steps, 5)):
+            inst.pool.copy_(pool_backup)
+            restore()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            one_step()
+            e1.record()
+            torch.cuda.synchronize()
+            if it >= 2:
+                ms2.append(e0.elapsed_time(e1))
+        lse_supplied = None
+        inplace_mode = False
+        del pool_backup
+        comp.check_status()
+        t2 = torch.tensor([sum(ms2) / len(ms2)], dtype=torch.float64, device=dev)
+        if dist is not None:
+            dist.all_reduce(t2, op=dist.ReduceOp.MAX)
         inplace_line = {"ms_per_step": float(tl.item()), "value": world * tokens / (float(tl.item()) * 1e-3), "unit": UNIT,
+                        "with_lse_supplied": {"ms_per_step": float(t2.item()),
+                                              "value": world * tokens / (float(t2.item()) * 1e-3), "unit": UNIT},
                         "compact_ms": cp, "rows_moved_fraction_of_kept": moved / max(1.0, rho * tokens * Hkv * comp.lpc),
                         "compact_gbs": moved_bytes / (cp * 1e-3) / 1e9,
                         "compact_frac_of_hbm_peak": moved_bytes / (cp * 1e-3) / 1e9 / pk["hbm_gbs"]}
@@ -708,9 +730,9 @@ def run_ours(args):
             "ties_at_threshold": ties_line,
             "clocks": clocks, "gpu_launches": launches, "wall_s_timed_region": t_wall,
         }
-        print(json.dumps(out))
     if dist is not None:
         dist.destroy_process_group()
+    return out if rank == 0 else None
 
 
 def main():
@@ -730,6 +752,10 @@ def main():
                     help="layer groups of the timed step, whose copies run inside the score kernels of the next group: "
                          "'auto' (three equal groups), comma-separated group sizes, or 'none' (one call per stage)")
     ap.add_argument("--lse", default="internal", choices=["internal", "supplied"])
+    ap.add_argument("--all-configs", action="store_true",
+                    help="after the timed workload, measure every configuration of the benchmark definition and the "
+                         "paper's kernel-table shapes (adds a per_config list; takes several minutes)")
+    ap.add_argument("--configs", default=None, help="like --all-configs for a subset: c1,c2,c3,c4,c5,table1")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-lrfu", action="store_true", help="skip the secondary LRFU-policy line")
@@ -740,8 +766,18 @@ def main():
         print("note: fewer than 3 warm-up steps", file=sys.stderr)
     if args.impl == "reference":
         run_reference(args)
-    else:
-        run_ours(args)
+        return
+    out = run_ours(args)
+    if out is not None and (args.all_configs or args.configs) and out["n_gpus"] == 1:
+        # every other configuration of the benchmark definition, one after the other on the freed device
+        import gc
+        from paper_2609_31395_b200 import config_bench
+        gc.collect()
+        torch.cuda.empty_cache()
+        out["per_config"] = config_bench.run_all(torch.device("cuda", 0), peaks(),
+                                                 args.configs.split(",") if args.configs else None)
+    if out is not None:
+        print(json.dumps(out))
 
 
 if __name__ == "__main__":

@@ -35,7 +35,7 @@ class Compressor:
 
     def __init__(self, pool: torch.Tensor, page_table, seq_len, free_list, free_count, n_q_heads: int,
                  sizes: StepSizes, layers_per_call: Optional[int] = None, want_lse: bool = False,
-                 want_ties: bool = False, want_mask: bool = False):
+                 want_ties: bool = False, want_mask: bool = False, lse_layers_per_call: Optional[int] = None):
         B.load()
         self.dev = pool.device
         self.pool = pool
@@ -46,6 +46,9 @@ class Compressor:
         self.sz = sizes
         NL, Hkv = self.pd.n_layers, self.pd.n_kv_heads
         self.lpc = NL if layers_per_call is None else max(1, min(NL, layers_per_call))
+        # layers per call of an LSE pass of its own (step_pipelined): it needs no score or index buffer, so it may
+        # cover more layers than the other passes
+        self.lse_lpc = self.lpc if lse_layers_per_call is None else max(self.lpc, min(NL, lse_layers_per_call))
         s = sizes
         self.score = torch.empty((self.lpc, Hkv, s.sum_tok), dtype=torch.float32, device=self.dev)
         self.sel_idx = torch.empty((self.lpc * Hkv, s.sel_stride), dtype=torch.int32, device=self.dev)
@@ -55,7 +58,7 @@ class Compressor:
         self.ties = torch.zeros((self.lpc * Hkv * s.n_req, 4), dtype=torch.int32, device=self.dev) if want_ties else None
         self.mask = (torch.zeros((self.lpc * Hkv, (s.sum_tok + 31) // 32), dtype=torch.int32, device=self.dev)
                      if want_mask else None)
-        self.ws_score = _ws(B.actkv_score_workspace_bytes(self.pd, s.n_req, self.lpc, n_q_heads, s.sum_win, s.max_win,
+        self.ws_score = _ws(B.actkv_score_workspace_bytes(self.pd, s.n_req, self.lse_lpc, n_q_heads, s.sum_win, s.max_win,
                                                           s.max_tok), self.dev)
         self.ws_select = _ws(B.actkv_select_workspace_bytes(self.lpc * Hkv, s.n_req, s.max_tok), self.dev)
         # (sized for the pipelined step as well: room for the resolved sources of one layer group)
@@ -179,18 +182,22 @@ class Compressor:
         launches = 1
         prev = None
         done = []               # groups whose statistics have been written to `stats` ([n_groups, 2] int32, optional)
+        if lse_in is None and (marks is not None or self.lse_lpc > self.lpc):
+            # the LSE pass of all layers first, in calls of its own (as long as the workspace allows: fewer, larger
+            # launches), then the pooled-score passes, which carry the copies
+            if self.lse is None:
+                self.lse = torch.empty((NL, s.sum_win, self.n_q_heads), dtype=torch.float32, device=self.dev)
+            for l0 in range(0, NL, self.lse_lpc):
+                l1 = min(NL, l0 + self.lse_lpc)
+                mark("begin")
+                self.run_lse(q, win_indptr, tok_indptr, sm_scale, causal, l0, l1, self.lse[l0:l1], stream)
+                mark("lse")
+                launches += 2
+            lse_in = self.lse
         for l0, l1 in groups:
             mark("begin")
             lse_g = None if lse_in is None else lse_in[l0:l1]
-            lse_out = None if self.lse is None else self.lse[l0:l1]
-            if marks is not None and lse_in is None:
-                # timed per kernel: the LSE pass as a call of its own (without a copy role), then the pooled-score
-                # pass with the copies inside
-                if self.lse is None:
-                    self.lse = torch.empty((NL, s.sum_win, self.n_q_heads), dtype=torch.float32, device=self.dev)
-                self.run_lse(q, win_indptr, tok_indptr, sm_scale, causal, l0, l1, self.lse[l0:l1], stream)
-                mark("lse")
-                lse_g, lse_out = self.lse[l0:l1], None
+            lse_out = None if (self.lse is None or lse_in is self.lse) else self.lse[l0:l1]
             B.actkv_score_overlap(self.pd, self.td, l0, l1, q[l0:l1], win_indptr, self.n_q_heads, lse_g, sm_scale, causal,
                                   tok_indptr, self.score[: l1 - l0], lse_out, s.sum_win, s.max_win, s.sum_tok, s.max_tok,
                                   self.ws_score, None if prev is None else self.ws_compact, self.status, stream)

@@ -38,10 +38,10 @@ def _reference(wl):
     return a, comp
 
 
-def _pipelined(wl, lpc, groups=None, lse_in=None):
+def _pipelined(wl, lpc, groups=None, lse_in=None, lse_lpc=None):
     b = synth.generate(wl, DEV)
     comp = H.Compressor(b.pool, b.page_table, b.seq_len, b.free_list, b.free_count, wl.n_q_heads, H.sizes_of(b),
-                        layers_per_call=lpc, want_lse=True)
+                        layers_per_call=lpc, want_lse=True, lse_layers_per_call=lse_lpc)
     comp.step_pipelined(b.q, b.win_indptr, b.tok_indptr, b.budget, wl.sm_scale, wl.causal, lse_in=lse_in, groups=groups)
     torch.cuda.synchronize()
     comp.check_status()
@@ -62,6 +62,10 @@ def test_pipelined_step_equals_the_one_call_step(causal):
     # with the LSE supplied (no LSE kernel: all copies ride on the pooled-score kernel or the drain)
     c, _ = _pipelined(wl, 2, lse_in=comp_a.lse)
     _same_state(a, c)
+    # the LSE pass of all layers first, in one call of its own, then the groups
+    d, comp_d = _pipelined(wl, 2, lse_lpc=7)
+    _same_state(a, d)
+    assert torch.equal(comp_a.lse, comp_d.lse)
 
 
 def test_uneven_groups_and_other_shapes():
