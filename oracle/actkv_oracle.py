@@ -18,9 +18,8 @@ compaction example and byte-permutation / conservation properties; closed forms 
 confidence monitor (uniform logits -> log V, two-point slope, numpy.polyfit, the budget chain
 from the Section 8.1 constants).
 
-Parity unpinned (conventions the paper leaves open, fixed by this build and listed in the
-design notes): the causal reading of the action window, per-KV-head selection, ascending
-survivor order, fresh-page allocation order and free-list discipline, nearest-rank percentile
+Parity unpinned (conventions the paper leaves open, fixed by this build): the causal reading of
+the action window, per-KV-head selection, ascending survivor order, fresh-page allocation order and free-list discipline, nearest-rank percentile
 and the x-axis of the line fit.
 """
 from __future__ import annotations
@@ -203,15 +202,6 @@ def select_unit(score_f32: np.ndarray, budget: int) -> np.ndarray:
     n = min(int(budget), L)
     order = np.lexsort((np.arange(L), -score_f32.astype(np.float64)))   # last key is primary
     return np.sort(np.asarray(order[:n], dtype=np.int64)).astype(np.int32)
-
-
-def select(score_all: np.ndarray, tok_indptr, budget) -> list:
-    """actkv_select: per (outer, request) list of kept indices; result[o][r] int32 array."""
-    score_all = np.asarray(score_all, dtype=np.float32)
-    n_outer = score_all.shape[0]
-    R = len(budget)
-    return [[select_unit(score_all[o, tok_indptr[r]:tok_indptr[r + 1]], budget[r]) for r in range(R)]
-            for o in range(n_outer)]
 
 
 # --------------------------------------------------------------------------------------------

@@ -234,7 +234,7 @@ def confidence_logits(n_req: int, rows_per_req: int, vocab: int, seed: int, devi
 
 
 # --------------------------------------------------------------------------------------------
-# The benchmark configurations (shapes of the paper's models and traces; see the design notes)
+# The benchmark configurations (shapes of the paper's models and traces)
 
 
 def config1(seed: int = 0) -> Workload:

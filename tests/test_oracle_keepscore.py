@@ -6,22 +6,24 @@ from oracle import actkv_oracle as O
 from conftest import read_golden
 
 
-def _brute_hits(score, p):
-    """Definition by hand with exact fractions: shortest descending prefix whose mass reaches p of the
-    total; the crossing entry is in."""
+def _plain_hits(score, p):
+    """The plain real-valued rule, with no quantisation anywhere: the float32 scores as the exact rationals
+    they are, p as the exact decimal, the shortest prefix of the entries ordered by (score descending, index
+    ascending) whose sum reaches p times the total; the crossing entry is in.  Also returns how far (as a
+    fraction of the total) the sums just before and just after the last hit are from the mark."""
     from fractions import Fraction
-    L = len(score)
-    mass = [int(np.floor(min(max(float(x), 0.0), 256.0) * 2**32)) for x in score]
-    total = sum(mass)
-    mark = Fraction(int(round(p * 10000)), 10000) * total
-    order = sorted(range(L), key=lambda i: (-float(score[i]), i))
-    hit, acc = set(), 0
+    vals = [max(Fraction(float(x)), Fraction(0)) for x in score]
+    total = sum(vals)
+    mark = Fraction(str(p)) * total
+    order = sorted(range(len(score)), key=lambda i: (-vals[i], i))
+    hit, acc, margin = [], Fraction(0), None
     for i in order:
-        if acc >= mark:
+        if acc >= mark or vals[i] == 0:
             break
-        hit.add(i)
-        acc += mass[i]
-    return sorted(hit)
+        hit.append(i)
+        margin = min(mark - acc, acc + vals[i] - mark) / total if total else None
+        acc += vals[i]
+    return sorted(hit), margin
 
 
 def test_paper_constants_present():
@@ -34,7 +36,27 @@ def test_hit_mask_against_brute_force_with_ties():
     for seed in range(6):
         s = (rng.integers(0, 9, 61).astype(np.float32) / 64.0)            # many exact ties, some zeros
         for p in (0.0, 0.5, 0.9, 0.99, 1.0):
-            assert np.nonzero(O.hit_mask_unit(s, p))[0].tolist() == _brute_hits(s, p)
+            # multiples of 1/64 have integer masses, so the integer rule and the real-valued rule coincide exactly,
+            # also when a prefix lands on the mark
+            assert np.nonzero(O.hit_mask_unit(s, p))[0].tolist() == _plain_hits(s, p)[0]
+
+
+def test_integer_masses_give_the_real_valued_top_p_set():
+    """The oracle counts mass in integers of 2^-32 so that the set does not depend on a summation order.  Against
+    the plain rule on the real values of the float32 scores: the same set whenever the mark is further from a
+    prefix sum than the truncation can move it (L x 2^-32 of mass), which random inputs always are."""
+    rng = np.random.default_rng(5)
+    checked = 0
+    for seed in range(8):
+        L = int(rng.integers(50, 400))
+        s = (rng.random(L) ** 6).astype(np.float32) * np.float32(0.05)       # skewed, pooled-probability sized
+        for p in (0.3, 0.9, 0.97):
+            want, margin = _plain_hits(s, p)
+            total = float(np.sum(s.astype(np.float64)))
+            if margin is not None and float(margin) * total > 4 * L * 2.0 ** -32:
+                assert np.nonzero(O.hit_mask_unit(s, p))[0].tolist() == want
+                checked += 1
+    assert checked >= 20
 
 
 def test_hit_mask_is_a_prefix_that_just_reaches_the_mark():
