@@ -70,7 +70,7 @@ def gather_rows(pool_bits: np.ndarray, layer: int, kv: int, head: int, slots: np
 
 
 def score_unit(q_unit: np.ndarray, k_unit: np.ndarray, sm_scale: float, causal: bool,
-               lse_in: np.ndarray | None = None):
+               lse_in: np.ndarray | None = None, window_left: int = 0):
     """Pooled action-region score of one (layer, request, KV head) unit.
 
     q_unit float64 [W, G, D]: the action-window queries of the G q-heads that share this KV
@@ -86,18 +86,21 @@ def score_unit(q_unit: np.ndarray, k_unit: np.ndarray, sm_scale: float, causal: 
     and row w sees j <= L - W + w (a decode step attends to the keys before it and itself
     being already cached); an invisible pair adds 0 and the divisor stays W, which is the
     running mean started from zero of Section 7.1's last paragraph.
+    window_left = S > 0: a sliding-window attention layer (Section 8.2 names such layers; the paper does
+    not say how they are scored): a query at cache position p attends to the S keys p - S < j <= p only.
+    With causal=True row w sits at p = L - W + w; with causal=False every row is taken to sit at the end of
+    the cache, p = L - 1.  The LSE runs over the same visible set, so a row's visible probabilities sum to 1.
 
     Returns (score float32 [L], lse float64 [W, G]).
     """
     W, G, D = q_unit.shape
     L = k_unit.shape[0]
     s = sm_scale * np.einsum("wgd,jd->wgj", q_unit, k_unit)          # [W, G, L]
-    if causal:
-        j = np.arange(L)[None, None, :]
-        w = np.arange(W)[:, None, None]
-        visible = j <= (L - W + w)
-    else:
-        visible = np.ones((W, 1, L), dtype=bool)
+    j = np.arange(L)[None, None, :]
+    pos = (L - W + np.arange(W))[:, None, None] if causal else np.full((W, 1, 1), L - 1)    # position of each row
+    visible = j <= pos
+    if window_left > 0:
+        visible = visible & (j > pos - window_left)
     visible = np.broadcast_to(visible, s.shape)
     if lse_in is None:
         s_masked = np.where(visible, s, -np.inf)
@@ -112,7 +115,7 @@ def score_unit(q_unit: np.ndarray, k_unit: np.ndarray, sm_scale: float, causal: 
 
 
 def score(pool_bits, page_table, seq_len, q_bits, win_indptr, n_q_heads, sm_scale, causal,
-          layers=None, lse_in=None, units=None):
+          layers=None, lse_in=None, units=None, window_left=0):
     """actkv_score over whole tensors (or over the listed units only).
 
     q_bits uint16 [NLs, sum_win, n_q_heads, D]; page_table int [R, max_pages]; seq_len [R];
@@ -140,7 +143,7 @@ def score(pool_bits, page_table, seq_len, q_bits, win_indptr, n_q_heads, sm_scal
         k_unit = bf16_bits_to_f64(gather_rows(pool_bits, layers[a], 0, h, slots))
         q_unit = bf16_bits_to_f64(q_bits[a, w0:w1, h * G:(h + 1) * G, :])
         li = None if lse_in is None else lse_in[a, w0:w1, h * G:(h + 1) * G]
-        sc, ls = score_unit(q_unit, k_unit, sm_scale, causal, li)
+        sc, ls = score_unit(q_unit, k_unit, sm_scale, causal, li, window_left)
         out[a, h, tok_indptr[r]:tok_indptr[r + 1]] = sc
         lse[a, w0:w1, h * G:(h + 1) * G] = ls
     return out, lse, tok_indptr

@@ -188,3 +188,62 @@ def test_planted_keys_are_retained_config1():
     for h in range(wl.n_kv_heads):
         kept = set(O.select_unit(out[0, h], wl.budgets[0]).tolist())
         assert planted <= kept
+
+
+# ---- sliding-window layers (window_left = S: a query at position p attends to keys p - S < j <= p) ----
+
+
+def _loops_windowed(q, k, scale, causal, S):
+    """The definition in pure-Python loops."""
+    W, G, D = q.shape
+    L = k.shape[0]
+    out = [0.0] * L
+    for w in range(W):
+        p = L - W + w if causal else L - 1
+        best = [0.0] * L
+        for g in range(G):
+            vis = [j for j in range(L) if j <= p and (S <= 0 or j > p - S)]
+            logit = {j: scale * sum(q[w, g, d] * k[j, d] for d in range(D)) for j in vis}
+            z = sum(math.exp(v) for v in logit.values())
+            for j in vis:
+                best[j] = max(best[j], math.exp(logit[j]) / z)
+        for j in range(L):
+            out[j] += best[j] / W
+    return np.array(out)
+
+
+@pytest.mark.parametrize("causal", [False, True])
+def test_sliding_window_against_python_loops(causal):
+    rng = np.random.default_rng(3)
+    q, k = _rand_unit(rng, 4, 2, 23, 5)
+    for S in (0, 1, 3, 7, 22, 23, 100):
+        got, lse = O.score_unit(q, k, 0.4, causal, window_left=S)
+        assert np.abs(got.astype(np.float64) - _loops_windowed(q, k, 0.4, causal, S)).max() < 1e-7
+        assert np.isfinite(lse).all()
+
+
+def test_sliding_window_closed_forms():
+    rng = np.random.default_rng(4)
+    W, G, L = 6, 3, 40
+    q, k = _rand_unit(rng, W, G, L, 8)
+    # S = 1, causal: a row sees its own key only, with probability 1 in every head -> each window position
+    # scores 1/W, every other key 0, and the LSE is the row's own logit
+    got, lse = O.score_unit(q, k, 0.3, True, window_left=1)
+    want = np.zeros(L)
+    want[L - W:] = 1.0 / W
+    assert np.abs(got - want).max() < 1e-7
+    own = 0.3 * np.einsum("wgd,wd->wg", q, k[L - W:])
+    assert np.abs(lse - own).max() < 1e-12
+    # a window at least as long as the cache changes nothing
+    for causal in (False, True):
+        full, lse_f = O.score_unit(q, k, 0.3, causal)
+        same, lse_s = O.score_unit(q, k, 0.3, causal, window_left=L + 5)
+        assert np.array_equal(full, same) and np.array_equal(lse_f, lse_s)
+    # not causal, one row, one head: the textbook softmax over the last S keys, 0 before them
+    S = 9
+    got, _ = O.score_unit(q[:1, :1], k, 0.3, False, window_left=S)
+    ref = torch.softmax(torch.from_numpy(0.3 * (k[L - S:] @ q[0, 0])), dim=0).numpy()
+    assert np.abs(got[L - S:] - ref).max() < 1e-7 and not got[:L - S].any()
+    # visible probabilities of a row sum to 1, so the unit's mass stays in [1, G]
+    got, _ = O.score_unit(q, k, 0.3, True, window_left=5)
+    assert 1.0 - 1e-6 <= got.sum() <= G + 1e-6 and not got[:L - W - 4].any()
