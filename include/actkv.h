@@ -167,6 +167,26 @@ int actkv_score(const actkv_pool_t* pool /* host */, const actkv_tables_t* table
                 void* ws, size_t ws_bytes, int32_t* status, actkv_stream_t stream);
 
 /* ---------------------------------------------------------------------------------------
+ * actkv_score_sliding — actkv_score for sliding-window attention layers (Section 8.2 names models
+ * that interleave such layers with full-attention ones; the paper does not say how they are scored,
+ * this is the reading taken here).
+ *
+ * window_left = S > 0: a query at cache position p attends to the S keys p - S < j <= p only.  With
+ * causal != 0 row w sits at p = L_r - W_r + w; with causal == 0 every row is taken to sit at the end
+ * of the cache, p = L_r - 1.  The LSE (computed here or supplied) runs over the same visible set.
+ * Keys no row sees score 0; whole key tiles of them are neither fetched nor multiplied.
+ * S = 0 is actkv_score.  One S per call: a model that alternates layer kinds hands each kind over as
+ * a pool view whose stride_layer skips the other.  All other arguments as actkv_score.
+ */
+int actkv_score_sliding(const actkv_pool_t* pool /* host */, const actkv_tables_t* tables /* host */,
+                        int32_t layer_begin, int32_t layer_end,
+                        const void* q, const int32_t* win_indptr, int32_t n_q_heads,
+                        const float* lse_in, float sm_scale, int32_t causal, int32_t window_left,
+                        const int32_t* tok_indptr, float* score_out, float* lse_out,
+                        int32_t sum_win, int32_t max_win, int32_t sum_tok, int32_t max_tok,
+                        void* ws, size_t ws_bytes, int32_t* status, actkv_stream_t stream);
+
+/* ---------------------------------------------------------------------------------------
  * actkv_score_path — which kernels actkv_score (streaming == 0) or actkv_score_accumulate
  * (streaming != 0) would run for this pool, group size, window bound, scale and query pointer:
  * 1 = the tensor-core kernels (tcgen05), 0 = the FMA kernels, negative = bad argument.

@@ -26,7 +26,7 @@ EXPORTS = ["actkv_budget_workspace_bytes", "actkv_budget", "actkv_score_workspac
            "actkv_keep_indptr", "actkv_select_workspace_bytes", "actkv_select",
            "actkv_compact_workspace_bytes", "actkv_compact", "actkv_compact_noalloc",
            "actkv_compact_noalloc_max_bytes", "actkv_step_host", "actkv_keepscore", "actkv_gather_f32",
-           "actkv_compact_inplace", "actkv_score_path", "actkv_debug_inject_stall",
+           "actkv_compact_inplace", "actkv_score_path", "actkv_debug_inject_stall", "actkv_score_sliding",
            "actkv_compact_deferred_workspace_bytes", "actkv_compact_begin", "actkv_compact_end", "actkv_score_overlap", "actkv_compact_stats",
            "actkv_version"]
 
@@ -158,6 +158,9 @@ def load():
     lib.actkv_compact_deferred_workspace_bytes.argtypes = [C.POINTER(PoolDesc), i32, i32, i32, i32]
     lib.actkv_compact_stats.restype = i32
     lib.actkv_compact_stats.argtypes = [vp, vp, vp]
+    lib.actkv_score_sliding.restype = i32
+    lib.actkv_score_sliding.argtypes = [C.POINTER(PoolDesc), C.POINTER(TablesDesc), i32, i32, vp, vp, i32, vp, f32, i32,
+                                        i32, vp, vp, vp, i32, i32, i32, i32, vp, sz, vp, vp]
     lib.actkv_score_path.restype = i32
     lib.actkv_score_path.argtypes = [C.POINTER(PoolDesc), i32, i32, f32, vp, i32]
     lib.actkv_debug_inject_stall.restype = i32
@@ -290,6 +293,19 @@ def actkv_compact_deferred_workspace_bytes(pool: PoolDesc, n_req, max_pages, n_l
 def actkv_compact_stats(ws, stats, stream=None):
     _check("actkv_compact_stats", load().actkv_compact_stats(_ptr(ws, None, "ws"), _ptr(stats, torch.int32, "stats"),
                                                              _stream(stream)))
+
+
+def actkv_score_sliding(pool: PoolDesc, tables: TablesDesc, layer_begin, layer_end, q, win_indptr, n_q_heads, lse_in,
+                        sm_scale, causal, window_left, tok_indptr, score_out, lse_out, sum_win, max_win, sum_tok, max_tok,
+                        ws, status, stream=None):
+    rc = load().actkv_score_sliding(C.byref(pool), C.byref(tables), layer_begin, layer_end, _ptr(q, torch.bfloat16, "q"),
+                                    _ptr(win_indptr, torch.int32, "win_indptr"), n_q_heads,
+                                    _ptr(lse_in, torch.float32, "lse_in"), float(sm_scale), int(bool(causal)),
+                                    int(window_left), _ptr(tok_indptr, torch.int32, "tok_indptr"),
+                                    _ptr(score_out, torch.float32, "score_out"), _ptr(lse_out, torch.float32, "lse_out"),
+                                    sum_win, max_win, sum_tok, max_tok, _ptr(ws, None, "ws"),
+                                    ws.numel() * ws.element_size(), _ptr(status, torch.int32, "status"), _stream(stream))
+    _check("actkv_score_sliding", rc)
 
 
 def actkv_score_path(pool: PoolDesc, n_q_heads, max_win, sm_scale, q, streaming=False) -> int:

@@ -62,7 +62,7 @@ static int score_impl(int mode, const actkv_pool_t* pool, const actkv_tables_t* 
                       const float* lse_in, float sm_scale, int32_t causal, const int32_t* tok_indptr,
                       float* score_out, float* lse_out, int32_t sum_win, int32_t max_win, int32_t sum_tok,
                       int32_t max_tok, void* ws, size_t ws_bytes, int32_t* status, actkv_stream_t stream,
-                      const int32_t* acc_steps = nullptr, void* copy_ws = nullptr) {
+                      const int32_t* acc_steps = nullptr, void* copy_ws = nullptr, int32_t window_left = 0) {
   using namespace actkv;
   if (!pool || !tables || !pool->base) return ACTKV_E_INVALID;
   if (layer_begin < 0 || layer_end > pool->n_layers || layer_begin > layer_end) return ACTKV_E_INVALID;
@@ -71,7 +71,7 @@ static int score_impl(int mode, const actkv_pool_t* pool, const actkv_tables_t* 
   if (n_q_heads <= 0 || n_q_heads % Hkv != 0) return ACTKV_E_INVALID;
   const int G = n_q_heads / Hkv;
   if (G > FMA_RQ) return ACTKV_E_INVALID;
-  if (R < 0 || sum_win < 0 || max_win < 0 || sum_tok < 0 || max_tok < 0) return ACTKV_E_INVALID;
+  if (R < 0 || sum_win < 0 || max_win < 0 || sum_tok < 0 || max_tok < 0 || window_left < 0) return ACTKV_E_INVALID;
   if (((uintptr_t)pool->base & 15) || pool->stride_layer % 8 || pool->stride_page % 8 || pool->stride_slot % 8 ||
       pool->stride_head % 8 || ((uintptr_t)q & 15))
     return ACTKV_E_INVALID;
@@ -124,6 +124,7 @@ static int score_impl(int mode, const actkv_pool_t* pool, const actkv_tables_t* 
   a.n_tiles = (max_tok + FMA_TK - 1) / FMA_TK;
   a.scale_log2 = sm_scale * kLog2e;
   a.causal = causal;
+  a.win_left = window_left;
   a.acc_steps = acc_steps;
   const int64_t units = (int64_t)nls * Hkv * R;
   // (the streaming update keeps a running mean in place, which the row-group launches of a window above
@@ -186,6 +187,17 @@ int actkv_score_overlap(const actkv_pool_t* pool, const actkv_tables_t* tables, 
   return score_impl(lse_in ? 2 : 3, pool, tables, layer_begin, layer_end, q, win_indptr, n_q_heads, lse_in, sm_scale,
                     causal, tok_indptr, score_out, lse_out, sum_win, max_win, sum_tok, max_tok, ws, ws_bytes, status,
                     stream, nullptr, pending_compact_ws);
+}
+
+int actkv_score_sliding(const actkv_pool_t* pool, const actkv_tables_t* tables, int32_t layer_begin,
+                        int32_t layer_end, const void* q, const int32_t* win_indptr, int32_t n_q_heads,
+                        const float* lse_in, float sm_scale, int32_t causal, int32_t window_left,
+                        const int32_t* tok_indptr, float* score_out, float* lse_out, int32_t sum_win,
+                        int32_t max_win, int32_t sum_tok, int32_t max_tok, void* ws, size_t ws_bytes,
+                        int32_t* status, actkv_stream_t stream) {
+  return score_impl(lse_in ? 2 : 3, pool, tables, layer_begin, layer_end, q, win_indptr, n_q_heads, lse_in, sm_scale,
+                    causal, tok_indptr, score_out, lse_out, sum_win, max_win, sum_tok, max_tok, ws, ws_bytes, status,
+                    stream, nullptr, nullptr, window_left);
 }
 
 int actkv_score_lse(const actkv_pool_t* pool, const actkv_tables_t* tables, int32_t layer_begin,

@@ -34,6 +34,7 @@ struct ScoreArgs {
   int32_t lse_chunk;             // keys per LSE partial of this launch (multiple of 128, >= LSE_CHUNK)
   float scale_log2;              // sm_scale * log2(e)
   int32_t causal;
+  int32_t win_left;              // sliding-window layer: a query at position p sees keys p - win_left < j <= p (0: all)
   const int32_t* acc_steps;      // accumulate mode (streaming, Algorithm 3 step 5): [R] action queries already
                                  // folded into score_out; nullptr: score_out is overwritten with this call's mean
 };
@@ -160,7 +161,7 @@ __global__ void __launch_bounds__(FMA_NT) score_fma_kernel(const ScoreArgs a) {
 #pragma unroll
         for (int k = 0; k < 4; ++k) {
           int j = t0 + tx + 16 * k;
-          bool vis = row_ok && j < L && j <= last_visible;
+          bool vis = row_ok && j < L && j <= last_visible && (a.win_left <= 0 || j > last_visible - a.win_left);
           t[k] = vis ? acc[i][k] * a.scale_log2 : -INFINITY;
         }
         if (PASS == 1) {

@@ -83,17 +83,17 @@ __device__ __forceinline__ float lse_fast32(const float* v, float c, float nmc, 
   return (s[0] + s[1]) + (s[2] + s[3]);
 }
 
-// The general form: the first nv (possibly <= 0 or >= 32) logits are visible; moves the reference to the
-// maximum seen so far.  Also the entry for a row's first logits (m = -inf, sum = 0).
-__device__ __forceinline__ void lse_slow32(const float* v, int nv, float c, float& m, float& sum) {
-  if (nv <= 0) return;
+// The general form: logits n_lo <= i < nv (any integers) are visible; moves the reference to the maximum seen
+// so far.  Also the entry for a row's first logits (m = -inf, sum = 0).
+__device__ __forceinline__ void lse_slow32(const float* v, int n_lo, int nv, float c, float& m, float& sum) {
+  if (nv <= 0 || n_lo >= 32 || n_lo >= nv) return;
   float gm = -INFINITY;
 #pragma unroll
-  for (int i = 0; i < 32; ++i) gm = fmaxf(gm, i < nv ? v[i] : -INFINITY);
+  for (int i = 0; i < 32; ++i) gm = fmaxf(gm, (i >= n_lo && i < nv) ? v[i] : -INFINITY);
   if (gm > m) { sum = (m == -INFINITY) ? 0.f : sum * exp2f((m - gm) * c); m = gm; }
   const float mc = m * c;
 #pragma unroll
-  for (int i = 0; i < 32; ++i) sum += (i < nv) ? exp2f(fmaf(v[i], c, -mc)) : 0.f;
+  for (int i = 0; i < 32; ++i) sum += (i >= n_lo && i < nv) ? exp2f(fmaf(v[i], c, -mc)) : 0.f;
 }
 
 constexpr int LSE_EPI_WARPS = 16;                // (TMEM lane quarter, accumulator, column half)
@@ -135,11 +135,12 @@ __device__ __forceinline__ int sel4(const int (&x)[4], int i) { return i == 0 ? 
 // for tensor memory the other keeps the special function unit busy.
 //   tq      tensor-memory address of the group's accumulator, this warp's lane quarter and first column
 //   nv_min  visible columns (from the warp's first column) of the most restricted row of this thread
-//   jm      last visible key of this thread's row in each row block; key0 = key of the warp's first column
+//   nlo_max columns (from the warp's first column) below the first visible key of the most restricted row
+//   jm, jl  last / first visible key of this thread's row in each row block; key0 = key of the warp's first column
 template <int NPOLY>
 __device__ __forceinline__ bool lse_job(LseBarriers* bars, volatile int* abort_flag, uint32_t tq, int grp, int job,
-                                        int mb, float2* st, int nv_min, const int (&jm)[4], int key0, float c, float c1,
-                                        int lane, long long wait_cycles) {
+                                        int mb, float2* st, int nv_min, int nlo_max, const int (&jm)[4], const int (&jl)[4],
+                                        int key0, float c, float c1, int lane, long long wait_cycles) {
   float v[64];
   float* va = v;
   float* vb = v + 32;
@@ -152,7 +153,7 @@ __device__ __forceinline__ bool lse_job(LseBarriers* bars, volatile int* abort_f
   tc_fence_before();
   __syncwarp();
   if (lane == 0) mbar_arrive(smem_u32(&bars->tmem_empty[grp]));
-  bool slow = __any_sync(0xffffffffu, nv_min < 64 || ms.x == -INFINITY);
+  bool slow = __any_sync(0xffffffffu, nv_min < 64 || nlo_max > 0 || ms.x == -INFINITY);
   if (!slow) {
     const float nmc = -ms.x * c, c0 = fmaf(nmc, 1.f / 252.f, 0.5f);
     const float ps = lse_fast32<NPOLY>(va, c, nmc, c1, c0) + lse_fast32<NPOLY>(vb, c, nmc, c1, c0);
@@ -160,9 +161,9 @@ __device__ __forceinline__ bool lse_job(LseBarriers* bars, volatile int* abort_f
     if (!slow) ms.y += ps;
   }
   if (slow) {
-    const int nv = sel4(jm, mb) - key0 + 1;
-    lse_slow32(va, nv, c, ms.x, ms.y);
-    lse_slow32(vb, nv - 32, c, ms.x, ms.y);
+    const int nv = sel4(jm, mb) - key0 + 1, nlo = sel4(jl, mb) - key0;
+    lse_slow32(va, nlo, nv, c, ms.x, ms.y);
+    lse_slow32(vb, nlo - 32, nv - 32, c, ms.x, ms.y);
   }
   *st = ms;
   return true;
@@ -198,9 +199,16 @@ score_tc_lse_kernel(const __grid_constant__ CUtensorMap kmap, const TcArgs ta) {
     return;
   }
   const int n_mb = (rows + 127) / 128;                   // 1..4
-  const int t_begin = key_begin / TK;
-  const int t_end = min((L + TK - 1) / TK, t_begin + a.lse_chunk / TK);
+  const int t_end = min((L + TK - 1) / TK, key_begin / TK + a.lse_chunk / TK);
+  // sliding-window layer: key tiles below the first key any row of the unit sees are not fetched at all
+  const int lo_all = a.win_left > 0 ? max(0, (a.causal ? L - W : L - 1) - a.win_left + 1) : 0;
+  const int t_begin = max(key_begin / TK, lo_all / TK);
   const int n_tiles = t_end - t_begin;
+  if (n_tiles <= 0) {                                    // no row sees a key of this chunk
+    for (int n = threadIdx.x; n < rows; n += blockDim.x)
+      a.partials[((int64_t)u * a.n_chunks + chunk) * a.rows_max + row0 + n] = make_float2(-INFINITY, 0.f);
+    return;
+  }
   const int n_jobs = n_tiles * n_mb;
   const int S = ta.n_stages;
 
@@ -342,22 +350,25 @@ score_tc_lse_kernel(const __grid_constant__ CUtensorMap kmap, const TcArgs ta) {
       if (lane == 0) mbar_arrive(smem_u32(&bars->q_ready));
     }
     // last key each of this thread's rows sees (padding rows: every key, their sums are dropped)
-    int jm[4];
+    // ... and the first one (0 unless the layer has a sliding window)
+    int jm[4], jl[4];
 #pragma unroll
     for (int mb = 0; mb < 4; ++mb) {
       const int n = mb * 128 + rib;
       jm[mb] = (a.causal && n < rows) ? (L - W + (row0 + n) / G) : (L - 1);
+      jl[mb] = (a.win_left > 0 && n < rows) ? max(0, jm[mb] - a.win_left + 1) : 0;
       bars->state[grp][mb][half][rib] = make_float2(-INFINITY, 0.f);
     }
     const int jfast = min(min(jm[0], jm[1]), min(jm[2], jm[3]));
+    const int jlmax = max(max(jl[0], jl[1]), max(jl[2], jl[3]));
     const float c = a.scale_log2, c1 = c * (1.f / 252.f);
     const uint32_t tq = tmem_base + ((uint32_t)(quarter * 32) << 16) + LSE_A_COLS + grp * 128 + half * 64;
     // (key tile, row block) of this group's jobs, carried along without divisions: job = tile * n_mb + mb
     int mb = grp % n_mb, key0 = (t_begin + grp / n_mb) * TK + half * 64;
     const int mb_step = 2 % n_mb, tile_step = 2 / n_mb;
     for (int job = grp; job < n_jobs; job += 2) {
-      epi_ok = lse_job<NPOLY>(bars, abort_flag, tq, grp, job, mb, &bars->state[grp][mb][half][rib], jfast - key0 + 1, jm, key0, c,
-                              c1, lane, ta.wait_cycles);
+      epi_ok = lse_job<NPOLY>(bars, abort_flag, tq, grp, job, mb, &bars->state[grp][mb][half][rib], jfast - key0 + 1,
+                              jlmax - key0, jm, jl, key0, c, c1, lane, ta.wait_cycles);
       if (!epi_ok) break;
       mb += mb_step;
       key0 += tile_step * TK;

@@ -101,8 +101,8 @@ score_tc_pool_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_cons
   // rows is taken MAX_ROWS (a whole number of action tokens) per launch, later launches add to the score
   const int row_begin = ta.row_begin, w_begin = row_begin / G;
   const int rows = min(W * G - row_begin, MAX_ROWS);
-  const int t_begin = kchunk * ta.tiles_per_cta;
-  if (t_begin * TK >= L) return;
+  const int t_first = kchunk * ta.tiles_per_cta;           // first key tile of this CTA's range
+  if (t_first * TK >= L) return;
   if (row_begin > 0 && rows <= 0) return;                   // this request's window ends before this row group
   if (W <= 0 && a.acc_steps != nullptr) return;            // accumulate mode: a request outside its action region
   if (W <= 0 || (a.causal && W > L)) {
@@ -114,7 +114,22 @@ score_tc_pool_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_cons
     if (threadIdx.x == 0 && kchunk == 0) report(a.status, ACTKV_E_INVALID, r, W * a.group > a.rows_max ? W : L);
     return;
   }
-  const int t_end = min((L + TK - 1) / TK, t_begin + ta.tiles_per_cta);
+  const int t_end = min((L + TK - 1) / TK, t_first + ta.tiles_per_cta);
+  // Sliding-window layer: a key below the first key any row of the unit sees scores 0; whole key tiles of
+  // them are written here and neither fetched nor multiplied.
+  const int lw = L - W;
+  const int win = a.win_left;
+  int t_vis = t_first;
+  if (win > 0) {
+    const int lo_all = max(0, (a.causal ? lw : L - 1) - win + 1);
+    t_vis = min(t_end, max(t_first, lo_all / TK));
+    float* out0 = a.score_out + ((int64_t)slab * Hkv + h) * a.sum_tok + a.tok_indptr[r];
+    if (row_begin == 0)
+      for (int key = t_first * TK + threadIdx.x; key < min(L, t_vis * TK); key += blockDim.x)
+        store_pooled(a, r, out0 + key, 0.f, 0.f, W);
+    if (t_vis >= t_end) return;
+  }
+  const int t_begin = t_vis;                               // first key tile that is fetched and multiplied
   const int n_tiles = t_end - t_begin;
   const int rows_pad = (rows + 127) & ~127;               // <= MAX_ROWS (checked by the host)
   const bool whole = rows > 128;                          // a job has up to 256 columns: two register loads (see the epilogue)
@@ -275,7 +290,6 @@ score_tc_pool_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_cons
     const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16);
     float acc = 0.f;
     if (whole) {
-      const int lw = L - W;
       bool pending = false;
       float acc_prev = 0.f;
       int key_prev = 0;
@@ -295,6 +309,7 @@ score_tc_pool_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_cons
       uint32_t fpar = 0;
       for (int job = wg; job < n_jobs; job += 2, it += it_step, key += it_step * TK, fpar ^= 1u) {
         const int w_min = a.causal ? max(0, key - lw) : 0;
+        const int w_end = win > 0 ? (a.causal ? min(W, key - lw + win) : (key >= L - win ? W : 0)) : W;
         if (!mbar_wait_warp(full_bar, fpar, abort_flag, ta.wait_cycles)) { ok = false; break; }
         tc_fence_after();
         {
@@ -308,8 +323,8 @@ score_tc_pool_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_cons
             __syncwarp();
             if (lane == 0) mbar_arrive(empty_bar);
           }
-          pool_fold64<G>(v[0], nl, wf, w_min, W, c, acc);
-          if (n_cg_job > 2) pool_fold64<G>(v[1], nl + 64, wf + 64 / G, w_min, W, c, acc);
+          pool_fold64<G>(v[0], nl, wf, w_min, w_end, c, acc);
+          if (n_cg_job > 2) pool_fold64<G>(v[1], nl + 64, wf + 64 / G, w_min, w_end, c, acc);
           if (n_cg_job > 4) {
             // columns [128, 256)
             tmem_ld64(tq + 128, v[0]);
@@ -318,8 +333,8 @@ score_tc_pool_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_cons
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(empty_bar);
-            pool_fold64<G>(v[0], nl + 128, wf + 128 / G, w_min, W, c, acc);
-            if (n_cg_job > 6) pool_fold64<G>(v[1], nl + 192, wf + 192 / G, w_min, W, c, acc);
+            pool_fold64<G>(v[0], nl + 128, wf + 128 / G, w_min, w_end, c, acc);
+            if (n_cg_job > 6) pool_fold64<G>(v[1], nl + 192, wf + 192 / G, w_min, w_end, c, acc);
           }
         }
         if (n_rc == 1) {
@@ -362,11 +377,12 @@ score_tc_pool_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_cons
       for (int job = wg; job < n_jobs; job += 2) {
         const int b = job & 1;
         const int key = (t_begin + job) * TK + quarter * 32 + lane;
-        const int w_min = a.causal ? max(0, key - (L - W)) : 0;
+        const int w_min = a.causal ? max(0, key - lw) : 0;
+        const int w_end = win > 0 ? (a.causal ? min(W, key - lw + win) : (key >= L - win ? W : 0)) : W;
         if (!mbar_wait_warp(smem_u32(&bars->tmem_full[b]), (uint32_t)(job >> 1) & 1u, abort_flag, ta.wait_cycles)) break;
         tc_fence_after();
         const int n_cg = (rows + 31) / 32;
-        pool_job<G>(taddr + b * 256, nlse, n_cg, w_begin, w_min, W, c, acc, smem_u32(&bars->tmem_empty[b]), lane);
+        pool_job<G>(taddr + b * 256, nlse, n_cg, w_begin, w_min, w_end, c, acc, smem_u32(&bars->tmem_empty[b]), lane);
         if (key < L) { if (row_begin > 0) out[key] += acc * inv_w; else store_pooled(a, r, out + key, acc, acc * inv_w, W); }
         acc = 0.f;
       }
