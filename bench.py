@@ -452,7 +452,13 @@ def run_ours(args):
         tj = json.load(open(tpath))
         ent = tj.get("kernels", {}).get(kernel_of[dom])
         if ent is not None and tj.get("library_version") == B.actkv_version():
-            traffic = ent["dram_bytes_per_unit"] * tokens * Hkv * NL / n_calls
+            per_unit = ent["dram_bytes_per_unit"]
+            ent2 = tj["kernels"].get(kernel_of[dom] + "_with_copies")
+            if pipelined and dom == "score" and ent2 is not None:
+                # every launch but the first carries the copies of the group before it
+                g0 = (pipe_groups[0][1] - pipe_groups[0][0]) / NL
+                per_unit = g0 * per_unit + (1.0 - g0) * ent2["dram_bytes_per_unit"]
+            traffic = per_unit * tokens * Hkv * NL / n_calls
             traffic_src = tj.get("capture")
     roofline.update({"kernel": dom, "kernel_name": kernel_of[dom], "launches_per_step": n_calls,
                      "ms_per_launch": stage_ms[dom] / n_calls,
