@@ -441,6 +441,8 @@ def run_ours(args):
     for s in stages.values():
         s["frac"] = None if s["achieved"] is None else s["achieved"] / s["peak"]
     dom = max(("lse", "score", "compact"), key=lambda k: stage_ms[k])
+    if pipelined and dom == "lse":
+        n_calls = -(-NL // pipe_comp.lse_lpc)      # the LSE pass of the pipelined step: all layers per launch
     roofline = dict(stages[dom])
     # DRAM bytes per (token, KV head, layer) of each kernel, measured with ncu on a small cut of the workload and kept
     # in a data file beside the capture's summary; scaled to one launch of this run by its unit count (traffic grows
@@ -508,7 +510,7 @@ def run_ours(args):
     # ---- the same step when the attention backend hands the LSE over (the paper's own mode, Section 7.1):
     # reported beside the headline, which computes the LSE itself
     lse_supplied_line = None
-    if args.lse == "internal":
+    if args.lse == "internal" and not args.no_secondary:
         lse_supplied = comp.lse.clone()
         ms = []
         for it in range(2 + min(args.steps, 5)):
@@ -532,7 +534,7 @@ def run_ours(args):
     # ---- the other form of the step (one score / select / compact call over all layers when the timed step is the
     # pipelined one, and the other way round), both LSE modes
     other_line = None
-    if pipe_groups is not None and not args.overlap:
+    if pipe_groups is not None and not args.overlap and not args.no_secondary:
         was = pipelined
         pipelined = not was
         other_line = {"form": "one call per stage over all layers" if was else "pipelined",
@@ -762,12 +764,17 @@ def main():
                     help="after the timed workload, measure every configuration of the benchmark definition and the "
                          "paper's kernel-table shapes (adds a per_config list; takes several minutes)")
     ap.add_argument("--configs", default=None, help="like --all-configs for a subset: c1,c2,c3,c4,c5,table1")
+    ap.add_argument("--no-secondary", action="store_true",
+                    help="only the timed step: none of the secondary lines (LSE supplied, other step form, LRFU, in place, "
+                         "streaming, monitor batch, end to end, CPU baseline); for launch lists")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-lrfu", action="store_true", help="skip the secondary LRFU-policy line")
     ap.add_argument("--no-inplace", action="store_true", help="skip the secondary in-place-compaction line")
     ap.add_argument("--no-stream", action="store_true", help="skip the secondary streaming-update line")
     args = ap.parse_args()
+    if args.no_secondary:
+        args.no_e2e = args.no_cpu_baseline = args.no_lrfu = args.no_inplace = args.no_stream = True
     if args.warmup < 3 and args.impl == "ours":
         print("note: fewer than 3 warm-up steps", file=sys.stderr)
     if args.impl == "reference":

@@ -391,13 +391,33 @@ __global__ void __launch_bounds__(TR_NT) trend_kernel(
     int rank = (int)ceil(p.b_percent * (double)M / 100.0);
     if (rank < 1) rank = 1;
     if (rank > M) rank = M;
-    // nearest-rank percentile: the value v with #(< v) < rank <= #(<= v)
-    for (int m = tid; m < M; m += TR_NT) {
-      const float v = Rp[m];
-      int lt = 0, le = 0;
-      for (int j = 0; j < M; ++j) { const float x = Rp[j]; lt += x < v; le += x <= v; }
-      if (lt < rank && rank <= le) s_q = v;            // every writer holds the same value
+    // nearest-rank percentile: the rank-th smallest value, i.e. the v with #(< v) < rank <= #(<= v), by a radix
+    // select over the order-preserving integer image of the values (four 8-bit digits, most significant first):
+    // 4 M steps for any history length (counting the values below each candidate would take M^2)
+    __shared__ uint32_t s_hist[256];
+    __shared__ uint32_t s_prefix, s_remaining;
+    if (tid == 0) { s_prefix = 0u; s_remaining = (uint32_t)rank; }
+    for (int pass = 0; pass < 4; ++pass) {
+      const int shift = 24 - 8 * pass;
+      const uint32_t himask = pass == 0 ? 0u : (0xffffffffu << (shift + 8));
+      s_hist[tid] = 0u;                                  // TR_NT == 256 bins
+      __syncthreads();
+      const uint32_t prefix = s_prefix;
+      for (int m = tid; m < M; m += TR_NT) {
+        const uint32_t k = okey(Rp[m]);
+        if ((k & himask) == prefix) atomicAdd(&s_hist[(k >> shift) & 255u], 1u);
+      }
+      __syncthreads();
+      if (tid == 0) {
+        uint32_t acc = 0, rem = s_remaining;
+        for (int d = 0; d < 256; ++d) {                  // ascending: the digit that holds the rem-th smallest
+          if (acc + s_hist[d] >= rem) { s_prefix = prefix | ((uint32_t)d << shift); s_remaining = rem - acc; break; }
+          acc += s_hist[d];
+        }
+      }
+      __syncthreads();
     }
+    if (tid == 0) s_q = okey_inv(s_prefix);
     __syncthreads();
     const float qv = s_q;
     // R = values <= q in time order; slope by one thread in float64 (|R| is small)

@@ -179,3 +179,27 @@ def test_trend_only_call_and_ties_at_top_k():
     lens = torch.tensor([512], dtype=torch.int32, device=DEV)
     got_B, got_a, st = _run(None, None, hist, lens, torch.tensor([512], dtype=torch.int32, device=DEV), p)
     assert st[0] == 0 and got_a[0] < 0 and got_B[0] == 896 and lens.cpu().tolist() == [512]
+
+
+def test_trend_on_a_history_of_the_maximum_length():
+    """hist_cap 65536 (the documented maximum): about 8000 pooled windows per request, with runs of equal values
+    (window-min pooling) and values drawn on a coarse grid so that the percentile falls among exact ties; the
+    percentile, the slope and the decision against the oracle run on the same stored history."""
+    cap, R = 65536, 3
+    g = torch.Generator().manual_seed(11)
+    hist = (torch.randint(0, 4000, (R, cap), generator=g).float() / 256.0 + 2.0)
+    hist[1] += torch.linspace(3.0, 0.0, cap)                    # a downward trend
+    hist[2] -= torch.linspace(3.0, 0.0, cap)                    # an upward trend
+    lens = torch.tensor([cap, 60001, 33333], dtype=torch.int32)
+    p = B.BudgetParams.paper_defaults()
+    budget_in = torch.tensor([512, 896, 30000], dtype=torch.int32)
+    hist_dev, lens_dev = hist.clone().to(DEV), lens.clone().to(DEV)
+    got_B, got_a, st = _run(None, None, hist_dev, lens_dev, budget_in.to(DEV), p)
+    assert st[0] == 0 and lens_dev.cpu().tolist() == lens.tolist()
+    op = _oracle_params(p)
+    for r in range(R):
+        Rr = O.trace_confidence(hist[r, :int(lens[r])].numpy(), op.w, op.s, op.b_percent)
+        a = O.fit_slope(Rr)
+        assert abs(got_a[r] - a) <= 1e-12 * max(1.0, abs(a))
+        assert got_B[r] == O.budget_update(int(budget_in[r]), a, op, None)
+    assert got_a[1] < 0 < got_a[2]
