@@ -587,6 +587,8 @@ def run_ours(args):
         lrfu_line = {"ms_per_step": float(tl.item()), "value": world * tokens / (float(tl.item()) * 1e-3), "unit": UNIT,
                      "keepscore_ms": ks, "keepscore_gbs": ks_bytes / (ks * 1e-3) / 1e9,
                      "keepscore_frac_of_hbm_peak": ks_bytes / (ks * 1e-3) / 1e9 / pk["hbm_gbs"],
+                     "keepscore_stage": "keep-score update and TopK in one launch (actkv_keepscore_select); the separate "
+                                        "select stage is empty",
                      "top_p": 0.9, "lambda": 0.5, "n_protect": 512}
         comp.check_status()
 
@@ -726,6 +728,8 @@ def run_ours(args):
                                    if pipelined else "none (one stream)"),
                        "l2": "inputs (KV pool %.1f GB) far larger than the 126 MB L2" % (inst.pool.numel() * 2 / 1e9)},
             "stage_ms": stage_ms, "hbm_roofline_frac_whole_step": hbm_frac_whole,
+            "hbm_roofline_frac_whole_step_of_nominal_8TBs": alg_bytes / (ms_max * 1e-3) / 8e12,
+            "hbm_roofline_target": {"north_star": 0.70, "met": bool(hbm_frac_whole >= 0.70)},
             "with_lse_supplied": lse_supplied_line, "other_step_form": other_line,
             "copy_items_taken_by_score_kernels": ([round(b / a, 3) if a else None for a, b in pipe_stats.cpu().tolist()]
                                                   if pipelined else None),

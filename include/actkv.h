@@ -19,9 +19,12 @@
  *     workspace too small, launch failure).  What only the device can see (a page id out of
  *     range, a free list that is too short) is written to the caller's `status[4]` int32 words:
  *     status[0] = first error code (0 while clean), status[1..2] = where (request / unit,
- *     offending value).  Kernels never trap; an out-of-range page id is replaced by page 0 for
- *     the access and reported.  When the plan step of actkv_compact reports ACTKV_E_NOFREE the
- *     copy and table-update steps of that call do nothing, so pool and tables stay unmodified.
+ *     offending value).  Kernels never trap.  An out-of-range page id met by a score kernel is
+ *     replaced by page 0 for the read and reported; a copy whose source or destination page id is
+ *     out of range is dropped and reported (nothing is read from or written to a page the request
+ *     does not own).  Once status[0] is set, actkv_select and the compaction calls of the same
+ *     step do nothing.  When the plan step of actkv_compact reports ACTKV_E_NOFREE the copy and
+ *     table-update steps of that call do nothing, so pool and tables stay unmodified.
  *   - All indices are int32.  Strides are in ELEMENTS (bf16), the head dimension is contiguous.
  *   - "unit" = one (layer, KV head, request); units are independent in score and select.
  *   - Arrays with a leading layer axis are RELATIVE to `layer_begin`: slab 0 belongs to layer
@@ -264,6 +267,22 @@ int actkv_keep_indptr(const int32_t* seq_len, const int32_t* budget, int32_t n_r
 int actkv_keepscore(float* score, const int32_t* tok_indptr, int32_t sum_tok, int32_t n_outer,
                     int32_t n_req, float top_p, float lambda, const int32_t* n_protect,
                     float* keep_score, uint32_t* hit_mask, int32_t* status, actkv_stream_t stream);
+
+/* ---------------------------------------------------------------------------------------
+ * actkv_keepscore_select — actkv_keepscore and actkv_select in one launch (Algorithm 1 steps 2-5):
+ * the ranking keys (updated keep-scores, +inf on the protected prefix) go straight into TopK
+ * without passing through memory, so the scores are read once.  Same results as the two calls
+ * (keep_score, hit_mask, sel_idx, keep_mask, tie_report), except that `score` is left as it was
+ * when every unit fits in shared memory (max_tok <= 45568 tokens); longer units run the two
+ * stages as two kernels and `score` then holds the ranking keys as after actkv_keepscore.
+ * max_tok: host upper bound on the unit lengths.  Other arguments as the two calls.
+ */
+int actkv_keepscore_select(float* score, const int32_t* tok_indptr, int32_t sum_tok, int32_t max_tok,
+                           int32_t n_outer, int32_t n_req, float top_p, float lambda,
+                           const int32_t* n_protect, float* keep_score, uint32_t* hit_mask,
+                           const int32_t* budget, const int32_t* keep_indptr, int32_t* sel_idx,
+                           int64_t sel_stride, uint32_t* keep_mask, actkv_tie_t* tie_report,
+                           int32_t* status, actkv_stream_t stream);
 
 /* ---------------------------------------------------------------------------------------
  * actkv_gather_f32 — the survivors' keep-scores move with them (Algorithm 1 step 5 returns KS'):

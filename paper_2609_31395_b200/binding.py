@@ -26,7 +26,7 @@ EXPORTS = ["actkv_budget_workspace_bytes", "actkv_budget", "actkv_score_workspac
            "actkv_keep_indptr", "actkv_select_workspace_bytes", "actkv_select",
            "actkv_compact_workspace_bytes", "actkv_compact", "actkv_compact_noalloc",
            "actkv_compact_noalloc_max_bytes", "actkv_step_host", "actkv_keepscore", "actkv_gather_f32",
-           "actkv_compact_inplace", "actkv_score_path", "actkv_debug_inject_stall", "actkv_score_sliding",
+           "actkv_compact_inplace", "actkv_score_path", "actkv_debug_inject_stall", "actkv_score_sliding", "actkv_keepscore_select",
            "actkv_compact_deferred_workspace_bytes", "actkv_compact_begin", "actkv_compact_end", "actkv_score_overlap", "actkv_compact_stats",
            "actkv_version"]
 
@@ -158,6 +158,8 @@ def load():
     lib.actkv_compact_deferred_workspace_bytes.argtypes = [C.POINTER(PoolDesc), i32, i32, i32, i32]
     lib.actkv_compact_stats.restype = i32
     lib.actkv_compact_stats.argtypes = [vp, vp, vp]
+    lib.actkv_keepscore_select.restype = i32
+    lib.actkv_keepscore_select.argtypes = [vp, vp, i32, i32, i32, i32, f32, f32, vp, vp, vp, vp, vp, vp, i64, vp, vp, vp, vp]
     lib.actkv_score_sliding.restype = i32
     lib.actkv_score_sliding.argtypes = [C.POINTER(PoolDesc), C.POINTER(TablesDesc), i32, i32, vp, vp, i32, vp, f32, i32,
                                         i32, vp, vp, vp, i32, i32, i32, i32, vp, sz, vp, vp]
@@ -293,6 +295,19 @@ def actkv_compact_deferred_workspace_bytes(pool: PoolDesc, n_req, max_pages, n_l
 def actkv_compact_stats(ws, stats, stream=None):
     _check("actkv_compact_stats", load().actkv_compact_stats(_ptr(ws, None, "ws"), _ptr(stats, torch.int32, "stats"),
                                                              _stream(stream)))
+
+
+def actkv_keepscore_select(score, tok_indptr, sum_tok, max_tok, n_outer, n_req, top_p, lam, n_protect, keep_score,
+                           hit_mask, budget, keep_indptr, sel_idx, sel_stride, keep_mask, tie_report, status, stream=None):
+    rc = load().actkv_keepscore_select(_ptr(score, torch.float32, "score"), _ptr(tok_indptr, torch.int32, "tok_indptr"),
+                                       sum_tok, max_tok, n_outer, n_req, float(top_p), float(lam),
+                                       _ptr(n_protect, torch.int32, "n_protect"),
+                                       _ptr(keep_score, torch.float32, "keep_score"), _ptr(hit_mask, None, "hit_mask"),
+                                       _ptr(budget, torch.int32, "budget"), _ptr(keep_indptr, torch.int32, "keep_indptr"),
+                                       _ptr(sel_idx, torch.int32, "sel_idx"), sel_stride, _ptr(keep_mask, None, "keep_mask"),
+                                       _ptr(tie_report, None, "tie_report"), _ptr(status, torch.int32, "status"),
+                                       _stream(stream))
+    _check("actkv_keepscore_select", rc)
 
 
 def actkv_score_sliding(pool: PoolDesc, tables: TablesDesc, layer_begin, layer_end, q, win_indptr, n_q_heads, lse_in,

@@ -165,14 +165,19 @@ static int step_enqueue(const actkv_pool_t* pool, const actkv_tables_t* tab, con
     ACTKV_TRY(actkv_select(io->score_dev, io->tok_indptr_dev, io->sum_tok, io->budget_dev, (l1 - l0) * Hkv, R,
                            io->keep_indptr_dev, io->sel_idx_dev, io->sel_stride, nullptr, nullptr, nullptr, 0,
                            io->status_dev, stream));
-    ACTKV_TRY(actkv_compact_begin(pool, tab, l0, l1, io->sel_idx_dev, io->sel_stride, io->keep_indptr_dev, io->budget_dev,
-                                  io->max_keep, g > 0 ? 1 : 0, io->ws_compact, io->ws_compact_bytes, io->status_dev, stream));
-    pl0 = l0;
-    pl1 = l1;
+    if (g == n_groups - 1) {
+      // nothing follows the last group that could carry its copies: the one-launch copy
+      ACTKV_TRY(actkv_compact(pool, tab, l0, l1, io->sel_idx_dev, io->sel_stride, io->keep_indptr_dev, io->budget_dev,
+                              io->max_keep, io->ws_compact, io->ws_compact_bytes, io->status_dev, stream));
+      pl0 = pl1 = -1;
+    } else {
+      ACTKV_TRY(actkv_compact_begin(pool, tab, l0, l1, io->sel_idx_dev, io->sel_stride, io->keep_indptr_dev, io->budget_dev,
+                                    io->max_keep, g > 0 ? 1 : 0, io->ws_compact, io->ws_compact_bytes, io->status_dev,
+                                    stream));
+      pl0 = l0;
+      pl1 = l1;
+    }
   }
-  if (pl0 >= 0)
-    ACTKV_TRY(actkv_compact_end(pool, tab, pl0, pl1, io->sel_idx_dev, io->sel_stride, io->keep_indptr_dev, io->budget_dev,
-                                io->max_keep, io->ws_compact, io->ws_compact_bytes, io->status_dev, stream));
 
   // ---- device -> host: the step's results ----
   ACTKV_TRY(d2h(io->page_table_out_host, tab->page_table, tbl_bytes, s));

@@ -12,7 +12,7 @@
 //      by index are hits (ordered sweep with a block scan, as in select);
 //   4. KS = lambda*KS + score*[hit], one float32 rounding per operation; the score buffer is
 //      overwritten with the ranking key: KS, or +inf for the protected prefix.
-#include "common.cuh"
+#include "select_core.cuh"
 
 namespace actkv {
 
@@ -50,10 +50,25 @@ constexpr size_t KS_SMEM = 232448 - 1024;                              // (nearl
 constexpr int KS_CAP = (int)((KS_SMEM - KS_BINS * 12) / 4);            // keys that fit beside the histogram
 // (chunk sums stay below 2^32 for units of up to 2^17 entries; the total mass needs 2^16 or fewer, see below)
 
+// What the fused form needs of actkv_select's arguments.
+struct FusedSelectArgs {
+  const int32_t* budget;
+  const int32_t* keep_indptr;
+  int32_t* sel_idx;
+  int64_t sel_stride;
+  uint32_t* keep_mask;
+  actkv_tie_t* tie;
+  int32_t* status;
+};
+
+// FUSED: the ranking keys go straight into TopK (the second half of select_kernel, on the keys in shared memory)
+// instead of back to the score array: one read of the scores, one launch.  Every unit must fit in shared memory.
+template <bool FUSED>
 __global__ void __launch_bounds__(KS_NT, 1) keepscore_kernel(
     float* __restrict__ score, const int32_t* __restrict__ tok_indptr, int32_t sum_tok, int32_t n_req,
     int32_t p_q, float lambda, const int32_t* __restrict__ n_protect, float* __restrict__ keep_score,
-    uint32_t* __restrict__ hit_mask) {
+    uint32_t* __restrict__ hit_mask, FusedSelectArgs fs) {
+  static_assert(KS_NT == SEL_NT && KS_BINS == SEL_BINS, "the fused form runs select's second half in this CTA");
   // A mass is below 2^41; its three 14-bit chunks are summed in three 32-bit histograms (native shared
   // atomics; a 64-bit shared atomic is a compare-and-swap loop) and put together when the bins are scanned.
   extern __shared__ __align__(16) uint32_t ks_smem[];
@@ -76,6 +91,17 @@ __global__ void __launch_bounds__(KS_NT, 1) keepscore_kernel(
   const int r = u % n_req, o = u / n_req;
   const int base = tok_indptr[r];
   const int L = tok_indptr[r + 1] - base;
+  int n_keep = 0;
+  if (FUSED) {
+    n_keep = min(max(fs.budget[r], 0), L);
+    // as actkv_select: nothing after an earlier error of the step, and no store past the index buffer
+    if (status_set(fs.status)) return;
+    if ((int64_t)fs.keep_indptr[r] + n_keep > fs.sel_stride) {
+      if (threadIdx.x == 0) report(fs.status, ACTKV_E_INVALID, r, n_keep);
+      return;
+    }
+    if (n_keep == 0 && fs.tie != nullptr && threadIdx.x == 0) fs.tie[u] = actkv_tie_t{0.f, 0, 0, 0};
+  }
   if (L <= 0) return;
   float* sc = score + (int64_t)o * sum_tok + base;
   float* ks = keep_score + (int64_t)o * sum_tok + base;
@@ -174,6 +200,10 @@ __global__ void __launch_bounds__(KS_NT, 1) keepscore_kernel(
   }
 
   // ---- ordered sweep: hits, keep-score update, ranking keys ----
+  if (FUSED) {                                           // the mass histograms are done with: first-digit counts of the ranking keys
+    __syncthreads();
+    for (int i = tid; i < KS_BINS; i += KS_NT) hist[i] = 0u;
+  }
   if (tid == 0) s_carry = 0ull;
   __syncthreads();
   const int np = n_protect ? n_protect[r] : 0;
@@ -213,7 +243,14 @@ __global__ void __launch_bounds__(KS_NT, 1) keepscore_kernel(
         const float decayed = mul_ieee(lambda, ks[i]);
         const float nk = hit ? add_ieee(decayed, x[k]) : decayed;
         ks[i] = nk;
-        sc[i] = (i < np) ? INFINITY : nk;                     // what TopK ranks
+        const float rank = (i < np) ? INFINITY : nk;          // what TopK ranks
+        if (FUSED) {
+          const uint32_t rk = ks_order_key(rank);
+          skeys[i] = rk;
+          atomicAdd(&hist[rk >> 20], 1u);
+        } else {
+          sc[i] = rank;
+        }
         if (hit && mrow) atomicOr(&mrow[(base + i) >> 5], 1u << ((base + i) & 31));
       }
       before += eq[k];
@@ -221,6 +258,11 @@ __global__ void __launch_bounds__(KS_NT, 1) keepscore_kernel(
     __syncthreads();
     if (tid == KS_NT - 1) s_carry = before;
     __syncthreads();
+  }
+  if (FUSED && n_keep > 0) {                             // uniform over the CTA
+    auto rank_key_at = [&](int i) -> uint32_t { return skeys[i]; };
+    select_threshold_and_emit(rank_key_at, hist, L, n_keep, fs.sel_idx + (int64_t)o * fs.sel_stride + fs.keep_indptr[r],
+                              fs.keep_mask ? fs.keep_mask + (int64_t)o * ((sum_tok + 31) / 32) : nullptr, base, fs.tie, u);
   }
 }
 
@@ -256,10 +298,39 @@ int actkv_keepscore(float* score, const int32_t* tok_indptr, int32_t sum_tok, in
   const int64_t units = (int64_t)n_outer * n_req;
   if (units > 0x7fffffffLL) return ACTKV_E_INVALID;
   const int32_t p_q = (int32_t)lrintf(top_p * 10000.f);
-  if (cudaFuncSetAttribute(actkv::keepscore_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)actkv::KS_SMEM) != cudaSuccess)
+  if (cudaFuncSetAttribute(actkv::keepscore_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)actkv::KS_SMEM) != cudaSuccess)
     return ACTKV_E_CUDA;
-  actkv::keepscore_kernel<<<(unsigned)units, actkv::KS_NT, actkv::KS_SMEM, (cudaStream_t)stream>>>(
-      score, tok_indptr, sum_tok, n_req, p_q, lambda, n_protect, keep_score, hit_mask);
+  actkv::keepscore_kernel<false><<<(unsigned)units, actkv::KS_NT, actkv::KS_SMEM, (cudaStream_t)stream>>>(
+      score, tok_indptr, sum_tok, n_req, p_q, lambda, n_protect, keep_score, hit_mask, actkv::FusedSelectArgs{});
+  ACTKV_CHECK_LAUNCH();
+  return ACTKV_OK;
+}
+
+int actkv_keepscore_select(float* score, const int32_t* tok_indptr, int32_t sum_tok, int32_t max_tok, int32_t n_outer,
+                           int32_t n_req, float top_p, float lambda, const int32_t* n_protect, float* keep_score,
+                           uint32_t* hit_mask, const int32_t* budget, const int32_t* keep_indptr, int32_t* sel_idx,
+                           int64_t sel_stride, uint32_t* keep_mask, actkv_tie_t* tie_report, int32_t* status,
+                           actkv_stream_t stream) {
+  if (n_outer < 0 || n_req < 0 || sum_tok < 0 || max_tok < 0 || sel_stride < 0) return ACTKV_E_INVALID;
+  if (!(top_p >= 0.f && top_p <= 1.f) || !(lambda >= 0.f && lambda <= 1.f)) return ACTKV_E_INVALID;
+  if (n_outer == 0 || n_req == 0 || sum_tok == 0) return ACTKV_OK;
+  if (!score || !tok_indptr || !keep_score || !budget || !keep_indptr || !sel_idx) return ACTKV_E_INVALID;
+  if (max_tok > actkv::KS_CAP) {
+    // a unit that does not fit in shared memory: the two stages as two kernels (the ranking keys go through `score`)
+    int rc = actkv_keepscore(score, tok_indptr, sum_tok, n_outer, n_req, top_p, lambda, n_protect, keep_score, hit_mask,
+                             status, stream);
+    if (rc != ACTKV_OK) return rc;
+    return actkv_select(score, tok_indptr, sum_tok, budget, n_outer, n_req, keep_indptr, sel_idx, sel_stride, keep_mask,
+                        tie_report, nullptr, 0, status, stream);
+  }
+  const int64_t units = (int64_t)n_outer * n_req;
+  if (units > 0x7fffffffLL) return ACTKV_E_INVALID;
+  const int32_t p_q = (int32_t)lrintf(top_p * 10000.f);
+  if (cudaFuncSetAttribute(actkv::keepscore_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)actkv::KS_SMEM) != cudaSuccess)
+    return ACTKV_E_CUDA;
+  actkv::FusedSelectArgs fs{budget, keep_indptr, sel_idx, sel_stride, keep_mask, tie_report, status};
+  actkv::keepscore_kernel<true><<<(unsigned)units, actkv::KS_NT, actkv::KS_SMEM, (cudaStream_t)stream>>>(
+      score, tok_indptr, sum_tok, n_req, p_q, lambda, n_protect, keep_score, hit_mask, fs);
   ACTKV_CHECK_LAUNCH();
   return ACTKV_OK;
 }

@@ -6,13 +6,10 @@
 // mantissa, and over the few dozen bins of the populated binades before) finds the n-th largest key
 // exactly; one ordered sweep with a block scan then emits the kept token indices in ascending order,
 // entries equal to the threshold being kept lowest index first.
-#include "common.cuh"
+#include "select_core.cuh"
 
 namespace actkv {
 
-constexpr int SEL_NT = 1024;
-constexpr int SEL_ITEMS = 4;
-constexpr int SEL_BINS = 4096;
 constexpr size_t SEL_SMEM = 232448 - 1024;                            // (nearly) all of an SM's shared memory: one CTA per SM
 constexpr int SEL_CAP = (int)((SEL_SMEM - SEL_BINS * 4) / 4);          // keys that fit beside the histogram
 
@@ -29,11 +26,6 @@ __global__ void __launch_bounds__(SEL_NT, 1) select_kernel(
   extern __shared__ __align__(16) uint32_t sel_smem[];
   uint32_t* hist = sel_smem;                             // [SEL_BINS]
   uint32_t* skeys = sel_smem + SEL_BINS;                 // [SEL_CAP]
-  __shared__ uint32_t warp_tot[SEL_NT / 32];
-  __shared__ uint32_t s_bin, s_remaining, s_eq_total;
-  __shared__ unsigned long long s_carry;
-  __shared__ unsigned long long wsum[SEL_NT / 32];
-
   const int u = blockIdx.x;
   const int r = u % n_req, o = u / n_req;
   const int base = tok_indptr[r];
@@ -93,130 +85,8 @@ __global__ void __launch_bounds__(SEL_NT, 1) select_kernel(
     if (tail0 + tid < L) take(tail0 + tid, sc[tail0 + tid]);
   }
 
-  // ---- radix select: n-th largest key -----------------------------------------------------
-  uint32_t prefix = 0, mask = 0, remaining = (uint32_t)n;
-#pragma unroll 1
-  for (int pass = 0; pass < 3; ++pass) {
-    const int shift = pass == 0 ? 20 : pass == 1 ? 8 : 0;
-    const uint32_t dmask = pass == 2 ? 255u : 4095u;
-    const int n_bins = (int)dmask + 1;
-    if (pass > 0) {
-      for (int i = tid; i < n_bins; i += SEL_NT) hist[i] = 0;
-      __syncthreads();
-      for (int i = tid; i < L; i += SEL_NT) {
-        const uint32_t k = key_at(i);
-        if ((k & mask) == prefix) atomicAdd(&hist[(k >> shift) & dmask], 1u);
-      }
-    }
-    __syncthreads();
-    // suffix sums over the bins, descending: thread t owns bins n_bins-1-4t .. n_bins-4-4t
-    const int per = n_bins / SEL_NT;                     // 4, or 0 for the 256-bin pass (then one bin for tid < 256)
-    uint32_t h[4] = {0, 0, 0, 0}, mine = 0;
-    if (per == 4) {
-#pragma unroll
-      for (int j = 0; j < 4; ++j) { h[j] = hist[n_bins - 1 - 4 * tid - j]; mine += h[j]; }
-    } else if (tid < n_bins) {
-      h[0] = hist[n_bins - 1 - tid];
-      mine = h[0];
-    }
-    uint32_t incl = mine;
-#pragma unroll
-    for (int d = 1; d < 32; d <<= 1) {
-      const uint32_t t = __shfl_up_sync(0xffffffffu, incl, d);
-      if (lane >= d) incl += t;
-    }
-    if (lane == 31) warp_tot[warp] = incl;
-    __syncthreads();
-    if (warp == 0) {                                     // exclusive prefix over the 32 warp totals
-      const uint32_t t = warp_tot[lane];
-      uint32_t in2 = t;
-#pragma unroll
-      for (int d = 1; d < 32; d <<= 1) {
-        const uint32_t y = __shfl_up_sync(0xffffffffu, in2, d);
-        if (lane >= d) in2 += y;
-      }
-      warp_tot[lane] = in2 - t;
-    }
-    __syncthreads();
-    uint32_t acc = incl - mine + warp_tot[warp];         // keys with a digit above this thread's first bin
-    const int first_bin = per == 4 ? n_bins - 1 - 4 * tid : n_bins - 1 - tid;
-#pragma unroll
-    for (int j = 0; j < 4; ++j) {
-      if (acc < remaining && acc + h[j] >= remaining) {  // exactly one bin over all threads crosses
-        s_bin = (uint32_t)(first_bin - j);
-        s_remaining = remaining - acc;
-        s_eq_total = h[j];
-      }
-      acc += h[j];
-    }
-    __syncthreads();
-    prefix |= s_bin << shift;
-    mask |= dmask << shift;
-    remaining = s_remaining;
-    __syncthreads();
-  }
-  const uint32_t thr = prefix;                           // key of the n-th largest score
-  const uint32_t need_eq = remaining;                    // entries equal to it that are kept
-  const uint32_t eq_total = s_eq_total;
-
-  // ---- ordered sweep: emit kept indices ascending ---------------------------------------------
-  if (tid == 0) s_carry = 0ull;
-  __syncthreads();
-  int32_t* out = sel_idx + (int64_t)o * sel_stride + keep_indptr[r];
-  uint32_t* mask_row = keep_mask ? keep_mask + (int64_t)o * ((sum_tok + 31) / 32) : nullptr;
-  for (int c0 = 0; c0 < L; c0 += SEL_NT * SEL_ITEMS) {
-    const int i0 = c0 + tid * SEL_ITEMS;
-    uint32_t gt[SEL_ITEMS], eq[SEL_ITEMS];
-    unsigned long long mine = 0ull;                      // high 32: #greater, low 32: #equal
-#pragma unroll
-    for (int k = 0; k < SEL_ITEMS; ++k) {
-      const int i = i0 + k;
-      uint32_t key = (i < L) ? key_at(i) : 0u;
-      gt[k] = (i < L) && key > thr;
-      eq[k] = (i < L) && key == thr;
-      mine += ((unsigned long long)gt[k] << 32) + eq[k];
-    }
-    unsigned long long incl = mine;
-#pragma unroll
-    for (int d = 1; d < 32; d <<= 1) {
-      unsigned long long t = __shfl_up_sync(0xffffffffu, incl, d);
-      if (lane >= d) incl += t;
-    }
-    if (lane == 31) wsum[warp] = incl;
-    __syncthreads();
-    if (warp == 0) {                                     // exclusive prefix over the 32 warp totals
-      const unsigned long long t = wsum[lane];
-      unsigned long long in2 = t;
-#pragma unroll
-      for (int d = 1; d < 32; d <<= 1) {
-        const unsigned long long y = __shfl_up_sync(0xffffffffu, in2, d);
-        if (lane >= d) in2 += y;
-      }
-      wsum[lane] = in2 - t;
-    }
-    __syncthreads();
-    unsigned long long before = s_carry + wsum[warp] + (incl - mine);
-    uint32_t gt_before = (uint32_t)(before >> 32), eq_before = (uint32_t)before;
-#pragma unroll
-    for (int k = 0; k < SEL_ITEMS; ++k) {
-      const int i = i0 + k;
-      const bool keep = gt[k] || (eq[k] && eq_before < need_eq);
-      if (keep) {
-        const uint32_t pos = gt_before + min(eq_before, need_eq);
-        out[pos] = i;
-        if (mask_row) atomicOr(&mask_row[(base + i) >> 5], 1u << ((base + i) & 31));
-      }
-      gt_before += gt[k];
-      eq_before += eq[k];
-    }
-    __syncthreads();
-    if (tid == SEL_NT - 1) s_carry = before + mine;
-    __syncthreads();
-  }
-  if (tie != nullptr && tid == 0) {
-    uint32_t b = (thr & 0x80000000u) ? (thr & 0x7fffffffu) : ~thr;
-    tie[u] = actkv_tie_t{__uint_as_float(b), (int32_t)need_eq, (int32_t)eq_total, n};
-  }
+  select_threshold_and_emit(key_at, hist, L, n, sel_idx + (int64_t)o * sel_stride + keep_indptr[r],
+                            keep_mask ? keep_mask + (int64_t)o * ((sum_tok + 31) / 32) : nullptr, base, tie, u);
 }
 
 __global__ void keep_indptr_kernel(const int32_t* seq_len, const int32_t* budget, int32_t n_req,

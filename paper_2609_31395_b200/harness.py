@@ -91,6 +91,14 @@ class Compressor:
         B.actkv_keepscore(self.score[: l1 - l0], tok_indptr, s.sum_tok, (l1 - l0) * Hkv, s.n_req, lrfu.top_p, lrfu.lam,
                           lrfu.n_protect, lrfu.keep_score[l0 * Hkv:l1 * Hkv], hit, self.status, stream)
 
+    def run_keepscore_select(self, lrfu: "LrfuState", tok_indptr, budget, l0, l1, stream=None):
+        """Keep-score update and TopK of layers [l0, l1) in one launch (actkv_keepscore_select)."""
+        Hkv, s = self.pd.n_kv_heads, self.sz
+        hit = None if lrfu.hit_mask is None else lrfu.hit_mask[l0 * Hkv:l1 * Hkv]
+        B.actkv_keepscore_select(self.score[: l1 - l0], tok_indptr, s.sum_tok, s.max_tok, (l1 - l0) * Hkv, s.n_req,
+                                 lrfu.top_p, lrfu.lam, lrfu.n_protect, lrfu.keep_score[l0 * Hkv:l1 * Hkv], hit, budget,
+                                 self.keep_indptr, self.sel_idx, s.sel_stride, self.mask, self.ties, self.status, stream)
+
     def run_gather_ks(self, lrfu: "LrfuState", tok_indptr, l0, l1, stream=None, idx=None):
         """Keep-scores of the survivors of layers [l0, l1), packed like the index lists (`idx`: the
         lists to follow, default the ascending ones; after an in-place compaction its new order)."""
@@ -122,11 +130,11 @@ class Compressor:
                           self.status, stream)
 
     def step(self, q, win_indptr, tok_indptr, budget, sm_scale, causal, lse_in=None, stream=None, marks=None,
-             lrfu: Optional["LrfuState"] = None, inplace: bool = False):
+             lrfu: Optional["LrfuState"] = None, inplace: bool = False, fused_lrfu: bool = True):
         """score -> select -> compact over all layers, `layers_per_call` layers at a time.
         Tables are rewritten by the last compact call; earlier calls see the old tables.
         `lrfu`: rank by the attention-aware LRFU keep-score instead of the raw pooled score
-        (score -> keepscore -> select -> gather keep-scores -> compact).
+        (score -> keepscore + select in one launch, or as two with fused_lrfu=False -> gather keep-scores -> compact).
         `inplace`: compact into the tail blocks of each request (Algorithm 4) instead of fresh pages.
         `marks`: optional callable(name) invoked between stages (the benchmark records CUDA events
         there); with it the LSE pass and the pooled-score pass run as two calls so that each can be
@@ -147,10 +155,14 @@ class Compressor:
             else:
                 self.run_score(q, win_indptr, tok_indptr, sm_scale, causal, l0, l1, lse_in, stream)
             mark("score")
-            if lrfu is not None:
-                self.run_keepscore(lrfu, tok_indptr, l0, l1, stream)
+            if lrfu is not None and fused_lrfu:
+                self.run_keepscore_select(lrfu, tok_indptr, budget, l0, l1, stream)
                 mark("keepscore")
-            self.run_select(tok_indptr, budget, l1 - l0, stream)
+            else:
+                if lrfu is not None:
+                    self.run_keepscore(lrfu, tok_indptr, l0, l1, stream)
+                    mark("keepscore")
+                self.run_select(tok_indptr, budget, l1 - l0, stream)
             if lrfu is not None and not inplace:
                 self.run_gather_ks(lrfu, tok_indptr, l0, l1, stream)
             mark("select")
@@ -211,15 +223,17 @@ class Compressor:
                 mark("compact")
             self.run_select(tok_indptr, budget, l1 - l0, stream)
             mark("select")
+            launches += (3 if lse_in is None else 1) + 1 + 1 + 1
+            if l1 == NL:
+                # nothing follows the last group that could carry its copies: the one-launch copy of actkv_compact
+                # (a CTA per destination page) is a little faster than draining a queue
+                self.run_compact(budget, l0, l1, stream)
+                mark("compact")
+                return launches + 2
             B.actkv_compact_begin(self.pd, self.td, l0, l1, self.sel_idx, s.sel_stride, self.keep_indptr, budget,
                                   s.max_keep, self.ws_compact, self.status, stream, reuse_plan=prev is not None)
             prev = (l0, l1)
-            launches += (3 if lse_in is None else 1) + 1 + 1 + 1
-        mark("begin")
-        B.actkv_compact_end(self.pd, self.td, prev[0], prev[1], self.sel_idx, s.sel_stride, self.keep_indptr, budget,
-                            s.max_keep, self.ws_compact, self.status, stream)
-        mark("compact")
-        return launches + 2
+        return launches
 
     def step_overlapped(self, q, win_indptr, tok_indptr, budget, sm_scale, causal, lse_in=None, marks=None):
         """The same step with select + compact of layer group g running on a second stream while

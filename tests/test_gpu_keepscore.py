@@ -242,3 +242,60 @@ def test_lrfu_trace_keepscores_travel_with_the_survivors(inplace):
         ks_gpu_prev = lrfu.kept[:, : int(ki[-1])].clone()
         ks_orc_prev, keep_prev = ks_orc_new, keep
     assert evicted_protected == 0
+
+
+@pytest.mark.parametrize("long_unit", [False, True])
+def test_fused_keepscore_select_matches_oracle_bit_exact(long_unit):
+    """actkv_keepscore_select: keep-score update and TopK in one launch.  Hit masks, keep-scores and index lists
+    bit-exact against the oracle run on the same float32 scores (the ranking keys never pass through memory, so the
+    index lists are held against the oracle's TopK of the oracle's keys); tie report and keep bitmap consistent;
+    with a unit longer than shared memory holds the call falls back to the two kernels and gives the same."""
+    rng = np.random.default_rng(21)
+    lens = [0, 5, 1500, 4096, 9001, 45568] + ([60001] if long_unit else [])
+    budgets = [3, 5, 400, 0, 9001, 12000] + ([15000] if long_unit else [])
+    protect = [0, 2, 100, 0, 5000, 7] + ([20000] if long_unit else [])            # one prefix longer than its budget
+    n_outer, lam, top_p, R = 3, 0.5, 0.9, len(lens)
+    sc, tok = _synthetic_scores(rng, n_outer, lens)
+    ks0 = (rng.random(sc.shape) ** 4).astype(np.float32)
+    ks0[:, ::5] = 0.0
+    sum_tok = int(tok[-1])
+    keep = [min(b, L) for b, L in zip(budgets, lens)]
+    ki = np.concatenate([[0], np.cumsum(keep)]).astype(np.int32)
+    d_sc = torch.from_numpy(sc.copy()).to(DEV)
+    d_ks = torch.from_numpy(ks0.copy()).to(DEV)
+    d_hit = torch.zeros((n_outer, (sum_tok + 31) // 32), dtype=torch.int32, device=DEV)
+    d_keep = torch.zeros_like(d_hit)
+    d_sel = torch.full((n_outer, int(ki[-1])), -1, dtype=torch.int32, device=DEV)
+    d_tie = torch.zeros((n_outer * R, 4), dtype=torch.int32, device=DEV)
+    status = torch.zeros(4, dtype=torch.int32, device=DEV)
+    B.actkv_keepscore_select(d_sc, torch.from_numpy(tok).to(DEV), sum_tok, max(lens), n_outer, R, top_p, lam,
+                             torch.tensor(protect, dtype=torch.int32, device=DEV), d_ks, d_hit,
+                             torch.tensor(budgets, dtype=torch.int32, device=DEV), torch.from_numpy(ki).to(DEV), d_sel,
+                             int(ki[-1]), d_keep, d_tie, status)
+    torch.cuda.synchronize()
+    assert status.cpu().tolist()[0] == 0
+    if not long_unit:
+        assert np.array_equal(_f32_bits(d_sc.cpu().numpy()), _f32_bits(sc)), "the fused form leaves the scores as they were"
+    got_ks, got_hit, got_sel = d_ks.cpu().numpy(), d_hit.cpu().numpy(), d_sel.cpu().numpy()
+    got_keep, got_tie = d_keep.cpu().numpy(), d_tie.cpu().numpy()
+    for o in range(n_outer):
+        for r, L in enumerate(lens):
+            a, b = int(tok[r]), int(tok[r + 1])
+            hit = O.hit_mask_unit(sc[o, a:b], top_p)
+            ks = O.keep_score_update(ks0[o, a:b], sc[o, a:b], hit, lam)
+            want = O.select_unit(O.rank_keys(ks, min(protect[r], L)), budgets[r])
+            assert np.array_equal(_unpack_hits(got_hit[o], a, b), hit), f"hit mask of unit ({o},{r})"
+            assert np.array_equal(_f32_bits(got_ks[o, a:b]), _f32_bits(ks)), f"keep-score of unit ({o},{r})"
+            assert np.array_equal(got_sel[o, ki[r]:ki[r + 1]], want), f"index list of unit ({o},{r})"
+            kept = np.zeros(L, dtype=bool)
+            kept[want] = True
+            assert np.array_equal(_unpack_hits(got_keep[o], a, b), kept)
+            assert got_tie[o * R + r, 3] == keep[r]
+    # a budget the index buffer was not sized for is reported and nothing is stored
+    status.zero_()
+    d_sel.fill_(-7)
+    big = torch.tensor([b + 50 for b in budgets], dtype=torch.int32, device=DEV)
+    B.actkv_keepscore_select(d_sc, torch.from_numpy(tok).to(DEV), sum_tok, max(lens), n_outer, R, top_p, lam, None, d_ks,
+                             None, big, torch.from_numpy(ki).to(DEV), d_sel, int(ki[-1]), None, None, status)
+    torch.cuda.synchronize()
+    assert status.cpu().tolist()[0] == B.E_INVALID

@@ -418,3 +418,32 @@ def test_keep_mask_bitmap():
         for r in range(wl.n_req):
             want[tok[r] + sel[o, ki[r]:ki[r + 1]]] = 1
         assert np.array_equal(bitsv, want)
+
+
+def test_select_reports_a_budget_beyond_the_index_buffer_and_stores_nothing_past_it():
+    """The budgets are device data (they may come straight from actkv_budget, which can scale them up); the host
+    sized the index buffer from what it knew.  A unit whose list would pass the end of its row is reported as
+    ACTKV_E_INVALID before anything is stored, and the guard words behind the buffer keep their pattern."""
+    rng = np.random.default_rng(3)
+    lens, R, n_outer = [300, 500], 2, 3
+    tok = np.array([0, 300, 800], dtype=np.int32)
+    sc = torch.from_numpy(rng.random((n_outer, 800)).astype(np.float32)).to(DEV)
+    sized_for = [100, 120]                                   # what the host sized the buffer for
+    actual = [100, 333]                                      # what the device-side budgets say
+    sel_stride = sum(sized_for)
+    buf = torch.full((n_outer * sel_stride + 64,), -99, dtype=torch.int32, device=DEV)
+    d_budget = torch.tensor(actual, dtype=torch.int32, device=DEV)
+    d_len = torch.tensor(lens, dtype=torch.int32, device=DEV)
+    ki = torch.zeros(R + 1, dtype=torch.int32, device=DEV)
+    status = torch.zeros(4, dtype=torch.int32, device=DEV)
+    B.actkv_keep_indptr(d_len, d_budget, R, ki)
+    ws = torch.empty(256, dtype=torch.uint8, device=DEV)
+    B.actkv_select(sc, torch.from_numpy(tok).to(DEV), 800, d_budget, n_outer, R, ki, buf[: n_outer * sel_stride].view(n_outer, sel_stride),
+                   sel_stride, None, None, ws, status)
+    torch.cuda.synchronize()
+    st = status.cpu().tolist()
+    assert st[0] == B.E_INVALID and st[1] == 1 and st[2] == 333
+    assert bool((buf[n_outer * sel_stride:] == -99).all())
+    # the request that fits was either written whole or, once the error was seen, not at all; never past its row
+    rows = buf[: n_outer * sel_stride].view(n_outer, sel_stride).cpu().numpy()
+    assert (rows[:, 100:] == -99).all()
