@@ -127,9 +127,6 @@ static int score_impl(int mode, const actkv_pool_t* pool, const actkv_tables_t* 
   a.win_left = window_left;
   a.acc_steps = acc_steps;
   const int64_t units = (int64_t)nls * Hkv * R;
-  // (the streaming update keeps a running mean in place, which the row-group launches of a window above
-  // 512 rows would break: such calls take the FMA path)
-
   const float* lse = lse_in;
   if (mode & 1) {
     float* lse_buf = lse_out ? lse_out : (float*)((char*)ws + lay.lse_off);
@@ -225,9 +222,7 @@ int actkv_score_path(const actkv_pool_t* pool, int32_t n_q_heads, int32_t max_wi
                      int32_t streaming) {
   if (!pool || pool->n_kv_heads <= 0 || n_q_heads <= 0 || n_q_heads % pool->n_kv_heads != 0) return ACTKV_E_INVALID;
   const int G = n_q_heads / pool->n_kv_heads;
-  const bool tcp = actkv::score_tc_supported(pool, G, max_win, sm_scale, q, streaming ? 1 : 64) &&
-                   !(streaming && max_win * actkv::tc::pow2_at_least(G) > actkv::tc::MAX_ROWS);
-  return tcp ? 1 : 0;
+  return actkv::score_tc_supported(pool, G, max_win, sm_scale, q, streaming ? 1 : 64) ? 1 : 0;
 }
 
 int actkv_debug_inject_stall(int32_t after_tile, int32_t wait_limit_us) {

@@ -285,7 +285,9 @@ score_tc_pool_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_cons
     const int wg = (warp - POOL_EPI_WARP0) >> 2;
     const int quarter = warp & 3;                 // TMEM lane quarter this warp may read
     const float c = a.scale_log2;
-    const float inv_w = 1.0f / (float)W;
+    // divisor of the mean: this call's W action tokens, plus, in the streaming form, the n already folded in (the
+    // first row group of a window forms (n Out + S) / (n + W) in store_pooled, later row groups add their S / (n + W))
+    const float inv_w = 1.0f / (float)(W + (a.acc_steps != nullptr ? a.acc_steps[r] : 0));
     float* out = a.score_out + ((int64_t)slab * Hkv + h) * a.sum_tok + a.tok_indptr[r];
     const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16);
     float acc = 0.f;

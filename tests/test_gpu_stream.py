@@ -163,3 +163,21 @@ def test_region_entry_ignores_old_state_and_argument_errors():
                              inst.tok_indptr, steps, score_io, 0, 0, sz.sum_tok, sz.max_tok, comp.ws_score, comp.status)
     torch.cuda.synchronize()
     assert (score_io == 0).all() and comp.status.cpu().tolist()[0] == 0
+
+
+def test_more_than_512_rows_per_call_on_the_tensor_core_path():
+    """75 queries x 8 heads = 600 window rows per call: the pooled-score kernel takes them in row groups of 512, the
+    first forming the running mean, the second adding its share with the same divisor; second call with 75 queries
+    already folded in."""
+    wl = synth.Workload("stream600", 2, 2, 8, [1500, 700, 333], [150, 75, 9], [400, 200, 100], causal=True,
+                        table_style="fragmented", seed=23, poison_tail=True)
+    inst = synth.generate(wl, DEV)
+    pd = B.pool_desc(inst.pool)
+    assert B.actkv_score_path(pd, wl.n_q_heads, 75, wl.sm_scale, inst.q, streaming=True) == 1
+    comp, score_io, n_calls = _run_stream(inst, chunk=75)
+    assert n_calls == 2
+    got = score_io.cpu().numpy()
+    want = _oracle_stream_all(inst, U.bits(inst.pool), comp.lse.cpu().numpy())
+    m = want > 0
+    assert U.max_rel(got[m], want[m]) <= U.SCORE_RTOL
+    assert not got[want == 0].any()
