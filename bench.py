@@ -477,6 +477,11 @@ def run_ours(args):
         ach = n_exp / (stage_ms["lse"] * 1e-3) / 1e9
         lse_exp = {"bound": "alu", "achieved": ach, "peak": exp_peak, "unit": "Gexp2/s", "frac": ach / exp_peak,
                    "kernel": "lse", "peak_source": "148 SMs x 16 MUFU results per clock x the maximum SM clock"}
+        if clocks.get("sm_mhz"):
+            # the same against the clock the SMs actually ran at under the power cap (median of the samples taken
+            # during the timed region, all phases of the step): how close the kernel is to the unit's limit there
+            lse_exp["frac_at_sampled_clock"] = ach / (148 * 16 * clocks["sm_mhz"] * 1e6 / 1e9)
+            lse_exp["sampled_sm_mhz"] = clocks["sm_mhz"]
 
     # ---- end to end: host buffers in, host results out, every step -------------------------------
     e2e = None
