@@ -45,3 +45,23 @@ def test_binding_refuses_cpu_tensors():
     with pytest.raises(TypeError):
         B.actkv_keep_indptr(torch.zeros(2, dtype=torch.int32), torch.zeros(2, dtype=torch.int32), 2,
                             torch.zeros(3, dtype=torch.int32))
+
+
+def test_host_side_checks_of_the_newer_entry_points_run_without_a_gpu():
+    import ctypes as C
+    lib = B.load()
+    pd = B.PoolDesc(1, 48, 1000, 16, 4, 128, 1, 1, 1, 1, 1)
+    base = lib.actkv_compact_workspace_bytes(8, 2188)
+    d1 = B.actkv_compact_deferred_workspace_bytes(pd, 8, 2188, 1, 9100)
+    d16 = B.actkv_compact_deferred_workspace_bytes(pd, 8, 2188, 16, 9100)
+    # base + one 32-entry table row per item: ceil(9100 / 16) pages x 8 requests x layers x (16 x 4 / 32) parts
+    assert d1 >= base + 569 * 8 * 2 * 128 and d16 >= base + 16 * 569 * 8 * 2 * 128 and d16 < base + 17 * 569 * 8 * 2 * 128 + 4096
+    # the fault-injection hook validates its arguments on the host
+    assert lib.actkv_debug_inject_stall(3, 0) == B.E_INVALID
+    assert lib.actkv_debug_inject_stall(-1, 0) == 0
+    # null descriptors are refused before anything is launched
+    null = C.c_void_p(None)
+    assert lib.actkv_compact_begin(None, None, 0, 1, null, 0, null, null, 0, 0, null, 0, null, null) == B.E_INVALID
+    assert lib.actkv_compact_end(None, None, 0, 1, null, 0, null, null, 0, null, 0, null, null) == B.E_INVALID
+    assert lib.actkv_compact_stats(null, null, null) == B.E_INVALID
+    assert lib.actkv_score_path(None, 32, 64, 0.1, null, 0) == B.E_INVALID
