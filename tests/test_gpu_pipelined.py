@@ -116,3 +116,34 @@ def test_begin_plus_end_is_compact_and_errors_leave_everything_untouched():
     torch.cuda.synchronize()
     comp.check_status()
     _same_state(a, b)
+
+
+@pytest.mark.parametrize("deferred", [False, True])
+def test_a_bad_page_id_in_a_table_stops_the_compaction_before_anything_is_modified(deferred):
+    """A page id outside the pool in a page table (of a page that holds evicted tokens only, so that no copy would
+    ever read it): reported by the plan, which checks every page it would push on the free list; pool, tables and
+    free list stay as they were."""
+    wl = synth.Workload("badpage", 2, 2, 4, [900, 333], [16, 8], [250, 100], table_style="fragmented", seed=55,
+                        poison_tail=True)
+    b = synth.generate(wl, DEV)
+    comp = H.Compressor(b.pool, b.page_table, b.seq_len, b.free_list, b.free_count, wl.n_q_heads, H.sizes_of(b))
+    B.actkv_keep_indptr(b.seq_len, b.budget, wl.n_req, comp.keep_indptr)
+    comp.run_score(b.q, b.win_indptr, b.tok_indptr, wl.sm_scale, wl.causal)
+    comp.run_select(b.tok_indptr, b.budget, wl.n_layers)
+    torch.cuda.synchronize()
+    comp.check_status()
+    b.page_table[1, 3] = b.pool.shape[2] + 5                       # out of range
+    snap = [U.bits(b.pool).copy()] + [t.clone() for t in (b.page_table, b.seq_len, b.free_list, b.free_count)]
+    args = (comp.pd, comp.td, 0, wl.n_layers, comp.sel_idx, comp.sz.sel_stride, comp.keep_indptr, b.budget,
+            comp.sz.max_keep, comp.ws_compact, comp.status)
+    if deferred:
+        B.actkv_compact_begin(*args)
+        B.actkv_compact_end(*args)
+    else:
+        B.actkv_compact(*args)
+    torch.cuda.synchronize()
+    st = comp.status.cpu().tolist()
+    assert st[0] == B.E_BADPAGE and st[1] == 1 and st[2] == b.pool.shape[2] + 5
+    assert np.array_equal(U.bits(b.pool), snap[0])
+    for t, s0 in zip((b.page_table, b.seq_len, b.free_list, b.free_count), snap[1:]):
+        assert torch.equal(t, s0)
