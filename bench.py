@@ -323,7 +323,7 @@ def run_ours(args):
         comp.status.zero_()
 
     lse_supplied = None
-    # The timed step hides the compaction of a layer group under the score kernels of the next group
+    # The timed step hides the compaction of a layer group under the pooled-score kernel of the next group
     # (actkv_compact_begin / actkv_score_overlap / actkv_compact_end) unless --pipeline none; the other form
     # (one score, one select and one compact call over all layers) is timed as a secondary line.
     pipelined = pipe_groups is not None and not args.overlap
@@ -728,7 +728,7 @@ def run_ours(args):
                        "layers_per_call": pipe_comp.lpc if pipelined else comp.lpc, "replicas": world,
                        "overlap": "select+compact of a layer group on a second stream under the score kernels "
                                   "of the next group" if args.overlap else
-                                  ("copies of a layer group inside the score kernels of the next one, groups of "
+                                  ("copies of a layer group inside the pooled-score kernel of the next one, groups of "
                                    + "+".join(str(l1 - l0) for l0, l1 in pipe_groups) + " layers (one stream)"
                                    if pipelined else "none (one stream)"),
                        "l2": "inputs (KV pool %.1f GB) far larger than the 126 MB L2" % (inst.pool.numel() * 2 / 1e9)},
@@ -766,7 +766,7 @@ def main():
                     help="run select + compact of a layer group on a second stream under the score kernels of the "
                          "next group (measured: no gain, the score CTAs fill the register file of every SM)")
     ap.add_argument("--pipeline", default="auto",
-                    help="layer groups of the timed step, whose copies run inside the score kernels of the next group: "
+                    help="layer groups of the timed step, whose copies run inside the pooled-score kernel of the next group: "
                          "'auto' (three equal groups), comma-separated group sizes, or 'none' (one call per stage)")
     ap.add_argument("--lse", default="internal", choices=["internal", "supplied"])
     ap.add_argument("--all-configs", action="store_true",

@@ -345,10 +345,10 @@ int actkv_compact(const actkv_pool_t* pool /* host */, const actkv_tables_t* tab
  * (Section 3.3: the three primitives are independent per layer; Section 7.2 / Algorithm 4: the
  *  copies of a planned compaction are order-free, their sources and destinations disjoint.)
  *
- * The score kernels are bound by the tensor pipe and leave most of the HBM bandwidth idle; the
+ * The pooled-score kernel is bound by the tensor pipe and leaves most of the HBM bandwidth idle; the
  * copy of a compaction is bound by HBM and needs no tensor pipe.  A step over many layers can
  * therefore run, for layer groups g = 0, 1, ...:
- *     actkv_score_overlap(group g, pending = ws)   score of g; spare warps of its kernels copy rows of g-1
+ *     actkv_score_overlap(group g, pending = ws)   score of g; spare warps of its pooled-score kernel copy rows of g-1
  *     actkv_compact_end(group g-1, ws)             copies whatever is left of g-1 (+ tables after the last layer)
  *     actkv_select(group g)
  *     actkv_compact_begin(group g, ws)             plan of g, published as a work queue in ws; copies nothing
@@ -366,9 +366,10 @@ int actkv_compact(const actkv_pool_t* pool /* host */, const actkv_tables_t* tab
  *   between; the plan does not depend on the layers), so only the job of this layer range is recorded.
  * actkv_score_overlap: actkv_score with one more argument, pending_compact_ws: the workspace of a
  *   begun compaction of OTHER layers of the same pool, or NULL (then it is actkv_score).  The
- *   result of the score does not depend on it.  On the tensor-core path four spare warps per CTA take
- *   items (one destination page of one request and layer) of the pending job from a queue for as
- *   long as their CTA is scoring; the FMA path ignores the argument.
+ *   result of the score does not depend on it.  On the tensor-core path four spare warps per CTA of the
+ *   pooled-score kernel take items (32 (slot, head) pairs of one destination page of one request and
+ *   layer) of the pending job from a queue for as long as their CTA is scoring; the LSE kernel (whose
+ *   epilogue needs every register of the SM) and the FMA path take none.
  * actkv_compact_end: the same arguments as the actkv_compact_begin it closes.  Copies every item
  *   not yet taken, then, when layer_end == pool->n_layers, updates the tables as actkv_compact does.
  * begin + end without a score call in between equals actkv_compact.  Pools the item copy does not

@@ -4,8 +4,8 @@
 // request in one layer: the K row and the V row of each (16 KB in, 16 KB out at head_dim 128).  Because the copies are order-free and touch nothing the
 // score kernels read or write (sources: old pages of layers already scored and selected; destinations:
 // pages still on the free list), any warp of any kernel may execute items: the spare warps of the
-// tensor-core score kernels of the NEXT layer group do (their kernels leave most of the HBM bandwidth
-// idle), and a drain kernel takes whatever is left.
+// tensor-core pooled-score kernel of the NEXT layer group do (it leaves most of the HBM bandwidth idle),
+// and a drain kernel takes whatever is left.
 #pragma once
 
 #include "common.cuh"

@@ -131,7 +131,7 @@ static int score_impl(int mode, const actkv_pool_t* pool, const actkv_tables_t* 
   if (mode & 1) {
     float* lse_buf = lse_out ? lse_out : (float*)((char*)ws + lay.lse_off);
     if (use_tc) {
-      int rc = score_tc_launch_lse(a, pool, max_tok, max_win, s, (CompactWs*)copy_ws);
+      int rc = score_tc_launch_lse(a, pool, max_tok, max_win, s);
       if (rc != ACTKV_OK) return rc;
     } else {
       const int64_t grid1 = units * a.n_chunks;

@@ -161,16 +161,18 @@ inline bool score_tc_supported(const actkv_pool_t* p, int G, int max_win, float 
 inline int score_tc_launch_lse_c(const CUtensorMap& kmap, const tc::TcArgs& ta, unsigned grid, size_t smem, cudaStream_t s) {
   constexpr int NPOLY = tc::LSE_NPOLY;
   const bool rgs = ta.n_rg > 1, d64 = ta.a.pool.head_dim == 64;
-  auto kern = rgs ? (d64 ? tc::score_tc_lse_kernel<NPOLY, true, 1> : tc::score_tc_lse_kernel<NPOLY, true, 2>)
-                  : (d64 ? tc::score_tc_lse_kernel<NPOLY, false, 1> : tc::score_tc_lse_kernel<NPOLY, false, 2>);
+  const bool win = ta.a.win_left > 0;
+  auto kern = win ? (rgs ? (d64 ? tc::score_tc_lse_kernel<NPOLY, true, 1, true> : tc::score_tc_lse_kernel<NPOLY, true, 2, true>)
+                         : (d64 ? tc::score_tc_lse_kernel<NPOLY, false, 1, true> : tc::score_tc_lse_kernel<NPOLY, false, 2, true>))
+                  : (rgs ? (d64 ? tc::score_tc_lse_kernel<NPOLY, true, 1, false> : tc::score_tc_lse_kernel<NPOLY, true, 2, false>)
+                         : (d64 ? tc::score_tc_lse_kernel<NPOLY, false, 1, false> : tc::score_tc_lse_kernel<NPOLY, false, 2, false>));
   if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return ACTKV_E_CUDA;
   kern<<<grid, tc::LSE_THREADS, smem, s>>>(kmap, ta);
   ACTKV_CHECK_LAUNCH();
   return ACTKV_OK;
 }
 
-inline int score_tc_launch_lse(ScoreArgs& a, const actkv_pool_t* pool, int max_tok, int max_win, cudaStream_t s,
-                               CompactWs* copy_ws) {
+inline int score_tc_launch_lse(ScoreArgs& a, const actkv_pool_t* pool, int max_tok, int max_win, cudaStream_t s) {
   (void)max_tok;
   CUtensorMap kmap, qmap;
   if (!tc::make_maps(pool, a.q, a.n_layers_sub, a.sum_win, a.n_q_heads, a.group, &kmap, &qmap)) return ACTKV_E_CUDA;
@@ -182,7 +184,7 @@ inline int score_tc_launch_lse(ScoreArgs& a, const actkv_pool_t* pool, int max_t
   ta.n_stages = 6;
   ta.tiles_per_cta = 0;
   ta.n_kchunks = 0;
-  ta.copy_ws = copy_ws;
+  ta.copy_ws = nullptr;              // (this kernel has no copy role)
   tc::apply_hook(ta);
   const int64_t units = (int64_t)a.n_layers_sub * a.pool.n_kv_heads * a.tab.n_req;
   const int64_t grid = units * a.n_chunks * ta.n_rg;

@@ -97,10 +97,13 @@ __device__ __forceinline__ void lse_slow32(const float* v, int n_lo, int nv, flo
 }
 
 constexpr int LSE_EPI_WARPS = 16;                // (TMEM lane quarter, accumulator, column half)
-constexpr int LSE_COPY_WARPS = 1;                // copy role (items of a pending compaction, when the launch carries one);
-                                                 // 20 warps of 96 registers are what the register file holds
-constexpr int LSE_COPY_WARP0 = 3 + LSE_EPI_WARPS;
-constexpr int LSE_THREADS = (3 + LSE_EPI_WARPS + LSE_COPY_WARPS) * 32;     // producer, two MMA issuers, epilogue, copy
+// Warp 0 is the producer, warps 1 and 2 the MMA issuers, warps 3..18 the epilogue: 19 warps leave each thread 104
+// registers.  The epilogue is sensitive to that: with a 20th warp (tried: a copy role for the items of a pending
+// compaction, as in the pooled-score kernel) the allocation is 96 and the pass 7-9 % slower, also when the
+// epilogue warpgroups take their 104 back from the control warps at run time; what the copies gained by hiding
+// under this kernel was less than that.
+constexpr int LSE_EPI_WARP0 = 3;
+constexpr int LSE_THREADS = (LSE_EPI_WARP0 + LSE_EPI_WARPS) * 32;
 constexpr int LSE_SLOTS = 2;                     // accumulators
 constexpr int LSE_A_COLS = 256;                  // TMEM columns holding the four Q blocks
 constexpr float LSE_BIG = 1099511627776.f;       // 2^40: a partial sum beyond it moves the reference
@@ -114,8 +117,6 @@ struct LseBarriers {
   uint64_t drained[2];
   uint32_t tmem_base;
   int abort_flag;
-  int prod_done;               // the producer has issued its last key tile: the copy role takes no more items
-  int pad;
   float2 state[2][4][2][128];  // (reference, sum) per (group, row block, column half, row in block)
 };
 
@@ -137,7 +138,9 @@ __device__ __forceinline__ int sel4(const int (&x)[4], int i) { return i == 0 ? 
 //   nv_min  visible columns (from the warp's first column) of the most restricted row of this thread
 //   nlo_max columns (from the warp's first column) below the first visible key of the most restricted row
 //   jm, jl  last / first visible key of this thread's row in each row block; key0 = key of the warp's first column
-template <int NPOLY>
+// WIN: the layer has a sliding window (a first visible key per row); kept out of the common instantiation, whose
+// epilogue should not carry the second bound.
+template <int NPOLY, bool WIN>
 __device__ __forceinline__ bool lse_job(LseBarriers* bars, volatile int* abort_flag, uint32_t tq, int grp, int job,
                                         int mb, float2* st, int nv_min, int nlo_max, const int (&jm)[4], const int (&jl)[4],
                                         int key0, float c, float c1, int lane, long long wait_cycles) {
@@ -153,7 +156,7 @@ __device__ __forceinline__ bool lse_job(LseBarriers* bars, volatile int* abort_f
   tc_fence_before();
   __syncwarp();
   if (lane == 0) mbar_arrive(smem_u32(&bars->tmem_empty[grp]));
-  bool slow = __any_sync(0xffffffffu, nv_min < 64 || nlo_max > 0 || ms.x == -INFINITY);
+  bool slow = __any_sync(0xffffffffu, nv_min < 64 || (WIN && nlo_max > 0) || ms.x == -INFINITY);
   if (!slow) {
     const float nmc = -ms.x * c, c0 = fmaf(nmc, 1.f / 252.f, 0.5f);
     const float ps = lse_fast32<NPOLY>(va, c, nmc, c1, c0) + lse_fast32<NPOLY>(vb, c, nmc, c1, c0);
@@ -161,7 +164,7 @@ __device__ __forceinline__ bool lse_job(LseBarriers* bars, volatile int* abort_f
     if (!slow) ms.y += ps;
   }
   if (slow) {
-    const int nv = sel4(jm, mb) - key0 + 1, nlo = sel4(jl, mb) - key0;
+    const int nv = sel4(jm, mb) - key0 + 1, nlo = WIN ? sel4(jl, mb) - key0 : 0;
     lse_slow32(va, nlo, nv, c, ms.x, ms.y);
     lse_slow32(vb, nlo - 32, nv - 32, c, ms.x, ms.y);
   }
@@ -172,7 +175,7 @@ __device__ __forceinline__ bool lse_job(LseBarriers* bars, volatile int* abort_f
 // ROW_GROUPS: the unit's window has more than MAX_ROWS rows and the grid has a row-group dimension (kept
 // out of the common instantiation, whose code should not change with it).
 // NH: 64-dim halves of the head dimension (head_dim = 64 NH); a K tile is NH x [128 keys][64 bf16].
-template <int NPOLY, bool ROW_GROUPS, int NH>
+template <int NPOLY, bool ROW_GROUPS, int NH, bool WIN>
 __global__ void __launch_bounds__(LSE_THREADS, 1)
 score_tc_lse_kernel(const __grid_constant__ CUtensorMap kmap, const TcArgs ta) {
   extern __shared__ __align__(1024) uint8_t smem[];
@@ -201,7 +204,7 @@ score_tc_lse_kernel(const __grid_constant__ CUtensorMap kmap, const TcArgs ta) {
   const int n_mb = (rows + 127) / 128;                   // 1..4
   const int t_end = min((L + TK - 1) / TK, key_begin / TK + a.lse_chunk / TK);
   // sliding-window layer: key tiles below the first key any row of the unit sees are not fetched at all
-  const int lo_all = a.win_left > 0 ? max(0, (a.causal ? L - W : L - 1) - a.win_left + 1) : 0;
+  const int lo_all = (WIN && a.win_left > 0) ? max(0, (a.causal ? L - W : L - 1) - a.win_left + 1) : 0;
   const int t_begin = max(key_begin / TK, lo_all / TK);
   const int n_tiles = t_end - t_begin;
   if (n_tiles <= 0) {                                    // no row sees a key of this chunk
@@ -232,7 +235,6 @@ score_tc_lse_kernel(const __grid_constant__ CUtensorMap kmap, const TcArgs ta) {
     mbar_init(smem_u32(&bars->drained[0]), 1);
     mbar_init(smem_u32(&bars->drained[1]), 1);
     bars->abort_flag = 0;
-    bars->prod_done = 0;
     fence_barrier_init();
   }
   if (warp == 1) {
@@ -245,7 +247,7 @@ score_tc_lse_kernel(const __grid_constant__ CUtensorMap kmap, const TcArgs ta) {
   const uint32_t tmem_base = bars->tmem_base;
 
   // epilogue identity (also used after the role split)
-  const int ew = warp - 3;                       // 0..15 for epilogue warps
+  const int ew = warp - LSE_EPI_WARP0;           // 0..15 for epilogue warps
   const int quarter = warp & 3;                  // TMEM lanes this warp may touch
   const int k = ew >> 2;                         // 0..3
   const int grp = k >> 1;                        // accumulator / job parity this warp serves
@@ -259,18 +261,7 @@ score_tc_lse_kernel(const __grid_constant__ CUtensorMap kmap, const TcArgs ta) {
     // (one producer: this pass needs a K tile per four jobs, far below what one warp delivers)
     if (ta.k5) k_tile_producer<true, NH>(&kmap, a, bars, k_smem, S, r, h, layer, L, t_begin, n_tiles, lane, abort_flag, 0, 1, ta.wait_cycles, ta.stall_tile);
     else k_tile_producer<false, NH>(&kmap, a, bars, k_smem, S, r, h, layer, L, t_begin, n_tiles, lane, abort_flag, 0, 1, ta.wait_cycles, ta.stall_tile);
-    if (lane == 0) bars->prod_done = 1;
-  } else if (warp >= LSE_COPY_WARP0) {
-    // ---------------- copy role: items of the pending compaction of another layer group ----------------
-    // Order-free copies between pages this kernel neither reads nor writes (Section 7.2), on the HBM
-    // bandwidth this pass leaves idle.  Items are taken until the producer has issued the CTA's last key tile.
-    volatile int* done = &bars->prod_done;
-    cj_copy_role<NH + 2, 16>(ta.copy_ws, lane, [&]() {
-      int go = 0;
-      if (lane == 0) go = (!*done && !*abort_flag) ? 1 : 0;
-      return __shfl_sync(0xffffffffu, go, 0) != 0;
-    });
-  } else if (warp <= 2) {
+  } else if (warp < LSE_EPI_WARP0) {
     // ---------------- MMA issuers: A = Q block in TMEM, B = K tile in shared memory ----------------
     // Two warps, one per accumulator: warp 1 issues the even jobs into accumulator 0, warp 2 the odd jobs
     // into accumulator 1.  Issuing is not free for the issuing thread (measured: about 50 cycles per
@@ -356,7 +347,7 @@ score_tc_lse_kernel(const __grid_constant__ CUtensorMap kmap, const TcArgs ta) {
     for (int mb = 0; mb < 4; ++mb) {
       const int n = mb * 128 + rib;
       jm[mb] = (a.causal && n < rows) ? (L - W + (row0 + n) / G) : (L - 1);
-      jl[mb] = (a.win_left > 0 && n < rows) ? max(0, jm[mb] - a.win_left + 1) : 0;
+      jl[mb] = (WIN && a.win_left > 0 && n < rows) ? max(0, jm[mb] - a.win_left + 1) : 0;
       bars->state[grp][mb][half][rib] = make_float2(-INFINITY, 0.f);
     }
     const int jfast = min(min(jm[0], jm[1]), min(jm[2], jm[3]));
@@ -367,7 +358,7 @@ score_tc_lse_kernel(const __grid_constant__ CUtensorMap kmap, const TcArgs ta) {
     int mb = grp % n_mb, key0 = (t_begin + grp / n_mb) * TK + half * 64;
     const int mb_step = 2 % n_mb, tile_step = 2 / n_mb;
     for (int job = grp; job < n_jobs; job += 2) {
-      epi_ok = lse_job<NPOLY>(bars, abort_flag, tq, grp, job, mb, &bars->state[grp][mb][half][rib], jfast - key0 + 1,
+      epi_ok = lse_job<NPOLY, WIN>(bars, abort_flag, tq, grp, job, mb, &bars->state[grp][mb][half][rib], jfast - key0 + 1,
                               jlmax - key0, jm, jl, key0, c, c1, lane, ta.wait_cycles);
       if (!epi_ok) break;
       mb += mb_step;
@@ -378,7 +369,7 @@ score_tc_lse_kernel(const __grid_constant__ CUtensorMap kmap, const TcArgs ta) {
   // ---------------- teardown ----------------
   tc_fence_before();
   __syncthreads();
-  if (warp >= 3 && warp < LSE_COPY_WARP0 && k == 0 && !*abort_flag) {
+  if (warp >= LSE_EPI_WARP0 && k == 0 && !*abort_flag) {
     // merge the four shares (group, column half) of each row, store (reference in log2 units, sum); (-inf, 0) when the
     // row saw no key of this chunk
     const float c = a.scale_log2;
