@@ -218,18 +218,21 @@ class Compressor:
                 if stats is not None:
                     B.actkv_compact_stats(self.ws_compact, stats[len(done)], stream)
                     done.append(prev)
+                    launches += 1
+                launches += 1                       # the drain kernel
                 B.actkv_compact_end(self.pd, self.td, prev[0], prev[1], self.sel_idx, s.sel_stride, self.keep_indptr,
                                     budget, s.max_keep, self.ws_compact, self.status, stream)
                 mark("compact")
             self.run_select(tok_indptr, budget, l1 - l0, stream)
             mark("select")
-            launches += (3 if lse_in is None else 1) + 1 + 1 + 1
+            launches += (3 if lse_in is None else 1) + 1      # score kernels, select
             if l1 == NL:
                 # nothing follows the last group that could carry its copies: the one-launch copy of actkv_compact
                 # (a CTA per destination page) is a little faster than draining a queue
                 self.run_compact(budget, l0, l1, stream)
                 mark("compact")
-                return launches + 2
+                return launches + 3                 # plan, copy, finalize
+            launches += 2                           # plan (or the job record when the plan is reused), resolve
             B.actkv_compact_begin(self.pd, self.td, l0, l1, self.sel_idx, s.sel_stride, self.keep_indptr, budget,
                                   s.max_keep, self.ws_compact, self.status, stream, reuse_plan=prev is not None)
             prev = (l0, l1)
