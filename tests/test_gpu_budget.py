@@ -48,7 +48,8 @@ def _compare(logits, tok, hist0, len0, budget_in, params, seq_len=None):
     gl = hist_len.cpu().numpy()
     assert np.array_equal(gl, ol)
     for r in range(R):
-        assert np.abs(gh[r, :gl[r]].astype(np.float64) - oh[r, :ol[r]]).max() <= T_ATOL
+        if gl[r]:
+            assert np.abs(gh[r, :gl[r]].astype(np.float64) - oh[r, :ol[r]]).max() <= T_ATOL
     # the decision part on the GPU's own stored history must match the oracle exactly
     borderline = 0
     for r in range(R):
@@ -203,3 +204,41 @@ def test_trend_on_a_history_of_the_maximum_length():
         assert abs(got_a[r] - a) <= 1e-12 * max(1.0, abs(a))
         assert got_B[r] == O.budget_update(int(budget_in[r]), a, op, None)
     assert got_a[1] < 0 < got_a[2]
+
+
+@pytest.mark.parametrize("seed", range(16))
+def test_random_monitor_calls(seed):
+    """Seeded random calls: ragged row counts per request (some with none), vocabularies that are not multiples
+    of the vector width, k from 1 to above the single-sweep limit, window / stride / percentile / scale drawn,
+    a history that already holds entries, clamps on or off; history, slope and decision against the oracle."""
+    rng = np.random.default_rng(9000 + seed)
+    R = int(rng.integers(1, 8))
+    V = int(rng.choice([37, 130, 1000, 4099, 32003, 151936]))
+    rows = [int(rng.choice([0, rng.integers(1, 30), rng.integers(30, 200)])) for _ in range(R)]
+    if V > 30000:
+        rows = [min(t, 60) for t in rows]
+    if sum(rows) == 0:
+        rows[0] = 5
+    tok = torch.tensor(np.concatenate([[0], np.cumsum(rows)]), dtype=torch.int32, device=DEV)
+    g = torch.Generator(device=DEV).manual_seed(9100 + seed)
+    sharp = torch.tensor(rng.uniform(0.3, 5.0, size=sum(rows)), dtype=torch.float32, device=DEV)
+    logits = torch.randn((sum(rows), V), generator=g, device=DEV) * sharp[:, None]
+    if rng.integers(0, 3) == 0:                                   # a few rows in adversarial order
+        n = min(3, sum(rows))
+        logits[:n] = torch.sort(logits[:n], dim=1).values
+    cap = int(rng.choice([256, 512, 1024]))
+    len0 = torch.tensor([int(rng.integers(0, cap - max(rows) + 1)) if rng.integers(0, 2) else 0 for _ in range(R)],
+                        dtype=torch.int32)
+    hist0 = torch.zeros((R, cap), dtype=torch.float32)
+    for r in range(R):
+        n = int(len0[r])
+        hist0[r, :n] = torch.tensor(rng.uniform(1.0, 9.0, size=n) + np.linspace(0, rng.uniform(-3, 3), n), dtype=torch.float32)
+    k = int(rng.choice([1, 5, 20, 20, 64, 65, 100]))
+    p = B.BudgetParams(min(k, V), int(rng.choice([8, 32, 64, 100])), int(rng.choice([1, 4, 8, 16])),
+                       float(rng.choice([5.0, 10.0, 25.0, 50.0])), float(rng.choice([1.25, 1.75, 2.0])), 30000,
+                       150000 if rng.integers(0, 2) else 0, 0)
+    if p.clamp_lo_ppm:
+        p.clamp_hi_ppm = 400000
+    seq_len = torch.tensor(rng.integers(100, 70000, size=R), dtype=torch.int32) if p.clamp_lo_ppm else None
+    budget_in = torch.tensor(rng.integers(1, 29000, size=R), dtype=torch.int32)
+    _compare(logits, tok, hist0, len0, budget_in, p, seq_len)
