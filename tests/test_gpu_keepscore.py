@@ -299,3 +299,49 @@ def test_fused_keepscore_select_matches_oracle_bit_exact(long_unit):
                              None, big, torch.from_numpy(ki).to(DEV), d_sel, int(ki[-1]), None, None, status)
     torch.cuda.synchronize()
     assert status.cpu().tolist()[0] == B.E_INVALID
+
+
+@pytest.mark.parametrize("seed", range(12))
+def test_random_keepscore_select(seed):
+    """Seeded random calls of the fused keep-score update + TopK: unit lengths from empty to beyond one sweep,
+    budgets 0 .. above the length, protected prefixes shorter and longer than the budget, top-p and decay drawn
+    (including their end points); hit masks, keep-scores and index lists bit-exact against the oracle."""
+    rng = np.random.default_rng(8000 + seed)
+    R = int(rng.integers(1, 7))
+    lens = [int(rng.choice([0, rng.integers(1, 40), rng.integers(40, 5000), rng.integers(5000, 30000)])) for _ in range(R)]
+    if max(lens) == 0:
+        lens[0] = 17
+    budgets = [int(rng.choice([0, 1, L, L + 3, max(1, L // 4), rng.integers(0, L + 1)])) for L in lens]
+    protect = [int(rng.choice([0, 0, 1, rng.integers(0, L + 1), L + 2])) for L in lens]
+    n_outer = int(rng.integers(1, 4))
+    top_p = float(rng.choice([0.0, 0.3, 0.9, 0.99, 1.0]))
+    lam = float(rng.choice([0.0, 0.5, 0.9, 1.0]))
+    sc, tok = _synthetic_scores(rng, n_outer, lens)
+    ks0 = (rng.random(sc.shape) ** 4).astype(np.float32)
+    ks0[:, ::3] = 0.0
+    sum_tok = int(tok[-1])
+    keep = [min(b, L) for b, L in zip(budgets, lens)]
+    ki = np.concatenate([[0], np.cumsum(keep)]).astype(np.int32)
+    stride = int(ki[-1]) + 3
+    d_sc = torch.from_numpy(sc.copy()).to(DEV)
+    d_ks = torch.from_numpy(ks0.copy()).to(DEV)
+    d_hit = torch.zeros((n_outer, (sum_tok + 31) // 32), dtype=torch.int32, device=DEV)
+    d_sel = torch.full((n_outer, stride), -1, dtype=torch.int32, device=DEV)
+    status = torch.zeros(4, dtype=torch.int32, device=DEV)
+    B.actkv_keepscore_select(d_sc, torch.from_numpy(tok).to(DEV), sum_tok, max(lens), n_outer, R, top_p, lam,
+                             torch.tensor(protect, dtype=torch.int32, device=DEV), d_ks, d_hit,
+                             torch.tensor(budgets, dtype=torch.int32, device=DEV), torch.from_numpy(ki).to(DEV), d_sel,
+                             stride, None, None, status)
+    torch.cuda.synchronize()
+    assert status.cpu().tolist()[0] == 0, status.cpu().tolist()
+    got_ks, got_hit, got_sel = d_ks.cpu().numpy(), d_hit.cpu().numpy(), d_sel.cpu().numpy()
+    for o in range(n_outer):
+        for r, L in enumerate(lens):
+            a, b = int(tok[r]), int(tok[r + 1])
+            hit = O.hit_mask_unit(sc[o, a:b], top_p)
+            ks = O.keep_score_update(ks0[o, a:b], sc[o, a:b], hit, lam)
+            want = O.select_unit(O.rank_keys(ks, min(protect[r], L)), budgets[r])
+            assert np.array_equal(_unpack_hits(got_hit[o], a, b), hit), f"hit mask of unit ({o},{r})"
+            assert np.array_equal(_f32_bits(got_ks[o, a:b]), _f32_bits(ks)), f"keep-score of unit ({o},{r})"
+            assert np.array_equal(got_sel[o, ki[r]:ki[r + 1]], want), f"index list of unit ({o},{r})"
+    assert (got_sel[:, ki[-1]:] == -1).all()
