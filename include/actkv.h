@@ -364,6 +364,8 @@ int actkv_compact(const actkv_pool_t* pool /* host */, const actkv_tables_t* tab
  *   and actkv_compact_end copies everything.  reuse_plan != 0: `ws` still holds the plan of an earlier
  *   actkv_compact_begin of the same step (same tables, budgets and max_keep, nothing finalized in
  *   between; the plan does not depend on the layers), so only the job of this layer range is recorded.
+ *   A workspace that holds no plan of this pool and these tables is reported (status ACTKV_E_INVALID) and
+ *   nothing is copied or finalized from it.
  * actkv_score_overlap: actkv_score with one more argument, pending_compact_ws: the workspace of a
  *   begun compaction of OTHER layers of the same pool, or NULL (then it is actkv_score).  The
  *   result of the score does not depend on it.  On the tensor-core path four spare warps per CTA of the

@@ -25,6 +25,7 @@ struct CompactJobArgs {
   int32_t deferred;
   uint32_t* src_tab;     // deferred: room for the resolved sources of every item
   int64_t src_tab_items; // ... in items (32 entries each)
+  const int32_t* tab_page_table;   // the tables of the call (a reused plan must be one of these tables)
 };
 
 __global__ void compact_plan_kernel(TablesView tab, int32_t page_size, int32_t n_pages,
@@ -113,7 +114,7 @@ __global__ void compact_plan_kernel(TablesView tab, int32_t page_size, int32_t n
     ws->vpr_shift = job.deferred ? job.vpr_shift : -1;
     ws->parts_per_page = jp;
     ws->role_items = 0;
-    ws->pad = 0;
+    ws->pad = CJ_PLAN_MARK;
   }
 }
 
@@ -125,6 +126,22 @@ __global__ void compact_stats_kernel(const CompactWs* ws, int32_t* out) {
 // A further layer range of a step whose plan is already in the workspace (the plan depends on the tables and
 // the budgets only, not on the layers): only the job is recorded anew.
 __global__ void compact_rejob_kernel(CompactWs* ws, CompactJobArgs job, int32_t* status) {
+  // the workspace must hold a plan of these very tables and this pool (a caller's mistake otherwise: reported,
+  // and nothing is copied or finalized from what happens to be in the workspace)
+  const bool mine = ws->pad == CJ_PLAN_MARK && ws->pool.base == job.pool.base && ws->tab.page_table == job.tab_page_table &&
+                    ws->status == status;
+  if (!mine) {
+    report(status, ACTKV_E_INVALID, -3, 0);
+    ws->pad = CJ_PLAN_MARK;
+    ws->plan_ok = 0;
+    ws->total_new = 0;
+    ws->n_items = 0;
+    ws->next_item = 0u;
+    ws->role_items = 0;
+    ws->vpr_shift = -1;
+    ws->parts_per_page = 1;
+    return;
+  }
   const bool ok = ws->plan_ok && !status_set(status);
   if (!ok) ws->plan_ok = 0;
   const int64_t items = (int64_t)ws->total_new * job.n_layers * ws->parts_per_page;
@@ -346,6 +363,7 @@ static int compact_plan(const actkv_pool_t* pool, const actkv_tables_t* tables, 
   job.src_tab = (uint32_t*)((char*)ws + base);
   job.src_tab_items = deferred ? (int64_t)((ws_bytes - base) / (32 * sizeof(uint32_t))) : 0;
   job.pool = make_view(pool);
+  job.tab_page_table = tables->page_table;
   job.sel_idx = sel_idx;
   job.sel_stride = sel_stride;
   job.keep_indptr = keep_indptr;

@@ -29,7 +29,7 @@ struct CompactWs {
   int32_t vpr_shift;     // log2 of the 16-byte vectors per row (3, 4, 5 for head_dim 64, 128, 256); -1: not deferrable
   int32_t parts_per_page;  // items per destination page: ceil(page_size x heads / 32)
   int32_t role_items;    // items executed by copy roles of other kernels (the rest went to the drain kernel)
-  int32_t pad;
+  int32_t pad;           // CJ_PLAN_MARK once a plan kernel has written this workspace
   uint32_t* src_tab;     // deferred copy: resolved sources, [n_items][32] (see cj_resolve_item)
   // followed by int32 new_off[R], push_off[R], item_off[R + 1], new_pages[R * max_pages]
 };
@@ -40,6 +40,7 @@ __host__ __device__ __forceinline__ int32_t* ws_item_off(CompactWs* w, int R) { 
 __host__ __device__ __forceinline__ int32_t* ws_new_pages(CompactWs* w, int R) { return ws_new_off(w) + 3 * R + 1; }
 
 constexpr uint32_t CJ_NONE = 0xffffffffu;
+constexpr int32_t CJ_PLAN_MARK = 0x414b5650;
 
 __device__ __forceinline__ uint4 ld_stream(const uint4* p) {
   uint4 v;

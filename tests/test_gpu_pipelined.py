@@ -147,3 +147,48 @@ def test_a_bad_page_id_in_a_table_stops_the_compaction_before_anything_is_modifi
     assert np.array_equal(U.bits(b.pool), snap[0])
     for t, s0 in zip((b.page_table, b.seq_len, b.free_list, b.free_count), snap[1:]):
         assert torch.equal(t, s0)
+
+
+def test_reusing_a_plan_that_is_not_there_is_reported_and_nothing_moves():
+    """actkv_compact_begin with reuse_plan on a workspace that holds no plan of these tables (never written, or
+    written for another pool): reported as an invalid call; neither begin + end nor a following score call with the
+    workspace as its pending compaction copies anything or touches the tables."""
+    wl = synth.Workload("noplan", 2, 2, 8, [900, 333], [16, 8], [250, 100], table_style="fragmented", seed=56,
+                        poison_tail=True)
+    b = synth.generate(wl, DEV)
+    comp = H.Compressor(b.pool, b.page_table, b.seq_len, b.free_list, b.free_count, wl.n_q_heads, H.sizes_of(b))
+    B.actkv_keep_indptr(b.seq_len, b.budget, wl.n_req, comp.keep_indptr)
+    comp.run_score(b.q, b.win_indptr, b.tok_indptr, wl.sm_scale, wl.causal)
+    comp.run_select(b.tok_indptr, b.budget, wl.n_layers)
+    torch.cuda.synchronize()
+    comp.check_status()
+    snap = [U.bits(b.pool).copy()] + [t.clone() for t in (b.page_table, b.seq_len, b.free_list, b.free_count)]
+    args = (comp.pd, comp.td, 0, wl.n_layers, comp.sel_idx, comp.sz.sel_stride, comp.keep_indptr, b.budget,
+            comp.sz.max_keep, comp.ws_compact, comp.status)
+    for fill in (0, 0x5A):
+        comp.ws_compact.fill_(fill)
+        comp.status.zero_()
+        B.actkv_compact_begin(*args, reuse_plan=True)
+        s = comp.sz
+        B.actkv_score_overlap(comp.pd, comp.td, 0, wl.n_layers, b.q, b.win_indptr, wl.n_q_heads, None, wl.sm_scale, wl.causal,
+                              b.tok_indptr, comp.score, None, s.sum_win, s.max_win, s.sum_tok, s.max_tok, comp.ws_score,
+                              comp.ws_compact, comp.status)
+        B.actkv_compact_end(*args)
+        torch.cuda.synchronize()
+        assert comp.status.cpu().tolist()[0] == B.E_INVALID
+        assert np.array_equal(U.bits(b.pool), snap[0])
+        for t, s0 in zip((b.page_table, b.seq_len, b.free_list, b.free_count), snap[1:]):
+            assert torch.equal(t, s0)
+    # a plan of another instance's tables in the workspace is refused as well
+    c = synth.generate(wl, DEV)
+    comp_c = H.Compressor(c.pool, c.page_table, c.seq_len, c.free_list, c.free_count, wl.n_q_heads, H.sizes_of(c))
+    comp.status.zero_()
+    B.actkv_compact_begin(comp_c.pd, comp_c.td, 0, wl.n_layers, comp.sel_idx, comp.sz.sel_stride, comp.keep_indptr, b.budget,
+                          comp.sz.max_keep, comp.ws_compact, comp.status)
+    B.actkv_compact_begin(*args, reuse_plan=True)
+    B.actkv_compact_end(*args)
+    torch.cuda.synchronize()
+    assert comp.status.cpu().tolist()[0] == B.E_INVALID
+    assert np.array_equal(U.bits(b.pool), snap[0])
+    for t, s0 in zip((b.page_table, b.seq_len, b.free_list, b.free_count), snap[1:]):
+        assert torch.equal(t, s0)
