@@ -336,6 +336,7 @@ def run_ours(args):
         pipe_comp.lse, pipe_comp.status = comp.lse, comp.status
     lrfu_state = None                          # set for the secondary LRFU-policy line only
     inplace_mode = False                       # set for the secondary in-place-compaction line only
+    inplace_pipe = False                       # ... its pipelined form
     stage_names = ["budget", "lse", "score", "select", "compact"]
 
     def one_step(events=None):
@@ -355,10 +356,10 @@ def run_ours(args):
         if args.overlap:
             n = comp.step_overlapped(inst.q, inst.win_indptr, inst.tok_indptr, bud, wl.sm_scale, wl.causal,
                                      lse_in=lse_supplied, marks=mark)
-        elif pipelined and lrfu_state is None and not inplace_mode:
+        elif pipelined and lrfu_state is None and (not inplace_mode or inplace_pipe):
             n = pipe_comp.step_pipelined(inst.q, inst.win_indptr, inst.tok_indptr, bud, wl.sm_scale, wl.causal,
                                          lse_in=lse_supplied, marks=(lambda nm: mark(nm)), groups=pipe_groups,
-                                         stats=pipe_stats)
+                                         stats=pipe_stats, inplace=inplace_mode)
         else:
             n = comp.step(inst.q, inst.win_indptr, inst.tok_indptr, bud, wl.sm_scale, wl.causal,
                           lse_in=lse_supplied, marks=(lambda nm: mark(nm)), lrfu=lrfu_state, inplace=inplace_mode)
@@ -693,6 +694,34 @@ def run_ours(args):
             torch.cuda.synchronize()
             if it >= 2:
                 ms2.append(e0.elapsed_time(e1))
+        # ... and both with the moves of a layer group inside the pooled-score kernel of the next one
+        pipe_ip = None
+        if pipelined:
+            inplace_pipe = True
+            tp = []
+            for mode in ("internal", "supplied"):
+                lse_supplied = comp.lse.clone() if mode == "supplied" else None
+                ms3 = []
+                for it in range(2 + min(args.steps, 5)):
+                    inst.pool.copy_(pool_backup)
+                    restore()
+                    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                    e0.record()
+                    one_step()
+                    e1.record()
+                    torch.cuda.synchronize()
+                    if it >= 2:
+                        ms3.append(e0.elapsed_time(e1))
+                t3 = torch.tensor([sum(ms3) / len(ms3)], dtype=torch.float64, device=dev)
+                if dist is not None:
+                    dist.all_reduce(t3, op=dist.ReduceOp.MAX)
+                tp.append(float(t3.item()))
+            inplace_pipe = False
+            pipe_comp.check_status()
+            pipe_ip = {"groups": [l1 - l0 for l0, l1 in pipe_groups],
+                       "ms_per_step": tp[0], "value": world * tokens / (tp[0] * 1e-3), "unit": UNIT,
+                       "with_lse_supplied": {"ms_per_step": tp[1], "value": world * tokens / (tp[1] * 1e-3), "unit": UNIT,
+                                             "hbm_roofline_frac_whole_step_fresh_page_bytes": alg_bytes / (tp[1] * 1e-3) / 1e9 / pk["hbm_gbs"]}}
         lse_supplied = None
         inplace_mode = False
         del pool_backup
@@ -705,7 +734,8 @@ def run_ours(args):
                                               "value": world * tokens / (float(t2.item()) * 1e-3), "unit": UNIT},
                         "compact_ms": cp, "rows_moved_fraction_of_kept": moved / max(1.0, rho * tokens * Hkv * comp.lpc),
                         "compact_gbs": moved_bytes / (cp * 1e-3) / 1e9,
-                        "compact_frac_of_hbm_peak": moved_bytes / (cp * 1e-3) / 1e9 / pk["hbm_gbs"]}
+                        "compact_frac_of_hbm_peak": moved_bytes / (cp * 1e-3) / 1e9 / pk["hbm_gbs"],
+                        "pipelined": pipe_ip}
 
     # ---- the oracle on the host cores (rank 0, single GPU only) ----------------------------------
     cpu_baseline = None

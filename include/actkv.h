@@ -430,6 +430,37 @@ int actkv_compact_inplace(const actkv_pool_t* pool /* host */, const actkv_table
                           const int32_t* budget, int32_t max_keep, int32_t* new_order,
                           int32_t* status, actkv_stream_t stream);
 
+/* actkv_compact_inplace_begin / actkv_compact_inplace_end — the same in-place compaction with the
+ * copies of one layer group hidden under the pooled-score kernel of the next one, as
+ * actkv_compact_begin / actkv_compact_end do for the fresh-page form (Section 3.3: the primitives
+ * are independent per layer; Algorithm 4: the moves of a plan are conflict-free, sources outside
+ * the region, destinations inside it, so their order is free).
+ *   begin: resolves every move of [layer_begin, layer_end) once into a table of (source,
+ *          destination) rows, 32 region slots per item, and publishes it in `ws` as the work queue
+ *          that actkv_score_overlap(pending_compact_ws = ws) serves; writes new_order (optional) as
+ *          actkv_compact_inplace does; copies nothing, leaves the tables alone.  sel_idx may be
+ *          reused once begin has run on the stream.
+ *   end:   the same arguments; copies every item not yet taken and, when layer_end ==
+ *          pool->n_layers, updates the tables as actkv_compact_inplace does.
+ * begin + end without a score call in between equals actkv_compact_inplace.  `ws` must have
+ * actkv_compact_inplace_deferred_workspace_bytes(pool, n_req, layer_end - layer_begin, max_keep)
+ * bytes for the copies to be deferred (8 bytes per kept row and layer); with less (at least the
+ * bytes of that call with max_keep = 0), or for a pool the item copy does not take (head_dim other
+ * than 64 / 128 / 256), nothing is deferred and end runs the one-launch copy itself, for which
+ * sel_idx must then still hold the lists. */
+size_t actkv_compact_inplace_deferred_workspace_bytes(const actkv_pool_t* pool /* host */, int32_t n_req,
+                                                      int32_t n_layers_sub, int32_t max_keep);
+int actkv_compact_inplace_begin(const actkv_pool_t* pool /* host */, const actkv_tables_t* tables /* host */,
+                                int32_t layer_begin, int32_t layer_end,
+                                const int32_t* sel_idx, int64_t sel_stride, const int32_t* keep_indptr,
+                                const int32_t* budget, int32_t max_keep, int32_t* new_order,
+                                void* ws, size_t ws_bytes, int32_t* status, actkv_stream_t stream);
+int actkv_compact_inplace_end(const actkv_pool_t* pool /* host */, const actkv_tables_t* tables /* host */,
+                              int32_t layer_begin, int32_t layer_end,
+                              const int32_t* sel_idx, int64_t sel_stride, const int32_t* keep_indptr,
+                              const int32_t* budget, int32_t max_keep, int32_t* new_order,
+                              void* ws, size_t ws_bytes, int32_t* status, actkv_stream_t stream);
+
 /* ---------------------------------------------------------------------------------------
  * actkv_step_host — one whole compression step (Algorithm 1 steps 1, 5, 6 with Algorithm 2 in
  * front) for a caller whose per-step inputs live in HOST memory.

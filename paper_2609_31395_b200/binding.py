@@ -28,6 +28,7 @@ EXPORTS = ["actkv_budget_workspace_bytes", "actkv_budget", "actkv_score_workspac
            "actkv_compact_noalloc_max_bytes", "actkv_step_host", "actkv_keepscore", "actkv_gather_f32",
            "actkv_compact_inplace", "actkv_score_path", "actkv_debug_inject_stall", "actkv_score_sliding", "actkv_keepscore_select",
            "actkv_compact_deferred_workspace_bytes", "actkv_compact_begin", "actkv_compact_end", "actkv_score_overlap", "actkv_compact_stats",
+           "actkv_compact_inplace_deferred_workspace_bytes", "actkv_compact_inplace_begin", "actkv_compact_inplace_end",
            "actkv_version"]
 
 
@@ -135,6 +136,11 @@ def load():
     lib.actkv_compact_inplace.restype = i32
     lib.actkv_compact_inplace.argtypes = [C.POINTER(PoolDesc), C.POINTER(TablesDesc), i32, i32, vp, i64, vp, vp, i32,
                                           vp, vp, vp]
+    lib.actkv_compact_inplace_deferred_workspace_bytes.restype = sz
+    lib.actkv_compact_inplace_deferred_workspace_bytes.argtypes = [C.POINTER(PoolDesc), i32, i32, i32]
+    for fn in (lib.actkv_compact_inplace_begin, lib.actkv_compact_inplace_end):
+        fn.restype = i32
+        fn.argtypes = [C.POINTER(PoolDesc), C.POINTER(TablesDesc), i32, i32, vp, i64, vp, vp, i32, vp, vp, sz, vp, vp]
     lib.actkv_gather_f32.restype = i32
     lib.actkv_gather_f32.argtypes = [vp, i64, vp, vp, i64, vp, i32, i32, i32, vp, i64, vp]
     lib.actkv_step_host.restype = i32
@@ -406,6 +412,32 @@ def actkv_compact_inplace(pool: PoolDesc, tables: TablesDesc, layer_begin, layer
                                       _ptr(new_order, torch.int32, "new_order"),
                                       _ptr(status, torch.int32, "status"), _stream(stream))
     _check("actkv_compact_inplace", rc)
+
+
+def actkv_compact_inplace_deferred_workspace_bytes(pool: PoolDesc, n_req, n_layers_sub, max_keep) -> int:
+    return load().actkv_compact_inplace_deferred_workspace_bytes(C.byref(pool), n_req, n_layers_sub, max_keep)
+
+
+def _inplace_deferred(fn_name, pool, tables, layer_begin, layer_end, sel_idx, sel_stride, keep_indptr, budget, max_keep,
+                      new_order, ws, status, stream):
+    rc = getattr(load(), fn_name)(C.byref(pool), C.byref(tables), layer_begin, layer_end,
+                                  _ptr(sel_idx, torch.int32, "sel_idx"), sel_stride,
+                                  _ptr(keep_indptr, torch.int32, "keep_indptr"), _ptr(budget, torch.int32, "budget"),
+                                  max_keep, _ptr(new_order, torch.int32, "new_order"), _ptr(ws, None, "ws"),
+                                  ws.numel() * ws.element_size(), _ptr(status, torch.int32, "status"), _stream(stream))
+    _check(fn_name, rc)
+
+
+def actkv_compact_inplace_begin(pool: PoolDesc, tables: TablesDesc, layer_begin, layer_end, sel_idx, sel_stride,
+                                keep_indptr, budget, max_keep, new_order, ws, status, stream=None):
+    _inplace_deferred("actkv_compact_inplace_begin", pool, tables, layer_begin, layer_end, sel_idx, sel_stride,
+                      keep_indptr, budget, max_keep, new_order, ws, status, stream)
+
+
+def actkv_compact_inplace_end(pool: PoolDesc, tables: TablesDesc, layer_begin, layer_end, sel_idx, sel_stride,
+                              keep_indptr, budget, max_keep, new_order, ws, status, stream=None):
+    _inplace_deferred("actkv_compact_inplace_end", pool, tables, layer_begin, layer_end, sel_idx, sel_stride,
+                      keep_indptr, budget, max_keep, new_order, ws, status, stream)
 
 
 def actkv_keepscore(score, tok_indptr, sum_tok, n_outer, n_req, top_p, lam, n_protect, keep_score, hit_mask, status,

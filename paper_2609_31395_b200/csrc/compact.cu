@@ -113,6 +113,9 @@ __global__ void compact_plan_kernel(TablesView tab, int32_t page_size, int32_t n
     ws->n_layers = job.n_layers;
     ws->vpr_shift = job.deferred ? job.vpr_shift : -1;
     ws->parts_per_page = jp;
+    ws->items_per_slab = (int32_t)max((int64_t)1, min((int64_t)total * jp, (int64_t)0x7fffffff));
+    ws->dst_tab = nullptr;
+    ws->pad2 = 0;
     ws->role_items = 0;
     ws->pad = CJ_PLAN_MARK;
   }
@@ -140,6 +143,8 @@ __global__ void compact_rejob_kernel(CompactWs* ws, CompactJobArgs job, int32_t*
     ws->role_items = 0;
     ws->vpr_shift = -1;
     ws->parts_per_page = 1;
+    ws->items_per_slab = 1;
+    ws->dst_tab = nullptr;
     return;
   }
   const bool ok = ws->plan_ok && !status_set(status);
@@ -150,6 +155,7 @@ __global__ void compact_rejob_kernel(CompactWs* ws, CompactJobArgs job, int32_t*
   ws->n_items = (ok && job.deferred && job.vpr_shift >= 0 && items <= 0x7fffffff && items <= job.src_tab_items)
                     ? (int32_t)items : 0;
   ws->src_tab = job.src_tab;
+  ws->dst_tab = nullptr;
   ws->sel_idx = job.sel_idx;
   ws->sel_stride = job.sel_stride;
   ws->keep_indptr = job.keep_indptr;
@@ -164,21 +170,6 @@ __global__ void __launch_bounds__(128) compact_resolve_kernel(CompactWs* ws) {
   const int64_t n = cj_count(ws);
   for (int64_t item = (int64_t)blockIdx.x * 4 + (threadIdx.x >> 5); item < n; item += (int64_t)gridDim.x * 4)
     cj_resolve_item(ws, (int)item, lane);
-}
-
-// What is left of a deferred copy: every warp takes items until the queue is empty.
-template <int VPR_SHIFT>
-__global__ void __launch_bounds__(128) compact_drain_kernel(CompactWs* ws) {
-  const int lane = threadIdx.x & 31;
-  if (ws->vpr_shift != VPR_SHIFT) return;
-  const uint32_t n = cj_count(ws);
-  if (n == 0) return;
-  uint32_t item = cj_pop(ws, lane);
-  while (item < n) {
-    const uint32_t next = cj_pop(ws, lane);              // asked for now, looked at after this item's copies
-    cj_copy_item<VPR_SHIFT, 16>(ws, (int)item, lane);
-    item = next;
-  }
 }
 
 constexpr int CP_NT = 128;
@@ -338,18 +329,6 @@ static int compact_check(const actkv_pool_t* pool, const actkv_tables_t* tables,
   return ACTKV_OK;
 }
 
-// log2 of the 16-byte vectors per row when the warp-level item copy takes this pool: head_dim 64, 128 or 256,
-// a layer (K and V) within 2^32 16-byte units; else -1.
-static int deferrable_shift(const actkv_pool_t* pool) {
-  const int vpr = pool->head_dim / 8;
-  const int shift = vpr == 8 ? 3 : vpr == 16 ? 4 : vpr == 32 ? 5 : -1;
-  if (shift < 0) return -1;
-  const int64_t extent = pool->stride_kv + (int64_t)pool->n_pages * pool->stride_page;       // elements, upper bound
-  if (pool->stride_kv < 0 || pool->stride_page < 0 || pool->stride_slot < 0 || pool->stride_head < 0) return -1;
-  if (extent / 8 >= 0xffffffffLL) return -1;
-  return shift;
-}
-
 static int compact_plan(const actkv_pool_t* pool, const actkv_tables_t* tables, int32_t layer_begin, int32_t layer_end,
                         const int32_t* sel_idx, int64_t sel_stride, const int32_t* keep_indptr, const int32_t* budget,
                         int32_t max_keep, void* ws, size_t ws_bytes, int32_t* status, cudaStream_t s, bool deferred,
@@ -482,15 +461,10 @@ int actkv_compact_end(const actkv_pool_t* pool, const actkv_tables_t* tables, in
     rc = compact_copy_all(pool, tables, layer_begin, layer_end, sel_idx, sel_stride, keep_indptr, budget, max_keep, ws, status, s);
     if (rc != ACTKV_OK) return rc;
   } else {
-    // every warp takes items until the queue is empty; at most eight CTAs of four warps per SM
+    // every warp takes items until the queue is empty
     const int64_t max_x = std::min<int64_t>((max_keep + pool->page_size - 1) / pool->page_size, tables->max_pages);
     const int64_t jp = ((int64_t)pool->page_size * pool->n_kv_heads + 31) / 32;
-    const int64_t items_max = max_x * tables->n_req * (layer_end - layer_begin) * jp;
-    const unsigned grid = (unsigned)std::max<int64_t>(1, std::min<int64_t>((items_max + 3) / 4, 148 * 8));
-    CompactWs* w = (CompactWs*)ws;
-    if (shift == 3) compact_drain_kernel<3><<<grid, 128, 0, s>>>(w);
-    else if (shift == 4) compact_drain_kernel<4><<<grid, 128, 0, s>>>(w);
-    else compact_drain_kernel<5><<<grid, 128, 0, s>>>(w);
+    launch_drain((CompactWs*)ws, shift, max_x * tables->n_req * (layer_end - layer_begin) * jp, s);
     ACTKV_CHECK_LAUNCH();
   }
   return compact_finalize(pool, tables, layer_end, budget, ws, status, s);

@@ -17,7 +17,11 @@
 //   finalize : page_table[r] <- its last X pages, seq_len[r] <- B, the first Y-X pages are pushed on
 //              the free-list stack (only on the call whose layer range ends at the pool's last layer).
 // On a device-detected error the tables stay as they were; only dead slots (holes) were written.
-#include "common.cuh"
+// The copy can also be deferred (actkv_compact_inplace_begin / _end): the moves of a layer group are resolved
+// once into a table of (source, destination) row offsets, 32 region slots per item, and published as the work
+// queue of compact_job.cuh, so that the spare warps of the pooled-score kernel of the NEXT layer group execute
+// them (sources and destinations lie in layers that kernel does not touch) and a drain kernel what is left.
+#include "compact_job.cuh"
 
 namespace actkv {
 
@@ -150,6 +154,148 @@ __global__ void __launch_bounds__(CI_NT) compact_inplace_copy_kernel(
   }
 }
 
+// ---- deferred form --------------------------------------------------------------------------------
+// Plan: items per request (32 region slots each; with an order output also the requests that are not
+// compacted, whose order is the identity list), their prefix sums, and the job record.
+__global__ void compact_inplace_plan_kernel(TablesView tab, PoolView pool, const int32_t* __restrict__ budget,
+                                            int32_t max_keep, int32_t want_order, int32_t layer_begin, int32_t n_layers,
+                                            int32_t vpr_shift, uint32_t* src_tab, uint32_t* dst_tab, int64_t tab_items,
+                                            CompactWs* ws, int32_t* status) {
+  if (threadIdx.x != 0) return;
+  const int R = tab.n_req, P = pool.page_size;
+  int32_t* item_off = ws_item_off(ws, R);
+  bool ok = !status_set(status);
+  int64_t off = 0;
+  for (int r = 0; r < R; ++r) {
+    item_off[r] = (int32_t)off;
+    const int32_t L = tab.seq_len[r];
+    const int32_t B = budget[r] < 0 ? 0 : budget[r];
+    if (L < 0) { report(status, ACTKV_E_INVALID, r, L); ok = false; continue; }
+    if (B >= L) {
+      if (want_order) off += (L + 31) / 32;
+      continue;
+    }
+    const int Y = (L + P - 1) / P;
+    if (Y > tab.max_pages || B > max_keep) { report(status, ACTKV_E_INVALID, r, Y > tab.max_pages ? L : B); ok = false; continue; }
+    off += (B + 31) / 32;
+  }
+  item_off[R] = (int32_t)off;
+  const int64_t per_slab = off * pool.n_kv_heads;
+  const int64_t items = per_slab * n_layers;
+  if (items > 0x7fffffff || items > tab_items) {         // (the host sized the tables for max_keep)
+    if (ok) report(status, ACTKV_E_WORKSPACE, -1, (int32_t)min(items, (int64_t)0x7fffffff));
+    ok = false;
+  }
+  ws->plan_ok = ok ? 1 : 0;
+  ws->total_new = (int32_t)off;                 // items of one (layer, head)
+  ws->next_item = 0u;
+  ws->n_items = ok ? (int32_t)items : 0;
+  ws->pool = pool;
+  ws->tab = tab;
+  ws->sel_idx = nullptr;
+  ws->sel_stride = 0;
+  ws->keep_indptr = nullptr;
+  ws->budget = budget;
+  ws->status = status;
+  ws->layer_begin = layer_begin;
+  ws->n_layers = n_layers;
+  ws->vpr_shift = vpr_shift;
+  ws->parts_per_page = 1;
+  ws->role_items = 0;
+  ws->pad = CJ_INPLACE_MARK;
+  ws->src_tab = src_tab;
+  ws->dst_tab = dst_tab;
+  ws->items_per_slab = (int32_t)max((int64_t)1, min(per_slab, (int64_t)0x7fffffff));
+  ws->pad2 = 0;
+}
+
+// One warp per item: the 32 region slots [32 chunk, 32 chunk + 32) of one (layer, head, request), classified as
+// in the one-launch kernel above; a hole's move goes into the table as (source, destination) offsets in 16-byte
+// units within the layer, everything else as CJ_NONE.
+__global__ void __launch_bounds__(128) compact_inplace_resolve_kernel(
+    CompactWs* ws, const int32_t* __restrict__ sel_idx, int64_t sel_stride, const int32_t* __restrict__ keep_indptr,
+    int32_t* __restrict__ new_order) {
+  const int lane = threadIdx.x & 31;
+  const int64_t n = cj_count(ws);
+  const PoolView& pool = ws->pool;
+  const TablesView& tab = ws->tab;
+  const int R = tab.n_req, H = pool.n_kv_heads, P = pool.page_size;
+  const int32_t* item_off = ws_item_off(ws, R);
+  const int per_head = ws->total_new, per_slab = ws->items_per_slab;
+  int32_t* status = ws->status;
+  for (int64_t item = (int64_t)blockIdx.x * 4 + (threadIdx.x >> 5); item < n; item += (int64_t)gridDim.x * 4) {
+    const int slab = (int)(item / per_slab), rem = (int)(item - (int64_t)slab * per_slab);
+    const int h = rem / per_head, rem2 = rem - h * per_head;
+    int lo = 0, hi = R;                                  // item_off[lo] <= rem2 < item_off[hi]
+    while (hi - lo > 1) {
+      const int mid = (lo + hi) >> 1;
+      if (item_off[mid] <= rem2) lo = mid; else hi = mid;
+    }
+    const int r = lo, chunk = rem2 - item_off[r];
+    const int z = slab * H + h;
+    const int32_t L = tab.seq_len[r];
+    const int32_t B = ws->budget[r] < 0 ? 0 : ws->budget[r];
+    const int32_t* sel = sel_idx + (int64_t)z * sel_stride + keep_indptr[r];
+    int32_t* ord = new_order ? new_order + (int64_t)z * sel_stride + keep_indptr[r] : nullptr;
+    uint32_t so = CJ_NONE, dof = CJ_NONE;
+    if (B >= L) {                                        // not compacting: the order is the identity list
+      const int i = chunk * 32 + lane;
+      if (ord && i < L) ord[i] = sel[i];
+    } else {
+      const int Y = (L + P - 1) / P, X = (B + P - 1) / P;
+      const int32_t start = (Y - X) * P, end = start + B;
+      const int32_t p0 = start + chunk * 32, p = p0 + lane;
+      int v = 0;
+      if (lane == 0) v = lower_bound_i32(sel, B, start);
+      if (lane == 1) v = lower_bound_i32(sel, B, end);
+      if (lane == 2) v = lower_bound_i32(sel, B, p0);
+      const int a = __shfl_sync(0xffffffffu, v, 0), c = __shfl_sync(0xffffffffu, v, 1), lb0 = __shfl_sync(0xffffffffu, v, 2);
+      const int m = a + (B - c);                         // survivors outside the region = holes inside it
+      // at most 32 kept indices fall in these 32 slots: they all sit in sel[lb0 .. lb0 + 32)
+      const int wn = min(32, B - lb0);
+      const int32_t win = lane < wn ? sel[lb0 + lane] : 0x7fffffff;
+      const int32_t nxt = __shfl_down_sync(0xffffffffu, win, 1);
+      if (lane + 1 < wn && nxt <= win) report(status, ACTKV_E_BADINDEX, r, nxt);      // must be strictly ascending
+      int w = 0;                                         // #kept in [p0, p)
+      bool kept = false;
+#pragma unroll
+      for (int k = 0; k < 32; ++k) {
+        const int32_t x = __shfl_sync(0xffffffffu, win, k);
+        w += (k < wn && x < p) ? 1 : 0;
+        kept = kept || (k < wn && x == p);
+      }
+      if (p < end) {
+        if (kept) {
+          if (ord) ord[p - start] = p;
+        } else {
+          const int j = (p - start) - (lb0 + w - a);     // rank of this hole
+          if (j < 0 || j >= m) {
+            report(status, ACTKV_E_BADINDEX, r, p);
+          } else {
+            const int32_t src_pos = j < a ? sel[j] : sel[c + (j - a)];
+            if ((uint32_t)src_pos >= (uint32_t)L || (src_pos >= start && src_pos < end)) {
+              report(status, ACTKV_E_BADINDEX, r, src_pos);
+            } else {
+              if (ord) ord[p - start] = src_pos;
+              // a move whose source or destination page id is out of range is dropped (and reported)
+              const int32_t sp = page_or_neg(tab, pool.n_pages, r, src_pos / P, status);
+              const int32_t dp = page_or_neg(tab, pool.n_pages, r, p / P, status);
+              if (sp >= 0 && dp >= 0) {
+                so = (uint32_t)(((int64_t)sp * pool.stride_page + (int64_t)(src_pos % P) * pool.stride_slot +
+                                 (int64_t)h * pool.stride_head) >> 3);
+                dof = (uint32_t)(((int64_t)dp * pool.stride_page + (int64_t)(p % P) * pool.stride_slot +
+                                  (int64_t)h * pool.stride_head) >> 3);
+              }
+            }
+          }
+        }
+      }
+    }
+    ws->src_tab[item * 32 + lane] = so;
+    ws->dst_tab[item * 32 + lane] = dof;
+  }
+}
+
 __global__ void compact_inplace_finalize_kernel(TablesView tab, int32_t page_size, int32_t n_pages,
                                                 const int32_t* __restrict__ budget, int32_t* status) {
   if (status_set(status)) return;
@@ -201,12 +347,11 @@ __global__ void compact_inplace_finalize_kernel(TablesView tab, int32_t page_siz
 
 }  // namespace actkv
 
-extern "C" {
+namespace actkv {
 
-int actkv_compact_inplace(const actkv_pool_t* pool, const actkv_tables_t* tables, int32_t layer_begin,
-                          int32_t layer_end, const int32_t* sel_idx, int64_t sel_stride,
-                          const int32_t* keep_indptr, const int32_t* budget, int32_t max_keep,
-                          int32_t* new_order, int32_t* status, actkv_stream_t stream) {
+static int inplace_check(const actkv_pool_t* pool, const actkv_tables_t* tables, int32_t layer_begin, int32_t layer_end,
+                         const int32_t* sel_idx, int64_t sel_stride, const int32_t* keep_indptr, const int32_t* budget,
+                         int32_t max_keep) {
   if (!pool || !tables || !pool->base) return ACTKV_E_INVALID;
   if (layer_begin < 0 || layer_end > pool->n_layers || layer_begin > layer_end) return ACTKV_E_INVALID;
   if (pool->page_size <= 0 || pool->head_dim <= 0 || pool->head_dim % 8 != 0 || pool->n_kv_heads <= 0)
@@ -222,31 +367,135 @@ int actkv_compact_inplace(const actkv_pool_t* pool, const actkv_tables_t* tables
     return ACTKV_E_INVALID;
   const int64_t nz = (int64_t)(layer_end - layer_begin) * pool->n_kv_heads;
   if (R > 65535 || nz > 65535) return ACTKV_E_INVALID;
-  cudaStream_t s = (cudaStream_t)stream;
-  actkv::PoolView pv = actkv::make_view(pool);
-  actkv::TablesView tv = actkv::make_view(tables);
+  return ACTKV_OK;
+}
+
+// The whole copy of a call in one launch.
+static int inplace_copy_all(const actkv_pool_t* pool, const actkv_tables_t* tables, int32_t layer_begin, int32_t layer_end,
+                            const int32_t* sel_idx, int64_t sel_stride, const int32_t* keep_indptr, const int32_t* budget,
+                            int32_t max_keep, int32_t* new_order, int32_t* status, cudaStream_t s) {
+  const int R = tables->n_req;
+  const int64_t nz = (int64_t)(layer_end - layer_begin) * pool->n_kv_heads;
+  PoolView pv = make_view(pool);
+  TablesView tv = make_view(tables);
   if (nz > 0 && max_keep > 0) {
-    dim3 grid((unsigned)((max_keep + actkv::CI_NT - 1) / actkv::CI_NT), (unsigned)R, (unsigned)nz);
+    dim3 grid((unsigned)((max_keep + CI_NT - 1) / CI_NT), (unsigned)R, (unsigned)nz);
     const int vpr = pool->head_dim / 8;
     if (vpr == 16)
-      actkv::compact_inplace_copy_kernel<4><<<grid, actkv::CI_NT, 0, s>>>(pv, tv, layer_begin, sel_idx, sel_stride,
-                                                                          keep_indptr, budget, max_keep, new_order, status);
+      compact_inplace_copy_kernel<4><<<grid, CI_NT, 0, s>>>(pv, tv, layer_begin, sel_idx, sel_stride, keep_indptr, budget,
+                                                            max_keep, new_order, status);
     else if (vpr == 8)
-      actkv::compact_inplace_copy_kernel<3><<<grid, actkv::CI_NT, 0, s>>>(pv, tv, layer_begin, sel_idx, sel_stride,
-                                                                          keep_indptr, budget, max_keep, new_order, status);
+      compact_inplace_copy_kernel<3><<<grid, CI_NT, 0, s>>>(pv, tv, layer_begin, sel_idx, sel_stride, keep_indptr, budget,
+                                                            max_keep, new_order, status);
     else if (vpr == 32)
-      actkv::compact_inplace_copy_kernel<5><<<grid, actkv::CI_NT, 0, s>>>(pv, tv, layer_begin, sel_idx, sel_stride,
-                                                                          keep_indptr, budget, max_keep, new_order, status);
+      compact_inplace_copy_kernel<5><<<grid, CI_NT, 0, s>>>(pv, tv, layer_begin, sel_idx, sel_stride, keep_indptr, budget,
+                                                            max_keep, new_order, status);
     else
-      actkv::compact_inplace_copy_kernel<-1><<<grid, actkv::CI_NT, 0, s>>>(pv, tv, layer_begin, sel_idx, sel_stride,
-                                                                           keep_indptr, budget, max_keep, new_order, status);
-    ACTKV_CHECK_LAUNCH();
-  }
-  if (layer_end == pool->n_layers) {
-    actkv::compact_inplace_finalize_kernel<<<1, 1024, 0, s>>>(tv, pool->page_size, pool->n_pages, budget, status);
+      compact_inplace_copy_kernel<-1><<<grid, CI_NT, 0, s>>>(pv, tv, layer_begin, sel_idx, sel_stride, keep_indptr, budget,
+                                                             max_keep, new_order, status);
     ACTKV_CHECK_LAUNCH();
   }
   return ACTKV_OK;
+}
+
+static int inplace_finalize(const actkv_pool_t* pool, const actkv_tables_t* tables, int32_t layer_end, const int32_t* budget,
+                            int32_t* status, cudaStream_t s) {
+  if (layer_end == pool->n_layers) {
+    compact_inplace_finalize_kernel<<<1, 1024, 0, s>>>(make_view(tables), pool->page_size, pool->n_pages, budget, status);
+    ACTKV_CHECK_LAUNCH();
+  }
+  return ACTKV_OK;
+}
+
+// Items of the largest job these arguments allow, per layer.
+static int64_t inplace_items_per_layer(const actkv_pool_t* pool, int32_t n_req, int32_t max_keep) {
+  return (int64_t)pool->n_kv_heads * n_req * (((int64_t)max_keep + 31) / 32);
+}
+static size_t inplace_ws_base(int32_t n_req) {
+  return align_up(sizeof(CompactWs) + sizeof(int32_t) * ((size_t)3 * n_req + 1), 256);
+}
+
+}  // namespace actkv
+
+extern "C" {
+
+int actkv_compact_inplace(const actkv_pool_t* pool, const actkv_tables_t* tables, int32_t layer_begin,
+                          int32_t layer_end, const int32_t* sel_idx, int64_t sel_stride,
+                          const int32_t* keep_indptr, const int32_t* budget, int32_t max_keep,
+                          int32_t* new_order, int32_t* status, actkv_stream_t stream) {
+  using namespace actkv;
+  int rc = inplace_check(pool, tables, layer_begin, layer_end, sel_idx, sel_stride, keep_indptr, budget, max_keep);
+  if (rc != ACTKV_OK || tables->n_req == 0) return rc;
+  cudaStream_t s = (cudaStream_t)stream;
+  rc = inplace_copy_all(pool, tables, layer_begin, layer_end, sel_idx, sel_stride, keep_indptr, budget, max_keep, new_order,
+                        status, s);
+  if (rc != ACTKV_OK) return rc;
+  return inplace_finalize(pool, tables, layer_end, budget, status, s);
+}
+
+size_t actkv_compact_inplace_deferred_workspace_bytes(const actkv_pool_t* pool, int32_t n_req, int32_t n_layers_sub,
+                                                      int32_t max_keep) {
+  if (!pool || n_req < 0 || n_layers_sub < 0 || max_keep < 0 || pool->n_kv_heads <= 0) return 0;
+  const int64_t items = actkv::inplace_items_per_layer(pool, n_req, max_keep) * n_layers_sub;
+  return actkv::inplace_ws_base(n_req) + 2 * actkv::align_up((size_t)items * 32 * sizeof(uint32_t), 256);
+}
+
+int actkv_compact_inplace_begin(const actkv_pool_t* pool, const actkv_tables_t* tables, int32_t layer_begin,
+                                int32_t layer_end, const int32_t* sel_idx, int64_t sel_stride,
+                                const int32_t* keep_indptr, const int32_t* budget, int32_t max_keep,
+                                int32_t* new_order, void* ws, size_t ws_bytes, int32_t* status, actkv_stream_t stream) {
+  using namespace actkv;
+  int rc = inplace_check(pool, tables, layer_begin, layer_end, sel_idx, sel_stride, keep_indptr, budget, max_keep);
+  if (rc != ACTKV_OK || tables->n_req == 0) return rc;
+  if (!ws || ws_bytes < inplace_ws_base(tables->n_req)) return ACTKV_E_WORKSPACE;
+  cudaStream_t s = (cudaStream_t)stream;
+  const int nl = layer_end - layer_begin;
+  const int shift = deferrable_shift(pool);
+  const int64_t items_max = inplace_items_per_layer(pool, tables->n_req, max_keep) * nl;
+  const bool deferred = shift >= 0 && items_max <= 0x7fffffff &&
+                        ws_bytes >= actkv_compact_inplace_deferred_workspace_bytes(pool, tables->n_req, nl, max_keep);
+  const size_t base = inplace_ws_base(tables->n_req);
+  const size_t tab_bytes = align_up((size_t)(deferred ? items_max : 0) * 32 * sizeof(uint32_t), 256);
+  uint32_t* src_tab = (uint32_t*)((char*)ws + base);
+  uint32_t* dst_tab = (uint32_t*)((char*)ws + base + tab_bytes);
+  // (not deferred: an empty job, so that a score call given this workspace finds nothing to do; actkv_compact_inplace_end
+  //  then copies everything itself)
+  compact_inplace_plan_kernel<<<1, 32, 0, s>>>(make_view(tables), make_view(pool), budget, max_keep,
+                                               new_order != nullptr ? 1 : 0, layer_begin, deferred ? nl : 0,
+                                               deferred ? shift : -1, src_tab, dst_tab, deferred ? items_max : 0,
+                                               (CompactWs*)ws, status);
+  ACTKV_CHECK_LAUNCH();
+  if (deferred && items_max > 0) {
+    const int64_t ctas = std::min<int64_t>(std::max<int64_t>(1, (items_max + 3) / 4), 1 << 20);
+    compact_inplace_resolve_kernel<<<(unsigned)ctas, 128, 0, s>>>((CompactWs*)ws, sel_idx, sel_stride, keep_indptr, new_order);
+    ACTKV_CHECK_LAUNCH();
+  }
+  return ACTKV_OK;
+}
+
+int actkv_compact_inplace_end(const actkv_pool_t* pool, const actkv_tables_t* tables, int32_t layer_begin,
+                              int32_t layer_end, const int32_t* sel_idx, int64_t sel_stride,
+                              const int32_t* keep_indptr, const int32_t* budget, int32_t max_keep,
+                              int32_t* new_order, void* ws, size_t ws_bytes, int32_t* status, actkv_stream_t stream) {
+  using namespace actkv;
+  int rc = inplace_check(pool, tables, layer_begin, layer_end, sel_idx, sel_stride, keep_indptr, budget, max_keep);
+  if (rc != ACTKV_OK || tables->n_req == 0) return rc;
+  if (!ws || ws_bytes < inplace_ws_base(tables->n_req)) return ACTKV_E_WORKSPACE;
+  cudaStream_t s = (cudaStream_t)stream;
+  const int nl = layer_end - layer_begin;
+  const int shift = deferrable_shift(pool);
+  const int64_t items_max = inplace_items_per_layer(pool, tables->n_req, max_keep) * nl;
+  const bool deferred = shift >= 0 && items_max <= 0x7fffffff &&
+                        ws_bytes >= actkv_compact_inplace_deferred_workspace_bytes(pool, tables->n_req, nl, max_keep);
+  if (!deferred) {
+    rc = inplace_copy_all(pool, tables, layer_begin, layer_end, sel_idx, sel_stride, keep_indptr, budget, max_keep, new_order,
+                          status, s);
+    if (rc != ACTKV_OK) return rc;
+  } else if (items_max > 0) {
+    launch_drain((CompactWs*)ws, shift, items_max, s);
+    ACTKV_CHECK_LAUNCH();
+  }
+  return inplace_finalize(pool, tables, layer_end, budget, status, s);
 }
 
 }  // extern "C"

@@ -29,8 +29,12 @@ struct CompactWs {
   int32_t vpr_shift;     // log2 of the 16-byte vectors per row (3, 4, 5 for head_dim 64, 128, 256); -1: not deferrable
   int32_t parts_per_page;  // items per destination page: ceil(page_size x heads / 32)
   int32_t role_items;    // items executed by copy roles of other kernels (the rest went to the drain kernel)
-  int32_t pad;           // CJ_PLAN_MARK once a plan kernel has written this workspace
+  int32_t pad;           // CJ_PLAN_MARK / CJ_INPLACE_MARK once a plan kernel has written this workspace
   uint32_t* src_tab;     // deferred copy: resolved sources, [n_items][32] (see cj_resolve_item)
+  uint32_t* dst_tab;     // deferred in-place copy: resolved destinations, [n_items][32]; nullptr for the fresh-page form,
+                         // whose destinations follow from the item number
+  int32_t items_per_slab;  // items of one layer (>= 1): the layer of an item is item / items_per_slab
+  int32_t pad2;
   // followed by int32 new_off[R], push_off[R], item_off[R + 1], new_pages[R * max_pages]
 };
 
@@ -40,7 +44,8 @@ __host__ __device__ __forceinline__ int32_t* ws_item_off(CompactWs* w, int R) { 
 __host__ __device__ __forceinline__ int32_t* ws_new_pages(CompactWs* w, int R) { return ws_new_off(w) + 3 * R + 1; }
 
 constexpr uint32_t CJ_NONE = 0xffffffffu;
-constexpr int32_t CJ_PLAN_MARK = 0x414b5650;
+constexpr int32_t CJ_PLAN_MARK = 0x414b5650;      // a fresh-page plan
+constexpr int32_t CJ_INPLACE_MARK = 0x414b5649;   // an in-place job
 
 __device__ __forceinline__ uint4 ld_stream(const uint4* p) {
   uint4 v;
@@ -107,18 +112,24 @@ __device__ __forceinline__ void cj_resolve_item(CompactWs* w, int item, int lane
 template <int VPR_SHIFT, int NFLY>
 __device__ __forceinline__ void cj_copy_item(CompactWs* w, int item, int lane) {
   const PoolView& pool = w->pool;
-  const int H = pool.n_kv_heads;
-  const int jp = w->parts_per_page;                    // items per destination page: ceil(P H / 32)
-  const int page_item = item / jp, j = item - page_item * jp;
-  const int total_new = w->total_new;
-  const int slab = page_item / total_new, rem = page_item - slab * total_new;
+  const int ips = w->items_per_slab;
+  const int slab = item / ips;
   // the two lookups of an item, independent of each other
   const uint32_t so = w->src_tab[(int64_t)item * 32 + lane];
-  const int32_t dst_page = ws_new_pages(w, w->tab.n_req)[rem];
-  const int i = lane + 32 * j;
-  const int slot = i / H, h = i - slot * H;
-  const uint32_t dof = (uint32_t)(((int64_t)dst_page * pool.stride_page + (int64_t)slot * pool.stride_slot +
-                                   (int64_t)h * pool.stride_head) >> 3);
+  uint32_t dof;
+  if (w->dst_tab != nullptr) {                         // (uniform over the job) in-place form: resolved destinations
+    dof = w->dst_tab[(int64_t)item * 32 + lane];
+  } else {
+    const int H = pool.n_kv_heads;
+    const int jp = w->parts_per_page;                  // items per destination page: ceil(P H / 32)
+    const int rem_item = item - slab * ips;
+    const int rem = rem_item / jp, j = rem_item - rem * jp;
+    const int32_t dst_page = ws_new_pages(w, w->tab.n_req)[rem];
+    const int i = lane + 32 * j;
+    const int slot = i / H, h = i - slot * H;
+    dof = (uint32_t)(((int64_t)dst_page * pool.stride_page + (int64_t)slot * pool.stride_slot +
+                      (int64_t)h * pool.stride_head) >> 3);
+  }
   uint4* lbase = reinterpret_cast<uint4*>(const_cast<__nv_bfloat16*>(pool.base) +
                                           (int64_t)(w->layer_begin + slab) * pool.stride_layer);
   constexpr int RPS = 32 >> VPR_SHIFT;                 // rows per step (one 16-byte vector per lane): 4, 2, 1
@@ -171,6 +182,42 @@ __device__ __forceinline__ void cj_copy_role(CompactWs* w, int lane, KeepGoing k
     item = next;
   }
   if (lane == 0 && done > 0) atomicAdd(&w->role_items, done);
+}
+
+// What is left of a deferred copy: every warp takes items until the queue is empty.
+template <int VPR_SHIFT>
+__global__ void __launch_bounds__(128) compact_drain_kernel(CompactWs* ws) {
+  const int lane = threadIdx.x & 31;
+  if (ws->vpr_shift != VPR_SHIFT) return;
+  const uint32_t n = cj_count(ws);
+  if (n == 0) return;
+  uint32_t item = cj_pop(ws, lane);
+  while (item < n) {
+    const uint32_t next = cj_pop(ws, lane);              // asked for now, looked at after this item's copies
+    cj_copy_item<VPR_SHIFT, 16>(ws, (int)item, lane);
+    item = next;
+  }
+}
+
+// Launches the drain kernel for a job of at most `items_max` items: at most eight CTAs of four warps per SM.
+inline void launch_drain(CompactWs* w, int shift, int64_t items_max, cudaStream_t s) {
+  const int64_t want = (items_max + 3) / 4;
+  const unsigned grid = (unsigned)(want < 1 ? 1 : (want > 148 * 8 ? 148 * 8 : want));
+  if (shift == 3) compact_drain_kernel<3><<<grid, 128, 0, s>>>(w);
+  else if (shift == 4) compact_drain_kernel<4><<<grid, 128, 0, s>>>(w);
+  else compact_drain_kernel<5><<<grid, 128, 0, s>>>(w);
+}
+
+// log2 of the 16-byte vectors per row when the warp-level item copy takes this pool: head_dim 64, 128 or 256,
+// a layer (K and V) within 2^32 16-byte units; else -1.
+inline int deferrable_shift(const actkv_pool_t* pool) {
+  const int vpr = pool->head_dim / 8;
+  const int shift = vpr == 8 ? 3 : vpr == 16 ? 4 : vpr == 32 ? 5 : -1;
+  if (shift < 0) return -1;
+  const int64_t extent = pool->stride_kv + (int64_t)pool->n_pages * pool->stride_page;       // elements, upper bound
+  if (pool->stride_kv < 0 || pool->stride_page < 0 || pool->stride_slot < 0 || pool->stride_head < 0) return -1;
+  if (extent / 8 >= 0xffffffffLL) return -1;
+  return shift;
 }
 
 }  // namespace actkv

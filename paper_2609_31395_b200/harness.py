@@ -64,7 +64,9 @@ class Compressor:
         # (sized for the pipelined step as well: room for the resolved sources of one layer group)
         self.ws_compact = _ws(max(B.actkv_compact_workspace_bytes(s.n_req, self.td.max_pages),
                                   B.actkv_compact_deferred_workspace_bytes(self.pd, s.n_req, self.td.max_pages, self.lpc,
-                                                                           s.max_keep)), self.dev)
+                                                                           s.max_keep),
+                                  B.actkv_compact_inplace_deferred_workspace_bytes(self.pd, s.n_req, self.lpc, s.max_keep)),
+                              self.dev)
 
     # -- single stages (whole layer range unless given) ------------------------------------------
     def run_score(self, q, win_indptr, tok_indptr, sm_scale, causal, l0=0, l1=None, lse_in=None, stream=None):
@@ -178,12 +180,13 @@ class Compressor:
         return launches
 
     def step_pipelined(self, q, win_indptr, tok_indptr, budget, sm_scale, causal, lse_in=None, stream=None, marks=None,
-                       groups=None, stats=None):
+                       groups=None, stats=None, inplace=False):
         """score -> select -> compact over all layers with the copies of layer group g running inside the
         score kernels of group g+1 (actkv_compact_begin / actkv_score_overlap / actkv_compact_end), all on one
         stream.  `groups`: list of (l0, l1) layer ranges, each at most `layers_per_call` long (default: equal
         groups of `layers_per_call`); the copies of the last group are not hidden, so a short last group
-        exposes less.  Results are those of step().  Returns the number of kernels launched."""
+        exposes less.  Results are those of step().  inplace: Algorithm 4's in-place compaction instead of fresh
+        pages (actkv_compact_inplace_begin / _end).  Returns the number of kernels launched."""
         NL, Hkv, s = self.pd.n_layers, self.pd.n_kv_heads, self.sz
         if groups is None:
             groups = [(l0, min(NL, l0 + self.lpc)) for l0 in range(0, NL, self.lpc)]
@@ -220,8 +223,13 @@ class Compressor:
                     done.append(prev)
                     launches += 1
                 launches += 1                       # the drain kernel
-                B.actkv_compact_end(self.pd, self.td, prev[0], prev[1], self.sel_idx, s.sel_stride, self.keep_indptr,
-                                    budget, s.max_keep, self.ws_compact, self.status, stream)
+                if inplace:
+                    B.actkv_compact_inplace_end(self.pd, self.td, prev[0], prev[1], self.sel_idx, s.sel_stride,
+                                                self.keep_indptr, budget, s.max_keep, None, self.ws_compact, self.status,
+                                                stream)
+                else:
+                    B.actkv_compact_end(self.pd, self.td, prev[0], prev[1], self.sel_idx, s.sel_stride, self.keep_indptr,
+                                        budget, s.max_keep, self.ws_compact, self.status, stream)
                 mark("compact")
             self.run_select(tok_indptr, budget, l1 - l0, stream)
             mark("select")
@@ -229,10 +237,20 @@ class Compressor:
             if l1 == NL:
                 # nothing follows the last group that could carry its copies: the one-launch copy of actkv_compact
                 # (a CTA per destination page) is a little faster than draining a queue
+                if inplace:
+                    B.actkv_compact_inplace(self.pd, self.td, l0, l1, self.sel_idx, s.sel_stride, self.keep_indptr, budget,
+                                            s.max_keep, None, self.status, stream)
+                    mark("compact")
+                    return launches + 2             # copy, finalize
                 self.run_compact(budget, l0, l1, stream)
                 mark("compact")
                 return launches + 3                 # plan, copy, finalize
             launches += 2                           # plan (or the job record when the plan is reused), resolve
+            if inplace:
+                B.actkv_compact_inplace_begin(self.pd, self.td, l0, l1, self.sel_idx, s.sel_stride, self.keep_indptr,
+                                              budget, s.max_keep, None, self.ws_compact, self.status, stream)
+                prev = (l0, l1)
+                continue
             B.actkv_compact_begin(self.pd, self.td, l0, l1, self.sel_idx, s.sel_stride, self.keep_indptr, budget,
                                   s.max_keep, self.ws_compact, self.status, stream, reuse_plan=prev is not None)
             prev = (l0, l1)

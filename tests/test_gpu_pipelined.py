@@ -192,3 +192,31 @@ def test_reusing_a_plan_that_is_not_there_is_reported_and_nothing_moves():
     assert np.array_equal(U.bits(b.pool), snap[0])
     for t, s0 in zip((b.page_table, b.seq_len, b.free_list, b.free_count), snap[1:]):
         assert torch.equal(t, s0)
+
+
+@pytest.mark.parametrize("causal", [False, True])
+def test_pipelined_in_place_step_equals_the_one_call_in_place_step(causal):
+    """Algorithm 4's in-place compaction with the moves of a layer group executed inside the pooled-score kernel of
+    the next group (actkv_compact_inplace_begin / actkv_score_overlap / actkv_compact_inplace_end): pool, tables and
+    free list bit for bit those of the one-call in-place step, which tests/test_gpu_compact_inplace.py holds
+    against the oracle."""
+    wl = synth.Workload("pipe-ip", 7, 2, 8, [1500, 333, 700, 90, 260], [32, 16, 24, 8, 32], [400, 100, 200, 90, 0],
+                        table_style="fragmented", causal=causal, seed=57, poison_tail=True)
+    a = synth.generate(wl, DEV)
+    comp_a = H.Compressor(a.pool, a.page_table, a.seq_len, a.free_list, a.free_count, wl.n_q_heads, H.sizes_of(a),
+                          want_lse=True)
+    comp_a.step(a.q, a.win_indptr, a.tok_indptr, a.budget, wl.sm_scale, wl.causal, inplace=True)
+    torch.cuda.synchronize()
+    comp_a.check_status()
+    for lpc, lse_in in ((2, None), (3, comp_a.lse)):
+        b = synth.generate(wl, DEV)
+        comp_b = H.Compressor(b.pool, b.page_table, b.seq_len, b.free_list, b.free_count, wl.n_q_heads, H.sizes_of(b),
+                              layers_per_call=lpc, want_lse=True)
+        stats = torch.zeros((8, 2), dtype=torch.int32, device=DEV)
+        comp_b.step_pipelined(b.q, b.win_indptr, b.tok_indptr, b.budget, wl.sm_scale, wl.causal, lse_in=lse_in, inplace=True,
+                              stats=stats)
+        torch.cuda.synchronize()
+        comp_b.check_status()
+        _same_state(a, b)
+        st = stats.cpu().numpy()
+        assert st[0, 0] > 0 and (st[:, 1] <= st[:, 0]).all()          # a queue was published for the first group

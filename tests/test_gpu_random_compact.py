@@ -1,7 +1,8 @@
-"""Seeded random cases of the three compaction forms called directly, with random ascending keep lists (not
+"""Seeded random cases of the compaction forms called directly, with random ascending keep lists (not
 from TopK) on random pool bits: the fresh-page compaction in one call (actkv_compact), the same split into
-actkv_compact_begin / actkv_compact_end (work queue, resolve table, drain kernel), and the in-place tail
-compaction (Algorithm 4), each against the oracle on every byte of the pool, the tables and the free list.
+actkv_compact_begin / actkv_compact_end (work queue, resolve table, drain kernel), the in-place tail
+compaction (Algorithm 4) in one call and split into actkv_compact_inplace_begin / _end, each against the oracle
+on every byte of the pool, the tables and the free list.
 Shapes the step never produces are drawn on purpose: pages of 4 to 64 tokens, 1 to 8 KV heads, head
 dimensions whose rows are not a power of two of 16-byte vectors, requests shorter than a page.
 """
@@ -51,7 +52,7 @@ def _check_fresh(inst, want_pool, want_t):
 
 
 @pytest.mark.parametrize("seed", range(24))
-@pytest.mark.parametrize("form", ["one call", "begin + end", "in place"])
+@pytest.mark.parametrize("form", ["one call", "begin + end", "in place", "in place, begin + end"])
 def test_random_compaction(seed, form):
     rng, P, Hkv, D, NL, lens, budgets = _draw(seed)
     inst, sel, ki, stride, max_keep = TI._direct_case(rng, lens, budgets, P, Hkv, D, NL)
@@ -67,6 +68,24 @@ def test_random_compaction(seed, form):
         torch.cuda.synchronize()
         assert status.cpu().tolist()[0] == 0, status.cpu().tolist()
         TI._check_against_oracle(inst, pool_before, tables_before, sel, ki, budgets, d_order.cpu().numpy())
+        return
+    if form == "in place, begin + end":
+        d_order = torch.full_like(d_sel, -9) if seed % 2 == 0 else None
+        ws = torch.empty(B.actkv_compact_inplace_deferred_workspace_bytes(pd, len(lens), 1, max_keep) + 16,
+                         dtype=torch.uint8, device=DEV)
+        ws.fill_(0x5A)
+        for l in range(NL):                               # layer by layer; the tables change with the last one
+            rows = slice(l * Hkv, (l + 1) * Hkv)
+            args = (pd, td, l, l + 1, d_sel[rows], stride, d_ki, d_bud, max_keep, None if d_order is None else d_order[rows],
+                    ws, status)
+            B.actkv_compact_inplace_begin(*args)
+            B.actkv_compact_inplace_end(*args)
+        torch.cuda.synchronize()
+        assert status.cpu().tolist()[0] == 0, status.cpu().tolist()
+        TI._check_against_oracle(inst, pool_before, tables_before, sel, ki, budgets,
+                                 None if d_order is None else d_order.cpu().numpy())
+        if d_order is not None:
+            assert (d_order.cpu().numpy()[:, ki[-1]:] == -9).all()
         return
     want_pool, want_t = _fresh_page_oracle(inst, pool_before, tables_before, sel, ki, budgets, NL)
     if form == "one call":
