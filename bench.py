@@ -356,10 +356,10 @@ def run_ours(args):
         if args.overlap:
             n = comp.step_overlapped(inst.q, inst.win_indptr, inst.tok_indptr, bud, wl.sm_scale, wl.causal,
                                      lse_in=lse_supplied, marks=mark)
-        elif pipelined and lrfu_state is None and (not inplace_mode or inplace_pipe):
+        elif pipelined and (not inplace_mode or inplace_pipe) and not (inplace_mode and lrfu_state is not None):
             n = pipe_comp.step_pipelined(inst.q, inst.win_indptr, inst.tok_indptr, bud, wl.sm_scale, wl.causal,
                                          lse_in=lse_supplied, marks=(lambda nm: mark(nm)), groups=pipe_groups,
-                                         stats=pipe_stats, inplace=inplace_mode)
+                                         stats=pipe_stats, inplace=inplace_mode, lrfu=lrfu_state)
         else:
             n = comp.step(inst.q, inst.win_indptr, inst.tok_indptr, bud, wl.sm_scale, wl.causal,
                           lse_in=lse_supplied, marks=(lambda nm: mark(nm)), lrfu=lrfu_state, inplace=inplace_mode)
@@ -595,8 +595,11 @@ def run_ours(args):
                      "keepscore_frac_of_hbm_peak": ks_bytes / (ks * 1e-3) / 1e9 / pk["hbm_gbs"],
                      "keepscore_stage": "keep-score update and TopK in one launch (actkv_keepscore_select); the separate "
                                         "select stage is empty",
-                     "top_p": 0.9, "lambda": 0.5, "n_protect": 512}
+                     "top_p": 0.9, "lambda": 0.5, "n_protect": 512,
+                     "form": "pipelined like the timed step" if pipelined else "one call per stage"}
         comp.check_status()
+        if pipe_comp is not None:
+            pipe_comp.check_status()
 
     # ---- streaming form (Algorithm 3 as triggered per decode step): one action query per request per call,
     # LSE supplied, running mean updated in place; all layers in one call.  Bound by the K reads.

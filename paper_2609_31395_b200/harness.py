@@ -180,13 +180,15 @@ class Compressor:
         return launches
 
     def step_pipelined(self, q, win_indptr, tok_indptr, budget, sm_scale, causal, lse_in=None, stream=None, marks=None,
-                       groups=None, stats=None, inplace=False):
+                       groups=None, stats=None, inplace=False, lrfu: Optional["LrfuState"] = None):
         """score -> select -> compact over all layers with the copies of layer group g running inside the
         score kernels of group g+1 (actkv_compact_begin / actkv_score_overlap / actkv_compact_end), all on one
         stream.  `groups`: list of (l0, l1) layer ranges, each at most `layers_per_call` long (default: equal
         groups of `layers_per_call`); the copies of the last group are not hidden, so a short last group
         exposes less.  Results are those of step().  inplace: Algorithm 4's in-place compaction instead of fresh
-        pages (actkv_compact_inplace_begin / _end).  Returns the number of kernels launched."""
+        pages (actkv_compact_inplace_begin / _end).  lrfu (fresh-page form only): rank by the LRFU keep-score, as
+        step() does.  Returns the number of kernels launched."""
+        assert lrfu is None or not inplace
         NL, Hkv, s = self.pd.n_layers, self.pd.n_kv_heads, self.sz
         if groups is None:
             groups = [(l0, min(NL, l0 + self.lpc)) for l0 in range(0, NL, self.lpc)]
@@ -231,7 +233,13 @@ class Compressor:
                     B.actkv_compact_end(self.pd, self.td, prev[0], prev[1], self.sel_idx, s.sel_stride, self.keep_indptr,
                                         budget, s.max_keep, self.ws_compact, self.status, stream)
                 mark("compact")
-            self.run_select(tok_indptr, budget, l1 - l0, stream)
+            if lrfu is not None:
+                self.run_keepscore_select(lrfu, tok_indptr, budget, l0, l1, stream)
+                mark("keepscore")
+                self.run_gather_ks(lrfu, tok_indptr, l0, l1, stream)
+                launches += 1
+            else:
+                self.run_select(tok_indptr, budget, l1 - l0, stream)
             mark("select")
             launches += (3 if lse_in is None else 1) + 1      # score kernels, select
             if l1 == NL:

@@ -220,3 +220,32 @@ def test_pipelined_in_place_step_equals_the_one_call_in_place_step(causal):
         _same_state(a, b)
         st = stats.cpu().numpy()
         assert st[0, 0] > 0 and (st[:, 1] <= st[:, 0]).all()          # a queue was published for the first group
+
+
+def test_pipelined_step_with_the_lrfu_policy_equals_the_one_call_form():
+    """Ranking by the LRFU keep-score (Section 5.1) in the pipelined step: pool, tables, persistent keep-scores and
+    the survivors' keep-scores bit for bit those of the one-call form (held against the oracle in
+    tests/test_gpu_keepscore.py)."""
+    wl = synth.Workload("pipe-lrfu", 5, 2, 8, [1500, 333, 700, 90], [32, 16, 24, 8], [400, 100, 200, 90],
+                        table_style="fragmented", seed=58, poison_tail=True)
+    out = []
+    for lpc in (None, 2):
+        a = synth.generate(wl, DEV)
+        sz = H.sizes_of(a)
+        comp = H.Compressor(a.pool, a.page_table, a.seq_len, a.free_list, a.free_count, wl.n_q_heads, sz, layers_per_call=lpc)
+        lrfu = H.LrfuState(wl.n_layers * wl.n_kv_heads, sz, DEV, 0.9, 0.5,
+                           torch.tensor([4, 0, 300, 7], dtype=torch.int32, device=DEV), want_hits=True)
+        lrfu.keep_score.uniform_(0.0, 1e-3, generator=torch.Generator(device=DEV).manual_seed(3))
+        if lpc is None:
+            comp.step(a.q, a.win_indptr, a.tok_indptr, a.budget, wl.sm_scale, wl.causal, lrfu=lrfu)
+        else:
+            comp.step_pipelined(a.q, a.win_indptr, a.tok_indptr, a.budget, wl.sm_scale, wl.causal, lrfu=lrfu)
+        torch.cuda.synchronize()
+        comp.check_status()
+        out.append((a, lrfu))
+    (a, la), (b, lb) = out
+    _same_state(a, b)
+    assert torch.equal(la.keep_score.view(torch.int32), lb.keep_score.view(torch.int32))
+    assert torch.equal(la.hit_mask, lb.hit_mask)
+    n_keep = sum(min(x, L) for x, L in zip(wl.budgets, wl.seq_lens))
+    assert torch.equal(la.kept[:, :n_keep].view(torch.int32), lb.kept[:, :n_keep].view(torch.int32))
