@@ -14,7 +14,7 @@ from paper_2609_31395_b200 import synth
 
 pytestmark = pytest.mark.gpu
 DEV = "cuda:0"
-SLEEP_CYCLES = 150_000_000          # about 0.1 s
+SLEEP_CYCLES = 800_000_000          # about 0.4 s: far longer than the host needs to queue a step
 
 
 def _wl():
