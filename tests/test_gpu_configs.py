@@ -394,3 +394,40 @@ def test_config5_agent_trace_25_rounds():
     print(f"c5: index lists of {ties['units']} sampled units differ from TopK of the oracle's scores in {ties['n']} entries "
           f"(within the tie tolerance)")
     assert 40000 <= min(final_uncompressed) and max(final_uncompressed) <= 90000
+
+
+def test_config3_in_the_launch_configuration_the_benchmark_times():
+    """The benchmark's timed step at full size: the LSE pass of all 48 layers in one launch, then three groups of
+    16 layers whose copies run inside the pooled-score kernel of the next group.  Scores of sampled units of the
+    last group (every head, several requests) against the oracle; every byte of the 35 GB pool, the tables and the
+    free list against the one-call step on a second copy of the inputs (the form the test above holds against the
+    oracle); the copy role must have taken items."""
+    wl = synth.config3()
+    a = synth.generate(wl, DEV)
+    comp_a = U.run_step(a)
+    comp_a.check_status()
+    b = synth.generate(wl, DEV)
+    pt_before, sl_before = b.page_table.clone(), b.seq_len.clone()
+    comp_b = H.Compressor(b.pool, b.page_table, b.seq_len, b.free_list, b.free_count, wl.n_q_heads, H.sizes_of(b),
+                          layers_per_call=16, want_lse=True, lse_layers_per_call=wl.n_layers)
+    stats = torch.zeros((3, 2), dtype=torch.int32, device=DEV)
+    comp_b.step_pipelined(b.q, b.win_indptr, b.tok_indptr, b.budget, wl.sm_scale, wl.causal,
+                          groups=[(0, 16), (16, 32), (32, 48)], stats=stats)
+    torch.cuda.synchronize()
+    comp_b.check_status()
+    st = stats.cpu().numpy()
+    assert (st[:2, 0] > 0).all() and (st[:2, 1] > 0).all(), st          # queues of the first two groups, served by the role
+    assert torch.equal(comp_a.lse, comp_b.lse)
+    assert torch.equal(a.pool.view(torch.int16), b.pool.view(torch.int16))
+    assert torch.equal(a.page_table, b.page_table) and torch.equal(a.seq_len, b.seq_len)
+    assert torch.equal(a.free_list, b.free_list) and torch.equal(a.free_count, b.free_count)
+    del a, comp_a
+    # the score buffer holds the last group (layers 32..47): slab 15 = layer 47, slab 0 = layer 32
+    wl_like = (wl.n_kv_heads, wl.group, wl.head_dim, wl.page_size, wl.causal, wl.sm_scale)
+    units = [(15, 0, 7), (15, 1, 0), (15, 2, 1), (15, 3, 2), (0, 0, 4), (0, 3, 6)]
+    # (the pool's old pages still hold the keys: fresh-page compaction leaves them as they were)
+    worst = _check_sampled_scores(b.pool, pt_before, sl_before, b.q[32:], b.win_indptr, b.tok_indptr, wl_like,
+                                  comp_b.score, units, layer_of_slab={s: 32 + s for s in range(16)},
+                                  budgets=wl.budgets, sel_idx=comp_b.sel_idx, keep_indptr=comp_b.keep_indptr)
+    print(f"c3, pipelined 16+16+16: score max-rel {worst:.2e} on {len(units)} sampled units of the last group; "
+          f"copy items served by the pooled-score kernels: {st[:2, 1].tolist()} of {st[:2, 0].tolist()}")
