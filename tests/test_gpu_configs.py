@@ -431,3 +431,44 @@ def test_config3_in_the_launch_configuration_the_benchmark_times():
                                   budgets=wl.budgets, sel_idx=comp_b.sel_idx, keep_indptr=comp_b.keep_indptr)
     print(f"c3, pipelined 16+16+16: score max-rel {worst:.2e} on {len(units)} sampled units of the last group; "
           f"copy items served by the pooled-score kernels: {st[:2, 1].tolist()} of {st[:2, 0].tolist()}")
+
+
+def test_config3_through_host_buffers_full_size():
+    """The end-to-end form the benchmark times (one actkv_step_host call, queries and tables from pinned host
+    memory, layer groups of 16) at full size (budgets given, no logits):
+    sampled scores of the last group against the oracle, two whole layers of the compaction against the oracle's
+    compaction of the GPU's lists, the tables that come back to the host, planted keys kept."""
+    wl = synth.config3()
+    b = synth.generate(wl, DEV)
+    tables_before = U.oracle_tables(b)
+    pt_before, sl_before = b.page_table.clone(), b.seq_len.clone()
+    snap = {l: b.pool[l].clone() for l in (32, 47)}
+    comp = H.Compressor(b.pool, b.page_table, b.seq_len, b.free_list, b.free_count, wl.n_q_heads, H.sizes_of(b),
+                        layers_per_call=16, want_lse=False, lse_layers_per_call=wl.n_layers)
+    comp.lse = torch.empty((wl.n_layers, comp.sz.sum_win, wl.n_q_heads), dtype=torch.float32, device=DEV)
+    runner = H.HostStepRunner(comp, b.q, b.win_indptr, b.tok_indptr, b.budget, wl.sm_scale, wl.causal)
+    b.page_table.fill_(-7)                       # the call must bring the tables from the host buffers
+    b.seq_len.zero_()
+    out = runner.run()
+    assert out["st"].tolist()[0] == 0
+    assert out["bud"].tolist() == wl.budgets
+    wl_like = (wl.n_kv_heads, wl.group, wl.head_dim, wl.page_size, wl.causal, wl.sm_scale)
+    units = [(15, 0, 7), (15, 1, 0), (15, 2, 1), (15, 3, 2), (0, 1, 4), (0, 2, 6)]
+    worst = _check_sampled_scores(b.pool, pt_before, sl_before, b.q[32:], b.win_indptr, b.tok_indptr, wl_like, comp.score,
+                                  units, layer_of_slab={s: 32 + s for s in range(16)}, budgets=wl.budgets,
+                                  sel_idx=comp.sel_idx, keep_indptr=comp.keep_indptr)
+    want_t = None
+    for l in (32, 47):
+        want_t = _check_layer_compaction(snap[l], b.pool[l], tables_before, comp.sel_idx, comp.keep_indptr, wl.budgets,
+                                         wl.n_kv_heads, l - 32)
+    _check_tables((b.page_table, b.seq_len, b.free_list, b.free_count), want_t)
+    fc = int(out["fc"])
+    assert fc == want_t.free_count
+    assert np.array_equal(out["pt"].numpy(), want_t.page_table) and np.array_equal(out["sl"].numpy(), want_t.seq_len)
+    assert np.array_equal(out["fl"].numpy()[:fc], want_t.free_list[:fc])
+    sel, ki = comp.sel_idx.cpu().numpy(), comp.keep_indptr.cpu().numpy()
+    for r in range(wl.n_req):
+        planted = b.planted[r].numpy()
+        for o in range(sel.shape[0]):
+            assert np.isin(planted, sel[o, ki[r]:ki[r + 1]]).all(), f"planted key evicted in unit ({o},{r})"
+    print(f"c3 through actkv_step_host: score max-rel {worst:.2e} on {len(units)} sampled units of the last group")
