@@ -75,7 +75,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     }
   }
 }
-// The same wait called by all 32 lanes of a converged warp, with ONE verdict for the warp: the callers go on
+// The same wait called by all 32 lanes of a converged warp, with ONE answer for the warp: the callers go on
 // to warp-collective instructions (tcgen05.ld, elect, __syncwarp) and must not split on a wait that some
 // lanes saw complete and others gave up on.
 __device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, volatile int* abort_flag, long long limit_cycles) {
