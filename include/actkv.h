@@ -519,6 +519,18 @@ int actkv_step_host(const actkv_pool_t* pool /* host */, const actkv_tables_t* t
                     const actkv_budget_params_t* params /* host, may be NULL without logits */,
                     const actkv_host_step_t* io /* host */, actkv_stream_t stream);
 
+/* actkv_step_device — the same whole step in one call for inputs that are ALREADY in device memory:
+ * the *_host members of `io` are ignored, q_dev / win_indptr_dev / tok_indptr_dev / budget_dev (and
+ * logits_dev / logit_indptr_dev for a budget update: logits_dev == NULL or n_rows == 0 skips it) and
+ * `tables` hold this step's inputs.  Runs actkv_budget, then (lse_supplied == 0) actkv_score_lse over
+ * all layers in as few launches as ws_score allows, writing lse_dev, or (lse_supplied != 0) takes
+ * lse_dev as the attention backend's LSE; then the layer groups as actkv_step_host does.  Everything
+ * is queued on `stream`; like the per-stage calls it neither synchronises nor copies, and status_dev
+ * is the caller's to clear and read. */
+int actkv_step_device(const actkv_pool_t* pool /* host */, const actkv_tables_t* tables /* host */,
+                      const actkv_budget_params_t* params /* host, may be NULL without logits */,
+                      const actkv_host_step_t* io /* host */, int32_t lse_supplied, actkv_stream_t stream);
+
 /* ---------------------------------------------------------------------------------------
  * actkv_compact_noalloc — actkv_compact without a caller-supplied workspace.
  * (The paper has no counterpart; this is a convenience of the library.)

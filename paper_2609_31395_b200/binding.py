@@ -25,7 +25,7 @@ EXPORTS = ["actkv_budget_workspace_bytes", "actkv_budget", "actkv_score_workspac
            "actkv_score_lse", "actkv_score_accumulate",
            "actkv_keep_indptr", "actkv_select_workspace_bytes", "actkv_select",
            "actkv_compact_workspace_bytes", "actkv_compact", "actkv_compact_noalloc",
-           "actkv_compact_noalloc_max_bytes", "actkv_step_host", "actkv_keepscore", "actkv_gather_f32",
+           "actkv_compact_noalloc_max_bytes", "actkv_step_host", "actkv_step_device", "actkv_keepscore", "actkv_gather_f32",
            "actkv_compact_inplace", "actkv_score_path", "actkv_debug_inject_stall", "actkv_score_sliding", "actkv_keepscore_select",
            "actkv_compact_deferred_workspace_bytes", "actkv_compact_begin", "actkv_compact_end", "actkv_score_overlap", "actkv_compact_stats",
            "actkv_compact_inplace_deferred_workspace_bytes", "actkv_compact_inplace_begin", "actkv_compact_inplace_end",
@@ -143,6 +143,9 @@ def load():
         fn.argtypes = [C.POINTER(PoolDesc), C.POINTER(TablesDesc), i32, i32, vp, i64, vp, vp, i32, vp, vp, sz, vp, vp]
     lib.actkv_gather_f32.restype = i32
     lib.actkv_gather_f32.argtypes = [vp, i64, vp, vp, i64, vp, i32, i32, i32, vp, i64, vp]
+    lib.actkv_step_device.restype = i32
+    lib.actkv_step_device.argtypes = [C.POINTER(PoolDesc), C.POINTER(TablesDesc), C.POINTER(BudgetParams),
+                                      C.POINTER(HostStep), i32, vp]
     lib.actkv_step_host.restype = i32
     lib.actkv_step_host.argtypes = [C.POINTER(PoolDesc), C.POINTER(TablesDesc), C.POINTER(BudgetParams),
                                     C.POINTER(HostStep), vp]
@@ -457,6 +460,13 @@ def actkv_gather_f32(src, src_stride, tok_indptr, sel_idx, sel_stride, keep_indp
                                  _ptr(keep_indptr, torch.int32, "keep_indptr"), n_outer, n_req, max_total_keep,
                                  _ptr(dst, torch.float32, "dst"), dst_stride, _stream(stream))
     _check("actkv_gather_f32", rc)
+
+
+def actkv_step_device(pool: PoolDesc, tables: TablesDesc, params: Optional[BudgetParams], io: HostStep, lse_supplied: bool,
+                      stream=None):
+    rc = load().actkv_step_device(C.byref(pool), C.byref(tables), None if params is None else C.byref(params),
+                                  C.byref(io), int(bool(lse_supplied)), _stream(stream))
+    _check("actkv_step_device", rc)
 
 
 def actkv_step_host(pool: PoolDesc, tables: TablesDesc, params: Optional[BudgetParams], io: HostStep, stream=None):

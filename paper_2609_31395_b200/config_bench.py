@@ -117,6 +117,30 @@ class _Fixed:
             return None
 
 
+    def timed_one_call(self, lse, reps: int) -> float:
+        """Whole-step milliseconds through actkv_step_device: the step as ONE call of the library on inputs that are
+        already on the device (`lse`: the supplied LSE, or None to have it computed)."""
+        if getattr(self, "runner", None) is None:
+            inst = self.inst
+            self.runner = H.HostStepRunner(self.comp, inst.q, inst.win_indptr, inst.tok_indptr, inst.budget, self.wl.sm_scale,
+                                           self.wl.causal)
+            self.runner.stage_inputs()
+        if lse is not None:
+            self.comp.lse.copy_(lse)
+        ms = []
+        for it in range(3 + reps):
+            self.restore()
+            e0, e1 = _event(), _event()
+            e0.record()
+            self.runner.run_device(lse_supplied=lse is not None)
+            e1.record()
+            torch.cuda.synchronize()
+            self.comp.check_status()
+            if it >= 3:
+                ms.append(e0.elapsed_time(e1))
+        return sum(ms) / len(ms)
+
+
 def _fixed_line(name: str, wl: synth.Workload, dev, pk: dict, reps: int, budget=None, scale_layers_to: Optional[int] = None,
                 inplace_too: bool = False, graph: bool = False) -> dict:
     fx = _Fixed(wl, dev, budget)
@@ -138,6 +162,7 @@ def _fixed_line(name: str, wl: synth.Workload, dev, pk: dict, reps: int, budget=
            "lse_supplied": _roofs(tokens, keep, upt, flops_pass, st_sup["total"], 1, pk)}
     if graph:
         out["graph_replay_ms_lse_internal"], out["graph_replay_ms_lse_supplied"] = g_int, g_sup
+        out["one_call_ms_lse_internal"], out["one_call_ms_lse_supplied"] = fx.timed_one_call(None, reps), fx.timed_one_call(lse, reps)
     if inplace_too:
         backup = fx.inst.pool.clone()
         st_ip = fx.timed(lse, reps, inplace=True, pool_backup=backup)
@@ -293,6 +318,8 @@ def _table1(dev, pk: dict, reps: int) -> List[dict]:
                           "us_graph_replay_lse_internal": None if gi is None else gi * 1e3,
                           "us_graph_replay_lse_supplied": None if gs is None else gs * 1e3,
                           "us_lse_internal": line["lse_internal"]["ms"] * 1e3, "us_lse_supplied": line["lse_supplied"]["ms"] * 1e3,
+                          "us_one_call_lse_internal": line["one_call_ms_lse_internal"] * 1e3,
+                          "us_one_call_lse_supplied": line["one_call_ms_lse_supplied"] * 1e3,
                           "stage_us_lse_internal": {k: v * 1e3 for k, v in line["stage_ms_lse_internal"].items()},
                           "tokens_per_s_lse_supplied": line["lse_supplied"]["tokens_per_s"],
                           "score_path": line["score_path"]})
@@ -305,7 +332,8 @@ def run_all(dev, pk: dict, only: Optional[List[str]] = None) -> List[dict]:
     out: List[dict] = []
     if "c1" in want:
         l1 = _fixed_line("c1_4k_x1", synth.config1(), dev, pk, reps=20, graph=True)
-        for k in ("graph_replay_ms_lse_internal", "graph_replay_ms_lse_supplied"):
+        for k in ("graph_replay_ms_lse_internal", "graph_replay_ms_lse_supplied", "one_call_ms_lse_internal",
+                  "one_call_ms_lse_supplied"):
             v = l1.pop(k)
             l1[k.replace("_ms_", "_us_")] = None if v is None else v * 1e3
         # a step of a few kernels on 17 MB that fit in L2: bound by launch latency, reported in microseconds

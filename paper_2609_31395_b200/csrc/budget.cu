@@ -487,9 +487,7 @@ int actkv_budget(const float* logits, const int32_t* tok_indptr, int32_t n_rows,
   float* pooled = (float*)((char*)ws + actkv::align_up((size_t)n_rows * 4, 256));
   if (n_rows > 0) {
     const size_t sm = sizeof(actkv::SweepSmem);
-    if (cudaFuncSetAttribute(actkv::token_conf_sweep_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm) !=
-        cudaSuccess)
-      return ACTKV_E_CUDA;
+    if (actkv::ensure_dyn_smem(actkv::token_conf_sweep_kernel, sm) != cudaSuccess) return ACTKV_E_CUDA;
     actkv::token_conf_sweep_kernel<<<(unsigned)n_rows, actkv::SW_NT, sm, s>>>(
         logits, tok_indptr, vocab, n_req, params->k, conf_hist, hist_len, hist_cap, redo, status);
     ACTKV_CHECK_LAUNCH();

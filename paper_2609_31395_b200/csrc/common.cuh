@@ -5,6 +5,8 @@
 #include <cuda_bf16.h>
 #include <stdint.h>
 
+#include <mutex>
+
 #include "../../include/actkv.h"
 
 #define ACTKV_CHECK_LAUNCH()                                   \
@@ -60,6 +62,52 @@ inline TablesView make_view(const actkv_tables_t* t) {
 }
 
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+// Per-kernel launch attributes are asked of the driver once per (kernel, device) and remembered: on steps of a few
+// dozen microseconds the attribute calls of every launch were a tenth of the time.
+struct KernelAttrCache {
+  struct Entry { const void* fn; int dev; int smem; int regs; };
+  static constexpr int kCap = 128;
+  Entry e[kCap];
+  int n = 0;
+  std::mutex m;
+  // entry of (fn, current device), created on first use; nullptr when the table is full or the device is unknown
+  Entry* find(const void* fn) {
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess) return nullptr;
+    for (int i = 0; i < n; ++i)
+      if (e[i].fn == fn && e[i].dev == dev) return &e[i];
+    if (n >= kCap) return nullptr;
+    e[n] = Entry{fn, dev, -1, -1};
+    return &e[n++];
+  }
+};
+inline KernelAttrCache& kernel_attr_cache() { static KernelAttrCache c; return c; }
+
+// cudaFuncSetAttribute(MaxDynamicSharedMemorySize) only when this kernel has not been given at least `bytes` yet.
+template <class K>
+inline cudaError_t ensure_dyn_smem(K kernel, size_t bytes) {
+  KernelAttrCache& c = kernel_attr_cache();
+  std::lock_guard<std::mutex> lock(c.m);
+  KernelAttrCache::Entry* en = c.find(reinterpret_cast<const void*>(kernel));
+  if (en != nullptr && en->smem >= (int)bytes) return cudaSuccess;
+  const cudaError_t rc = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
+  if (rc == cudaSuccess && en != nullptr) en->smem = (int)bytes;
+  return rc;
+}
+
+// Registers per thread the kernel was compiled to (cudaFuncGetAttributes, remembered); -1 on failure.
+template <class K>
+inline int kernel_num_regs(K kernel) {
+  KernelAttrCache& c = kernel_attr_cache();
+  std::lock_guard<std::mutex> lock(c.m);
+  KernelAttrCache::Entry* en = c.find(reinterpret_cast<const void*>(kernel));
+  if (en != nullptr && en->regs >= 0) return en->regs;
+  cudaFuncAttributes fa;
+  if (cudaFuncGetAttributes(&fa, kernel) != cudaSuccess) return -1;
+  if (en != nullptr) en->regs = fa.numRegs;
+  return fa.numRegs;
+}
 
 // Page id of logical page `lp` of request r; out-of-range ids are reported and replaced by 0.
 __device__ __forceinline__ int32_t checked_page(const TablesView& t, int32_t n_pages, int32_t r,

@@ -69,19 +69,63 @@ int wait(cudaStream_t s, cudaEvent_t e) { return cudaStreamWaitEvent(s, e, 0) ==
 
 }  // namespace
 
+// The passes that follow the LSE pass, in layer groups of layers_per_call layers: pooled score, select, compaction.
+// The budgets are first needed by the first select (`budget_ready`: an event to wait for before it, or nullptr).
+// With several layer groups the copies of group g run inside the pooled-score kernel of group g + 1
+// (actkv_compact_begin / actkv_score_overlap / actkv_compact_end); one index buffer suffices because the copies of
+// g are closed before the select of g + 1.
+static int step_groups(const actkv_pool_t* pool, const actkv_tables_t* tab, const actkv_host_step_t* io,
+                       actkv_stream_t stream, cudaEvent_t budget_ready) {
+  cudaStream_t s = (cudaStream_t)stream;
+  const int R = tab->n_req, NL = pool->n_layers, Hkv = pool->n_kv_heads;
+  const int lpc_post = io->layers_per_call > 0 && io->layers_per_call < NL ? io->layers_per_call : NL;
+  const int n_groups = (NL + lpc_post - 1) / lpc_post;
+  const size_t q_layer_bytes = (size_t)io->sum_win * io->n_q_heads * pool->head_dim * 2;
+  int pl0 = -1, pl1 = -1;                      // the group whose compaction is pending
+  for (int g = 0; g < n_groups; ++g) {
+    const int l0 = g * lpc_post, l1 = l0 + lpc_post < NL ? l0 + lpc_post : NL;
+    ACTKV_TRY(actkv_score_overlap(pool, tab, l0, l1, (const char*)io->q_dev + (size_t)l0 * q_layer_bytes, io->win_indptr_dev,
+                                  io->n_q_heads, io->lse_dev + (size_t)l0 * io->sum_win * io->n_q_heads, io->sm_scale,
+                                  io->causal, io->tok_indptr_dev, io->score_dev, nullptr, io->sum_win, io->max_win,
+                                  io->sum_tok, io->max_tok, io->ws_score, io->ws_score_bytes,
+                                  pl0 >= 0 ? io->ws_compact : nullptr, io->status_dev, stream));
+    if (pl0 >= 0)
+      ACTKV_TRY(actkv_compact_end(pool, tab, pl0, pl1, io->sel_idx_dev, io->sel_stride, io->keep_indptr_dev, io->budget_dev,
+                                  io->max_keep, io->ws_compact, io->ws_compact_bytes, io->status_dev, stream));
+    if (g == 0) {
+      if (budget_ready != nullptr) ACTKV_TRY(wait(s, budget_ready));
+      ACTKV_TRY(actkv_keep_indptr(tab->seq_len, io->budget_dev, R, io->keep_indptr_dev, stream));
+    }
+    ACTKV_TRY(actkv_select(io->score_dev, io->tok_indptr_dev, io->sum_tok, io->budget_dev, (l1 - l0) * Hkv, R,
+                           io->keep_indptr_dev, io->sel_idx_dev, io->sel_stride, nullptr, nullptr, nullptr, 0,
+                           io->status_dev, stream));
+    if (g == n_groups - 1) {
+      // nothing follows the last group that could carry its copies: the one-launch copy
+      ACTKV_TRY(actkv_compact(pool, tab, l0, l1, io->sel_idx_dev, io->sel_stride, io->keep_indptr_dev, io->budget_dev,
+                              io->max_keep, io->ws_compact, io->ws_compact_bytes, io->status_dev, stream));
+      pl0 = pl1 = -1;
+    } else {
+      ACTKV_TRY(actkv_compact_begin(pool, tab, l0, l1, io->sel_idx_dev, io->sel_stride, io->keep_indptr_dev, io->budget_dev,
+                                    io->max_keep, g > 0 ? 1 : 0, io->ws_compact, io->ws_compact_bytes, io->status_dev,
+                                    stream));
+      pl0 = l0;
+      pl1 = l1;
+    }
+  }
+  return ACTKV_OK;
+}
+
 static int step_enqueue(const actkv_pool_t* pool, const actkv_tables_t* tab, const actkv_budget_params_t* params,
                         const actkv_host_step_t* io, actkv_stream_t stream, StepStreams* st) {
   cudaStream_t s = (cudaStream_t)stream;
-  const int R = tab->n_req, NL = pool->n_layers, Hkv = pool->n_kv_heads;
+  const int R = tab->n_req, NL = pool->n_layers;
   const bool with_budget = io->logits_host != nullptr && io->n_rows > 0;
   int lpc = io->layers_per_call > 0 && io->layers_per_call < kDefaultGroupLayers ? io->layers_per_call
                                                                                  : kDefaultGroupLayers;
   if (lpc > NL) lpc = NL;
   if ((NL + lpc - 1) / lpc + 1 > kMaxGroups) return ACTKV_E_INVALID;
-  // The passes that follow the LSE work on resident queries: as many layers per call as the caller's score
-  // and index buffers hold (layers_per_call; all layers when it is left open).
-  const int lpc_post = io->layers_per_call > 0 && io->layers_per_call < NL ? io->layers_per_call : NL;
-  const int n_groups = (NL + lpc_post - 1) / lpc_post;
+  // (The passes that follow the LSE work on resident queries: as many layers per call as the caller's score
+  // and index buffers hold: step_groups.)
   // Groups of the query copies and LSE passes: a short first group, so that the first kernel starts
   // after a quarter of a group's transfer time, then groups of lpc layers.
   int lse_bound[kMaxGroups + 1];
@@ -144,40 +188,7 @@ static int step_enqueue(const actkv_pool_t* pool, const actkv_tables_t* tab, con
                               io->lse_dev + (size_t)l0 * io->sum_win * io->n_q_heads, io->sum_win, io->max_win,
                               io->sum_tok, io->max_tok, io->ws_score, io->ws_score_bytes, io->status_dev, stream));
   }
-  // ---- then the other passes; the budgets are first needed by the first select.  With several layer groups the
-  // copies of group g run inside the pooled-score kernels of group g + 1 (actkv_compact_begin / actkv_score_overlap /
-  // actkv_compact_end); one index buffer suffices because the copies of g are closed before the select of g + 1. ----
-  int pl0 = -1, pl1 = -1;                      // the group whose compaction is pending
-  for (int g = 0; g < n_groups; ++g) {
-    const int l0 = g * lpc_post, l1 = l0 + lpc_post < NL ? l0 + lpc_post : NL;
-    ACTKV_TRY(actkv_score_overlap(pool, tab, l0, l1, (const char*)io->q_dev + (size_t)l0 * q_layer_bytes, io->win_indptr_dev,
-                                  io->n_q_heads, io->lse_dev + (size_t)l0 * io->sum_win * io->n_q_heads, io->sm_scale,
-                                  io->causal, io->tok_indptr_dev, io->score_dev, nullptr, io->sum_win, io->max_win,
-                                  io->sum_tok, io->max_tok, io->ws_score, io->ws_score_bytes,
-                                  pl0 >= 0 ? io->ws_compact : nullptr, io->status_dev, stream));
-    if (pl0 >= 0)
-      ACTKV_TRY(actkv_compact_end(pool, tab, pl0, pl1, io->sel_idx_dev, io->sel_stride, io->keep_indptr_dev, io->budget_dev,
-                                  io->max_keep, io->ws_compact, io->ws_compact_bytes, io->status_dev, stream));
-    if (g == 0) {
-      if (with_budget) ACTKV_TRY(wait(s, st->budget));
-      ACTKV_TRY(actkv_keep_indptr(tab->seq_len, io->budget_dev, R, io->keep_indptr_dev, stream));
-    }
-    ACTKV_TRY(actkv_select(io->score_dev, io->tok_indptr_dev, io->sum_tok, io->budget_dev, (l1 - l0) * Hkv, R,
-                           io->keep_indptr_dev, io->sel_idx_dev, io->sel_stride, nullptr, nullptr, nullptr, 0,
-                           io->status_dev, stream));
-    if (g == n_groups - 1) {
-      // nothing follows the last group that could carry its copies: the one-launch copy
-      ACTKV_TRY(actkv_compact(pool, tab, l0, l1, io->sel_idx_dev, io->sel_stride, io->keep_indptr_dev, io->budget_dev,
-                              io->max_keep, io->ws_compact, io->ws_compact_bytes, io->status_dev, stream));
-      pl0 = pl1 = -1;
-    } else {
-      ACTKV_TRY(actkv_compact_begin(pool, tab, l0, l1, io->sel_idx_dev, io->sel_stride, io->keep_indptr_dev, io->budget_dev,
-                                    io->max_keep, g > 0 ? 1 : 0, io->ws_compact, io->ws_compact_bytes, io->status_dev,
-                                    stream));
-      pl0 = l0;
-      pl1 = l1;
-    }
-  }
+  ACTKV_TRY(step_groups(pool, tab, io, stream, with_budget ? st->budget : nullptr));
 
   // ---- device -> host: the step's results ----
   ACTKV_TRY(d2h(io->page_table_out_host, tab->page_table, tbl_bytes, s));
@@ -205,4 +216,39 @@ extern "C" int actkv_step_host(const actkv_pool_t* pool, const actkv_tables_t* t
   ok = (cudaStreamSynchronize((cudaStream_t)stream) == cudaSuccess) && ok;
   if (rc != ACTKV_OK) return rc;
   return ok ? ACTKV_OK : ACTKV_E_CUDA;
+}
+
+// The same step for inputs that are already in device memory: nothing is copied, no stream of the library's own is
+// used and the call does not synchronise.
+extern "C" int actkv_step_device(const actkv_pool_t* pool, const actkv_tables_t* tab,
+                                 const actkv_budget_params_t* params, const actkv_host_step_t* io,
+                                 int32_t lse_supplied, actkv_stream_t stream) {
+  if (!pool || !tab || !io) return ACTKV_E_INVALID;
+  if (tab->n_req <= 0 || pool->n_layers <= 0 || io->sum_win <= 0 || io->sum_tok <= 0) return ACTKV_E_INVALID;
+  const bool with_budget = io->logits_dev != nullptr && io->n_rows > 0;
+  if (with_budget && !params) return ACTKV_E_INVALID;
+  if (!io->lse_dev || !io->q_dev || !io->budget_dev) return ACTKV_E_INVALID;
+  const int R = tab->n_req, NL = pool->n_layers;
+  if (with_budget)
+    ACTKV_TRY(actkv_budget(io->logits_dev, io->logit_indptr_dev, io->n_rows, io->vocab, io->conf_hist_dev,
+                           io->hist_len_dev, io->hist_cap, params, tab->seq_len, io->budget_dev, io->budget_dev, nullptr,
+                           R, io->ws_budget, io->ws_budget_bytes, io->status_dev, stream));
+  if (!lse_supplied) {
+    // as many layers per LSE launch as the score workspace holds (fewer, larger launches waste less)
+    int per = NL;
+    for (int parts = 1; parts <= NL; ++parts) {
+      per = (NL + parts - 1) / parts;
+      if (actkv_score_workspace_bytes(pool, R, per, io->n_q_heads, io->sum_win, io->max_win, io->max_tok) <= io->ws_score_bytes)
+        break;
+    }
+    const size_t q_layer_bytes = (size_t)io->sum_win * io->n_q_heads * pool->head_dim * 2;
+    for (int l0 = 0; l0 < NL; l0 += per) {
+      const int l1 = l0 + per < NL ? l0 + per : NL;
+      ACTKV_TRY(actkv_score_lse(pool, tab, l0, l1, (const char*)io->q_dev + (size_t)l0 * q_layer_bytes, io->win_indptr_dev,
+                                io->n_q_heads, io->sm_scale, io->causal, io->tok_indptr_dev,
+                                io->lse_dev + (size_t)l0 * io->sum_win * io->n_q_heads, io->sum_win, io->max_win,
+                                io->sum_tok, io->max_tok, io->ws_score, io->ws_score_bytes, io->status_dev, stream));
+    }
+  }
+  return step_groups(pool, tab, io, stream, nullptr);
 }

@@ -298,7 +298,7 @@ int actkv_keepscore(float* score, const int32_t* tok_indptr, int32_t sum_tok, in
   const int64_t units = (int64_t)n_outer * n_req;
   if (units > 0x7fffffffLL) return ACTKV_E_INVALID;
   const int32_t p_q = (int32_t)lrintf(top_p * 10000.f);
-  if (cudaFuncSetAttribute(actkv::keepscore_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)actkv::KS_SMEM) != cudaSuccess)
+  if (actkv::ensure_dyn_smem(actkv::keepscore_kernel<false>, actkv::KS_SMEM) != cudaSuccess)
     return ACTKV_E_CUDA;
   actkv::keepscore_kernel<false><<<(unsigned)units, actkv::KS_NT, actkv::KS_SMEM, (cudaStream_t)stream>>>(
       score, tok_indptr, sum_tok, n_req, p_q, lambda, n_protect, keep_score, hit_mask, actkv::FusedSelectArgs{});
@@ -326,7 +326,7 @@ int actkv_keepscore_select(float* score, const int32_t* tok_indptr, int32_t sum_
   const int64_t units = (int64_t)n_outer * n_req;
   if (units > 0x7fffffffLL) return ACTKV_E_INVALID;
   const int32_t p_q = (int32_t)lrintf(top_p * 10000.f);
-  if (cudaFuncSetAttribute(actkv::keepscore_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)actkv::KS_SMEM) != cudaSuccess)
+  if (actkv::ensure_dyn_smem(actkv::keepscore_kernel<true>, actkv::KS_SMEM) != cudaSuccess)
     return ACTKV_E_CUDA;
   actkv::FusedSelectArgs fs{budget, keep_indptr, sel_idx, sel_stride, keep_mask, tie_report, status};
   actkv::keepscore_kernel<true><<<(unsigned)units, actkv::KS_NT, actkv::KS_SMEM, (cudaStream_t)stream>>>(

@@ -138,7 +138,7 @@ static int score_impl(int mode, const actkv_pool_t* pool, const actkv_tables_t* 
       if (grid1 > 0x7fffffffLL) return ACTKV_E_INVALID;
       const size_t sm1 = score_fma_smem_bytes(D, lay.rows_max, 1);
       if (sm1 > 200 * 1024) return ACTKV_E_INVALID;
-      if (cudaFuncSetAttribute(score_fma_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm1) != cudaSuccess)
+      if (ensure_dyn_smem(score_fma_kernel<1>, sm1) != cudaSuccess)
         return ACTKV_E_CUDA;
       score_fma_kernel<1><<<(unsigned)grid1, FMA_NT, sm1, s>>>(a);
       ACTKV_CHECK_LAUNCH();
@@ -158,7 +158,7 @@ static int score_impl(int mode, const actkv_pool_t* pool, const actkv_tables_t* 
   const int64_t grid2 = units * a.n_tiles;
   if (grid2 > 0x7fffffffLL) return ACTKV_E_INVALID;
   const size_t sm2 = score_fma_smem_bytes(D, lay.rows_max, 2);
-  if (cudaFuncSetAttribute(score_fma_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm2) != cudaSuccess)
+  if (ensure_dyn_smem(score_fma_kernel<2>, sm2) != cudaSuccess)
     return ACTKV_E_CUDA;
   score_fma_kernel<2><<<(unsigned)grid2, FMA_NT, sm2, s>>>(a);
   ACTKV_CHECK_LAUNCH();

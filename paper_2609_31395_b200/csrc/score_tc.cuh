@@ -166,7 +166,7 @@ inline int score_tc_launch_lse_c(const CUtensorMap& kmap, const tc::TcArgs& ta, 
                          : (d64 ? tc::score_tc_lse_kernel<NPOLY, false, 1, true> : tc::score_tc_lse_kernel<NPOLY, false, 2, true>))
                   : (rgs ? (d64 ? tc::score_tc_lse_kernel<NPOLY, true, 1, false> : tc::score_tc_lse_kernel<NPOLY, true, 2, false>)
                          : (d64 ? tc::score_tc_lse_kernel<NPOLY, false, 1, false> : tc::score_tc_lse_kernel<NPOLY, false, 2, false>));
-  if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return ACTKV_E_CUDA;
+  if (ensure_dyn_smem(kern, smem) != cudaSuccess) return ACTKV_E_CUDA;
   kern<<<grid, tc::LSE_THREADS, smem, s>>>(kmap, ta);
   ACTKV_CHECK_LAUNCH();
   return ACTKV_OK;
@@ -199,9 +199,8 @@ inline int score_tc_launch_pool_g(const CUtensorMap& kmap, const CUtensorMap& qm
   auto kern = ta.a.pool.head_dim == 64 ? tc::score_tc_pool_kernel<G, 1> : tc::score_tc_pool_kernel<G, 2>;
   // The warpgroups of this kernel re-divide the registers the launch allocates; the epilogue warpgroups would
   // wait for ever for registers that a smaller allocation does not have, so the allocation is checked first.
-  cudaFuncAttributes fa;
-  if (cudaFuncGetAttributes(&fa, kern) != cudaSuccess || fa.numRegs < tc::POOL_REGS_ENTRY) return ACTKV_E_CUDA;
-  if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return ACTKV_E_CUDA;
+  if (kernel_num_regs(kern) < tc::POOL_REGS_ENTRY) return ACTKV_E_CUDA;
+  if (ensure_dyn_smem(kern, smem) != cudaSuccess) return ACTKV_E_CUDA;
   kern<<<grid, tc::POOL_THREADS, smem, s>>>(kmap, qmap, ta);
   ACTKV_CHECK_LAUNCH();
   return ACTKV_OK;

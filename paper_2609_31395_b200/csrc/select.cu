@@ -119,7 +119,7 @@ int actkv_select(const float* score, const int32_t* tok_indptr, int32_t sum_tok,
   if (!score || !tok_indptr || !budget || !keep_indptr || !sel_idx) return ACTKV_E_INVALID;
   const int64_t units = (int64_t)n_outer * n_req;
   if (units > 0x7fffffffLL) return ACTKV_E_INVALID;
-  if (cudaFuncSetAttribute(actkv::select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)actkv::SEL_SMEM) != cudaSuccess)
+  if (actkv::ensure_dyn_smem(actkv::select_kernel, actkv::SEL_SMEM) != cudaSuccess)
     return ACTKV_E_CUDA;
   actkv::select_kernel<<<(unsigned)units, actkv::SEL_NT, actkv::SEL_SMEM, (cudaStream_t)stream>>>(
       score, tok_indptr, sum_tok, budget, n_req, keep_indptr, sel_idx, sel_stride, keep_mask,

@@ -421,6 +421,17 @@ class HostStepRunner:
         B.actkv_step_host(self.comp.pd, self.comp.td, self.params, self.io, stream)
         return self.h_out
 
+    def stage_inputs(self):
+        """Puts the step's inputs into the device staging buffers (for run_device; tables are the caller's)."""
+        for k in ("q", "win", "tok", "bud", "lg", "lgi"):
+            if k in self.d:
+                self.d[k].copy_(self.h_in[k], non_blocking=True)
+
+    def run_device(self, lse_supplied=False, stream=None):
+        """The whole step as ONE call on inputs already in device memory (actkv_step_device): asynchronous, no
+        copies; results are in the caller's pool, tables, free list and `self.d["bud"]`."""
+        B.actkv_step_device(self.comp.pd, self.comp.td, self.params, self.io, lse_supplied, stream)
+
 
 def sizes_of(inst, sel_stride: Optional[int] = None) -> StepSizes:
     """StepSizes for a synth.Instance (host-known lengths)."""

@@ -447,3 +447,46 @@ def test_select_reports_a_budget_beyond_the_index_buffer_and_stores_nothing_past
     # the request that fits was either written whole or, once the error was seen, not at all; never past its row
     rows = buf[: n_outer * sel_stride].view(n_outer, sel_stride).cpu().numpy()
     assert (rows[:, 100:] == -99).all()
+
+
+@pytest.mark.parametrize("lse_supplied", [False, True])
+def test_step_device_is_the_step_in_one_call(lse_supplied):
+    """actkv_step_device (inputs already in device memory, one asynchronous call) against the per-stage calls, with the
+    budgets coming from the confidence monitor inside the call."""
+    wl = synth.Workload("onecall", 5, 2, 8, [1500, 333, 700, 90], [32, 16, 24, 8], [400, 100, 200, 90],
+                        table_style="fragmented", seed=15, poison_tail=True)
+    R, T, V = wl.n_req, 70, 2048
+    logits, ltok = synth.confidence_logits(R, T, V, seed=9, device=DEV)
+    p = B.BudgetParams.paper_defaults()
+    # reference: monitor, then the step with those budgets, stage by stage
+    a = synth.generate(wl, DEV)
+    hist, hlen = torch.zeros((R, 256), dtype=torch.float32, device=DEV), torch.zeros(R, dtype=torch.int32, device=DEV)
+    bud_a = torch.zeros(R, dtype=torch.int32, device=DEV)
+    st = torch.zeros(4, dtype=torch.int32, device=DEV)
+    ws = torch.empty(B.actkv_budget_workspace_bytes(R * T, R, 256) + 256, dtype=torch.uint8, device=DEV)
+    B.actkv_budget(logits, ltok, R * T, V, hist, hlen, 256, p, a.seq_len, a.budget, bud_a, None, R, ws, st)
+    torch.cuda.synchronize()
+    budgets = bud_a.cpu().tolist()
+    sz = H.StepSizes(R, sum(wl.windows), max(wl.windows), sum(wl.seq_lens), max(wl.seq_lens),
+                     sum(min(b, L) for b, L in zip(budgets, wl.seq_lens)), max(min(b, L) for b, L in zip(budgets, wl.seq_lens)))
+    comp_a = H.Compressor(a.pool, a.page_table, a.seq_len, a.free_list, a.free_count, wl.n_q_heads, sz, want_lse=True)
+    comp_a.step(a.q, a.win_indptr, a.tok_indptr, bud_a, wl.sm_scale, wl.causal)
+    torch.cuda.synchronize()
+    comp_a.check_status()
+    # the same in one call, layer groups of two
+    b = synth.generate(wl, DEV)
+    comp_b = H.Compressor(b.pool, b.page_table, b.seq_len, b.free_list, b.free_count, wl.n_q_heads, sz, layers_per_call=2,
+                          want_lse=True, lse_layers_per_call=wl.n_layers)
+    runner = H.HostStepRunner(comp_b, b.q, b.win_indptr, b.tok_indptr, b.budget, wl.sm_scale, wl.causal, logits=logits,
+                              logit_indptr=ltok, hist_cap=256, params=p)
+    runner.stage_inputs()
+    if lse_supplied:
+        comp_b.lse.copy_(comp_a.lse)
+    runner.run_device(lse_supplied=lse_supplied)
+    torch.cuda.synchronize()
+    comp_b.check_status()
+    assert runner.d["bud"].cpu().tolist() == budgets
+    assert torch.equal(a.pool.view(torch.int16), b.pool.view(torch.int16))
+    assert torch.equal(a.page_table, b.page_table) and torch.equal(a.seq_len, b.seq_len)
+    assert torch.equal(a.free_list, b.free_list) and torch.equal(a.free_count, b.free_count)
+    assert torch.equal(comp_a.lse, comp_b.lse)
