@@ -9,9 +9,14 @@
 
 #include "../../include/actkv.h"
 
+// (a failed launch also drops the remembered launch attributes: after a device reset by the caller the kernels have
+//  lost them, and the next call asks the driver again)
 #define ACTKV_CHECK_LAUNCH()                                   \
   do {                                                         \
-    if (cudaGetLastError() != cudaSuccess) return ACTKV_E_CUDA; \
+    if (cudaGetLastError() != cudaSuccess) {                   \
+      ::actkv::forget_kernel_attrs();                          \
+      return ACTKV_E_CUDA;                                     \
+    }                                                          \
   } while (0)
 
 namespace actkv {
@@ -83,6 +88,11 @@ struct KernelAttrCache {
   }
 };
 inline KernelAttrCache& kernel_attr_cache() { static KernelAttrCache c; return c; }
+inline void forget_kernel_attrs() {
+  KernelAttrCache& c = kernel_attr_cache();
+  std::lock_guard<std::mutex> lock(c.m);
+  c.n = 0;
+}
 
 // cudaFuncSetAttribute(MaxDynamicSharedMemorySize) only when this kernel has not been given at least `bytes` yet.
 template <class K>
